@@ -1,0 +1,175 @@
+"""ctypes wrapper around the plain-C fp64 oracle (cadd_oracle.c).
+
+TEST INFRASTRUCTURE.  Only tests, the smoke check and the benchmark's CPU-baseline leg may use
+this module; the product path (the package and its CUDA library) never does.  Inputs are torch
+CPU tensors; outputs are torch CPU tensors allocated here.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "cadd_oracle.c")
+_LIB = os.path.join(_HERE, "libcadd_oracle.so")
+
+DT_BF16, DT_FP32 = 0, 1
+COST_QUADRATIC, COST_TABLE = 0, 1
+FLAG_FIXED_BUDGET = 4
+ROWS_LIVE, ROWS_DENSE = 0, 1
+ST_NONFINITE, ST_FEWER_THAN_K, ST_CAP_HIT, ST_FRONTIER_EXHAUSTED = 1, 2, 4, 8
+ST_L_EFF_CLAMPED, ST_COST_NONPOSITIVE, ST_BAD_N_NODES = 16, 32, 64
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain C, -O2, OpenMP over requests)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+                               "-ffp-contract=off", "-o", _LIB, _SRC, "-lm"])
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.cadd_oracle_row_argmax.restype = C.c_int32
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().cadd_oracle_num_threads())
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return DT_BF16
+    if t.dtype == torch.float32:
+        return DT_FP32
+    raise TypeError(f"unsupported logits dtype {t.dtype}")
+
+
+def _p(t: Optional[torch.Tensor]):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+@dataclass
+class OracleTree:
+    n_nodes: torch.Tensor
+    token_ids: torch.Tensor
+    parent_idx: torch.Tensor
+    depth: torch.Tensor
+    position_ids: torch.Tensor
+    node_logprob: torch.Tensor
+    phi: torch.Tensor
+    theta: torch.Tensor
+    mask_bits: torch.Tensor
+    mask_dense: Optional[torch.Tensor]
+    topk_token: torch.Tensor
+    topk_logprob: torch.Tensor
+    status: torch.Tensor
+    logZ: torch.Tensor
+    pop_gap: torch.Tensor
+    stop_gap: torch.Tensor
+    theta_curve: torch.Tensor
+    node_rank: torch.Tensor
+
+
+def row_softmax_topk(row: torch.Tensor, K: int):
+    """O1+O2 for one row: returns (m, logZ, tok[K], a[K], lp[K], k_eff, nonfinite, has_pinf)."""
+    assert row.dim() == 1 and row.is_contiguous() and row.device.type == "cpu"
+    tok = torch.empty(K, dtype=torch.int32)
+    a = torch.empty(K, dtype=torch.float64)
+    lp = torch.empty(K, dtype=torch.float64)
+    m, lz = C.c_double(), C.c_double()
+    ke, nf, pinf = C.c_int32(), C.c_int32(), C.c_int32()
+    lib().cadd_oracle_row_softmax_topk(_p(row), _dt(row), C.c_int64(row.numel()), K,
+                                       C.byref(m), C.byref(lz), _p(tok), _p(a), _p(lp),
+                                       C.byref(ke), C.byref(nf), C.byref(pinf))
+    return m.value, lz.value, tok, a, lp, ke.value, nf.value, pinf.value
+
+
+def build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[int] = None, *,
+               l_eff=None, bonus_token=None, ctx_len=None,
+               cost_kind: int = COST_QUADRATIC, cost_coef=None, cost_table=None, table_idx=None,
+               t_draft=None, flags: int = 0, dense_mask: bool = False) -> OracleTree:
+    """O1-O4 for a batch of requests; draft_logits is a CPU tensor [batch, L, V] (V contiguous)."""
+    x = draft_logits
+    assert x.device.type == "cpu" and x.dim() == 3 and x.stride(2) == 1
+    batch, L, V = x.shape
+    R = B_max + 1 if R is None else R
+    W = (R + 31) // 32
+    i32 = lambda *s: torch.empty(*s, dtype=torch.int32)
+    f64 = lambda *s: torch.empty(*s, dtype=torch.float64)
+    out = OracleTree(
+        n_nodes=i32(batch), token_ids=i32(batch, R), parent_idx=i32(batch, R), depth=i32(batch, R),
+        position_ids=i32(batch, R), node_logprob=f64(batch, R), phi=f64(batch), theta=f64(batch),
+        mask_bits=torch.empty(batch, R, W, dtype=torch.int32),
+        mask_dense=torch.empty(batch, R, R, dtype=torch.uint8) if dense_mask else None,
+        topk_token=i32(batch, L, K), topk_logprob=f64(batch, L, K), status=i32(batch),
+        logZ=f64(batch, L), pop_gap=f64(batch, R), stop_gap=f64(batch), theta_curve=f64(batch, R),
+        node_rank=i32(batch, R))
+    cv = lambda t, dt: None if t is None else t.to("cpu", dt).contiguous()
+    l_eff, bonus_token, ctx_len = cv(l_eff, torch.int32), cv(bonus_token, torch.int32), cv(ctx_len, torch.int32)
+    cost_coef, cost_table = cv(cost_coef, torch.float64), cv(cost_table, torch.float64)
+    table_idx, t_draft = cv(table_idx, torch.int32), cv(t_draft, torch.float64)
+    if cost_kind == COST_TABLE:
+        assert cost_table is not None and table_idx is not None and t_draft is not None
+        assert cost_table.shape[1] == B_max + 1
+    else:
+        assert cost_coef is not None and tuple(cost_coef.shape) == (batch, 4)
+    rc = lib().cadd_oracle_build_tree(
+        batch, L, C.c_int64(V), K, B_max, R, _dt(x), _p(x), C.c_int64(x.stride(0)), C.c_int64(x.stride(1)),
+        _p(l_eff), _p(bonus_token), _p(ctx_len), cost_kind, _p(cost_coef), _p(cost_table), _p(table_idx),
+        _p(t_draft), C.c_uint32(flags),
+        _p(out.n_nodes), _p(out.token_ids), _p(out.parent_idx), _p(out.depth), _p(out.position_ids),
+        _p(out.node_logprob), _p(out.phi), _p(out.theta), _p(out.mask_bits), _p(out.mask_dense),
+        _p(out.topk_token), _p(out.topk_logprob), _p(out.status),
+        _p(out.logZ), _p(out.pop_gap), _p(out.stop_gap), _p(out.theta_curve), _p(out.node_rank))
+    if rc != 0:
+        raise ValueError(f"cadd_oracle_build_tree rejected its arguments (rc={rc})")
+    return out
+
+
+@dataclass
+class OracleVerify:
+    node_argmax: torch.Tensor
+    accepted_len: torch.Tensor
+    accepted_nodes: torch.Tensor
+    next_bonus: torch.Tensor
+    status: torch.Tensor
+
+
+def row_argmax(row: torch.Tensor) -> int:
+    assert row.dim() == 1 and row.is_contiguous() and row.device.type == "cpu"
+    return int(lib().cadd_oracle_row_argmax(_p(row), _dt(row), C.c_int64(row.numel())))
+
+
+def verify_tree(target_logits: torch.Tensor, L: int, n_nodes, token_ids, parent_idx,
+                rows_mode: int = ROWS_LIVE) -> OracleVerify:
+    """O5+O6 for a batch; target_logits is a CPU tensor [batch, R, V] (V contiguous)."""
+    y = target_logits
+    assert y.device.type == "cpu" and y.dim() == 3 and y.stride(2) == 1
+    batch, R, V = y.shape
+    n_nodes = n_nodes.to("cpu", torch.int32).contiguous()
+    token_ids = token_ids.to("cpu", torch.int32).contiguous()
+    parent_idx = parent_idx.to("cpu", torch.int32).contiguous()
+    assert tuple(token_ids.shape) == (batch, R)
+    out = OracleVerify(torch.empty(batch, R, dtype=torch.int32), torch.empty(batch, dtype=torch.int32),
+                       torch.empty(batch, L, dtype=torch.int32), torch.empty(batch, dtype=torch.int32),
+                       torch.empty(batch, dtype=torch.int32))
+    rc = lib().cadd_oracle_verify_tree(
+        batch, C.c_int64(V), R, L, _dt(y), _p(y), C.c_int64(y.stride(0)), C.c_int64(y.stride(1)), rows_mode,
+        _p(n_nodes), _p(token_ids), _p(parent_idx),
+        _p(out.node_argmax), _p(out.accepted_len), _p(out.accepted_nodes), _p(out.next_bonus), _p(out.status))
+    if rc != 0:
+        raise ValueError(f"cadd_oracle_verify_tree rejected its arguments (rc={rc})")
+    return out
