@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the CaDDTree hot path: tree build + tree verify rounds per second on B200.
+
+A *step* is one decoding round of the whole hot path over one batch of synthetic input:
+    cadd_build_tree   (softmax + top-K over every live draft position, expansion, emission)
+    cadd_verify_tree  (argmax over every target row, accepted-path walk)
+The default workload is benchmark configuration 2 (batch 32, L 16, V 151936, bf16, K 8, B_max 256) with
+verification over the dense [batch, B_max+1, V] target tensor.  Inputs are seeded synthetic logits
+(paper_2606_01813_b200.synth); they are far larger than L2, so no flush is needed between steps.
+
+`python bench.py --gpus N --steps K --warmup W` prints ONE JSON line (rank 0).  With N > 1 (under
+torchrun) every rank runs an independent replica of the workload (requests are independent; there is no
+exchange step), and the value is the rounds all ranks completed per second of the slowest rank.
+`--impl reference` times the CPU oracle instead (the only baseline there is: the paper ships no code).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2606_01813_b200 import synth
+
+METRIC = "tree build+verify rounds/sec"
+UNIT = "rounds/s"
+KERNELS_PER_STEP = 4          # softmax_topk_partial, expand_emit, row_argmax, accept_walk
+
+# DRAM traffic of one row_argmax launch as a multiple of its algorithmic bytes, from the ncu capture
+# summarised in profiles/ (None until a capture exists).
+ARGMAX_TRAFFIC_RATIO = None
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device):
+        self.proc = None
+        self.path = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+            self.out.close()
+            rows = [l.strip().split(", ") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
+            sm, mx, reasons = [], [], set()
+            for r in rows:
+                if len(r) < 8:
+                    continue
+                try:
+                    sm.append(float(r[1])); mx.append(float(r[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                    if val.strip().lower() == "active":
+                        reasons.add(name)
+            if sm:
+                res = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+        except Exception:
+            pass
+        return res
+
+
+def cost_kwargs(G, c):
+    if c.kind == synth.COST_TABLE:
+        return dict(cost_kind=G.COST_TABLE, cost_table=c.table, table_idx=c.table_idx, t_draft=c.t_draft)
+    return dict(cost_kind=G.COST_QUADRATIC, cost_coef=c.coef)
+
+
+def run_ours(args, rank, world):
+    from paper_2606_01813_b200 import binding as G
+    from paper_2606_01813_b200 import build as cuda_build
+    cuda_build.build()                       # no-op when libcadd.so is current; raises if it cannot be built
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    cfg = synth.CONFIGS[args.workload]
+    seed = synth.config_seed(cfg) + 17 * rank
+    rows_mode = G.ROWS_DENSE if args.rows_mode == "dense" else G.ROWS_LIVE
+    flags = G.FLAG_FIXED_BUDGET if cfg.fixed_budget else 0
+
+    # ---- inputs resident in HBM ----
+    d = synth.make_draft_inputs(cfg, seed, device=str(dev))
+    c = synth.make_cost_inputs(cfg, seed)
+    kw = dict(l_eff=d.l_eff.to(dev), bonus_token=d.bonus_token.to(dev), ctx_len=d.ctx_len.to(dev), flags=flags)
+    ck = {k: (v.to(dev) if torch.is_tensor(v) else v) for k, v in cost_kwargs(G, c).items()}
+    ws = torch.empty(G.cadd_build_workspace_bytes(cfg.batch, cfg.L, cfg.V, cfg.K, cfg.B_max, cfg.R, cfg.torch_dtype),
+                     dtype=torch.uint8, device=dev)
+    tree = G.cadd_build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, workspace=ws, **kw, **ck)
+    torch.cuda.synchronize()
+    y = synth.make_target_logits(cfg, seed, d, tree.depth.cpu(), device=str(dev))
+    verdict = G.cadd_verify_tree(y, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode)
+    torch.cuda.synchronize()
+
+    def step():
+        G.cadd_build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=tree, **kw, **ck)
+        G.cadd_verify_tree(y, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, out=verdict)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----
+    K, Wm = args.steps, max(args.warmup, 3)
+    sampler = ClockSampler(dev) if rank == 0 else None
+    for _ in range(Wm):
+        step()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * K)]
+    barrier()
+    t_wall0 = time.perf_counter()
+    for i in range(K):
+        ev[3 * i].record()
+        G.cadd_build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=tree, **kw, **ck)
+        ev[3 * i + 1].record()
+        G.cadd_verify_tree(y, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, out=verdict)
+        ev[3 * i + 2].record()
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    # keep the GPU busy long enough for a few clock samples if the timed region was very short
+    if sampler is not None:
+        t_end = time.perf_counter() + max(0.0, 0.6 - t_wall)
+        while time.perf_counter() < t_end:
+            step()
+        torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler is not None else None
+    total_ms = ev[0].elapsed_time(ev[3 * K - 1])
+    build_ms = sum(ev[3 * i].elapsed_time(ev[3 * i + 1]) for i in range(K)) / K
+    verify_ms = sum(ev[3 * i + 1].elapsed_time(ev[3 * i + 2]) for i in range(K)) / K
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms = float(t.item())
+    value = world * K / (total_ms * 1e-3)
+
+    # ---- algorithmic bytes (logit bytes the kernels must read) ----
+    n_star = tree.n_nodes.cpu()
+    es = cfg.elem_bytes
+    build_bytes = int(d.l_eff.clamp(0, cfg.L).sum().item()) * cfg.V * es
+    rows_read = cfg.batch * cfg.R if rows_mode == G.ROWS_DENSE else int((n_star + 1).sum().item())
+    verify_bytes = rows_read * cfg.V * es
+    peak, peak_kind = measured_peak_gbs()
+    achieved = verify_bytes / (verify_ms * 1e-3) / 1e9
+    roofline = {"kernel": "row_argmax (+accept_walk, timed together)", "bound": "hbm", "achieved": round(achieved, 1),
+                "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(achieved / peak, 4),
+                "traffic": None if ARGMAX_TRAFFIC_RATIO is None else int(verify_bytes * ARGMAX_TRAFFIC_RATIO),
+                "algorithmic_bytes": verify_bytes, "ms": round(verify_ms, 4)}
+    build_gbs = build_bytes / (build_ms * 1e-3) / 1e9
+    build_info = {"kernels": "softmax_topk_partial + expand_emit", "ms": round(build_ms, 4), "algorithmic_bytes": build_bytes,
+                  "achieved": round(build_gbs, 1), "unit": "GB/s", "frac": round(build_gbs / peak, 4)}
+
+    # ---- end to end through the public API with HOST buffers ----
+    e2e = None
+    if not args.no_e2e:
+        hx = d.logits.cpu().pin_memory()
+        hy = torch.empty(y.shape, dtype=y.dtype, pin_memory=True)
+        hy.copy_(y)
+        h_tree = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (tree.n_nodes, tree.token_ids, tree.parent_idx, tree.depth)]
+        h_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (verdict.accepted_len, verdict.accepted_nodes, verdict.next_bonus)]
+        dx = torch.empty_like(d.logits)
+        dy = torch.empty_like(y)
+
+        def e2e_step():
+            dx.copy_(hx, non_blocking=True)
+            G.cadd_build_tree(dx, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=tree, **kw, **ck)
+            for h, t in zip(h_tree, (tree.n_nodes, tree.token_ids, tree.parent_idx, tree.depth)):
+                h.copy_(t, non_blocking=True)
+            dy.copy_(hy, non_blocking=True)
+            G.cadd_verify_tree(dy, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, out=verdict)
+            for h, t in zip(h_out, (verdict.accepted_len, verdict.accepted_nodes, verdict.next_bonus)):
+                h.copy_(t, non_blocking=True)
+
+        ke = max(1, min(K, args.e2e_steps))
+        e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(ke):
+            e2e_step()
+        e1.record()
+        barrier()
+        ems = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ems], device=dev, dtype=torch.float64)
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            ems = float(t.item())
+        h2d = hx.numel() * hx.element_size() + hy.numel() * hy.element_size()
+        d2h = sum(h.numel() * h.element_size() for h in h_tree + h_out)
+        e2e = {"value": round(world * ke / (ems * 1e-3), 3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": ke, "ms_per_step": round(ems / ke, 3)}
+        del hx, hy, dx, dy
+
+    # ---- the oracle timed on this machine's host cores, on a bounded sample (rank 0, N = 1 only) ----
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = oracle_sample(cfg, d, c, y, tree, rows_mode == G.ROWS_DENSE, args.cpu_requests)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": f"config {cfg.index} ({cfg.name}): batch={cfg.batch} L={cfg.L} V={cfg.V} {cfg.dtype} "
+                                   f"K={cfg.K} B_max={cfg.B_max} R={cfg.R}, verify rows_mode={args.rows_mode}",
+                       "l2": "inputs larger than L2 (no flush needed)", "parallelism": f"replicas x{world}",
+                       "n_star_mean": round(float(n_star.float().mean()), 2), "n_star_max": int(n_star.max()),
+                       "accepted_mean": round(float(verdict.accepted_len.float().mean().item()), 2)},
+            "roofline": roofline, "build": build_info, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "gpu_launches": KERNELS_PER_STEP * K, "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def oracle_sample(cfg, d, c, y, tree, dense, n_req):
+    """Time the CPU oracle, as it stands, on the first n_req requests of the workload."""
+    from oracle import cadd_oracle as O
+    nb = min(n_req, cfg.batch)
+    x = d.logits[:nb].cpu()
+    yy = y[:nb].cpu()
+    kw = dict(l_eff=d.l_eff[:nb], bonus_token=d.bonus_token[:nb], ctx_len=d.ctx_len[:nb],
+              flags=O.FLAG_FIXED_BUDGET if cfg.fixed_budget else 0)
+    if c.kind == synth.COST_TABLE:
+        kw.update(cost_kind=O.COST_TABLE, cost_table=c.table, table_idx=c.table_idx[:nb], t_draft=c.t_draft[:nb])
+    else:
+        kw.update(cost_coef=c.coef[:nb])
+    t0 = time.perf_counter()
+    ot = O.build_tree(x, cfg.K, cfg.B_max, cfg.R, **kw)
+    O.verify_tree(yy, cfg.L, ot.n_nodes, ot.token_ids, ot.parent_idx, O.ROWS_DENSE if dense else O.ROWS_LIVE)
+    dt = time.perf_counter() - t0
+    same = bool(torch.equal(ot.n_nodes, tree.n_nodes[:nb].cpu()) and torch.equal(ot.token_ids, tree.token_ids[:nb].cpu()))
+    return {"value": round((nb / cfg.batch) / dt, 4), "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"{nb} of {cfg.batch} requests of the same workload (one build + verify), {dt:.2f} s; "
+                      f"value scaled to whole rounds", "trees_match_gpu": same}
+
+
+def run_reference(args, rank, world):
+    """The reference arm: there is no reference implementation (the paper ships none), so the oracle is
+    timed on the host cores, each step a bounded sample of the workload."""
+    if rank != 0:
+        return
+    from oracle import cadd_oracle as O
+    O.build()
+    cfg = synth.CONFIGS[args.workload]
+    nb = min(args.cpu_requests, cfg.batch)
+    small = synth.scaled(cfg, batch=nb)
+    seed = synth.config_seed(cfg)
+    d = synth.make_draft_inputs(small, seed)
+    c = synth.make_cost_inputs(small, seed)
+    kw = dict(l_eff=d.l_eff, bonus_token=d.bonus_token, ctx_len=d.ctx_len, flags=O.FLAG_FIXED_BUDGET if cfg.fixed_budget else 0)
+    if c.kind == synth.COST_TABLE:
+        kw.update(cost_kind=O.COST_TABLE, cost_table=c.table, table_idx=c.table_idx, t_draft=c.t_draft)
+    else:
+        kw.update(cost_coef=c.coef)
+    dense = args.rows_mode == "dense"
+    ot = O.build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, **kw)
+    y = synth.make_target_logits(small, seed, d, ot.depth)
+
+    def step():
+        t = O.build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, **kw)
+        O.verify_tree(y, cfg.L, t.n_nodes, t.token_ids, t.parent_idx, O.ROWS_DENSE if dense else O.ROWS_LIVE)
+
+    K, Wm = args.steps, args.warmup
+    for _ in range(Wm):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(K):
+        step()
+    dt = time.perf_counter() - t0
+    value = K * (nb / cfg.batch) / dt
+    sample = f"each step = {nb} of {cfg.batch} requests of the workload (build + verify), value scaled to whole rounds"
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": Wm, "ms_per_step": round(dt / K * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"config {cfg.index} ({cfg.name}): batch={cfg.batch} L={cfg.L} V={cfg.V} {cfg.dtype} "
+                                   f"K={cfg.K} B_max={cfg.B_max} R={cfg.R}, verify rows_mode={args.rows_mode}"},
+            "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--rows-mode", default="dense", choices=["dense", "live"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-requests", type=int, default=8)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args, rank, world)
+    else:
+        args.steps = 500 if args.steps is None else args.steps
+        args.warmup = 10 if args.warmup is None else args.warmup
+        run_ours(args, rank, world)
+
+
+if __name__ == "__main__":
+    main()

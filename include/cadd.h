@@ -1,0 +1,171 @@
+/*
+ * cadd.h — C ABI of the B200 (sm_100a) implementation of the per-round hot path of CaDDTree
+ * ("Cost-Aware Diffusion Draft Trees for Speculative Decoding"): batched cost-aware draft-tree
+ * construction and tree verification.
+ *
+ * Conventions that hold for every call below
+ *   - Every data pointer is a DEVICE pointer owned by the caller, unless a comment says HOST.
+ *     The argument structs themselves live in HOST memory and are read during the call only.
+ *   - The library allocates nothing, frees nothing, never synchronises the device and never
+ *     touches a stream other than the one passed in.  Work is enqueued on `cuda_stream`
+ *     (a cudaStream_t cast to void*; NULL = the legacy default stream) and the call returns
+ *     immediately.  Results are valid once that stream reaches the end of the enqueued work.
+ *   - Scratch memory is passed in (`workspace`, `workspace_bytes`); its size comes from the
+ *     *_workspace_bytes query.  Its contents need no initialisation and are undefined after
+ *     the call.  Two calls that may overlap on the device need distinct workspaces.
+ *   - Return value: CADD_OK, or a negative code for an error detected on the host before any
+ *     kernel was launched (nothing is written in that case).  Conditions found on the device
+ *     are reported per request in the `status` output as CADD_STATUS_* bit flags.
+ *   - Index arithmetic is 64-bit; strides are counted in ELEMENTS of the logits dtype; the
+ *     vocabulary axis is contiguous.
+ *   - There is no CPU fallback: a machine without a CUDA device gets CADD_ERR_LAUNCH.
+ *
+ * Notation follows the paper: V vocabulary size, L draft block length (= maximum depth),
+ * K candidates kept per position, n the number of DRAFT nodes of the tree (the root, i.e. the
+ * bonus token, is row 0 and is not counted), B_max the cap on n, R >= B_max + 1 the row
+ * capacity of the per-request node arrays, C_d the drafting cost, C_v(n) the verification cost.
+ */
+#ifndef CADD_H_
+#define CADD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CADD_ABI_VERSION 1
+
+/* ---- return codes (host side, synchronous) ---- */
+#define CADD_OK              0
+#define CADD_ERR_NULL       -1   /* a required pointer is NULL */
+#define CADD_ERR_STRUCT_SIZE -2  /* struct_size does not match this library */
+#define CADD_ERR_SHAPE      -3   /* batch<1, L not in [1,64], K not in [1,64], V<1 or V>=2^31, B_max not in [0,2048], R<B_max+1 */
+#define CADD_ERR_DTYPE      -4   /* logits_dtype / cost_kind / rows_mode out of range */
+#define CADD_ERR_ALIGN      -5   /* logits base pointer not aligned to its element size, or a double/int array misaligned */
+#define CADD_ERR_WORKSPACE  -6   /* workspace NULL, misaligned (256 B) or smaller than the query says */
+#define CADD_ERR_LAUNCH     -7   /* a CUDA runtime call failed (wraps cudaGetLastError) */
+
+/* ---- per-request status bits (device side, written to `status`) ---- */
+#define CADD_STATUS_NONFINITE_INPUT      1   /* a NaN or +Inf draft logit was seen (NaN orders as -Inf; +Inf => empty tree) */
+#define CADD_STATUS_FEWER_THAN_K_FINITE  2   /* some live position has fewer than K finite logits */
+#define CADD_STATUS_CAP_HIT              4   /* expansion ended because n reached B_max */
+#define CADD_STATUS_FRONTIER_EXHAUSTED   8   /* expansion ended because no candidate was left */
+#define CADD_STATUS_L_EFF_CLAMPED       16   /* l_eff[b] was outside [0, L] */
+#define CADD_STATUS_COST_NONPOSITIVE    32   /* C_d + C_v(n) <= 0 (or not finite) was met; expansion stopped there */
+#define CADD_STATUS_BAD_N_NODES         64   /* verify: n_nodes[b] was outside [0, R-1] and was clamped */
+
+#define CADD_DTYPE_BF16 0
+#define CADD_DTYPE_FP32 1
+
+#define CADD_COST_QUADRATIC 0    /* C_v(n) = a + b n + c n^2, per request */
+#define CADD_COST_TABLE     1    /* C_v(n) = cost_table[table_idx[b]][n], n = 0..B_max */
+
+#define CADD_FLAG_EMIT_DENSE_MASK 1u   /* also write mask_dense */
+#define CADD_FLAG_EMIT_TOPK       2u   /* also write topk_token / topk_logprob */
+#define CADD_FLAG_FIXED_BUDGET    4u   /* ignore the stopping rule: expand to B_max (DDTree; the paper's constant-cost ablation, Table 2) */
+
+#define CADD_ROWS_LIVE  0        /* verify reads target rows 0..n_nodes[b] only */
+#define CADD_ROWS_DENSE 1        /* verify takes the argmax of all R rows */
+
+/*
+ * Arguments of cadd_build_tree: one decoding round's tree construction for `batch` requests.
+ * Implements Eq. 1 (per-position marginals q_i = softmax(l_i)), the top-K lists Algorithm 1
+ * requires, Algorithm 1 itself (best-first expansion over log prefix probabilities, Eq. 5, with
+ * the greedy stopping rule of Eq. 11 / Corollary 1 on the surrogate throughput of Eq. 7), and the
+ * draft-tree data structure with its ancestor mask (Section 3.3).
+ *
+ * Ordering rules (the paper is silent on ties): candidates of a position are ranked by
+ * (logit descending, token id ascending); nodes are popped by (score descending, depth ascending,
+ * token id ascending, parent row ascending).  Row 0 of every per-request array is the root.
+ * Row j >= 1 is the j-th popped node.  Rows above n_nodes[b] are padding: token -1, parent -1,
+ * depth 0, position 0, log-prob 0, empty mask row.
+ */
+typedef struct cadd_build_args {
+    uint32_t struct_size;          /* = sizeof(cadd_build_args) */
+    uint32_t flags;                /* CADD_FLAG_* */
+    int32_t  batch, L, K, B_max, R;
+    int32_t  logits_dtype;         /* CADD_DTYPE_* */
+    int64_t  V;
+    const void* draft_logits;      /* [batch, L, V]; element (b,i,v) at b*stride_b + i*stride_l + v */
+    int64_t  stride_b, stride_l;   /* in elements */
+    const int32_t* l_eff;          /* [batch] live positions per request, NULL => L (rows i >= l_eff[b] are never read) */
+    const int32_t* bonus_token;    /* [batch] token of the root, NULL => -1 */
+    const int32_t* ctx_len;        /* [batch] context length, NULL => 0; position_ids = ctx_len + depth */
+    int32_t  cost_kind;            /* CADD_COST_* */
+    int32_t  n_tables;             /* TABLE: number of rows of cost_table */
+    const double*  cost_coef;      /* QUADRATIC: [batch,4] = (C_d, a, b, c) */
+    const double*  cost_table;     /* TABLE: [n_tables, B_max+1] */
+    const int32_t* table_idx;      /* TABLE: [batch], each in [0, n_tables) */
+    const double*  t_draft;        /* TABLE: [batch] C_d */
+    /* outputs; n_nodes, token_ids, parent_idx, depth are required, the rest may be NULL */
+    int32_t* n_nodes;              /* [batch] n* */
+    int32_t* token_ids;            /* [batch,R] */
+    int32_t* parent_idx;           /* [batch,R] row of the parent, -1 for the root and padding */
+    int32_t* depth;                /* [batch,R] */
+    int32_t* position_ids;         /* [batch,R] */
+    double*  node_logprob;         /* [batch,R] log prefix probability sigma of each node (root 0) */
+    double*  phi;                  /* [batch] expected accepted draft tokens Phi*(n*) (Eq. 6) */
+    double*  theta;                /* [batch] surrogate throughput (1+Phi)/(C_d+C_v(n*)) (Eq. 7) */
+    uint32_t* mask_bits;           /* [batch,R,ceil(R/32)] bit c of row j set iff c == j or c is an ancestor of j */
+    uint8_t*  mask_dense;          /* [batch,R,R] same as bytes, written only with CADD_FLAG_EMIT_DENSE_MASK */
+    int32_t* topk_token;           /* [batch,L,K] written only with CADD_FLAG_EMIT_TOPK; -1 where absent */
+    double*  topk_logprob;         /* [batch,L,K] log q_i^(k); -Inf where absent */
+    int32_t* status;               /* [batch] CADD_STATUS_* bits */
+    void*    workspace;            /* >= cadd_build_workspace_bytes, 256-byte aligned */
+    size_t   workspace_bytes;
+} cadd_build_args;
+
+/*
+ * Arguments of cadd_verify_tree: greedy verification of the built trees (Section 3.1: a draft token
+ * is accepted iff it equals the argmax of the target distribution given its prefix; Section 3.3: the
+ * path with the longest accepted prefix is kept and the next bonus token follows it).
+ * Step 1: node_argmax[b,j] = argmax_v target_logits[b,j,v], ties to the lowest v, NaN ordered as -Inf.
+ * Step 2: walk from the root, at each node moving to the child whose token equals that node's argmax.
+ * next_bonus[b] is the argmax at the last accepted node.
+ */
+typedef struct cadd_verify_args {
+    uint32_t struct_size;          /* = sizeof(cadd_verify_args) */
+    uint32_t flags;                /* reserved, 0 */
+    int32_t  batch, L, R;
+    int32_t  logits_dtype;         /* CADD_DTYPE_* */
+    int32_t  rows_mode;            /* CADD_ROWS_* */
+    int32_t  reserved0;
+    int64_t  V;
+    const void* target_logits;     /* [batch, R, V]; element (b,j,v) at b*stride_b + j*stride_row + v */
+    int64_t  stride_b, stride_row; /* in elements */
+    const int32_t* n_nodes;        /* [batch]   from cadd_build_tree */
+    const int32_t* token_ids;      /* [batch,R] from cadd_build_tree */
+    const int32_t* parent_idx;     /* [batch,R] from cadd_build_tree */
+    /* outputs, all required except status */
+    int32_t* node_argmax;          /* [batch,R]; -1 for rows not read in LIVE mode */
+    int32_t* accepted_len;         /* [batch] alpha >= 0 */
+    int32_t* accepted_nodes;       /* [batch,L] rows of the accepted path in order, -1 padded */
+    int32_t* next_bonus;           /* [batch] */
+    int32_t* status;               /* [batch] CADD_STATUS_* bits, may be NULL */
+    void*    workspace;            /* >= cadd_verify_workspace_bytes (may be 0 => NULL allowed) */
+    size_t   workspace_bytes;
+} cadd_verify_args;
+
+/* ABI version of the loaded library (CADD_ABI_VERSION it was built with). */
+int cadd_version(void);
+
+/* Static, NUL-terminated description of a return code; never NULL, never freed. */
+const char* cadd_status_string(int code);
+
+/* Scratch sizes: pure host arithmetic on the shape fields (batch, L, K, B_max, R, V, dtype);
+ * pointers in the struct are ignored.  *out (HOST) receives the byte count. */
+int cadd_build_workspace_bytes(const cadd_build_args* a, size_t* out);
+int cadd_verify_workspace_bytes(const cadd_verify_args* a, size_t* out);
+
+/* Tree construction (Eq. 1, Algorithm 1, Section 3.3).  Asynchronous on `cuda_stream`. */
+int cadd_build_tree(const cadd_build_args* a, void* cuda_stream);
+
+/* Tree verification (Sections 3.1 and 3.3).  Asynchronous on `cuda_stream`. */
+int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CADD_H_ */

@@ -86,8 +86,9 @@ static double logit_at(const void *base, int dtype, int64_t idx)
  *   Z     = sum_v exp(x_v - m)      (ascending v)
  *   tok[k], a[k] = x_(k) - m, lp[k] = a[k] - log Z   for the K_eff best under
  *           (x descending, v ascending); K_eff = min(K, number of finite logits).
- * NaN and -Inf logits carry no mass and are never candidates; NaN or +Inf raise `nonfinite`,
- * +Inf additionally `has_pinf` (the caller then returns the empty tree).
+ * NaN and infinite logits carry no mass, are never candidates and do not enter m (m is the
+ * largest finite logit); NaN or +Inf raise `nonfinite`, +Inf additionally `has_pinf` (the caller
+ * then returns the empty tree; the lists reported for such a row are those of its finite logits).
  */
 int cadd_oracle_row_softmax_topk(const void *row, int dtype, int64_t V, int K,
                                  double *m_out, double *logZ_out,
@@ -99,7 +100,7 @@ int cadd_oracle_row_softmax_topk(const void *row, int dtype, int64_t V, int K,
     for (int64_t v = 0; v < V; ++v) {
         double x = logit_at(row, dtype, v);
         if (isnan(x)) { nf = 1; continue; }
-        if (isinf(x) && x > 0) { nf = 1; pinf = 1; }
+        if (isinf(x) && x > 0) { nf = 1; pinf = 1; continue; }   /* invalid input: flagged, kept out of m */
         if (x > m) m = x;
     }
     double Z = 0.0;

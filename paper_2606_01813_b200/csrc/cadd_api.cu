@@ -1,0 +1,222 @@
+// Host side of the C ABI declared in cadd.h: argument validation, workspace carve-up, kernel launches.
+// No allocation, no synchronisation, no state kept between calls.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cadd.h"
+#include "common.cuh"
+#include "expand_emit.cuh"
+#include "softmax_topk.cuh"
+#include "verify.cuh"
+
+namespace cadd {
+
+constexpr int kPreciseMin = 16;   // candidates per position whose exponentials are taken in fp64 (>= K)
+
+static inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+struct BuildPlan {
+    int KP;          // candidates kept per (row, segment)
+    int S;           // segments per row
+    size_t partial_bytes;
+    ExpandLayout lay;
+};
+
+static int sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 148;
+    return n;
+}
+
+static int check_build_shape(const cadd_build_args* a) {
+    if (!a) return CADD_ERR_NULL;
+    if (a->struct_size != sizeof(cadd_build_args)) return CADD_ERR_STRUCT_SIZE;
+    if (a->batch < 1 || a->L < 1 || a->L > 64 || a->K < 1 || a->K > 64 || a->V < 1 || a->V >= ((int64_t)1 << 31) ||
+        a->B_max < 0 || a->B_max > 2048 || a->R < a->B_max + 1)
+        return CADD_ERR_SHAPE;
+    if ((int64_t)a->batch * a->L * 8 >= ((int64_t)1 << 31) || (int64_t)a->batch * a->R >= ((int64_t)1 << 31)) return CADD_ERR_SHAPE;
+    if (a->logits_dtype != CADD_DTYPE_BF16 && a->logits_dtype != CADD_DTYPE_FP32) return CADD_ERR_DTYPE;
+    if (a->cost_kind != CADD_COST_QUADRATIC && a->cost_kind != CADD_COST_TABLE) return CADD_ERR_DTYPE;
+    return CADD_OK;
+}
+
+// Segments per row.  Whole rows are cheapest per element (one threshold warm-up per CTA), but the
+// grid must fill the resident-CTA slots of the machine evenly: take the smallest cut whose last wave
+// is at least 85 % full (else the fullest), never making a segment shorter than 4 iterations.
+constexpr int kMaxSegments = 8;
+static BuildPlan plan_build(const cadd_build_args* a, int slots) {
+    BuildPlan pl;
+    pl.KP = a->K > kPreciseMin ? a->K : kPreciseMin;
+    const int epc = a->logits_dtype == CADD_DTYPE_BF16 ? 8 : 4;
+    const int64_t rows = (int64_t)a->batch * a->L;
+    const int64_t chunks = a->V / epc;
+    int64_t cap = chunks / (4 * kTopkUnroll * kThreads);
+    if (cap > kMaxSegments) cap = kMaxSegments;
+    if (cap < 1) cap = 1;
+    int best = 1;
+    double best_eff = 0.0;
+    for (int S = 1; S <= (int)cap; ++S) {
+        const int64_t items = rows * S;
+        const int64_t waves = (items + slots - 1) / slots;
+        const double eff = (double)items / (double)(waves * slots);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = S; }
+        if (eff >= 0.85) { best = S; break; }
+    }
+    pl.S = best;
+    pl.partial_bytes = (size_t)rows * pl.S * seg_partial_stride(pl.KP);
+    pl.lay = expand_layout(a->L, a->K, pl.KP, pl.S, a->B_max);
+    return pl;
+}
+
+// Resident CTAs of the softmax/top-K kernel on the current device (occupancy x SM count).
+static int topk_slots(int dtype) {
+    int per_sm = 0;
+    cudaError_t e = dtype == CADD_DTYPE_BF16
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, kThreads, 0)
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, kThreads, 0);
+    if (e != cudaSuccess || per_sm < 1) { cudaGetLastError(); per_sm = 3; }
+    return per_sm * sm_count();
+}
+
+static size_t build_workspace_bytes(const BuildPlan& pl) { return (pl.partial_bytes + 255) & ~(size_t)255; }
+
+}  // namespace cadd
+
+using namespace cadd;
+
+extern "C" {
+
+int cadd_version(void) { return CADD_ABI_VERSION; }
+
+const char* cadd_status_string(int code) {
+    switch (code) {
+        case CADD_OK: return "ok";
+        case CADD_ERR_NULL: return "a required pointer is NULL";
+        case CADD_ERR_STRUCT_SIZE: return "struct_size does not match this library";
+        case CADD_ERR_SHAPE: return "shape out of range";
+        case CADD_ERR_DTYPE: return "unknown dtype, cost kind or rows mode";
+        case CADD_ERR_ALIGN: return "pointer or stride misaligned";
+        case CADD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case CADD_ERR_LAUNCH: return "CUDA launch failed";
+        default: return "unknown code";
+    }
+}
+
+int cadd_build_workspace_bytes(const cadd_build_args* a, size_t* out) {
+    int rc = check_build_shape(a);
+    if (rc != CADD_OK) return rc;
+    if (!out) return CADD_ERR_NULL;
+    // the SM count only steers how rows are cut; size for the largest cut so the answer is device independent
+    BuildPlan pl = plan_build(a, 148 * 3);
+    BuildPlan worst = pl;
+    worst.S = kMaxSegments;
+    worst.partial_bytes = (size_t)a->batch * a->L * kMaxSegments * seg_partial_stride(pl.KP);
+    *out = build_workspace_bytes(worst);
+    return CADD_OK;
+}
+
+int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
+    int rc = check_build_shape(a);
+    if (rc != CADD_OK) return rc;
+    if (!a->draft_logits || !a->n_nodes || !a->token_ids || !a->parent_idx || !a->depth) return CADD_ERR_NULL;
+    if (a->cost_kind == CADD_COST_QUADRATIC && !a->cost_coef) return CADD_ERR_NULL;
+    if (a->cost_kind == CADD_COST_TABLE && (!a->cost_table || !a->table_idx || !a->t_draft || a->n_tables < 1)) return CADD_ERR_NULL;
+    if ((a->flags & CADD_FLAG_EMIT_DENSE_MASK) && !a->mask_dense) return CADD_ERR_NULL;
+    if ((a->flags & CADD_FLAG_EMIT_TOPK) && !a->topk_token && !a->topk_logprob) return CADD_ERR_NULL;
+    const size_t es = a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
+    if (!aligned(a->draft_logits, es)) return CADD_ERR_ALIGN;
+    if (!aligned(a->cost_coef, 8) || !aligned(a->cost_table, 8) || !aligned(a->t_draft, 8) || !aligned(a->node_logprob, 8) ||
+        !aligned(a->phi, 8) || !aligned(a->theta, 8) || !aligned(a->topk_logprob, 8))
+        return CADD_ERR_ALIGN;
+    if (!aligned(a->n_nodes, 4) || !aligned(a->token_ids, 4) || !aligned(a->parent_idx, 4) || !aligned(a->depth, 4) ||
+        !aligned(a->position_ids, 4) || !aligned(a->mask_bits, 4) || !aligned(a->topk_token, 4) || !aligned(a->status, 4) ||
+        !aligned(a->l_eff, 4) || !aligned(a->bonus_token, 4) || !aligned(a->ctx_len, 4) || !aligned(a->table_idx, 4))
+        return CADD_ERR_ALIGN;
+    if (a->stride_l < a->V || a->stride_b < 0) return CADD_ERR_SHAPE;
+
+    const BuildPlan pl = plan_build(a, topk_slots(a->logits_dtype));
+    if (!a->workspace || !aligned(a->workspace, 256) || a->workspace_bytes < build_workspace_bytes(pl)) return CADD_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    TopkParams tp;
+    tp.logits = a->draft_logits; tp.V = a->V; tp.stride_b = a->stride_b; tp.stride_l = a->stride_l;
+    tp.L = a->L; tp.S = pl.S; tp.KP = pl.KP; tp.l_eff = a->l_eff; tp.partials = (unsigned char*)a->workspace;
+    const unsigned items = (unsigned)((int64_t)a->batch * a->L * pl.S);
+    if (a->logits_dtype == CADD_DTYPE_BF16) softmax_topk_partial_kernel<CADD_DTYPE_BF16><<<items, kThreads, 0, st>>>(tp);
+    else softmax_topk_partial_kernel<CADD_DTYPE_FP32><<<items, kThreads, 0, st>>>(tp);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+
+    ExpandParams ep;
+    ep.batch = a->batch; ep.L = a->L; ep.K = a->K; ep.KP = pl.KP; ep.S = pl.S; ep.B_max = a->B_max; ep.R = a->R;
+    ep.flags = a->flags; ep.partials = (const unsigned char*)a->workspace;
+    ep.l_eff = a->l_eff; ep.bonus_token = a->bonus_token; ep.ctx_len = a->ctx_len;
+    ep.cost_kind = a->cost_kind; ep.cost_coef = a->cost_coef; ep.cost_table = a->cost_table;
+    ep.table_idx = a->table_idx; ep.t_draft = a->t_draft;
+    ep.n_nodes = a->n_nodes; ep.token_ids = a->token_ids; ep.parent_idx = a->parent_idx; ep.depth = a->depth;
+    ep.position_ids = a->position_ids; ep.node_logprob = a->node_logprob; ep.phi = a->phi; ep.theta = a->theta;
+    ep.mask_bits = a->mask_bits; ep.mask_dense = a->mask_dense; ep.topk_token = a->topk_token;
+    ep.topk_logprob = a->topk_logprob; ep.status = a->status;
+    if (pl.lay.total > 48 * 1024) {
+        if (cudaFuncSetAttribute(expand_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.lay.total) != cudaSuccess) {
+            cudaGetLastError();
+            return CADD_ERR_LAUNCH;
+        }
+    }
+    expand_emit_kernel<<<a->batch, kThreads, pl.lay.total, st>>>(ep);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    return CADD_OK;
+}
+
+static int check_verify_shape(const cadd_verify_args* a) {
+    if (!a) return CADD_ERR_NULL;
+    if (a->struct_size != sizeof(cadd_verify_args)) return CADD_ERR_STRUCT_SIZE;
+    if (a->batch < 1 || a->L < 1 || a->L > 64 || a->R < 1 || a->V < 1 || a->V >= ((int64_t)1 << 31) ||
+        (int64_t)a->batch * a->R >= ((int64_t)1 << 31))
+        return CADD_ERR_SHAPE;
+    if (a->logits_dtype != CADD_DTYPE_BF16 && a->logits_dtype != CADD_DTYPE_FP32) return CADD_ERR_DTYPE;
+    if (a->rows_mode != CADD_ROWS_LIVE && a->rows_mode != CADD_ROWS_DENSE) return CADD_ERR_DTYPE;
+    return CADD_OK;
+}
+
+int cadd_verify_workspace_bytes(const cadd_verify_args* a, size_t* out) {
+    int rc = check_verify_shape(a);
+    if (rc != CADD_OK) return rc;
+    if (!out) return CADD_ERR_NULL;
+    *out = 0;
+    return CADD_OK;
+}
+
+int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream) {
+    int rc = check_verify_shape(a);
+    if (rc != CADD_OK) return rc;
+    if (!a->target_logits || !a->n_nodes || !a->token_ids || !a->parent_idx || !a->node_argmax || !a->accepted_len ||
+        !a->accepted_nodes || !a->next_bonus)
+        return CADD_ERR_NULL;
+    const size_t es = a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
+    if (!aligned(a->target_logits, es)) return CADD_ERR_ALIGN;
+    if (!aligned(a->n_nodes, 4) || !aligned(a->token_ids, 4) || !aligned(a->parent_idx, 4) || !aligned(a->node_argmax, 4) ||
+        !aligned(a->accepted_len, 4) || !aligned(a->accepted_nodes, 4) || !aligned(a->next_bonus, 4) || !aligned(a->status, 4))
+        return CADD_ERR_ALIGN;
+    if (a->stride_row < a->V || a->stride_b < 0) return CADD_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    ArgmaxParams ap;
+    ap.logits = a->target_logits; ap.V = a->V; ap.stride_b = a->stride_b; ap.stride_row = a->stride_row;
+    ap.R = a->R; ap.rows_mode = a->rows_mode; ap.n_nodes = a->n_nodes; ap.node_argmax = a->node_argmax;
+    const unsigned rows = (unsigned)((int64_t)a->batch * a->R);
+    if (a->logits_dtype == CADD_DTYPE_BF16) row_argmax_kernel<CADD_DTYPE_BF16><<<rows, kThreads, 0, st>>>(ap);
+    else row_argmax_kernel<CADD_DTYPE_FP32><<<rows, kThreads, 0, st>>>(ap);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+
+    WalkParams wp;
+    wp.batch = a->batch; wp.L = a->L; wp.R = a->R; wp.n_nodes = a->n_nodes; wp.token_ids = a->token_ids;
+    wp.parent_idx = a->parent_idx; wp.node_argmax = a->node_argmax; wp.accepted_len = a->accepted_len;
+    wp.accepted_nodes = a->accepted_nodes; wp.next_bonus = a->next_bonus; wp.status = a->status;
+    const int wpb = 4;
+    accept_walk_kernel<<<(a->batch + wpb - 1) / wpb, wpb * 32, 0, st>>>(wp);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    return CADD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,211 @@
+"""GPU parity tests: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cadd_oracle as O
+from paper_2606_01813_b200 import binding as G
+from paper_2606_01813_b200 import synth
+from parity_util import compare_build, compare_verify, run_both_build, to_cpu, LOGZ_TOL
+
+pytestmark = pytest.mark.gpu
+
+
+def quad_coef(batch, t_draft, a, b, c):
+    return torch.tensor([[t_draft, a, b, c]] * batch, dtype=torch.float64)
+
+
+def cost_kwargs(c: synth.CostInputs):
+    if c.kind == synth.COST_TABLE:
+        return dict(cost_kind=G.COST_TABLE, cost_table=c.table, table_idx=c.table_idx, t_draft=c.t_draft)
+    return dict(cost_kind=G.COST_QUADRATIC, cost_coef=c.coef)
+
+
+def round_trip(cfg, seed, rows_mode=G.ROWS_LIVE, dense_mask=False):
+    """One full round (build, target logits for the built tree, verify) on both sides."""
+    d = synth.make_draft_inputs(cfg, seed)
+    c = synth.make_cost_inputs(cfg, seed)
+    flags = (G.FLAG_FIXED_BUDGET if cfg.fixed_budget else 0) | (G.FLAG_EMIT_DENSE_MASK if dense_mask else 0)
+    gt, ot = run_both_build(d.logits, cfg.K, cfg.B_max, cfg.R, l_eff=d.l_eff, bonus_token=d.bonus_token,
+                            ctx_len=d.ctx_len, flags=flags, **cost_kwargs(c))
+    diag = compare_build(gt, ot, cfg.K)
+    if dense_mask:
+        assert torch.equal(to_cpu(gt.mask_dense), ot.mask_dense)
+    y = synth.make_target_logits(cfg, seed, d, ot.depth)
+    ov = O.verify_tree(y, cfg.L, ot.n_nodes, ot.token_ids, ot.parent_idx, rows_mode=rows_mode)
+    dev = lambda t: t.cuda()
+    gv = G.cadd_verify_tree(y.cuda(), cfg.L, dev(ot.n_nodes), dev(ot.token_ids), dev(ot.parent_idx), rows_mode=rows_mode)
+    torch.cuda.synchronize()
+    compare_verify(gv, ov)
+    return diag, ot, ov
+
+
+def test_library_reports_version():
+    assert G.cadd_version() == 1
+    assert G.cadd_status_string(0) == "ok"
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+@pytest.mark.parametrize("rows_mode", [G.ROWS_LIVE, G.ROWS_DENSE])
+def test_config1_full_round(seed, rows_mode):
+    diag, ot, ov = round_trip(synth.CONFIGS["c1"], seed, rows_mode, dense_mask=True)
+    assert not diag["exempt"]
+    assert diag["max_logZ_err"] < LOGZ_TOL
+
+
+# Reduced-size versions of configs 2-5: same generators, dtype, V and structure, fewer requests so the
+# oracle finishes in seconds.  V = 151936 spans many tiles, several segments and is not a power of two.
+SMALL = {
+    "c2": dict(batch=3),
+    "c3": dict(batch=3, B_max=128),
+    "c4": dict(batch=2, L=8, B_max=96),
+    "c4_stress": dict(batch=2, L=8, B_max=200),
+    "c5": dict(batch=6),
+}
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_reduced_configs_full_round(name):
+    cfg = synth.scaled(synth.CONFIGS[name], **SMALL[name])
+    diag, ot, ov = round_trip(cfg, synth.config_seed(cfg), G.ROWS_LIVE)
+    print(name, "n*", ot.n_nodes.tolist(), "alpha", ov.accepted_len.tolist(), diag)
+    assert len(diag["exempt"]) <= 1
+    assert diag["max_logZ_err"] < LOGZ_TOL
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("V", [1, 2, 7, 8, 9, 63, 257, 1000, 4099, 40000])
+def test_random_small_cases(dtype, V):
+    rng = np.random.default_rng(V)
+    for trial in range(6):
+        batch, L = int(rng.integers(1, 5)), int(rng.integers(1, 9))
+        K, B = int(rng.integers(1, 12)), int(rng.integers(0, 90))
+        g = torch.Generator().manual_seed(1000 * V + trial)
+        scale = float(rng.uniform(0.5, 5))
+        x = torch.randn(batch, L, V, generator=g) * scale
+        if trial % 2:
+            x = torch.round(x * 2) / 2                    # heavy ties
+        x = x.to(dtype)
+        coef = torch.tensor([[rng.uniform(0.1, 1), rng.uniform(0.2, 2), rng.uniform(1e-3, 5e-2), rng.uniform(0, 1e-3)]
+                             for _ in range(batch)], dtype=torch.float64)
+        flags = G.FLAG_FIXED_BUDGET if trial % 3 == 0 else 0
+        R = B + 1 + int(rng.integers(0, 40))
+        gt, ot = run_both_build(x, K, B, R, cost_coef=coef, flags=flags,
+                                ctx_len=torch.arange(batch, dtype=torch.int32) * 7)
+        diag = compare_build(gt, ot, K)
+        assert not diag["exempt"], diag
+        assert diag["max_logZ_err"] < 1e-6
+
+
+def test_unaligned_rows_and_strides():
+    """Row starts that are not 16-byte aligned (odd V, offset base) go through the scalar head/tail path."""
+    g = torch.Generator().manual_seed(5)
+    for dtype in (torch.bfloat16, torch.float32):
+        for V in (1001, 4099):
+            big = (torch.randn(3, 4, V + 13, generator=g) * 3).to(dtype)
+            x = big[:, :, 5:5 + V]                         # strided view, unaligned rows
+            coef = quad_coef(3, 0.3, 1.0, 0.002, 0.00002)
+            ot = O.build_tree(x.contiguous(), 8, 64, cost_coef=coef)
+            gt = G.cadd_build_tree(big.cuda()[:, :, 5:5 + V], 8, 64, cost_coef=coef, flags=G.FLAG_EMIT_TOPK)
+            torch.cuda.synchronize()
+            compare_build(gt, ot, 8)
+            y = (torch.randn(3, 65, V + 3, generator=g)).to(dtype)
+            ov = O.verify_tree(y[:, :, 1:1 + V].contiguous(), 4, ot.n_nodes, ot.token_ids, ot.parent_idx, rows_mode=O.ROWS_DENSE)
+            gv = G.cadd_verify_tree(y.cuda()[:, :, 1:1 + V], 4, ot.n_nodes.cuda(), ot.token_ids.cuda(), ot.parent_idx.cuda(),
+                                    rows_mode=G.ROWS_DENSE)
+            torch.cuda.synchronize()
+            compare_verify(gv, ov)
+
+
+def test_nonfinite_and_degenerate_inputs():
+    g = torch.Generator().manual_seed(9)
+    x = (torch.randn(6, 4, 3000, generator=g) * 2).to(torch.bfloat16)
+    x[0, 1, 5] = float("inf")                  # +Inf: empty tree
+    x[1, 0, 3] = float("nan")                  # NaN: ordered as -Inf
+    x[1, 2, 100:2000] = float("nan")
+    x[2, 1, :] = -float("inf")                 # a position with no finite logit
+    x[3, :, 7:] = -float("inf")                # only 7 finite logits per row: fewer than K
+    x[4] = 0.5                                 # all logits equal: order fixed by the tie-break alone
+    x[5, :, :] = torch.sort(x[5].float(), dim=-1).values.to(torch.bfloat16)   # ascending: every element a new best
+    coef = quad_coef(6, 0.3, 1.0, 0.002, 0.00002)
+    for flags in (0, G.FLAG_FIXED_BUDGET):
+        gt, ot = run_both_build(x, 9, 50, 60, cost_coef=coef, flags=flags,
+                                l_eff=torch.tensor([4, 4, 4, 4, 9, -1], dtype=torch.int32))
+        diag = compare_build(gt, ot, 9)
+        assert not diag["exempt"]
+    coef_bad = quad_coef(6, -2.0, 1.0, 0.002, 0.0)
+    gt, ot = run_both_build(x, 9, 50, 60, cost_coef=coef_bad)
+    compare_build(gt, ot, 9)
+    assert all(int(s) & G.STATUS_COST_NONPOSITIVE for s in to_cpu(gt.status))
+
+
+def test_table_cost_and_limits():
+    g = torch.Generator().manual_seed(10)
+    x = (torch.randn(2, 64, 500, generator=g) * 2).to(torch.float32)      # L = 64, K = 64: the limits of the ABI
+    n = torch.arange(301, dtype=torch.float64)
+    table = torch.stack([0.9 + 0.01 * n + 0.0004 * n * n, 0.5 + 0.002 * n])
+    kw = dict(cost_kind=G.COST_TABLE, cost_table=table, table_idx=torch.tensor([1, 0], dtype=torch.int32),
+              t_draft=torch.tensor([0.3, 0.2], dtype=torch.float64))
+    for flags in (0, G.FLAG_FIXED_BUDGET):
+        gt, ot = run_both_build(x, 64, 300, **kw, flags=flags)
+        assert not compare_build(gt, ot, 64)["exempt"]
+    x = (torch.randn(1, 3, 300, generator=g)).to(torch.bfloat16)          # B_max = 2048: the largest cap
+    gt, ot = run_both_build(x, 16, 2048, cost_coef=quad_coef(1, 1.0, 1.0, 0.0, 0.0), flags=G.FLAG_FIXED_BUDGET)
+    assert not compare_build(gt, ot, 16)["exempt"]
+    assert int(ot.n_nodes[0]) == 2048
+
+
+def test_argmax_ties_nan_and_walk():
+    g = torch.Generator().manual_seed(11)
+    batch, R, V, L = 3, 40, 151936, 6
+    y = torch.randn(batch, R, V, generator=g).to(torch.bfloat16)           # bf16 N(0,1): frequent exact ties at the top
+    y[0, 3, :] = float("nan")
+    y[0, 4, :] = -float("inf")
+    y[0, 5, 100] = float("nan"); y[0, 5, 7] = 9.0; y[0, 5, 150000] = 9.0
+    y[1, 2, V - 1] = 50.0
+    y[1, 3, 0] = 50.0
+    y[2, 0, :] = 0.0; y[2, 0, 5] = -0.0
+    x = (torch.randn(batch, L, 40, generator=g) * 2).to(torch.float32)
+    ot = O.build_tree(x, 4, R - 1, cost_coef=quad_coef(batch, 1.0, 1.0, 0.0, 0.0), flags=O.FLAG_FIXED_BUDGET)
+    for b in range(batch):                      # make the walk non-trivial: target agrees with the tree often
+        for j in range(R):
+            kids = [c for c in range(1, R) if int(ot.parent_idx[b, c]) == j]
+            if kids and j % 7 != 6 and not (b == 0 and j in (3, 4, 5)) and not (b == 2 and j == 0):
+                y[b, j, int(ot.token_ids[b, kids[0]])] = 60.0
+    for mode in (G.ROWS_LIVE, G.ROWS_DENSE):
+        n_nodes = ot.n_nodes.clone()
+        if mode == G.ROWS_LIVE:
+            n_nodes[1] = 17
+        ov = O.verify_tree(y, L, n_nodes, ot.token_ids, ot.parent_idx, rows_mode=mode)
+        gv = G.cadd_verify_tree(y.cuda(), L, n_nodes.cuda(), ot.token_ids.cuda(), ot.parent_idx.cuda(), rows_mode=mode)
+        torch.cuda.synchronize()
+        compare_verify(gv, ov)
+        assert int(ov.accepted_len.max()) >= 3
+    bad = ot.n_nodes.clone(); bad[0] = -5; bad[2] = 1000
+    ov = O.verify_tree(y, L, bad, ot.token_ids, ot.parent_idx)
+    gv = G.cadd_verify_tree(y.cuda(), L, bad.cuda(), ot.token_ids.cuda(), ot.parent_idx.cuda())
+    torch.cuda.synchronize()
+    compare_verify(gv, ov)
+    assert int(ov.status[0]) & O.ST_BAD_N_NODES
+
+
+def test_deterministic_and_reused_buffers():
+    cfg = synth.scaled(synth.CONFIGS["c2"], batch=2)
+    d = synth.make_draft_inputs(cfg, 3)
+    c = synth.make_cost_inputs(cfg, 3)
+    x = d.logits.cuda()
+    ws = torch.empty(G.cadd_build_workspace_bytes(cfg.batch, cfg.L, cfg.V, cfg.K, cfg.B_max, cfg.R, x.dtype),
+                     dtype=torch.uint8, device="cuda")
+    ws.fill_(0xAB)                              # scratch needs no initialisation
+    t1 = G.cadd_build_tree(x, cfg.K, cfg.B_max, cost_coef=c.coef, workspace=ws, flags=G.FLAG_EMIT_TOPK)
+    t2 = G.cadd_build_tree(x, cfg.K, cfg.B_max, cost_coef=c.coef, workspace=ws, flags=G.FLAG_EMIT_TOPK, out=None)
+    torch.cuda.synchronize()
+    for f in ("n_nodes", "token_ids", "parent_idx", "depth", "position_ids", "mask_bits", "topk_token", "status"):
+        assert torch.equal(getattr(t1, f), getattr(t2, f)), f
+    # evicted top-K candidates are folded into the partition sums in the order shared-memory atomics
+    # happened to hand out buffer slots (each thread folds with its own fp32 reference exponent), so
+    # floating-point outputs repeat to about 1e-10 in log space, not bit for bit
+    for f in ("node_logprob", "phi", "theta", "topk_logprob"):
+        a, b = getattr(t1, f), getattr(t2, f)
+        fin = torch.isfinite(a)
+        assert torch.equal(fin, torch.isfinite(b)) and torch.allclose(a[fin], b[fin], rtol=0, atol=2e-9), f
