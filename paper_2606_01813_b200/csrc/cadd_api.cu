@@ -72,9 +72,15 @@ static BuildPlan plan_build(const cadd_build_args* a, int slots) {
 // Resident CTAs of the softmax/top-K kernel on the current device (occupancy x SM count).
 static int topk_slots(int dtype) {
     int per_sm = 0;
+    if (cudaFuncSetAttribute(dtype == CADD_DTYPE_BF16 ? (const void*)softmax_topk_partial_kernel<CADD_DTYPE_BF16>
+                                                       : (const void*)softmax_topk_partial_kernel<CADD_DTYPE_FP32>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)topk_smem_bytes()) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
     cudaError_t e = dtype == CADD_DTYPE_BF16
-        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, kThreads, 0)
-        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, kThreads, 0);
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, kThreads, topk_smem_bytes())
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, kThreads, topk_smem_bytes());
     if (e != cudaSuccess || per_sm < 1) { cudaGetLastError(); per_sm = 3; }
     return per_sm * sm_count();
 }
@@ -135,7 +141,9 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
         return CADD_ERR_ALIGN;
     if (a->stride_l < a->V || a->stride_b < 0) return CADD_ERR_SHAPE;
 
-    const BuildPlan pl = plan_build(a, topk_slots(a->logits_dtype));
+    const int slots = topk_slots(a->logits_dtype);
+    if (slots < 1) return CADD_ERR_LAUNCH;
+    const BuildPlan pl = plan_build(a, slots);
     if (!a->workspace || !aligned(a->workspace, 256) || a->workspace_bytes < build_workspace_bytes(pl)) return CADD_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
@@ -143,8 +151,8 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
     tp.logits = a->draft_logits; tp.V = a->V; tp.stride_b = a->stride_b; tp.stride_l = a->stride_l;
     tp.L = a->L; tp.S = pl.S; tp.KP = pl.KP; tp.l_eff = a->l_eff; tp.partials = (unsigned char*)a->workspace;
     const unsigned items = (unsigned)((int64_t)a->batch * a->L * pl.S);
-    if (a->logits_dtype == CADD_DTYPE_BF16) softmax_topk_partial_kernel<CADD_DTYPE_BF16><<<items, kThreads, 0, st>>>(tp);
-    else softmax_topk_partial_kernel<CADD_DTYPE_FP32><<<items, kThreads, 0, st>>>(tp);
+    if (a->logits_dtype == CADD_DTYPE_BF16) softmax_topk_partial_kernel<CADD_DTYPE_BF16><<<items, kThreads, topk_smem_bytes(), st>>>(tp);
+    else softmax_topk_partial_kernel<CADD_DTYPE_FP32><<<items, kThreads, topk_smem_bytes(), st>>>(tp);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
 
     ExpandParams ep;

@@ -71,6 +71,14 @@ template <> struct Elem<CADD_DTYPE_BF16> {
         uint32_t bits = *reinterpret_cast<uint32_t*>(&m);
         return fmaxf(__uint_as_float(bits << 16), __uint_as_float(bits & 0xffff0000u));
     }
+    // maximum over four chunks (32 elements), NaN ignored
+    static __device__ __forceinline__ float max4(const uint4& a, const uint4& b, const uint4& c, const uint4& d) {
+        auto h = [](uint32_t x) { return *reinterpret_cast<const __nv_bfloat162*>(&x); };
+        auto m4 = [&](const uint4& w) { return __hmax2(__hmax2(h(w.x), h(w.y)), __hmax2(h(w.z), h(w.w))); };
+        __nv_bfloat162 m = __hmax2(__hmax2(m4(a), m4(b)), __hmax2(m4(c), m4(d)));
+        uint32_t bits = *reinterpret_cast<uint32_t*>(&m);
+        return fmaxf(__uint_as_float(bits << 16), __uint_as_float(bits & 0xffff0000u));
+    }
 };
 template <> struct Elem<CADD_DTYPE_FP32> {
     static constexpr int ES = 4;
@@ -83,6 +91,9 @@ template <> struct Elem<CADD_DTYPE_FP32> {
     static __device__ __forceinline__ float chunk_max(const uint4& w) {
         return fmaxf(fmaxf(__uint_as_float(w.x), __uint_as_float(w.y)),
                      fmaxf(__uint_as_float(w.z), __uint_as_float(w.w)));
+    }
+    static __device__ __forceinline__ float max4(const uint4& a, const uint4& b, const uint4& c, const uint4& d) {
+        return fmaxf(fmaxf(chunk_max(a), chunk_max(b)), fmaxf(chunk_max(c), chunk_max(d)));
     }
 };
 
