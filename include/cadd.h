@@ -46,6 +46,7 @@ extern "C" {
 #define CADD_ERR_ALIGN      -5   /* logits base pointer not aligned to its element size, or a double/int array misaligned */
 #define CADD_ERR_WORKSPACE  -6   /* workspace NULL, misaligned (256 B) or smaller than the query says */
 #define CADD_ERR_LAUNCH     -7   /* a CUDA runtime call failed (wraps cudaGetLastError) */
+#define CADD_ERR_STATIC_SCRATCH -8  /* cadd_build_tree_static_scratch: the problem needs more scratch than CADD_STATIC_SCRATCH_BYTES */
 
 /* ---- per-request status bits (device side, written to `status`) ---- */
 #define CADD_STATUS_NONFINITE_INPUT      1   /* a NaN or +Inf draft logit was seen (NaN orders as -Inf; +Inf => empty tree) */
@@ -164,6 +165,37 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream);
 
 /* Tree verification (Sections 3.1 and 3.3).  Asynchronous on `cuda_stream`. */
 int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream);
+
+/*
+ * cadd_build_tree for callers that cannot provide scratch memory.  (The paper has no counterpart to
+ * this entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where device allocation is off limits, for example a plugin inside a
+ * serving engine that owns the whole memory pool and forbids cudaMalloc after start-up, a real-time
+ * loop that must not take the allocator's locks, or a host language binding that can pass input and
+ * output tensors but has no allocator of its own to size a workspace with.  Such a caller still passes
+ * every input and output of cadd_build_args; the fields `workspace` and `workspace_bytes` are ignored.
+ *
+ * Where the scratch comes from: a fixed array of CADD_STATIC_SCRATCH_BYTES bytes that is part of the
+ * library's device image.  Every GPU on which the library is used holds those bytes from first use
+ * until the process ends.  The call itself allocates and frees nothing.
+ *
+ * Limits and rules
+ *   - Problems whose cadd_build_workspace_bytes() exceeds CADD_STATIC_SCRATCH_BYTES are refused with
+ *     CADD_ERR_STATIC_SCRATCH before anything is launched (8 MiB covers all five benchmark shapes,
+ *     e.g. batch 256 x L 16 x K 8, or batch 64 x L 32 x K 32).
+ *   - The first call on each device looks up the array's device address (a one-time, synchronous
+ *     runtime query made with that device current).  Make that first call outside any CUDA stream
+ *     capture; later calls only enqueue kernels.
+ *   - All calls on one device share the one array.  It needs no clearing between calls (every byte a
+ *     call reads was written earlier in the same call), but two calls that may run on the GPU at the
+ *     same time -- different streams, or different host threads -- would overwrite each other's
+ *     scratch: keep such calls on one stream or otherwise ordered.  Results are the same as those of
+ *     cadd_build_tree given a private workspace.
+ *   - Return codes and `status` bits otherwise as for cadd_build_tree.
+ */
+#define CADD_STATIC_SCRATCH_BYTES (8u << 20)
+int cadd_build_tree_static_scratch(const cadd_build_args* a, void* cuda_stream);
 
 #ifdef __cplusplus
 }

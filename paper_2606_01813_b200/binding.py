@@ -26,7 +26,9 @@ FLAG_EMIT_DENSE_MASK, FLAG_EMIT_TOPK, FLAG_FIXED_BUDGET = 1, 2, 4
 ROWS_LIVE, ROWS_DENSE = 0, 1
 
 EXPORTS = ("cadd_version", "cadd_status_string", "cadd_build_workspace_bytes", "cadd_verify_workspace_bytes",
-           "cadd_build_tree", "cadd_verify_tree")
+           "cadd_build_tree", "cadd_verify_tree", "cadd_build_tree_static_scratch")
+ERR_STATIC_SCRATCH = -8
+STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class BuildArgs(C.Structure):
@@ -77,6 +79,7 @@ def lib() -> C.CDLL:
         l.cadd_verify_workspace_bytes.argtypes = [C.POINTER(VerifyArgs), C.POINTER(C.c_size_t)]
         l.cadd_build_tree.argtypes = [C.POINTER(BuildArgs), C.c_void_p]
         l.cadd_verify_tree.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
+        l.cadd_build_tree_static_scratch.argtypes = [C.POINTER(BuildArgs), C.c_void_p]
         _lib = l
     return _lib
 
@@ -261,4 +264,60 @@ def cadd_verify_tree(target_logits: torch.Tensor, L: int, n_nodes: torch.Tensor,
         rc = lib().cadd_verify_tree(C.byref(a), _stream_ptr(stream))
     if rc != OK:
         raise CaddError(rc)
+    return out
+
+
+def cadd_build_tree_static_scratch(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[int] = None, *,
+                                   l_eff=None, bonus_token=None, ctx_len=None,
+                                   cost_kind: int = COST_QUADRATIC, cost_coef=None, cost_table=None,
+                                   table_idx=None, t_draft=None, flags: int = 0, out: Tree = None,
+                                   stream: Optional[torch.cuda.Stream] = None) -> Tree:
+    """cadd_build_tree without a workspace argument: the library uses its built-in scratch array.
+
+    For callers that may not allocate device memory (for instance code running inside a host
+    application that owns the memory pool): pass every input on the device already and a preallocated
+    `out`; the call then allocates nothing.  (If `out` is omitted it is allocated here with torch, which
+    is a convenience for tests.)  Shapes whose scratch need exceeds STATIC_SCRATCH_BYTES raise CaddError
+    with code ERR_STATIC_SCRATCH.  Calls on one device share the scratch: do not let two of them overlap
+    on the GPU.  The first call per device performs a one-time address look-up and belongs outside any
+    stream capture."""
+    x = draft_logits
+    if not x.is_cuda:
+        raise ValueError("draft_logits must be a CUDA tensor (there is no CPU path)")
+    if x.dim() != 3 or x.stride(2) != 1:
+        raise ValueError("draft_logits must be [batch, L, V] with a contiguous vocabulary axis")
+    dev = x.device
+    batch, L, V = x.shape
+    R = B_max + 1 if R is None else R
+    a = _build_args(x, K, B_max, R, flags, cost_kind)
+    a.draft_logits = x.data_ptr()
+    a.stride_b, a.stride_l = x.stride(0), x.stride(1)
+    keep = [_dev(l_eff, dev, torch.int32), _dev(bonus_token, dev, torch.int32), _dev(ctx_len, dev, torch.int32),
+            _dev(cost_coef, dev, torch.float64), _dev(cost_table, dev, torch.float64),
+            _dev(table_idx, dev, torch.int32), _dev(t_draft, dev, torch.float64)]
+    a.l_eff, a.bonus_token, a.ctx_len = _ptr(keep[0]), _ptr(keep[1]), _ptr(keep[2])
+    a.cost_coef, a.cost_table, a.table_idx, a.t_draft = _ptr(keep[3]), _ptr(keep[4]), _ptr(keep[5]), _ptr(keep[6])
+    a.n_tables = 0 if keep[4] is None else keep[4].shape[0]
+    if out is None:
+        W = (R + 31) // 32
+        i32 = lambda *s: torch.empty(*s, dtype=torch.int32, device=dev)
+        f64 = lambda *s: torch.empty(*s, dtype=torch.float64, device=dev)
+        out = Tree(n_nodes=i32(batch), token_ids=i32(batch, R), parent_idx=i32(batch, R), depth=i32(batch, R),
+                   position_ids=i32(batch, R), node_logprob=f64(batch, R), phi=f64(batch), theta=f64(batch),
+                   mask_bits=i32(batch, R, W),
+                   mask_dense=torch.empty(batch, R, R, dtype=torch.uint8, device=dev) if flags & FLAG_EMIT_DENSE_MASK else None,
+                   topk_token=i32(batch, L, K) if flags & FLAG_EMIT_TOPK else None,
+                   topk_logprob=f64(batch, L, K) if flags & FLAG_EMIT_TOPK else None,
+                   status=i32(batch))
+    a.n_nodes, a.token_ids, a.parent_idx, a.depth = _ptr(out.n_nodes), _ptr(out.token_ids), _ptr(out.parent_idx), _ptr(out.depth)
+    a.position_ids, a.node_logprob, a.phi, a.theta = _ptr(out.position_ids), _ptr(out.node_logprob), _ptr(out.phi), _ptr(out.theta)
+    a.mask_bits, a.mask_dense = _ptr(out.mask_bits), _ptr(out.mask_dense)
+    a.topk_token, a.topk_logprob, a.status = _ptr(out.topk_token), _ptr(out.topk_logprob), _ptr(out.status)
+    with torch.cuda.device(dev):
+        rc = lib().cadd_build_tree_static_scratch(C.byref(a), _stream_ptr(stream))
+    if rc != OK:
+        raise CaddError(rc)
+    for t in keep:
+        if t is not None:
+            t.record_stream(torch.cuda.current_stream() if stream is None else stream)
     return out

@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libcadd.so")
-SOURCES = [os.path.join(CSRC, "cadd_api.cu")]
+SOURCES = [os.path.join(CSRC, "cadd_api.cu"), os.path.join(CSRC, "cadd_static_scratch.cu")]
 
 
 def _newest_source_mtime() -> float:

@@ -105,6 +105,7 @@ const char* cadd_status_string(int code) {
         case CADD_ERR_ALIGN: return "pointer or stride misaligned";
         case CADD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case CADD_ERR_LAUNCH: return "CUDA launch failed";
+        case CADD_ERR_STATIC_SCRATCH: return "problem needs more scratch than the built-in static array holds";
         default: return "unknown code";
     }
 }
