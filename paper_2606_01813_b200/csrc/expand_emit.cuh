@@ -6,13 +6,17 @@
 //            sorted top-K list (token, a = logit - row max) and log Z, all in fp64
 //   phase 1  one thread: running log-partition sums S_d and the reachable depth
 //   phase 2  warp 0: the pop loop.  The frontier (Algorithm 1's heap) is striped over the 32 lanes;
-//            each lane caches the best entry of its stripe, a pop is a 128-bit warp arg-max
-//            (four redux.sync steps) followed by a rescan of the winner's stripe only.  Nodes are
-//            popped speculatively in groups; the group's exp(sigma), prefix sums Phi and throughput
-//            tests are then evaluated lane-parallel, and the first failing test fixes n*.  The pop
-//            order does not depend on the cost model, so this yields exactly Algorithm 1's tree.
-//   phase 3  all warps: write token / parent / depth / position / log-prob rows, padding, and the
-//            packed (and optionally dense) ancestor mask.
+//            each lane caches the best entry of its stripe in registers.  A pop is a warp arg-max over
+//            the cached bests on a 128-bit key (score, then the packed tie-break), taken 32 bits at a
+//            time with redux.sync and stopped as soon as one lane is left.  The popped entry's next
+//            sibling overwrites it in place, only the winner lane rescans its stripe, the first child
+//            goes to the next lane round-robin.  Nodes are popped speculatively in groups; the group's
+//            exp(sigma), prefix sums Phi and throughput tests are then evaluated lane-parallel, and the
+//            first failing test fixes n*.  The pop order does not depend on the cost model, so this
+//            yields exactly Algorithm 1's tree.
+//   phase 3  all threads: write token / parent / depth / position / log-prob rows and padding; zero
+//            the mask rows with coalesced stores, then one thread per node walks its ancestors and
+//            writes the few non-zero words (bytes for the dense form).
 #pragma once
 #include "common.cuh"
 #include "softmax_topk.cuh"
@@ -47,18 +51,29 @@ struct ExpandParams {
 };
 
 constexpr int kExpandWarps = kThreads / 32;
-constexpr int kMaskRowWords = 65;      // words that can hold a set bit: rows 0..2048
+
+// Tie-break half of a frontier / node key.  Smaller packed value = earlier in the pop order
+// (depth, then token id, then parent row); the rank within the position's top-K list rides along in
+// the low bits (it never decides: depth, token and parent already identify a node).
+__device__ __forceinline__ uint64_t pack_tiebreak(int depth, int token, int parent, int rank) {
+    return ((uint64_t)depth << 50) | ((uint64_t)(uint32_t)token << 19) | ((uint64_t)parent << 7) | (uint64_t)rank;
+}
+__device__ __forceinline__ int tb_depth(uint64_t tb) { return (int)(tb >> 50); }
+__device__ __forceinline__ int tb_token(uint64_t tb) { return (int)((tb >> 19) & 0x7fffffffu); }
+__device__ __forceinline__ int tb_parent(uint64_t tb) { return (int)((tb >> 7) & 0xfffu); }
+__device__ __forceinline__ int tb_rank(uint64_t tb) { return (int)(tb & 0x7fu); }
 
 // Dynamic shared memory layout of the expansion kernel (byte offsets), same arithmetic on host and device.
 struct ExpandLayout {
-    size_t a_list, lz, S, nA, nSig, region, tok_list, nTok, keff, maskrow, nPar, nDep, nRank, total;
-    int fr_slots;      // frontier slots per lane
+    size_t a_list, lz, S, nHi, nLo, region, tok_list, keff, total;
+    int fr_cap;        // frontier slots per lane
 };
 __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int KP, int S, int B_max) {
     ExpandLayout o;
     const size_t NR = (size_t)B_max + 1;
-    o.fr_slots = (2 * B_max + 1 + 31) / 32 + 1;
-    size_t frontier = (size_t)o.fr_slots * 32 * (8 + 8 + 4);
+    // every pop adds at most one entry (the sibling reuses the popped slot, the child is dealt round-robin)
+    o.fr_cap = (B_max + 1 + 31) / 32 + 1;
+    size_t frontier = (size_t)o.fr_cap * 32 * (8 + 8 + 8);
     size_t scratch = (size_t)kExpandWarps * S * KP * 8;
     size_t region = frontier > scratch ? frontier : scratch;
     region = (region + 7) & ~(size_t)7;
@@ -66,16 +81,11 @@ __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int KP, int 
     o.a_list = p;   p += (size_t)L * K * 8;
     o.lz = p;       p += (size_t)L * 8;
     o.S = p;        p += ((size_t)L + 1) * 8;
-    o.nA = p;       p += NR * 8;
-    o.nSig = p;     p += NR * 8;
+    o.nHi = p;      p += NR * 8;
+    o.nLo = p;      p += NR * 8;
     o.region = p;   p += region;
     o.tok_list = p; p += (size_t)L * K * 4;
-    o.nTok = p;     p += NR * 4;
     o.keff = p;     p += ((size_t)L + 2) * 4;
-    o.maskrow = p;  p += (size_t)kExpandWarps * kMaskRowWords * 4;
-    o.nPar = p;     p += NR * 2;  p = (p + 3) & ~(size_t)3;
-    o.nDep = p;     p += NR;
-    o.nRank = p;    p += NR;
     o.total = (p + 15) & ~(size_t)15;
     return o;
 }
@@ -92,18 +102,13 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
     double* a_list = (double*)(smem + lay.a_list);
     double* lz = (double*)(smem + lay.lz);
     double* Sd = (double*)(smem + lay.S);
-    double* nA = (double*)(smem + lay.nA);
-    double* nSig = (double*)(smem + lay.nSig);
+    uint64_t* nHi = (uint64_t*)(smem + lay.nHi);          // ordered image of the node's score sigma
+    uint64_t* nLo = (uint64_t*)(smem + lay.nLo);          // ~pack_tiebreak(depth, token, parent, rank)
     int32_t* tok_list = (int32_t*)(smem + lay.tok_list);
-    int32_t* nTok = (int32_t*)(smem + lay.nTok);
     int32_t* keff = (int32_t*)(smem + lay.keff);          // keff[d], d = 1..L
-    uint32_t* maskrow = (uint32_t*)(smem + lay.maskrow);
-    uint16_t* nPar = (uint16_t*)(smem + lay.nPar);
-    uint8_t* nDep = (uint8_t*)(smem + lay.nDep);
-    uint8_t* nRank = (uint8_t*)(smem + lay.nRank);
-    uint64_t* fHi = (uint64_t*)(smem + lay.region);
-    uint64_t* fLo = fHi + (size_t)lay.fr_slots * 32;
-    uint32_t* fPay = (uint32_t*)(fLo + (size_t)lay.fr_slots * 32);
+    uint64_t* fHi = (uint64_t*)(smem + lay.region);       // frontier, lane-major: [lane * fr_cap + slot]
+    uint64_t* fLo = fHi + (size_t)lay.fr_cap * 32;
+    double* fAp = (double*)(fLo + (size_t)lay.fr_cap * 32);  // the entry's parent's sum of (logit - row max)
 
     __shared__ int s_status, s_pinf, s_Lr, s_n;
     __shared__ double s_phi, s_theta;
@@ -181,7 +186,6 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         }
     }
     __syncthreads();
-
     // ---------------- phase 1: S_d and the reachable depth ----------------
     if (tid == 0) {
         Sd[0] = 0.0;
@@ -191,10 +195,9 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
             if (keff[d] == 0 && Lr == Le) Lr = d - 1;
         }
         s_Lr = Lr;
-        nA[0] = 0.0; nSig[0] = 0.0; nTok[0] = -1; nPar[0] = 0; nDep[0] = 0; nRank[0] = 0;
+        nHi[0] = ord64(0.0); nLo[0] = ~0ull;
     }
     __syncthreads();
-
     // ---------------- phase 2: the pop loop (warp 0) ----------------
     if (warp == 0) {
         const int Lr = s_Lr;
@@ -218,25 +221,39 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         else theta_prev = 1.0 / den0;
         if (s_pinf) ok = false;
 
-        // lane-private view of the frontier
-        int cnt = 0, bslot = -1;
-        uint64_t bhi = 0, blo = 0;
-        uint32_t brank = 0;
+        // Lane-private view of the frontier.  This lane's stripe holds cnt entries in shared memory; its
+        // best entry (b1) and, when b2ok, its exact second best (b2) are cached in registers, so that most
+        // pops need no look at the stripe at all.  (0,0) stands for "no entry": every real key is larger.
+        const int fbase = lane * lay.fr_cap;
+        int cnt = 0, b1slot = 0, b2slot = 0;
+        uint64_t b1hi = 0, b1lo = 0, b2hi = 0, b2lo = 0;
+        double b1ap = 0.0;
+        bool b2ok = true;
         int fsize = 0;
         unsigned pushctr = 0;
-        auto push = [&](double sigma, int d, int token, int parent, int rank) {
-            const uint64_t hi = ord64(sigma);
-            const uint64_t lo = ~(((uint64_t)d << 43) | ((uint64_t)(uint32_t)token << 12) | (uint64_t)parent);
-            const int t = pushctr & 31;
-            ++pushctr;
-            ++fsize;
-            if (lane == t) {
-                const int slot = cnt++;
-                fHi[slot * 32 + lane] = hi; fLo[slot * 32 + lane] = lo; fPay[slot * 32 + lane] = (uint32_t)rank;
-                if (bslot < 0 || hi > bhi || (hi == bhi && lo > blo)) { bhi = hi; blo = lo; bslot = slot; brank = rank; }
+        auto key_gt = [](uint64_t ahi, uint64_t alo, uint64_t bhi, uint64_t blo) { return ahi > bhi || (ahi == bhi && alo > blo); };
+        // recompute b1 and b2 from the stripe (only this lane runs it, reading its own earlier writes)
+        auto rescan_top2 = [&]() {
+            b1hi = b1lo = b2hi = b2lo = 0; b1slot = b2slot = 0;
+            for (int s2 = 0; s2 < cnt; ++s2) {
+                const uint64_t hi = fHi[fbase + s2], lo = fLo[fbase + s2];
+                if (key_gt(hi, lo, b1hi, b1lo)) { b2hi = b1hi; b2lo = b1lo; b2slot = b1slot; b1hi = hi; b1lo = lo; b1slot = s2; }
+                else if (key_gt(hi, lo, b2hi, b2lo)) { b2hi = hi; b2lo = lo; b2slot = s2; }
             }
+            b1ap = cnt > 0 ? fAp[fbase + b1slot] : 0.0;
+            b2ok = true;
         };
-        if (ok && Lr >= 1) push(a_list[0] - Sd[1], 1, tok_list[0], 0, 1);
+        if (ok && Lr >= 1) {                                // Algorithm 1, line 3: the heap starts with node (1)
+            if (lane == 0) {
+                b1hi = ord64(a_list[0] - Sd[1]);
+                b1lo = ~pack_tiebreak(1, tok_list[0], 0, 1);
+                b1ap = 0.0;
+                fHi[fbase] = b1hi; fLo[fbase] = b1lo; fAp[fbase] = 0.0;
+                cnt = 1;
+            }
+            fsize = 1;
+            pushctr = 1;
+        }
 
         int n = 0, popped = 0;
         bool stopped = false;
@@ -244,62 +261,115 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
             const int G = popped < 16 ? 8 : 32;
             int g = 0;
             while (g < G && popped < B_max && fsize > 0) {
-                // 128-bit arg-max over the lanes' cached bests
-                const bool has = cnt > 0;
-                uint32_t v = has ? (uint32_t)(bhi >> 32) : 0u;
+                // ---- arg-max of the 128-bit keys cached per lane, 32 bits at a time ----
+                uint32_t v = (uint32_t)(b1hi >> 32);        // empty lanes hold 0
                 uint32_t mx = __reduce_max_sync(kFullMask, v);
-                bool alive = has && v == mx;
-                v = alive ? (uint32_t)bhi : 0u;
-                mx = __reduce_max_sync(kFullMask, v);
-                alive = alive && v == mx;
-                v = alive ? (uint32_t)(blo >> 32) : 0u;
-                mx = __reduce_max_sync(kFullMask, v);
-                alive = alive && v == mx;
-                v = alive ? (uint32_t)blo : 0u;
-                mx = __reduce_max_sync(kFullMask, v);
-                alive = alive && v == mx;
-                const int win = __ffs(__ballot_sync(kFullMask, alive)) - 1;
-                const uint64_t whi = __shfl_sync(kFullMask, bhi, win);
-                const uint64_t wlo = __shfl_sync(kFullMask, blo, win);
-                const int r = (int)__shfl_sync(kFullMask, brank, win);
-                if (lane == win) {                          // remove the entry, rescan this stripe
-                    const int last = --cnt;
-                    if (bslot != last) {
-                        fHi[bslot * 32 + lane] = fHi[last * 32 + lane];
-                        fLo[bslot * 32 + lane] = fLo[last * 32 + lane];
-                        fPay[bslot * 32 + lane] = fPay[last * 32 + lane];
+                unsigned m = __ballot_sync(kFullMask, cnt > 0 && v == mx);
+                if (m & (m - 1)) {
+                    v = ((m >> lane) & 1u) ? (uint32_t)b1hi : 0u;
+                    mx = __reduce_max_sync(kFullMask, v);
+                    m &= __ballot_sync(kFullMask, v == mx);
+                    if (m & (m - 1)) {                      // equal scores: the tie-break decides
+                        v = ((m >> lane) & 1u) ? (uint32_t)(b1lo >> 32) : 0u;
+                        mx = __reduce_max_sync(kFullMask, v);
+                        m &= __ballot_sync(kFullMask, v == mx);
+                        if (m & (m - 1)) {
+                            v = ((m >> lane) & 1u) ? (uint32_t)b1lo : 0u;
+                            mx = __reduce_max_sync(kFullMask, v);
+                            m &= __ballot_sync(kFullMask, v == mx);
+                        }
                     }
-                    bslot = -1; bhi = 0; blo = 0;
-                    for (int s = 0; s < cnt; ++s) {
-                        const uint64_t hi = fHi[s * 32 + lane], lo = fLo[s * 32 + lane];
-                        if (bslot < 0 || hi > bhi || (hi == bhi && lo > blo)) { bhi = hi; blo = lo; bslot = s; }
-                    }
-                    if (bslot >= 0) brank = fPay[bslot * 32 + lane];
                 }
-                --fsize;
+                const int win = __ffs(m) - 1;
+                const uint64_t whi = __shfl_sync(kFullMask, b1hi, win);
+                const uint64_t wlo = __shfl_sync(kFullMask, b1lo, win);
+                const double Apar = __shfl_sync(kFullMask, b1ap, win);
                 const uint64_t tb = ~wlo;
-                const int d = (int)(tb >> 43);
-                const int token = (int)((tb >> 12) & 0x7fffffffu);
-                const int par = (int)(tb & 0xfffu);
-                const double A = nA[par] + a_list[(d - 1) * K + (r - 1)];
+                const int d = tb_depth(tb), par = tb_parent(tb), r = tb_rank(tb);
                 const int j = ++popped;
-                if (lane == 0) {
-                    nA[j] = A; nSig[j] = unord64(whi); nTok[j] = token;
-                    nPar[j] = (uint16_t)par; nDep[j] = (uint8_t)d; nRank[j] = (uint8_t)r;
+                // ---- the popped node and its two successors (Algorithm 1, lines 12-19); every lane forms
+                //      both successor keys so that all shared-memory reads are issued together ----
+                const double* arow = a_list + (d - 1) * K;
+                const double a_cur = arow[r - 1];
+                const int rs = r < K ? r : K - 1;                       // index of the next sibling (clamped)
+                const int dc = d < L ? d : L - 1;                       // row of the first child (clamped)
+                const double a_sib = arow[rs], a_chi = a_list[dc * K];
+                const int tok_sib = tok_list[(d - 1) * K + rs], tok_chi = tok_list[dc * K];
+                const double S_d = Sd[d], S_c = Sd[dc + 1];
+                const bool has_sib = r < keff[d];
+                const bool has_child = d < Lr;
+                const double A = Apar + a_cur;
+                const uint64_t sib_hi = ord64((Apar + a_sib) - S_d);
+                const uint64_t sib_lo = ~pack_tiebreak(d, tok_sib, par, r + 1);
+                const uint64_t chi_hi = ord64((A + a_chi) - S_c);
+                const uint64_t chi_lo = ~pack_tiebreak(d + 1, tok_chi, j, 1);
+                if (lane == 1) nHi[j] = whi;
+                if (lane == 2) nLo[j] = wlo;
+                const bool w = lane == win;
+                if (has_sib) {
+                    // The next sibling takes the popped entry's slot (same parent).  Written without
+                    // divergent branches: every lane evaluates the selects, only the winner's take effect.
+                    const int s1 = b1slot;
+                    if (w) { fHi[fbase + s1] = sib_hi; fLo[fbase + s1] = sib_lo; }
+                    if (w && cnt > 1 && !b2ok) {
+                        rescan_top2();                      // rare: the second best was not known
+                    } else {
+                        // an empty b2 is (0,0), so a lone sibling always wins
+                        const bool sib_wins = key_gt(sib_hi, sib_lo, b2hi, b2lo);
+                        const bool promote = w && !sib_wins;        // the cached second best moves up and the
+                        const bool keep = w && sib_wins;            // sibling becomes a candidate second
+                        const double ap2 = promote ? fAp[fbase + b2slot] : b1ap;
+                        const uint64_t o2hi = b2hi, o2lo = b2lo;
+                        const int o2slot = b2slot;
+                        b1hi = keep ? sib_hi : (promote ? o2hi : b1hi);
+                        b1lo = keep ? sib_lo : (promote ? o2lo : b1lo);
+                        b1slot = promote ? o2slot : b1slot;
+                        b1ap = ap2;
+                        b2hi = promote ? sib_hi : b2hi;
+                        b2lo = promote ? sib_lo : b2lo;
+                        b2slot = promote ? s1 : b2slot;
+                        b2ok = promote ? (cnt == 2) : b2ok;
+                    }
+                } else if (w) {                             // no sibling: the last entry moves into the hole
+                    const int s1 = b1slot;
+                    const int last = --cnt;
+                    if (s1 != last) {
+                        fHi[fbase + s1] = fHi[fbase + last]; fLo[fbase + s1] = fLo[fbase + last]; fAp[fbase + s1] = fAp[fbase + last];
+                        if (b2slot == last) b2slot = s1;
+                    }
+                    if (cnt == 0) { b1hi = b1lo = b2hi = b2lo = 0; b2ok = true; }
+                    else if (!b2ok) rescan_top2();
+                    else {
+                        b1hi = b2hi; b1lo = b2lo; b1slot = b2slot; b1ap = fAp[fbase + b2slot];
+                        b2hi = b2lo = 0;
+                        b2ok = cnt == 1;
+                    }
                 }
-                __syncwarp();
-                if (r + 1 <= keff[d])                       // next sibling
-                    push((nA[par] + a_list[(d - 1) * K + r]) - Sd[d], d, tok_list[(d - 1) * K + r], par, r + 1);
-                if (d < Lr)                                 // first child
-                    push((A + a_list[d * K]) - Sd[d + 1], d + 1, tok_list[d * K], j, 1);
+                if (has_child) {                            // the first child goes to the next lane in turn
+                    const bool mine = lane == (int)(pushctr & 31);
+                    ++pushctr;
+                    if (mine) { fHi[fbase + cnt] = chi_hi; fLo[fbase + cnt] = chi_lo; fAp[fbase + cnt] = A; }
+                    const bool first = mine && key_gt(chi_hi, chi_lo, b1hi, b1lo);   // new best: the old best is the exact second
+                    const bool second = mine && !first && b2ok && key_gt(chi_hi, chi_lo, b2hi, b2lo);
+                    b2hi = first ? b1hi : (second ? chi_hi : b2hi);
+                    b2lo = first ? b1lo : (second ? chi_lo : b2lo);
+                    b2slot = first ? b1slot : (second ? cnt : b2slot);
+                    b2ok = first ? true : b2ok;
+                    b1hi = first ? chi_hi : b1hi;
+                    b1lo = first ? chi_lo : b1lo;
+                    b1slot = first ? cnt : b1slot;
+                    b1ap = first ? A : b1ap;
+                    cnt += mine ? 1 : 0;
+                }
+                fsize += (int)has_sib + (int)has_child - 1;
                 ++g;
             }
+            __syncwarp();                                   // the node records written above are read below
             if (g == 0) break;
-            __syncwarp();
             // evaluate the group: rows n+1 .. n+g, one per lane
             const int j = n + 1 + lane;
             const bool act = lane < g;
-            const double delta = act ? exp(nSig[j]) : 0.0;
+            const double delta = act ? exp(unord64(nHi[j])) : 0.0;
             double cum = delta;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -335,7 +405,6 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         }
     }
     __syncthreads();
-
     // ---------------- phase 3: emission ----------------
     const int n = s_n;
     const int ctx = p.ctx_len ? p.ctx_len[b] : 0;
@@ -351,7 +420,10 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         int t = -1, par = -1, d = 0, pos = 0;
         double lp = 0.0;
         if (j == 0) { t = bonus; pos = ctx; }
-        else if (j <= n) { t = nTok[j]; par = nPar[j]; d = nDep[j]; pos = ctx + d; lp = nSig[j]; }
+        else if (j <= n) {
+            const uint64_t tb = ~nLo[j];
+            t = tb_token(tb); par = tb_parent(tb); d = tb_depth(tb); pos = ctx + d; lp = unord64(nHi[j]);
+        }
         p.token_ids[o] = t;
         p.parent_idx[o] = par;
         p.depth[o] = d;
@@ -359,32 +431,42 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         if (p.node_logprob) p.node_logprob[o] = lp;
     }
     const bool dense = (p.flags & CADD_FLAG_EMIT_DENSE_MASK) && p.mask_dense;
-    if (p.mask_bits || dense) {
-        const int W = (R + 31) >> 5;
-        uint32_t* mr = maskrow + warp * kMaskRowWords;
-        for (int j = warp; j < R; j += kExpandWarps) {
-            for (int w = lane; w < kMaskRowWords; w += 32) mr[w] = 0;
-            __syncwarp();
-            if (j <= n && lane == 0) {                      // self and ancestors: at most L+1 bits
-                int cur = j;
-                for (;;) {
-                    mr[cur >> 5] |= 1u << (cur & 31);
-                    if (cur == 0) break;
-                    cur = nPar[cur];
-                }
+    const int W = (R + 31) >> 5;
+    // all rows zero first (coalesced), then the few non-zero words / bytes of the live rows
+    if (p.mask_bits) {
+        uint32_t* base = p.mask_bits + (int64_t)b * R * W;
+        for (int64_t q = tid; q < (int64_t)R * W; q += kThreads) base[q] = 0u;
+    }
+    if (dense) {
+        uint8_t* base = p.mask_dense + (int64_t)b * R * R;
+        const int64_t total = (int64_t)R * R;
+        int64_t head = (4 - (int64_t)((uintptr_t)base & 3)) & 3;
+        if (head > total) head = total;
+        const int64_t words = (total - head) >> 2;
+        if (tid < head) base[tid] = 0;
+        uint32_t* mid = (uint32_t*)(base + head);
+        for (int64_t q = tid; q < words; q += kThreads) mid[q] = 0u;
+        for (int64_t q = head + words * 4 + tid; q < total; q += kThreads) base[q] = 0;
+    }
+    __syncthreads();
+    for (int j = tid; j <= n; j += kThreads) {              // self and ancestors: at most L+1 bits, rows descending
+        uint32_t* wrow = p.mask_bits ? p.mask_bits + ((int64_t)b * R + j) * W : nullptr;
+        uint8_t* brow = dense ? p.mask_dense + ((int64_t)b * R + j) * R : nullptr;
+        int cur = j, word = j >> 5;
+        uint32_t acc = 0;
+        for (;;) {
+            acc |= 1u << (cur & 31);
+            if (brow) brow[cur] = 1;
+            if (cur == 0) break;
+            const int next = tb_parent(~nLo[cur]);
+            if ((next >> 5) != word) {
+                if (wrow) wrow[word] = acc;
+                acc = 0;
+                word = next >> 5;
             }
-            __syncwarp();
-            if (p.mask_bits) {
-                uint32_t* dst = p.mask_bits + ((int64_t)b * R + j) * W;
-                for (int w = lane; w < W; w += 32) dst[w] = w < kMaskRowWords ? mr[w] : 0u;
-            }
-            if (dense) {
-                uint8_t* dst = p.mask_dense + ((int64_t)b * R + j) * R;
-                for (int c = lane; c < R; c += 32)
-                    dst[c] = (c >> 5) < kMaskRowWords ? (uint8_t)((mr[c >> 5] >> (c & 31)) & 1u) : (uint8_t)0;
-            }
-            __syncwarp();
+            cur = next;
         }
+        if (wrow) wrow[word] = acc;
     }
 }
 
