@@ -56,6 +56,7 @@ extern "C" {
 #define CADD_STATUS_L_EFF_CLAMPED       16   /* l_eff[b] was outside [0, L] */
 #define CADD_STATUS_COST_NONPOSITIVE    32   /* C_d + C_v(n) <= 0 (or not finite) was met; expansion stopped there */
 #define CADD_STATUS_BAD_N_NODES         64   /* verify: n_nodes[b] was outside [0, R-1] and was clamped */
+#define CADD_STATUS_INTERNAL_TIMEOUT   128   /* a bounded wait on an asynchronous copy ran out; build returns the empty tree, verify leaves -2 in node_argmax */
 
 #define CADD_DTYPE_BF16 0
 #define CADD_DTYPE_FP32 1

@@ -214,8 +214,14 @@ int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream) {
     ap.logits = a->target_logits; ap.V = a->V; ap.stride_b = a->stride_b; ap.stride_row = a->stride_row;
     ap.R = a->R; ap.rows_mode = a->rows_mode; ap.n_nodes = a->n_nodes; ap.node_argmax = a->node_argmax;
     const unsigned rows = (unsigned)((int64_t)a->batch * a->R);
-    if (a->logits_dtype == CADD_DTYPE_BF16) row_argmax_kernel<CADD_DTYPE_BF16><<<rows, kThreads, 0, st>>>(ap);
-    else row_argmax_kernel<CADD_DTYPE_FP32><<<rows, kThreads, 0, st>>>(ap);
+    const void* kfn = a->logits_dtype == CADD_DTYPE_BF16 ? (const void*)row_argmax_kernel<CADD_DTYPE_BF16>
+                                                          : (const void*)row_argmax_kernel<CADD_DTYPE_FP32>;
+    if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)argmax_smem_bytes()) != cudaSuccess) {
+        cudaGetLastError();
+        return CADD_ERR_LAUNCH;
+    }
+    if (a->logits_dtype == CADD_DTYPE_BF16) row_argmax_kernel<CADD_DTYPE_BF16><<<rows, kThreads, argmax_smem_bytes(), st>>>(ap);
+    else row_argmax_kernel<CADD_DTYPE_FP32><<<rows, kThreads, argmax_smem_bytes(), st>>>(ap);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
 
     WalkParams wp;

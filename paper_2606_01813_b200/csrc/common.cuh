@@ -11,15 +11,6 @@ namespace cadd {
 constexpr int kThreads = 256;              // threads per CTA in every streaming kernel
 constexpr unsigned kFullMask = 0xffffffffu;
 
-// ---- 16-byte streaming load: read-once data, keep it out of L1 ----
-__device__ __forceinline__ uint4 ld_stream16(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-
 // ---- order-preserving integer images of IEEE values ----
 // ord32(a) < ord32(b)  <=>  a < b as floats, for non-NaN a, b with -0 canonicalised to +0 by the caller.
 __device__ __forceinline__ uint32_t ord32(uint32_t bits) {

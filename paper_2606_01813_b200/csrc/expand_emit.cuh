@@ -179,6 +179,7 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
             if (ke < K) st |= CADD_STATUS_FEWER_THAN_K_FINITE;
             if (st) atomicOr(&s_status, st);
             if (fl & kPartPosInf) s_pinf = 1;
+            if (fl & kPartTimeout) { atomicOr(&s_status, CADD_STATUS_INTERNAL_TIMEOUT); s_pinf = 1; }   // empty tree
         }
         if (emit) for (int k = lane; k < K; k += 32) {
             if (out_tok) out_tok[k] = k < ke ? tok_list[i * K + k] : -1;

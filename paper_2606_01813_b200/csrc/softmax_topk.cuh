@@ -10,25 +10,30 @@
 // only ever cover the part of the mass that is spread over many small terms.
 //
 // Data path: one elected thread streams the segment into a ring of shared-memory tiles with bulk
-// asynchronous copies (cp.async.bulk, completion on an mbarrier; no multicast), so several tiles are
-// always in flight per CTA while the other threads compute from shared memory.
+// asynchronous copies (cp.async.bulk, completion on an mbarrier; no multicast); a second set of mbarriers
+// tells it when all eight warps are done with a stage.  Warps advance through the tiles on their own:
+// there is no CTA-wide barrier in the steady state.
 //
-// Hot loop per 16-byte chunk (8 bf16 / 4 fp32): chunk max (packed), one compare against the CTA's
-// running KP-th best value; per element two FMAs (x*log2e split in hi+lo, minus an integer reference
-// exponent; issued as packed fma.rn.f32x2), one ex2.approx, and packed adds; the fp32 sum of one chunk
-// goes to an fp64 accumulator.  A chunk whose maximum reaches the threshold value pushes its
-// candidates into a shared buffer and keeps them out of the sum; when the buffer holds 2*KP entries
-// the CTA ranks them, keeps the KP best, raises the threshold and folds the evicted ones into the sums.
+// Hot loop per thread and tile (four 16-byte chunks = 32 bf16 / 16 fp32): one packed max over all
+// elements and one compare against the CTA's running KP-th best value; per element two FMAs
+// (x*log2e split in hi+lo, minus an integer reference exponent; issued as packed fma.rn.f32x2), one
+// ex2.approx, packed adds; the fp32 sum of the tile goes to an fp64 accumulator.  An element that reaches
+// the threshold is appended to a shared ring of candidate keys and replaced by -Inf in the register copy,
+// so that it is left out of the sum exactly.  Whenever KP new candidates have gathered, ONE warp (whichever
+// gets the lock) merges them into the sorted list of the KP best, folds the losers into its sums and
+// publishes the new threshold; the other warps keep streaming with the old one (a stale threshold only
+// means a few extra candidates).
+//
+// If the candidate ring overflows (pathological inputs such as an ascending row) or a non-finite value
+// poisons the sums, the segment is redone by the careful path: element by element from global memory,
+// with a CTA-wide barrier protocol.  Slow, but correct for every input.
 #pragma once
 #include "common.cuh"
+#include "tile_ring.cuh"
 
 namespace cadd {
 
-constexpr int kTopkUnroll = 4;            // chunks per thread per tile
-constexpr int kTileChunks = kTopkUnroll * kThreads;   // 16-byte chunks per tile (16 KB)
-constexpr int kStages = 3;                // tiles in flight per CTA
-constexpr int kSpinLimit = 1 << 18;       // bounded mbarrier wait (each try may itself block for a while)
-constexpr int kCandCap = 512;             // candidate buffer entries per CTA
+constexpr int kCandCap = 512;             // candidate ring entries per CTA (power of two)
 constexpr int kMaxKP = 64;
 
 constexpr uint32_t kPartNonfinite = 1u;   // NaN or +Inf seen
@@ -90,48 +95,27 @@ __device__ __forceinline__ void fold_scalar(ThreadSum& s, float x) {   // x fini
 
 // Shared state of one CTA.
 struct TopkShared {
-    uint64_t keys[kCandCap];
-    uint64_t win[kMaxKP];
+    uint64_t keys[kCandCap]; // fast path: ring of candidate keys (0 = not written yet); careful path: plain buffer
+    uint64_t win[kMaxKP];    // the KP best candidates so far, sorted, best first
     unsigned hist[256];
-    unsigned count;          // pushes so far (may exceed kCandCap: the excess was not stored)
-    unsigned nwin;
-    uint64_t thr_key;        // candidates must beat this key (0 = none yet)
-    float thr_val;           // its logit value (-Inf = none yet)
+    unsigned count;          // careful path: entries in keys[]
+    unsigned nwin;           // entries in win[]
+    uint64_t thr_key;        // candidates must beat this key (0 = none yet); only ever rises
+    float thr_val;           // careful path: its logit value
     uint64_t sel_prefix;
     unsigned sel_need;
+    unsigned pushed;         // fast path: candidates appended so far
+    unsigned consumed;       // fast path: candidates merged so far (changed under the lock only)
+    unsigned lock;           // fast path: 1 while a warp merges
+    unsigned overflow;       // fast path: the ring was full at some push
+    unsigned timeout;        // a bounded wait ran out
     double red_d[kThreads / 32];
     float red_f[kThreads / 32];
     unsigned red_u[kThreads / 32];
-    unsigned timeout;        // set when a bounded wait ran out
     alignas(8) uint64_t full[kStages];                 // mbarriers: tile landed
+    unsigned released[kStages];                        // warps done with the stage's current tile
     alignas(128) uint4 ring[kStages][kTileChunks];     // tiles of logits
 };
-
-// ---- mbarrier / bulk-copy primitives (shared::cta addresses, no cluster, no multicast) ----
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
-    unsigned ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Wait for a phase with an iteration limit; false = gave up (the caller flags an error and leaves).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity) {
-    for (int it = 0; it < kSpinLimit; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// 1-D bulk copy global -> this CTA's shared memory; both addresses 16-byte aligned, bytes % 16 == 0.
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
 
 // ---- packed fp32x2 arithmetic (one instruction for two lanes of a register pair) ----
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
@@ -176,21 +160,78 @@ __device__ __forceinline__ bool slow_element(TopkShared& sh, ThreadSum& s, uint3
     return false;
 }
 
-// Hot-loop handling of one element whose value reached the threshold value.  Kept out of line so that
-// the chunk loop stays small.  Returns a bit set: kTakeExclude = keep it out of the fast sum,
-// kTakeDropped = buffer full, retry after the next refresh, kTakeRefresh = the buffer now holds 2*KP
-// entries or more, plus partial flags shifted left by 8.
-constexpr uint32_t kTakeExclude = 1u, kTakeDropped = 2u, kTakeRefresh = 4u;
-__device__ __noinline__ uint32_t take_candidate(TopkShared& sh, float x, uint32_t id, uint64_t thrk, int KP) {
+// Fast-path handling of one element whose value reached the threshold value.  Kept out of line so that
+// the tile loop stays small.  Returns kTakeExclude when the element was appended to the candidate ring
+// (or is +-Inf) and must be kept out of the fast sum, plus partial flags shifted left by 8.
+constexpr uint32_t kTakeExclude = 1u;
+__device__ __noinline__ uint32_t take_candidate(TopkShared& sh, float x, uint32_t id, uint64_t thrk) {
     const uint32_t bits = __float_as_uint(x);
     if ((bits & 0x7f800000u) == 0x7f800000u)               // +Inf (-Inf only while no threshold is set)
         return kTakeExclude | (bits == 0x7f800000u ? (kPartNonfinite | kPartPosInf) << 8 : 0u);
     const uint64_t key = make_key(x, id);
     if (key <= thrk) return 0u;                            // equal value, higher id than the threshold key
-    const unsigned pos = atomicAdd(&sh.count, 1u);
-    if (pos >= (unsigned)kCandCap) return kTakeExclude | kTakeDropped | kTakeRefresh;
-    sh.keys[pos] = key;
-    return kTakeExclude | (pos + 1 >= 2u * (unsigned)KP ? kTakeRefresh : 0u);
+    const unsigned pos = atomicAdd(&sh.pushed, 1u);
+    if (pos - *(volatile unsigned*)&sh.consumed >= (unsigned)kCandCap) {
+        sh.overflow = 1;                                   // no room: the segment will be redone carefully
+        return 0u;
+    }
+    *(volatile uint64_t*)&sh.keys[pos & (kCandCap - 1)] = key;
+    return kTakeExclude;
+}
+
+// One warp merges the candidates appended since the last merge (at most 32 per call) into the sorted list
+// of the KP best, folds the losers into its lanes' sums and raises the threshold.  The caller holds the lock.
+// ok = false if an entry that was announced never showed up within the spin limit.
+struct MergeResult { ThreadSum s; bool ok; };
+__device__ __noinline__ MergeResult warp_merge_candidates(TopkShared& sh, ThreadSum s, int KP) {
+    const int lane = threadIdx.x & 31;
+    const unsigned c0 = *(volatile unsigned*)&sh.consumed;
+    const unsigned avail = *(volatile unsigned*)&sh.pushed - c0;
+    const unsigned m = avail < 32u ? avail : 32u;
+    bool ok = true;
+    uint64_t kn = 0;                                       // this lane's new candidate
+    if ((unsigned)lane < m) {
+        volatile uint64_t* slot = &sh.keys[(c0 + lane) & (kCandCap - 1)];
+        int spins = 0;
+        while ((kn = *slot) == 0ull && spins < kSpinLimit && !*(volatile unsigned*)&sh.overflow) ++spins;   // its writer is about to store it
+        if (kn == 0ull) ok = false;
+        *slot = 0ull;                                      // the ring entry is free again
+    }
+    ok = __all_sync(kFullMask, ok);
+    const int nold = (int)sh.nwin;
+    const uint64_t k0 = lane < nold ? sh.win[lane] : 0ull;  // the current list is sorted: win[i] has rank i
+    const uint64_t k1 = lane + 32 < nold ? sh.win[lane + 32] : 0ull;
+    // New rank of an old key = its old rank + the number of new keys above it; rank of a new key = the
+    // number of old and new keys above it.  Every new key is broadcast once (keys are unique; 0 = absent).
+    int r0 = lane, r1 = lane + 32, rn = 0;
+    for (int j = 0; j < (int)m; ++j) {
+        const uint64_t bn = __shfl_sync(kFullMask, kn, j);
+        r0 += bn > k0;
+        r1 += bn > k1;
+        int above = __popc(__ballot_sync(kFullMask, k0 > bn)) + __popc(__ballot_sync(kFullMask, kn > bn));
+        if (nold > 32) above += __popc(__ballot_sync(kFullMask, k1 > bn));
+        if (lane == j) rn = above;
+    }
+    __syncwarp();
+    if (k0) { if (r0 < KP) sh.win[r0] = k0; else fold_scalar(s, key_value(k0)); }
+    if (k1) { if (r1 < KP) sh.win[r1] = k1; else fold_scalar(s, key_value(k1)); }
+    if (kn) { if (rn < KP) sh.win[rn] = kn; else fold_scalar(s, key_value(kn)); }
+    __syncwarp();
+    if (lane == 0) {
+        const int total = nold + (int)m;
+        const int nw = total < KP ? total : KP;
+        sh.nwin = nw;
+        if (nw == KP) {
+            const uint64_t kth = sh.win[KP - 1];
+            if (kth > sh.thr_key) *(volatile uint64_t*)&sh.thr_key = kth;
+        }
+        __threadfence_block();
+        *(volatile unsigned*)&sh.consumed = c0 + m;
+    }
+    __syncwarp();
+    MergeResult res;
+    res.s = s; res.ok = ok;
+    return res;
 }
 
 // The thread's sum is passed and returned by value so that it stays in registers in the hot loop.
@@ -351,9 +392,10 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkParams p) {
     using E = Elem<DT>;
     static_assert(kTopkUnroll == 4, "the tile loop below is written for four chunks per thread");
+    static_assert((kCandCap & (kCandCap - 1)) == 0, "the candidate ring is indexed with a mask");
     extern __shared__ unsigned char topk_smem_raw[];
     TopkShared& sh = *reinterpret_cast<TopkShared*>(((uintptr_t)topk_smem_raw + 127) & ~(uintptr_t)127);
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int item = blockIdx.x;
     const int rowi = item / p.S;
     const int seg = item - rowi * p.S;
@@ -371,162 +413,109 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
     const int KP = p.KP;
     const int n_tiles = (c_end - c_begin + kTileChunks - 1) / kTileChunks;
 
+    for (int q = tid; q < kCandCap; q += kThreads) sh.keys[q] = 0ull;
     if (tid == 0) {
-        for (int q = 0; q < kStages; ++q) mbar_init(&sh.full[q], 1);
-        sh.timeout = 0;
+        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
+        sh.timeout = 0; sh.overflow = 0; sh.lock = 0; sh.pushed = 0; sh.consumed = 0; sh.nwin = 0;
+        sh.count = 0; sh.thr_key = 0; sh.thr_val = -INFINITY;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    // the elected thread issues tile t of this attempt into stage (seq % kStages)
-    auto issue_tile = [&](int t, unsigned seq) {
+    // one thread issues tile t into stage t % kStages: thread 0 for the first kStages tiles, afterwards
+    // lane 0 of whichever warp is the last to finish with the tile that occupied the stage
+    auto issue_tile = [&](int t) {
         const int c0 = c_begin + t * kTileChunks;
         const unsigned bytes = (unsigned)min(kTileChunks, c_end - c0) * 16u;
-        const unsigned st = seq % kStages;
+        const unsigned st = (unsigned)t % kStages;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic reads of the stage are done
         mbar_arrive_expect_tx(&sh.full[st], bytes);
         bulk_load(&sh.ring[st][0], body + c0, bytes, &sh.full[st]);
     };
+    if (tid == 0)
+        for (int t = 0; t < kStages && t < n_tiles; ++t) issue_tile(t);
 
     const uint64_t l2e_hi2 = pack2(kLog2eHi, kLog2eHi), l2e_lo2 = pack2(kLog2eLo, kLog2eLo);
-    unsigned seq0 = 0;             // sequence number of tile 0 of the current attempt
-    bool careful = false;          // second attempt: every element goes through slow_element
-    double W = 0.0, Cmax = 0.0;
+    ThreadSum s{0.0, -INFINITY, 0.0f};
     uint32_t flags = 0;
-    for (;;) {
-        if (tid == 0) {
-            sh.count = 0; sh.thr_key = 0; sh.thr_val = -INFINITY;
-            for (int t = 0; t < kStages && t < n_tiles; ++t) issue_tile(t, seq0 + t);
+
+    // ================= fast path: warps advance on their own =================
+    {
+        // ragged ends of the row, one element per thread (segment 0 takes the head, the last one the tail)
+        bool dummy = false;
+        if (seg == 0 && tid < sp.head) slow_element(sh, s, flags, dummy, E::load(row, tid), (uint32_t)tid);
+        if (seg == p.S - 1 && tid < sp.tail) {
+            const int64_t e = p.V - sp.tail + tid;
+            slow_element(sh, s, flags, dummy, E::load(row, e), (uint32_t)e);
+        }
+        // (slow_element appends to keys[0..count): at most 14 entries, moved into the ring below)
+        __syncthreads();
+        if (tid == 0) { sh.pushed = sh.count; sh.count = 0; }
+
+        // Seed the threshold from tile 0: at least KP finite elements are >= the smallest of KP' group maxima
+        // (groups of 256/KP' consecutive threads, KP' = KP rounded up to a power of two), each thread
+        // contributing the maximum of its chunks of the tile.  Elements equal to the seed stay candidates.
+        bool landed = true;
+        if (n_tiles > 0) {
+            landed = mbar_wait_bounded(&sh.full[0], 0);
+            float gm = -INFINITY;
+            if (landed) {
+#pragma unroll
+                for (int u = 0; u < kTopkUnroll; ++u)
+                    if (c_begin + u * kThreads + tid < c_end) gm = fmaxf(gm, E::chunk_max(sh.ring[0][u * kThreads + tid]));
+            }
+            if (!(fabsf(gm) < INFINITY)) gm = -INFINITY;           // NaN or Inf: no help from this thread
+            const int gs = KP <= 16 ? 16 : (KP <= 32 ? 8 : 4);
+            for (int o = gs >> 1; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(kFullMask, gm, o));
+            float* seeds = (float*)sh.hist;
+            if ((tid & (gs - 1)) == 0) seeds[tid / gs] = gm;
+            if (!landed) sh.timeout = 1;
         }
         __syncthreads();
-        ThreadSum s{0.0, -INFINITY, 0.0f};
-        flags = 0;
-        bool want_refresh = false;
-        uint32_t dropped = 0;
-        // ragged ends of the row, one element per thread
-        if (seg == 0 && tid < sp.head)
-            slow_element(sh, s, flags, want_refresh, E::load(row, tid), (uint32_t)tid);
-        if (seg == p.S - 1 && tid < sp.tail) {
-            int64_t e = p.V - sp.tail + tid;
-            slow_element(sh, s, flags, want_refresh, E::load(row, e), (uint32_t)e);
-        }
-
-        float thrv = -INFINITY;
-        uint64_t thrk = 0, negc2 = 0;
-        auto reload_threshold = [&]() {                             // both only change inside a refresh
-            thrv = sh.thr_val;
-            thrk = sh.thr_key;
-            if (thrv > s.tmax + 60.0f) raise_reference(s, thrv);    // keeps 2^(x*log2e - c) in range for x < thrv
-            negc2 = pack2(s.negc, s.negc);
-        };
-        // Push the candidates of a chunk (value >= threshold value, key above the threshold key) and replace
-        // them by -Inf in the register copy, so that the common arithmetic leaves them out of the sum exactly.
-        auto extract_candidates = [&](uint4& w, int c, int bit0) {
-            const uint32_t id0 = (uint32_t)(sp.head + (int64_t)c * E::EPC);
-            float f[E::EPC];
-            E::unpack(w, f);
+        if (tid < 32 && n_tiles > 0 && c_end - c_begin >= kThreads) {
+            const int gs = KP <= 16 ? 16 : (KP <= 32 ? 8 : 4);
+            const int ng = kThreads / gs;
+            const float* seeds = (const float*)sh.hist;
+            float v = INFINITY;
+            for (int q = tid; q < ng; q += 32) v = fminf(v, seeds[q]);
 #pragma unroll
-            for (int q = 0; q < E::EPC; ++q) {
-                if (f[q] >= thrv) {
-                    const uint32_t r = take_candidate(sh, f[q], id0 + q, thrk, KP);
-                    if (r & kTakeExclude) mask_out<DT>(w, q);
-                    if (r & kTakeDropped) dropped |= 1u << (bit0 + q);
-                    if (r & kTakeRefresh) want_refresh = true;
-                    flags |= r >> 8;
-                }
-            }
-        };
-        // one chunk with all checks (tile 0, ragged tiles, the careful attempt)
-        auto checked_chunk = [&](uint4 w, int c, int bit0) {
-            if (careful) {                                          // rare: re-read element by element
-                const uint32_t id0 = (uint32_t)(sp.head + (int64_t)c * E::EPC);
-#pragma unroll 1
-                for (int q = 0; q < E::EPC; ++q)
-                    if (slow_element(sh, s, flags, want_refresh, E::load(row, id0 + q), id0 + q)) dropped |= 1u << (bit0 + q);
-                return;
-            }
-            if (E::chunk_max(w) >= thrv) extract_candidates(w, c, bit0);
-            float lo, hi;
-            unpack2(chunk_exp_sum2<DT>(w, l2e_hi2, l2e_lo2, negc2), lo, hi);
-            s.acc += (double)(lo + hi);
-        };
-        // end of a step: refresh the candidate buffer when asked to, retry dropped elements
-        auto settle = [&](bool force, int cbase) {
-            if (!__syncthreads_or(want_refresh || dropped != 0 || force)) return;
-            want_refresh = false;
-            for (;;) {
-                s = refresh_candidates(sh, s, KP);
-                uint32_t again = 0;
-                while (dropped) {                                   // retry what did not fit
-                    int bit = __ffs(dropped) - 1;
-                    dropped &= dropped - 1;
-                    int u = bit / E::EPC, q = bit - u * E::EPC;
-                    int64_t el = sp.head + (int64_t)(cbase + u * kThreads + tid) * E::EPC + q;
-                    if (slow_element(sh, s, flags, want_refresh, E::load(row, el), (uint32_t)el)) again |= 1u << bit;
-                }
-                dropped = again;
-                if (!__syncthreads_or(dropped != 0 || want_refresh)) break;
-                want_refresh = false;
-            }
-            reload_threshold();
-        };
+            for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(kFullMask, v, o));
+            if (tid == 0 && v > -INFINITY) sh.thr_key = make_key(v, 0xffffffffu);   // the lowest key carrying this value
+        }
+        __syncthreads();
 
-        bool failed = false;
-        for (int t = 0; t < n_tiles; ++t) {
-            const unsigned seq = seq0 + t;
-            const unsigned st = seq % kStages;
-            // every thread waits for the tile; a thread that gives up raises a flag which all threads read
-            // after the next barrier, so that the decision to leave is uniform
-            bool landed = mbar_wait_bounded(&sh.full[st], (seq / kStages) & 1u);
-            if (!landed) sh.timeout = 1;
+        const bool timed_out = sh.timeout != 0;
+        unsigned st = 0, phase = 0;
+        for (int t = 0; t < n_tiles && !timed_out; ++t, st = (st + 1 == kStages ? 0u : st + 1), phase ^= (st == 0 ? 1u : 0u)) {
+            const bool here = __all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase));
+            if (!here) { sh.timeout = 1; break; }
+            const uint64_t thrk = *(volatile uint64_t*)&sh.thr_key;          // only ever rises; stale is safe
+            const float thrv = thrk ? key_value(thrk) : -INFINITY;
+            if (thrv > s.tmax + 60.0f) raise_reference(s, thrv);             // keeps 2^(x*log2e - c) in range for x < thrv
+            const uint64_t negc2 = pack2(s.negc, s.negc);
             const int cbase = c_begin + t * kTileChunks;
             const uint4* tile = &sh.ring[st][tid];
-            const int c3 = cbase + 3 * kThreads + tid;
-
-            if (t == 0) {
-                landed = __syncthreads_and(landed) != 0;            // the steps below have barriers of their own
-                if (!landed) { failed = true; break; }
-                if (!careful && c_end - c_begin >= kThreads) {
-                    // Seed the threshold: at least KP finite elements are >= the smallest of KP' group maxima
-                    // (groups of 256/KP' consecutive threads, KP' = KP rounded up to a power of two), each
-                    // thread contributing the maximum of its chunks of this tile.  Elements equal to the
-                    // seed value stay candidates.
-                    float gm = -INFINITY;
+            // append the candidates of a chunk and replace them by -Inf in the register copy
+            auto extract_candidates = [&](uint4& w, int c) {
+                const uint32_t id0 = (uint32_t)(sp.head + (int64_t)c * E::EPC);
+                float f[E::EPC];
+                E::unpack(w, f);
 #pragma unroll
-                    for (int u = 0; u < kTopkUnroll; ++u)
-                        if (cbase + u * kThreads + tid < c_end) gm = fmaxf(gm, E::chunk_max(tile[u * kThreads]));
-                    if (!(fabsf(gm) < INFINITY)) gm = -INFINITY;   // NaN or Inf: no help from this thread
-                    const int gs = KP <= 16 ? 16 : (KP <= 32 ? 8 : 4);
-                    for (int o = gs >> 1; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(kFullMask, gm, o));
-                    float* seeds = (float*)sh.hist;
-                    if ((tid & (gs - 1)) == 0) seeds[tid / gs] = gm;
-                    __syncthreads();
-                    if (tid < 32) {
-                        const int ng = kThreads / gs;
-                        float v = INFINITY;
-                        for (int q = tid; q < ng; q += 32) v = fminf(v, seeds[q]);
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(kFullMask, v, o));
-                        if (tid == 0 && v > -INFINITY) {
-                            sh.thr_val = v;
-                            sh.thr_key = make_key(v, 0xffffffffu); // the lowest key carrying this value
-                        }
+                for (int q = 0; q < E::EPC; ++q) {
+                    if (f[q] >= thrv) {
+                        const uint32_t r = take_candidate(sh, f[q], id0 + q, thrk);
+                        if (r & kTakeExclude) mask_out<DT>(w, q);
+                        flags |= r >> 8;
                     }
-                    __syncthreads();
                 }
-                reload_threshold();
-#pragma unroll 1
-                for (int u = 0; u < kTopkUnroll; ++u) {
-                    const int c = cbase + u * kThreads + tid;
-                    if (c < c_end) checked_chunk(tile[u * kThreads], c, u * E::EPC);
-                }
-            } else if (landed && !careful && c3 < c_end) {
-                // lean path: four whole chunks per thread, one test for all 32 (16) elements
+            };
+            if (cbase + 3 * kThreads + tid < c_end) {
+                // whole tile for this thread: one test for all 32 (16) elements
                 uint4 w0 = tile[0], w1 = tile[kThreads], w2 = tile[2 * kThreads], w3 = tile[3 * kThreads];
                 if (E::max4(w0, w1, w2, w3) >= thrv) {              // rare: some element is a candidate
-                    extract_candidates(w0, cbase + tid, 0);
-                    extract_candidates(w1, cbase + kThreads + tid, E::EPC);
-                    extract_candidates(w2, cbase + 2 * kThreads + tid, 2 * E::EPC);
-                    extract_candidates(w3, c3, 3 * E::EPC);
+                    if (E::chunk_max(w0) >= thrv) extract_candidates(w0, cbase + tid);
+                    if (E::chunk_max(w1) >= thrv) extract_candidates(w1, cbase + kThreads + tid);
+                    if (E::chunk_max(w2) >= thrv) extract_candidates(w2, cbase + 2 * kThreads + tid);
+                    if (E::chunk_max(w3) >= thrv) extract_candidates(w3, cbase + 3 * kThreads + tid);
                 }
                 const uint64_t a = add2(chunk_exp_sum2<DT>(w0, l2e_hi2, l2e_lo2, negc2),
                                         chunk_exp_sum2<DT>(w1, l2e_hi2, l2e_lo2, negc2));
@@ -535,37 +524,60 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
                 float lo, hi;
                 unpack2(add2(a, c2), lo, hi);
                 s.acc += (double)(lo + hi);
-            } else if (landed) {                                    // ragged last tile, or the careful attempt
+            } else {                                                // ragged last tile
 #pragma unroll 1
                 for (int u = 0; u < kTopkUnroll; ++u) {
                     const int c = cbase + u * kThreads + tid;
-                    if (c < c_end) checked_chunk(tile[u * kThreads], c, u * E::EPC);
+                    if (c >= c_end) break;
+                    uint4 w = tile[u * kThreads];
+                    if (E::chunk_max(w) >= thrv) extract_candidates(w, c);
+                    float lo, hi;
+                    unpack2(chunk_exp_sum2<DT>(w, l2e_hi2, l2e_lo2, negc2), lo, hi);
+                    s.acc += (double)(lo + hi);
                 }
             }
-            settle(t == 0, cbase);                                  // always sharpen the threshold after tile 0
-            if (sh.timeout) { failed = true; break; }               // written before the barrier in settle(): uniform
-            if (tid == 0 && t + kStages < n_tiles) issue_tile(t + kStages, seq + kStages);   // the stage is free again
+            __syncwarp();
+            // This warp is done with the stage (its loads from it have returned: their values were consumed
+            // above); the last warp to say so refills the stage at once.
+            if (lane == 0) {
+                if (atomicAdd(&sh.released[st], 1u) == kThreads / 32 - 1) {
+                    atomicExch(&sh.released[st], 0u);
+                    if (t + kStages < n_tiles) issue_tile(t + kStages);
+                }
+            }
+            // enough new candidates: one warp merges them and raises the threshold
+            int go = 0;
+            if (lane == 0 && *(volatile unsigned*)&sh.pushed - *(volatile unsigned*)&sh.consumed >= (unsigned)min(2 * KP, 32))
+                go = atomicCAS(&sh.lock, 0u, 1u) == 0u;
+            if (__shfl_sync(kFullMask, go, 0)) {
+                const MergeResult mr = warp_merge_candidates(sh, s, KP);
+                s = mr.s;
+                if (!mr.ok && !*(volatile unsigned*)&sh.overflow) sh.timeout = 1;
+                __syncwarp();
+                if (lane == 0) { __threadfence_block(); atomicExch(&sh.lock, 0u); }
+            }
         }
-        if (failed) {
-            // give copies still in flight a bounded chance to land before this CTA's shared memory is released
-            if (tid == 0)
-                for (int q = 0; q < kStages; ++q) mbar_wait_bounded(&sh.full[q], 0);
-            flags |= kPartTimeout;
-            __syncthreads();
-            if (tid == 0) sh.count = 0;
-            __syncthreads();
-            W = 0.0; Cmax = 0.0;
-            break;
+        __syncthreads();
+        // drain: warp 0 merges what is left (nobody appends any more)
+        if (warp == 0 && !sh.overflow && !sh.timeout) {
+            for (int guard = 0; guard < 4 * kCandCap; ++guard) {
+                if (*(volatile unsigned*)&sh.pushed == *(volatile unsigned*)&sh.consumed) break;
+                const MergeResult mr = warp_merge_candidates(sh, s, KP);
+                s = mr.s;
+                if (!mr.ok) { sh.timeout = 1; break; }
+            }
         }
-        seq0 += n_tiles;
-        s = refresh_candidates(sh, s, KP);                          // leaves min(KP, candidates) keys, sorted
+        __syncthreads();
+    }
 
-        // CTA combine: common reference C = max c_t, W = sum acc_t * 2^(c_t - C)
+    // CTA combine: common reference C = max c_t, W = sum acc_t * 2^(c_t - C)
+    double W, Cmax;
+    auto combine = [&]() {
         float c_t = (s.acc != 0.0) ? -s.negc : -INFINITY;
         float cm = c_t;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(kFullMask, cm, o));
-        if ((tid & 31) == 0) sh.red_f[tid >> 5] = cm;
+        if (lane == 0) sh.red_f[warp] = cm;
         __syncthreads();
         cm = sh.red_f[0];
 #pragma unroll
@@ -576,31 +588,81 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
         uint32_t fl = flags;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) fl |= __shfl_xor_sync(kFullMask, fl, o);
-        if ((tid & 31) == 0) { sh.red_d[tid >> 5] = part; sh.red_u[tid >> 5] = fl; }
+        if (lane == 0) { sh.red_d[warp] = part; sh.red_u[warp] = fl; }
         __syncthreads();
         W = 0.0; flags = 0;
 #pragma unroll
         for (int q = 0; q < kThreads / 32; ++q) { W += sh.red_d[q]; flags |= sh.red_u[q]; }
         Cmax = (cm == -INFINITY) ? 0.0 : (double)cm;
-        // A NaN that slipped through the fast path poisons W: redo the segment element by element.
-        if (careful || (W == W && W < INFINITY)) break;
-        careful = true;
         __syncthreads();
+    };
+    combine();
+    const bool timed_out = sh.timeout != 0;
+    const bool redo = !timed_out && (sh.overflow != 0 || !(W == W && W < INFINITY));
+
+    // ================= careful path: element by element from global memory, CTA-wide protocol =================
+    if (redo) {
+        __syncthreads();
+        if (tid == 0) { sh.count = 0; sh.nwin = 0; sh.thr_key = 0; sh.thr_val = -INFINITY; }
+        __syncthreads();
+        s = ThreadSum{0.0, -INFINITY, 0.0f};
+        flags = 0;
+        bool want_refresh = false;
+        if (seg == 0 && tid < sp.head) slow_element(sh, s, flags, want_refresh, E::load(row, tid), (uint32_t)tid);
+        if (seg == p.S - 1 && tid < sp.tail) {
+            const int64_t e = p.V - sp.tail + tid;
+            slow_element(sh, s, flags, want_refresh, E::load(row, e), (uint32_t)e);
+        }
+        for (int cbase = c_begin; cbase < c_end; cbase += kThreads) {
+            const int c = cbase + tid;
+            uint32_t dropped = 0;
+            if (c < c_end) {
+                const int64_t e0 = sp.head + (int64_t)c * E::EPC;
+#pragma unroll 1
+                for (int q = 0; q < E::EPC; ++q)
+                    if (slow_element(sh, s, flags, want_refresh, E::load(row, e0 + q), (uint32_t)(e0 + q))) dropped |= 1u << q;
+            }
+            if (__syncthreads_or(want_refresh || dropped != 0)) {
+                want_refresh = false;
+                for (;;) {
+                    s = refresh_candidates(sh, s, KP);
+                    uint32_t again = 0;
+                    while (dropped) {                               // retry what did not fit
+                        const int q = __ffs(dropped) - 1;
+                        dropped &= dropped - 1;
+                        const int64_t e = sp.head + (int64_t)c * E::EPC + q;
+                        if (slow_element(sh, s, flags, want_refresh, E::load(row, e), (uint32_t)e)) again |= 1u << q;
+                    }
+                    dropped = again;
+                    if (!__syncthreads_or(dropped != 0 || want_refresh)) break;
+                    want_refresh = false;
+                }
+            }
+        }
+        s = refresh_candidates(sh, s, KP);                          // leaves min(KP, candidates) keys in keys[]
+        __syncthreads();
+        // sort them into win[] by counting
+        const int cnt = (int)sh.count;
+        if (tid < cnt) {
+            const uint64_t k = sh.keys[tid];
+            int rank = 0;
+            for (int q = 0; q < cnt; ++q) rank += sh.keys[q] > k;
+            sh.win[rank] = k;
+        }
+        if (tid == 0) sh.nwin = cnt;
+        __syncthreads();
+        combine();
     }
 
-    // write the record: the surviving keys are already sorted, best first
+    // write the record: win[] is sorted, best first
     unsigned char* rec = p.partials + (size_t)item * seg_partial_stride(KP);
     uint64_t* out_keys = (uint64_t*)(rec + sizeof(SegPartial));
-    const int cnt = (int)sh.count;
-    if (tid < cnt) {
-        const uint64_t k = sh.keys[tid];
-        int rank = 0;
-        for (int q = 0; q < cnt; ++q) rank += sh.keys[q] > k;      // (also sorts the cnt <= KP early-out case)
-        out_keys[rank] = k;
-    }
+    const int cnt = timed_out ? 0 : (int)sh.nwin;
+    if (tid < cnt) out_keys[tid] = sh.win[tid];
     if (tid == 0) {
         SegPartial h;
-        h.W = W * kEx2BiasFix; h.C = Cmax; h.cnt = cnt; h.flags = flags; h.pad[0] = h.pad[1] = 0;
+        h.W = timed_out ? 0.0 : W * kEx2BiasFix; h.C = timed_out ? 0.0 : Cmax; h.cnt = cnt;
+        h.flags = flags | (timed_out ? kPartTimeout : 0u); h.pad[0] = h.pad[1] = 0;
         *(SegPartial*)rec = h;
     }
 }

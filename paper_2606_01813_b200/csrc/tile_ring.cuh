@@ -1,0 +1,48 @@
+// Building blocks of the shared-memory tile ring used by the streaming kernels: a thread issues 1-D bulk
+// asynchronous copies (cp.async.bulk) of 16 KB tiles into a small ring of stages; each stage has an mbarrier
+// that completes when the tile's bytes have landed (complete_tx).  No cluster, no multicast: every copy goes
+// into the issuing CTA's own shared memory.  Every wait is bounded.
+#pragma once
+#include "common.cuh"
+
+namespace cadd {
+
+constexpr int kTopkUnroll = 4;            // chunks per thread per tile
+constexpr int kTileChunks = kTopkUnroll * kThreads;   // 16-byte chunks per tile (16 KB)
+constexpr int kStages = 3;                // tiles in flight per CTA
+constexpr int kSpinLimit = 1 << 16;       // bounded waits: tries of up to ~2 us each (mbarrier), or plain polls
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// One try: the hardware may park the thread for up to `hint_ns` while the phase is incomplete, so a waiting
+// warp does not burn issue slots.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity, unsigned hint_ns = 2000u) {
+    unsigned ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
+// Wait for a phase with an iteration limit; false = gave up (the caller flags an error and leaves).
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity) {
+    for (int it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(200);          // a waiting warp must not take issue slots from the warps that still work
+    }
+    return false;
+}
+// 1-D bulk copy global -> this CTA's shared memory; both addresses 16-byte aligned, bytes % 16 == 0.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+
+}  // namespace cadd

@@ -2,6 +2,7 @@
 // (greedy acceptance, Section 3.1; longest accepted prefix and next bonus token, Section 3.3).
 #pragma once
 #include "common.cuh"
+#include "tile_ring.cuh"
 
 namespace cadd {
 
@@ -13,17 +14,31 @@ struct ArgmaxParams {
     int32_t* node_argmax;      // [batch, R]
 };
 
-constexpr int kArgmaxUnroll = 4;   // 16-byte loads in flight per thread
+// Shared memory of row_argmax_kernel.
+struct ArgmaxRing {
+    alignas(8) uint64_t full[kStages];                 // mbarriers: tile landed
+    unsigned released[kStages];                        // warps done with the stage's current tile
+    unsigned timeout;
+    float red_m[kThreads / 32];
+    int64_t red_p[kThreads / 32];
+    alignas(128) uint4 ring[kStages][kTileChunks];
+};
+inline size_t argmax_smem_bytes() { return sizeof(ArgmaxRing) + 128; }
 
-// One CTA per (request, row): stream the row once, keep per thread the running maximum and the
-// first position (chunk start or scalar element) where it was reached, reduce over the CTA, then
-// find the first maximal element inside that one chunk.  HBM-bound: 9 instructions per 16 bytes.
+// One CTA per (request, row).  One thread streams the row's 16-byte chunks into a ring of 16 KB
+// shared-memory tiles with cp.async.bulk + mbarrier (no multicast); the last warp to finish a tile refills
+// its stage, so (kStages - 1) x 16 KB stay in flight per CTA (4 CTAs per SM) without living in registers.
+// Each thread keeps the running maximum (packed bf16 max, NaN ignored) and the first position (chunk start or
+// scalar element) where it was reached; the CTA reduces (value descending, position ascending) and one warp
+// finds the first maximal element inside that one chunk.  HBM-bound: ~9 instructions per 16 bytes.
 template <int DT>
-__global__ void __launch_bounds__(kThreads) row_argmax_kernel(ArgmaxParams p) {
+__global__ void __launch_bounds__(kThreads, 4) row_argmax_kernel(ArgmaxParams p) {
     using E = Elem<DT>;
+    extern __shared__ unsigned char argmax_smem_raw[];
+    ArgmaxRing& sh = *reinterpret_cast<ArgmaxRing*>(((uintptr_t)argmax_smem_raw + 127) & ~(uintptr_t)127);
     const int b = blockIdx.x / p.R;
     const int j = blockIdx.x - b * p.R;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t* out = p.node_argmax + (int64_t)b * p.R + j;
     if (p.rows_mode == CADD_ROWS_LIVE) {
         int n = p.n_nodes[b];
@@ -35,6 +50,26 @@ __global__ void __launch_bounds__(kThreads) row_argmax_kernel(ArgmaxParams p) {
     }
     const char* row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)j * p.stride_row) * E::ES;
     const RowSplit sp = split_row<DT>(row, p.V);
+    const uint4* body = (const uint4*)(row + (int64_t)sp.head * E::ES);
+    const int nc = sp.n_chunks;
+    const int n_tiles = (nc + kTileChunks - 1) / kTileChunks;
+
+    if (tid == 0) {
+        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
+        sh.timeout = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    auto issue_tile = [&](int t) {
+        const int c0 = t * kTileChunks;
+        const unsigned bytes = (unsigned)min(kTileChunks, nc - c0) * 16u;
+        const unsigned st = (unsigned)t % kStages;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive_expect_tx(&sh.full[st], bytes);
+        bulk_load(&sh.ring[st][0], body + c0, bytes, &sh.full[st]);
+    };
+    if (tid == 0)
+        for (int t = 0; t < kStages && t < n_tiles; ++t) issue_tile(t);
 
     float rm = -INFINITY;            // running maximum (NaN never enters: only strict '>' updates it)
     int64_t rpos = INT64_MAX;        // first position where rm was reached
@@ -42,22 +77,25 @@ __global__ void __launch_bounds__(kThreads) row_argmax_kernel(ArgmaxParams p) {
         float x = E::load(row, tid);
         if (x > rm) { rm = x; rpos = tid; }
     }
-    const uint4* body = (const uint4*)(row + (int64_t)sp.head * E::ES);
-    const int nc = sp.n_chunks;
-    int c = tid;
-    for (; c + (kArgmaxUnroll - 1) * kThreads < nc; c += kArgmaxUnroll * kThreads) {
-        uint4 w[kArgmaxUnroll];
+    unsigned st = 0, phase = 0;
+    for (int t = 0; t < n_tiles; ++t) {
+        if (!__all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase))) { sh.timeout = 1; break; }
+        const uint4* tile = &sh.ring[st][tid];
+        const int cbase = t * kTileChunks + tid;
 #pragma unroll
-        for (int u = 0; u < kArgmaxUnroll; ++u) w[u] = ld_stream16(body + c + u * kThreads);
-#pragma unroll
-        for (int u = 0; u < kArgmaxUnroll; ++u) {
-            float cm = E::chunk_max(w[u]);
-            if (cm > rm) { rm = cm; rpos = sp.head + (int64_t)(c + u * kThreads) * E::EPC; }
+        for (int u = 0; u < kTopkUnroll; ++u) {
+            const int c = cbase + u * kThreads;
+            if (c < nc) {
+                const float cm = E::chunk_max(tile[u * kThreads]);
+                if (cm > rm) { rm = cm; rpos = sp.head + (int64_t)c * E::EPC; }
+            }
         }
-    }
-    for (; c < nc; c += kThreads) {
-        float cm = E::chunk_max(ld_stream16(body + c));
-        if (cm > rm) { rm = cm; rpos = sp.head + (int64_t)c * E::EPC; }
+        __syncwarp();
+        if (lane == 0 && atomicAdd(&sh.released[st], 1u) == kThreads / 32 - 1) {   // last warp refills the stage
+            atomicExch(&sh.released[st], 0u);
+            if (t + kStages < n_tiles) issue_tile(t + kStages);
+        }
+        if (++st == kStages) { st = 0; phase ^= 1u; }
     }
     if (tid < sp.tail) {
         int64_t i = p.V - sp.tail + tid;
@@ -72,13 +110,11 @@ __global__ void __launch_bounds__(kThreads) row_argmax_kernel(ArgmaxParams p) {
         int64_t op = __shfl_xor_sync(kFullMask, rpos, o);
         if (om > rm || (om == rm && op < rpos)) { rm = om; rpos = op; }
     }
-    __shared__ float s_m[kThreads / 32];
-    __shared__ int64_t s_p[kThreads / 32];
-    if ((tid & 31) == 0) { s_m[tid >> 5] = rm; s_p[tid >> 5] = rpos; }
+    if (lane == 0) { sh.red_m[warp] = rm; sh.red_p[warp] = rpos; }
     __syncthreads();
     if (tid < 32) {
-        rm = tid < kThreads / 32 ? s_m[tid] : -INFINITY;
-        rpos = tid < kThreads / 32 ? s_p[tid] : INT64_MAX;
+        rm = tid < kThreads / 32 ? sh.red_m[tid] : -INFINITY;
+        rpos = tid < kThreads / 32 ? sh.red_p[tid] : INT64_MAX;
 #pragma unroll
         for (int o = 4; o > 0; o >>= 1) {
             float om = __shfl_xor_sync(kFullMask, rm, o);
@@ -87,7 +123,6 @@ __global__ void __launch_bounds__(kThreads) row_argmax_kernel(ArgmaxParams p) {
         }
         rm = __shfl_sync(kFullMask, rm, 0);
         rpos = __shfl_sync(kFullMask, rpos, 0);
-        // first element equal to the maximum within the EPC elements starting at rpos
         int32_t ans = 0;                                  // every logit is -Inf or NaN: lowest id
         if (rpos != INT64_MAX) {
             int64_t i = rpos + tid;
@@ -95,6 +130,7 @@ __global__ void __launch_bounds__(kThreads) row_argmax_kernel(ArgmaxParams p) {
             unsigned m = __ballot_sync(kFullMask, hit);
             ans = (int32_t)(rpos + (__ffs(m) - 1));
         }
+        if (sh.timeout) ans = -2;                         // a bulk copy never landed: the walk kernel flags the request
         if (tid == 0) *out = ans;
     }
 }
@@ -127,6 +163,10 @@ __global__ void __launch_bounds__(128) accept_walk_kernel(WalkParams p) {
     int32_t* acc = p.accepted_nodes + (int64_t)b * p.L;
     for (int i = lane; i < p.L; i += 32) acc[i] = -1;
     __syncwarp();
+    for (int c = lane; c <= n; c += 32)                    // -2 marks a row whose bulk copy never landed
+        if (gmx[c] == -2) st |= CADD_STATUS_INTERNAL_TIMEOUT;
+    st |= __shfl_xor_sync(kFullMask, st, 16); st |= __shfl_xor_sync(kFullMask, st, 8); st |= __shfl_xor_sync(kFullMask, st, 4);
+    st |= __shfl_xor_sync(kFullMask, st, 2); st |= __shfl_xor_sync(kFullMask, st, 1);
     int cur = 0, alpha = 0;
     while (alpha < p.L) {
         const int32_t g = gmx[cur];
