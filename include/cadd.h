@@ -35,7 +35,7 @@
 extern "C" {
 #endif
 
-#define CADD_ABI_VERSION 1
+#define CADD_ABI_VERSION 2
 
 /* ---- return codes (host side, synchronous) ---- */
 #define CADD_OK              0
@@ -63,6 +63,11 @@ extern "C" {
 
 #define CADD_COST_QUADRATIC 0    /* C_v(n) = a + b n + c n^2, per request */
 #define CADD_COST_TABLE     1    /* C_v(n) = cost_table[table_idx[b]][n], n = 0..B_max */
+#define CADD_COST_TABLE_INTERP 2 /* context interpolation at inference (Eq. 13): cost_table row j is the fitted cost at
+                                    context length ctx_grid[j]; with L_j <= ctx_len[b] < L_{j+1} and
+                                    alpha = (ctx_len[b] - L_j) / (L_{j+1} - L_j),
+                                    C_v(n) = (1 - alpha) cost_table[j][n] + alpha cost_table[j+1][n];
+                                    outside the grid the nearest table is used */
 
 #define CADD_FLAG_EMIT_DENSE_MASK 1u   /* also write mask_dense */
 #define CADD_FLAG_EMIT_TOPK       2u   /* also write topk_token / topk_logprob */
@@ -96,11 +101,12 @@ typedef struct cadd_build_args {
     const int32_t* bonus_token;    /* [batch] token of the root, NULL => -1 */
     const int32_t* ctx_len;        /* [batch] context length, NULL => 0; position_ids = ctx_len + depth */
     int32_t  cost_kind;            /* CADD_COST_* */
-    int32_t  n_tables;             /* TABLE: number of rows of cost_table */
+    int32_t  n_tables;             /* TABLE, TABLE_INTERP: number of rows of cost_table */
     const double*  cost_coef;      /* QUADRATIC: [batch,4] = (C_d, a, b, c) */
     const double*  cost_table;     /* TABLE: [n_tables, B_max+1] */
     const int32_t* table_idx;      /* TABLE: [batch], each in [0, n_tables) */
-    const double*  t_draft;        /* TABLE: [batch] C_d */
+    const double*  t_draft;        /* TABLE, TABLE_INTERP: [batch] C_d */
+    const int32_t* ctx_grid;       /* TABLE_INTERP: [n_tables] strictly ascending context lengths of the tables */
     /* outputs; n_nodes, token_ids, parent_idx, depth are required, the rest may be NULL */
     int32_t* n_nodes;              /* [batch] n* */
     int32_t* token_ids;            /* [batch,R] */
@@ -110,6 +116,8 @@ typedef struct cadd_build_args {
     double*  node_logprob;         /* [batch,R] log prefix probability sigma of each node (root 0) */
     double*  phi;                  /* [batch] expected accepted draft tokens Phi*(n*) (Eq. 6) */
     double*  theta;                /* [batch] surrogate throughput (1+Phi)/(C_d+C_v(n*)) (Eq. 7) */
+    double*  theta_curve;          /* [batch,R] optional: theta*(n) for n = 0..n_nodes[b] (Prop. 1), 0 above; with
+                                      CADD_FLAG_FIXED_BUDGET this is the whole budget sweep of one expansion */
     uint32_t* mask_bits;           /* [batch,R,ceil(R/32)] bit c of row j set iff c == j or c is an ancestor of j */
     uint8_t*  mask_dense;          /* [batch,R,R] same as bytes, written only with CADD_FLAG_EMIT_DENSE_MASK */
     int32_t* topk_token;           /* [batch,L,K] written only with CADD_FLAG_EMIT_TOPK; -1 where absent */

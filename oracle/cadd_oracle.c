@@ -46,7 +46,7 @@
 #endif
 
 enum { ORC_BF16 = 0, ORC_FP32 = 1 };
-enum { ORC_COST_QUADRATIC = 0, ORC_COST_TABLE = 1 };
+enum { ORC_COST_QUADRATIC = 0, ORC_COST_TABLE = 1, ORC_COST_TABLE_INTERP = 2 };
 enum { ORC_FLAG_FIXED_BUDGET = 4 };
 enum { ORC_ROWS_LIVE = 0, ORC_ROWS_DENSE = 1 };
 enum {
@@ -151,11 +151,24 @@ static int cand_before(const cand_t *x, const cand_t *y)
     return x->parent < y->parent;
 }
 
-static double cost_verify(int cost_kind, const double *coef4, const double *table_row, int n)
+/* The verification cost C_v(n; l) of one request.  QUADRATIC: a + b n + c n^2.  TABLE: one table row.
+ * TABLE_INTERP (context interpolation at inference, Eq. 13): with L_j <= l < L_{j+1} and
+ * alpha = (l - L_j) / (L_{j+1} - L_j),  C_v(n; l) = (1 - alpha) C_v(n; L_j) + alpha C_v(n; L_{j+1});
+ * outside the profiled range the nearest table is used. */
+typedef struct {
+    int kind;
+    const double *coef4;      /* QUADRATIC */
+    const double *row0;       /* TABLE: the row; TABLE_INTERP: the row of L_j */
+    const double *row1;       /* TABLE_INTERP: the row of L_{j+1} */
+    double alpha;             /* TABLE_INTERP */
+} cost_model_t;
+
+static double cost_verify(const cost_model_t *cm, int n)
 {
-    if (cost_kind == ORC_COST_TABLE) return table_row[n];
+    if (cm->kind == ORC_COST_TABLE) return cm->row0[n];
+    if (cm->kind == ORC_COST_TABLE_INTERP) return (1.0 - cm->alpha) * cm->row0[n] + cm->alpha * cm->row1[n];
     double x = (double)n;
-    return coef4[1] + coef4[2] * x + coef4[3] * (x * x);
+    return cm->coef4[1] + cm->coef4[2] * x + cm->coef4[3] * (x * x);
 }
 
 /*
@@ -173,7 +186,7 @@ int cadd_oracle_build_tree(
     int dtype, const void *draft_logits, int64_t stride_b, int64_t stride_l,
     const int32_t *l_eff_in, const int32_t *bonus_token, const int32_t *ctx_len,
     int cost_kind, const double *cost_coef, const double *cost_table, const int32_t *table_idx,
-    const double *t_draft, uint32_t flags,
+    const double *t_draft, int n_tables, const int32_t *ctx_grid, uint32_t flags,
     int32_t *n_nodes, int32_t *token_ids, int32_t *parent_idx, int32_t *depth,
     int32_t *position_ids, double *node_logprob, double *phi_out, double *theta_out,
     uint32_t *mask_bits, uint8_t *mask_dense, int32_t *topk_token, double *topk_logprob,
@@ -223,10 +236,21 @@ int cadd_oracle_build_tree(
         }
 
         /* ---- O3: Algorithm 1 ---- */
-        const double *coef4 = (cost_kind == ORC_COST_QUADRATIC) ? cost_coef + (size_t)b * 4 : NULL;
-        const double *trow = (cost_kind == ORC_COST_TABLE)
-                                 ? cost_table + (size_t)table_idx[b] * (B_max + 1) : NULL;
-        const double C_d = (cost_kind == ORC_COST_QUADRATIC) ? coef4[0] : t_draft[b];
+        cost_model_t cm = { cost_kind, NULL, NULL, NULL, 0.0 };
+        if (cost_kind == ORC_COST_QUADRATIC) cm.coef4 = cost_coef + (size_t)b * 4;
+        else if (cost_kind == ORC_COST_TABLE) cm.row0 = cost_table + (size_t)table_idx[b] * (B_max + 1);
+        else {                                   /* Eq. 13: the two profiled context lengths around l */
+            const int l = ctx_len ? ctx_len[b] : 0;
+            int jlo = 0;
+            while (jlo + 1 < n_tables && ctx_grid[jlo + 1] <= l) ++jlo;      /* largest j with L_j <= l (or 0) */
+            int jhi = (jlo + 1 < n_tables) ? jlo + 1 : jlo;
+            if (l <= ctx_grid[0]) { jlo = jhi = 0; }
+            cm.row0 = cost_table + (size_t)jlo * (B_max + 1);
+            cm.row1 = cost_table + (size_t)jhi * (B_max + 1);
+            cm.alpha = (jhi == jlo) ? 0.0
+                                    : ((double)l - (double)ctx_grid[jlo]) / ((double)ctx_grid[jhi] - (double)ctx_grid[jlo]);
+        }
+        const double C_d = (cost_kind == ORC_COST_QUADRATIC) ? cm.coef4[0] : t_draft[b];
 
         cand_t *node = (cand_t *)calloc((size_t)R + 1, sizeof(cand_t));   /* rows 1..n */
         cand_t *H = (cand_t *)malloc(sizeof(cand_t) * ((size_t)B_max + 2));
@@ -235,7 +259,7 @@ int cadd_oracle_build_tree(
         int hn = 0, n = 0;
         double Phi = 0.0, theta_prev = 0.0;
         double min_margin = INFINITY, stop_margin = -1.0;
-        double den0 = C_d + cost_verify(cost_kind, coef4, trow, 0);
+        double den0 = C_d + cost_verify(&cm, 0);
         int ok = 1;
         if (!(den0 > 0.0)) { st |= ORC_ST_COST_NONPOSITIVE; ok = 0; }
         else theta_prev = 1.0 / den0;
@@ -255,7 +279,7 @@ int cadd_oracle_build_tree(
             for (int i = 0; i < hn; ++i)
                 if (H[i].sigma < s.sigma && H[i].sigma > runner) runner = H[i].sigma;
             double delta = exp(s.sigma);
-            double den = C_d + cost_verify(cost_kind, coef4, trow, n + 1);
+            double den = C_d + cost_verify(&cm, n + 1);
             if (!(den > 0.0)) { st |= ORC_ST_COST_NONPOSITIVE; stopped_by_rule = 1; break; }
             double theta_new = (1.0 + Phi + delta) / den;
             double margin = fabs(theta_new - theta_prev) / theta_prev;

@@ -19,7 +19,7 @@ _SRC = os.path.join(_HERE, "cadd_oracle.c")
 _LIB = os.path.join(_HERE, "libcadd_oracle.so")
 
 DT_BF16, DT_FP32 = 0, 1
-COST_QUADRATIC, COST_TABLE = 0, 1
+COST_QUADRATIC, COST_TABLE, COST_TABLE_INTERP = 0, 1, 2
 FLAG_FIXED_BUDGET = 4
 ROWS_LIVE, ROWS_DENSE = 0, 1
 ST_NONFINITE, ST_FEWER_THAN_K, ST_CAP_HIT, ST_FRONTIER_EXHAUSTED = 1, 2, 4, 8
@@ -100,7 +100,7 @@ def row_softmax_topk(row: torch.Tensor, K: int):
 def build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[int] = None, *,
                l_eff=None, bonus_token=None, ctx_len=None,
                cost_kind: int = COST_QUADRATIC, cost_coef=None, cost_table=None, table_idx=None,
-               t_draft=None, flags: int = 0, dense_mask: bool = False) -> OracleTree:
+               t_draft=None, ctx_grid=None, flags: int = 0, dense_mask: bool = False) -> OracleTree:
     """O1-O4 for a batch of requests; draft_logits is a CPU tensor [batch, L, V] (V contiguous)."""
     x = draft_logits
     assert x.device.type == "cpu" and x.dim() == 3 and x.stride(2) == 1
@@ -121,7 +121,13 @@ def build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[int] 
     l_eff, bonus_token, ctx_len = cv(l_eff, torch.int32), cv(bonus_token, torch.int32), cv(ctx_len, torch.int32)
     cost_coef, cost_table = cv(cost_coef, torch.float64), cv(cost_table, torch.float64)
     table_idx, t_draft = cv(table_idx, torch.int32), cv(t_draft, torch.float64)
-    if cost_kind == COST_TABLE:
+    ctx_grid = cv(ctx_grid, torch.int32)
+    n_tables = 0 if cost_table is None else int(cost_table.shape[0])
+    if cost_kind == COST_TABLE_INTERP:
+        assert cost_table is not None and ctx_grid is not None and t_draft is not None
+        assert cost_table.shape[1] == B_max + 1 and ctx_grid.numel() == n_tables
+        assert bool((ctx_grid[1:] > ctx_grid[:-1]).all())
+    elif cost_kind == COST_TABLE:
         assert cost_table is not None and table_idx is not None and t_draft is not None
         assert cost_table.shape[1] == B_max + 1
     else:
@@ -129,7 +135,7 @@ def build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[int] 
     rc = lib().cadd_oracle_build_tree(
         batch, L, C.c_int64(V), K, B_max, R, _dt(x), _p(x), C.c_int64(x.stride(0)), C.c_int64(x.stride(1)),
         _p(l_eff), _p(bonus_token), _p(ctx_len), cost_kind, _p(cost_coef), _p(cost_table), _p(table_idx),
-        _p(t_draft), C.c_uint32(flags),
+        _p(t_draft), n_tables, _p(ctx_grid), C.c_uint32(flags),
         _p(out.n_nodes), _p(out.token_ids), _p(out.parent_idx), _p(out.depth), _p(out.position_ids),
         _p(out.node_logprob), _p(out.phi), _p(out.theta), _p(out.mask_bits), _p(out.mask_dense),
         _p(out.topk_token), _p(out.topk_logprob), _p(out.status),

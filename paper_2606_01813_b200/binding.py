@@ -21,7 +21,7 @@ ERR_NULL, ERR_STRUCT_SIZE, ERR_SHAPE, ERR_DTYPE, ERR_ALIGN, ERR_WORKSPACE, ERR_L
 STATUS_NONFINITE_INPUT, STATUS_FEWER_THAN_K_FINITE, STATUS_CAP_HIT, STATUS_FRONTIER_EXHAUSTED = 1, 2, 4, 8
 STATUS_L_EFF_CLAMPED, STATUS_COST_NONPOSITIVE, STATUS_BAD_N_NODES, STATUS_INTERNAL_TIMEOUT = 16, 32, 64, 128
 DTYPE_BF16, DTYPE_FP32 = 0, 1
-COST_QUADRATIC, COST_TABLE = 0, 1
+COST_QUADRATIC, COST_TABLE, COST_TABLE_INTERP = 0, 1, 2
 FLAG_EMIT_DENSE_MASK, FLAG_EMIT_TOPK, FLAG_FIXED_BUDGET = 1, 2, 4
 ROWS_LIVE, ROWS_DENSE = 0, 1
 
@@ -40,8 +40,10 @@ class BuildArgs(C.Structure):
         ("l_eff", C.c_void_p), ("bonus_token", C.c_void_p), ("ctx_len", C.c_void_p),
         ("cost_kind", C.c_int32), ("n_tables", C.c_int32),
         ("cost_coef", C.c_void_p), ("cost_table", C.c_void_p), ("table_idx", C.c_void_p), ("t_draft", C.c_void_p),
+        ("ctx_grid", C.c_void_p),
         ("n_nodes", C.c_void_p), ("token_ids", C.c_void_p), ("parent_idx", C.c_void_p), ("depth", C.c_void_p),
         ("position_ids", C.c_void_p), ("node_logprob", C.c_void_p), ("phi", C.c_void_p), ("theta", C.c_void_p),
+        ("theta_curve", C.c_void_p),
         ("mask_bits", C.c_void_p), ("mask_dense", C.c_void_p), ("topk_token", C.c_void_p),
         ("topk_logprob", C.c_void_p), ("status", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
@@ -137,6 +139,7 @@ class Tree:
     topk_token: Optional[torch.Tensor]
     topk_logprob: Optional[torch.Tensor]
     status: torch.Tensor
+    theta_curve: Optional[torch.Tensor] = None
 
 
 @dataclass
@@ -175,7 +178,7 @@ def cadd_build_workspace_bytes(batch: int, L: int, V: int, K: int, B_max: int, R
 def cadd_build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[int] = None, *,
                     l_eff=None, bonus_token=None, ctx_len=None,
                     cost_kind: int = COST_QUADRATIC, cost_coef=None, cost_table=None, table_idx=None,
-                    t_draft=None, flags: int = 0, out: Optional[Tree] = None,
+                    t_draft=None, ctx_grid=None, theta_curve: bool = False, flags: int = 0, out: Optional[Tree] = None,
                     workspace: Optional[torch.Tensor] = None,
                     stream: Optional[torch.cuda.Stream] = None) -> Tree:
     """Build the draft trees of a batch (Eq. 1, Algorithm 1, Section 3.3) on the current CUDA stream.
@@ -197,9 +200,10 @@ def cadd_build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[
     a.stride_b, a.stride_l = x.stride(0), x.stride(1)
     keep = [_dev(l_eff, dev, torch.int32), _dev(bonus_token, dev, torch.int32), _dev(ctx_len, dev, torch.int32),
             _dev(cost_coef, dev, torch.float64), _dev(cost_table, dev, torch.float64),
-            _dev(table_idx, dev, torch.int32), _dev(t_draft, dev, torch.float64)]
+            _dev(table_idx, dev, torch.int32), _dev(t_draft, dev, torch.float64), _dev(ctx_grid, dev, torch.int32)]
     a.l_eff, a.bonus_token, a.ctx_len = _ptr(keep[0]), _ptr(keep[1]), _ptr(keep[2])
     a.cost_coef, a.cost_table, a.table_idx, a.t_draft = _ptr(keep[3]), _ptr(keep[4]), _ptr(keep[5]), _ptr(keep[6])
+    a.ctx_grid = _ptr(keep[7])
     a.n_tables = 0 if keep[4] is None else keep[4].shape[0]
     if out is None:
         W = (R + 31) // 32
@@ -211,9 +215,10 @@ def cadd_build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[
                    mask_dense=torch.empty(batch, R, R, dtype=torch.uint8, device=dev) if flags & FLAG_EMIT_DENSE_MASK else None,
                    topk_token=i32(batch, L, K) if flags & FLAG_EMIT_TOPK else None,
                    topk_logprob=f64(batch, L, K) if flags & FLAG_EMIT_TOPK else None,
-                   status=i32(batch))
+                   status=i32(batch), theta_curve=f64(batch, R) if theta_curve else None)
     a.n_nodes, a.token_ids, a.parent_idx, a.depth = _ptr(out.n_nodes), _ptr(out.token_ids), _ptr(out.parent_idx), _ptr(out.depth)
     a.position_ids, a.node_logprob, a.phi, a.theta = _ptr(out.position_ids), _ptr(out.node_logprob), _ptr(out.phi), _ptr(out.theta)
+    a.theta_curve = _ptr(out.theta_curve)
     a.mask_bits, a.mask_dense = _ptr(out.mask_bits), _ptr(out.mask_dense)
     a.topk_token, a.topk_logprob, a.status = _ptr(out.topk_token), _ptr(out.topk_logprob), _ptr(out.status)
     if workspace is None:
@@ -270,7 +275,7 @@ def cadd_verify_tree(target_logits: torch.Tensor, L: int, n_nodes: torch.Tensor,
 def cadd_build_tree_static_scratch(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[int] = None, *,
                                    l_eff=None, bonus_token=None, ctx_len=None,
                                    cost_kind: int = COST_QUADRATIC, cost_coef=None, cost_table=None,
-                                   table_idx=None, t_draft=None, flags: int = 0, out: Tree = None,
+                                   table_idx=None, t_draft=None, ctx_grid=None, flags: int = 0, out: Tree = None,
                                    stream: Optional[torch.cuda.Stream] = None) -> Tree:
     """cadd_build_tree without a workspace argument: the library uses its built-in scratch array.
 
@@ -294,9 +299,10 @@ def cadd_build_tree_static_scratch(draft_logits: torch.Tensor, K: int, B_max: in
     a.stride_b, a.stride_l = x.stride(0), x.stride(1)
     keep = [_dev(l_eff, dev, torch.int32), _dev(bonus_token, dev, torch.int32), _dev(ctx_len, dev, torch.int32),
             _dev(cost_coef, dev, torch.float64), _dev(cost_table, dev, torch.float64),
-            _dev(table_idx, dev, torch.int32), _dev(t_draft, dev, torch.float64)]
+            _dev(table_idx, dev, torch.int32), _dev(t_draft, dev, torch.float64), _dev(ctx_grid, dev, torch.int32)]
     a.l_eff, a.bonus_token, a.ctx_len = _ptr(keep[0]), _ptr(keep[1]), _ptr(keep[2])
     a.cost_coef, a.cost_table, a.table_idx, a.t_draft = _ptr(keep[3]), _ptr(keep[4]), _ptr(keep[5]), _ptr(keep[6])
+    a.ctx_grid = _ptr(keep[7])
     a.n_tables = 0 if keep[4] is None else keep[4].shape[0]
     if out is None:
         W = (R + 31) // 32

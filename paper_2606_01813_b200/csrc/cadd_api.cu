@@ -37,7 +37,7 @@ static int check_build_shape(const cadd_build_args* a) {
         return CADD_ERR_SHAPE;
     if ((int64_t)a->batch * a->L * 8 >= ((int64_t)1 << 31) || (int64_t)a->batch * a->R >= ((int64_t)1 << 31)) return CADD_ERR_SHAPE;
     if (a->logits_dtype != CADD_DTYPE_BF16 && a->logits_dtype != CADD_DTYPE_FP32) return CADD_ERR_DTYPE;
-    if (a->cost_kind != CADD_COST_QUADRATIC && a->cost_kind != CADD_COST_TABLE) return CADD_ERR_DTYPE;
+    if (a->cost_kind != CADD_COST_QUADRATIC && a->cost_kind != CADD_COST_TABLE && a->cost_kind != CADD_COST_TABLE_INTERP) return CADD_ERR_DTYPE;
     return CADD_OK;
 }
 
@@ -129,16 +129,18 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
     if (!a->draft_logits || !a->n_nodes || !a->token_ids || !a->parent_idx || !a->depth) return CADD_ERR_NULL;
     if (a->cost_kind == CADD_COST_QUADRATIC && !a->cost_coef) return CADD_ERR_NULL;
     if (a->cost_kind == CADD_COST_TABLE && (!a->cost_table || !a->table_idx || !a->t_draft || a->n_tables < 1)) return CADD_ERR_NULL;
+    if (a->cost_kind == CADD_COST_TABLE_INTERP && (!a->cost_table || !a->ctx_grid || !a->t_draft || a->n_tables < 1)) return CADD_ERR_NULL;
     if ((a->flags & CADD_FLAG_EMIT_DENSE_MASK) && !a->mask_dense) return CADD_ERR_NULL;
     if ((a->flags & CADD_FLAG_EMIT_TOPK) && !a->topk_token && !a->topk_logprob) return CADD_ERR_NULL;
     const size_t es = a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
     if (!aligned(a->draft_logits, es)) return CADD_ERR_ALIGN;
     if (!aligned(a->cost_coef, 8) || !aligned(a->cost_table, 8) || !aligned(a->t_draft, 8) || !aligned(a->node_logprob, 8) ||
-        !aligned(a->phi, 8) || !aligned(a->theta, 8) || !aligned(a->topk_logprob, 8))
+        !aligned(a->phi, 8) || !aligned(a->theta, 8) || !aligned(a->theta_curve, 8) || !aligned(a->topk_logprob, 8))
         return CADD_ERR_ALIGN;
     if (!aligned(a->n_nodes, 4) || !aligned(a->token_ids, 4) || !aligned(a->parent_idx, 4) || !aligned(a->depth, 4) ||
         !aligned(a->position_ids, 4) || !aligned(a->mask_bits, 4) || !aligned(a->topk_token, 4) || !aligned(a->status, 4) ||
-        !aligned(a->l_eff, 4) || !aligned(a->bonus_token, 4) || !aligned(a->ctx_len, 4) || !aligned(a->table_idx, 4))
+        !aligned(a->l_eff, 4) || !aligned(a->bonus_token, 4) || !aligned(a->ctx_len, 4) || !aligned(a->table_idx, 4) ||
+        !aligned(a->ctx_grid, 4))
         return CADD_ERR_ALIGN;
     if (a->stride_l < a->V || a->stride_b < 0) return CADD_ERR_SHAPE;
 
@@ -161,9 +163,9 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
     ep.flags = a->flags; ep.partials = (const unsigned char*)a->workspace;
     ep.l_eff = a->l_eff; ep.bonus_token = a->bonus_token; ep.ctx_len = a->ctx_len;
     ep.cost_kind = a->cost_kind; ep.cost_coef = a->cost_coef; ep.cost_table = a->cost_table;
-    ep.table_idx = a->table_idx; ep.t_draft = a->t_draft;
+    ep.table_idx = a->table_idx; ep.t_draft = a->t_draft; ep.ctx_grid = a->ctx_grid; ep.n_tables = a->n_tables;
     ep.n_nodes = a->n_nodes; ep.token_ids = a->token_ids; ep.parent_idx = a->parent_idx; ep.depth = a->depth;
-    ep.position_ids = a->position_ids; ep.node_logprob = a->node_logprob; ep.phi = a->phi; ep.theta = a->theta;
+    ep.position_ids = a->position_ids; ep.node_logprob = a->node_logprob; ep.phi = a->phi; ep.theta = a->theta; ep.theta_curve = a->theta_curve;
     ep.mask_bits = a->mask_bits; ep.mask_dense = a->mask_dense; ep.topk_token = a->topk_token;
     ep.topk_logprob = a->topk_logprob; ep.status = a->status;
     if (pl.lay.total > 48 * 1024) {

@@ -35,6 +35,8 @@ struct ExpandParams {
     const double* cost_table;
     const int32_t* table_idx;
     const double* t_draft;
+    const int32_t* ctx_grid;
+    int n_tables;
     int32_t* n_nodes;
     int32_t* token_ids;
     int32_t* parent_idx;
@@ -43,6 +45,7 @@ struct ExpandParams {
     double* node_logprob;
     double* phi;
     double* theta;
+    double* theta_curve;
     uint32_t* mask_bits;
     uint8_t* mask_dense;
     int32_t* topk_token;
@@ -90,10 +93,20 @@ __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int KP, int 
     return o;
 }
 
-__device__ __forceinline__ double cost_verify(int kind, const double* q, const double* trow, int n) {
-    if (kind == CADD_COST_TABLE) return trow[n];
-    double x = (double)n;
-    return q[1] + q[2] * x + q[3] * (x * x);
+// The verification cost C_v(n) of one request: quadratic, one table row, or two table rows blended by
+// context length (Eq. 13).
+struct CostModel {
+    int kind;
+    double q[4];            // QUADRATIC: (C_d, a, b, c)
+    const double* row0;     // TABLE: the row; TABLE_INTERP: the row of L_j
+    const double* row1;     // TABLE_INTERP: the row of L_{j+1}
+    double alpha;           // TABLE_INTERP
+};
+__device__ __forceinline__ double cost_verify(const CostModel& cm, int n) {
+    if (cm.kind == CADD_COST_TABLE) return cm.row0[n];
+    if (cm.kind == CADD_COST_TABLE_INTERP) return (1.0 - cm.alpha) * cm.row0[n] + cm.alpha * cm.row1[n];
+    const double x = (double)n;
+    return cm.q[1] + cm.q[2] * x + cm.q[3] * (x * x);
 }
 
 __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
@@ -111,7 +124,7 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
     double* fAp = (double*)(fLo + (size_t)lay.fr_cap * 32);  // the entry's parent's sum of (logit - row max)
 
     __shared__ int s_status, s_pinf, s_Lr, s_n;
-    __shared__ double s_phi, s_theta;
+    __shared__ double s_phi, s_theta, s_theta0;
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -204,20 +217,31 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         const int Lr = s_Lr;
         const int B_max = p.B_max;
         const bool fixed = (p.flags & CADD_FLAG_FIXED_BUDGET) != 0;
-        double q4[4] = {0, 0, 0, 0};
-        const double* trow = nullptr;
+        CostModel cm;
+        cm.kind = p.cost_kind; cm.row0 = cm.row1 = nullptr; cm.alpha = 0.0;
+        cm.q[0] = cm.q[1] = cm.q[2] = cm.q[3] = 0.0;
         double C_d;
         if (p.cost_kind == CADD_COST_QUADRATIC) {
-            for (int c = 0; c < 4; ++c) q4[c] = p.cost_coef[(int64_t)b * 4 + c];
-            C_d = q4[0];
-        } else {
-            trow = p.cost_table + (int64_t)p.table_idx[b] * (B_max + 1);
+            for (int c = 0; c < 4; ++c) cm.q[c] = p.cost_coef[(int64_t)b * 4 + c];
+            C_d = cm.q[0];
+        } else if (p.cost_kind == CADD_COST_TABLE) {
+            cm.row0 = p.cost_table + (int64_t)p.table_idx[b] * (B_max + 1);
+            C_d = p.t_draft[b];
+        } else {                                            // Eq. 13: the two profiled context lengths around l
+            const int l = p.ctx_len ? p.ctx_len[b] : 0;
+            int jlo = 0;
+            while (jlo + 1 < p.n_tables && p.ctx_grid[jlo + 1] <= l) ++jlo;
+            int jhi = jlo + 1 < p.n_tables ? jlo + 1 : jlo;
+            if (l <= p.ctx_grid[0]) jlo = jhi = 0;
+            cm.row0 = p.cost_table + (int64_t)jlo * (B_max + 1);
+            cm.row1 = p.cost_table + (int64_t)jhi * (B_max + 1);
+            cm.alpha = jhi == jlo ? 0.0 : ((double)l - (double)p.ctx_grid[jlo]) / ((double)p.ctx_grid[jhi] - (double)p.ctx_grid[jlo]);
             C_d = p.t_draft[b];
         }
         int st = 0;
         bool ok = true;
         double theta_prev = 0.0, Phi = 0.0;
-        const double den0 = C_d + cost_verify(p.cost_kind, q4, trow, 0);
+        const double den0 = C_d + cost_verify(cm, 0);
         if (!(den0 > 0.0)) { st |= CADD_STATUS_COST_NONPOSITIVE; ok = false; }
         else theta_prev = 1.0 / den0;
         if (s_pinf) ok = false;
@@ -378,13 +402,15 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
                 if (lane >= o) cum += t;
             }
             const double Phi_j = Phi + cum;
-            const double den = act ? C_d + cost_verify(p.cost_kind, q4, trow, j) : 1.0;
+            const double den = act ? C_d + cost_verify(cm, j) : 1.0;
             const bool bad = !(den > 0.0);
             const double theta_j = (1.0 + Phi_j) / den;
             double theta_jm1 = __shfl_up_sync(kFullMask, theta_j, 1);
             if (lane == 0) theta_jm1 = theta_prev;
             const bool stop = act && (bad || (!fixed && theta_j <= theta_jm1));
             const unsigned sm = __ballot_sync(kFullMask, stop);
+            if (p.theta_curve && act && (sm == 0 || lane < __ffs(sm) - 1))
+                p.theta_curve[(int64_t)b * R + j] = theta_j;        // theta*(n) of every accepted n (Prop. 1)
             if (sm) {
                 const int f = __ffs(sm) - 1;                // rows n+1 .. n+f are accepted
                 if (__shfl_sync(kFullMask, (int)bad, f)) st |= CADD_STATUS_COST_NONPOSITIVE;
@@ -401,7 +427,7 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         }
         if (ok && !stopped) st |= (fsize == 0) ? CADD_STATUS_FRONTIER_EXHAUSTED : CADD_STATUS_CAP_HIT;
         if (lane == 0) {
-            s_n = n; s_phi = Phi; s_theta = theta_prev;
+            s_n = n; s_phi = Phi; s_theta = theta_prev; s_theta0 = (den0 > 0.0) ? 1.0 / den0 : 0.0;
             if (st) atomicOr(&s_status, st);
         }
     }
@@ -415,7 +441,10 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         if (p.phi) p.phi[b] = s_phi;
         if (p.theta) p.theta[b] = s_theta;
         if (p.status) p.status[b] = s_status;
+        if (p.theta_curve) p.theta_curve[(int64_t)b * R] = s_theta0;
     }
+    if (p.theta_curve)
+        for (int j = n + 1 + tid; j < R; j += kThreads) p.theta_curve[(int64_t)b * R + j] = 0.0;
     for (int j = tid; j < R; j += kThreads) {
         const int64_t o = (int64_t)b * R + j;
         int t = -1, par = -1, d = 0, pos = 0;

@@ -26,6 +26,7 @@ import torch
 
 COST_QUADRATIC = 0
 COST_TABLE = 1
+COST_TABLE_INTERP = 2
 
 
 @dataclass(frozen=True)
@@ -232,3 +233,16 @@ def make_target_logits(cfg: WorkloadConfig, seed: int, draft: DraftInputs, depth
                 bst[b, r0:r1].to(device=device, dtype=torch.float32)
             out[b, r0:r1] = y.to(cfg.torch_dtype)
     return out
+
+
+def make_context_cost_tables(B_max: int, grid=(0, 1024, 2048, 3072, 4096, 5120, 6144, 7168, 8192),
+                             abc: Tuple[float, float, float] = (1.0, 0.002, 0.00002)):
+    """Verification-cost tables at a grid of context lengths, shaped like the paper's profile (Figure 3:
+    convex and increasing in the node count; longer contexts shift the curve up and steepen it).
+    Returns (tables [len(grid), B_max+1] float64, grid int32)."""
+    a, b, c = abc
+    n = torch.arange(B_max + 1, dtype=torch.float64)
+    rows = []
+    for j, _ in enumerate(grid):
+        rows.append(a * (1.0 + 0.10 * j) + b * (1.0 + 0.15 * j) * n + c * (1.0 + 0.10 * j) * n * n)
+    return torch.stack(rows), torch.tensor(grid, dtype=torch.int32)

@@ -41,7 +41,7 @@ def round_trip(cfg, seed, rows_mode=G.ROWS_LIVE, dense_mask=False):
 
 
 def test_library_reports_version():
-    assert G.cadd_version() == 1
+    assert G.cadd_version() == 2
     assert G.cadd_status_string(0) == "ok"
 
 
@@ -209,3 +209,25 @@ def test_deterministic_and_reused_buffers():
         a, b = getattr(t1, f), getattr(t2, f)
         fin = torch.isfinite(a)
         assert torch.equal(fin, torch.isfinite(b)) and torch.allclose(a[fin], b[fin], rtol=0, atol=2e-9), f
+
+
+def test_context_interpolated_cost_and_theta_curve():
+    """Table cost blended by context length (Eq. 13) and the theta*(n) curve output, against the oracle."""
+    B = 200
+    tables, grid = synth.make_context_cost_tables(B)
+    gen = torch.Generator().manual_seed(77)
+    x = (torch.randn(8, 6, 5000, generator=gen) * 3).to(torch.bfloat16)
+    ctx = torch.tensor([0, 512, 1024, 2300, 5000, 8191, 8192, 30000], dtype=torch.int32)
+    td = torch.full((8,), 0.25, dtype=torch.float64)
+    for flags in (0, G.FLAG_FIXED_BUDGET):
+        kw = dict(ctx_len=ctx, cost_kind=G.COST_TABLE_INTERP, cost_table=tables, ctx_grid=grid, t_draft=td)
+        ot = O.build_tree(x, 6, B, flags=flags, **kw)
+        gt = G.cadd_build_tree(x.cuda(), 6, B, flags=flags | G.FLAG_EMIT_TOPK, theta_curve=True, **kw)
+        torch.cuda.synchronize()
+        assert not compare_build(gt, ot, 6)["exempt"]
+        np.testing.assert_allclose(to_cpu(gt.theta_curve).numpy(), ot.theta_curve.numpy(), rtol=1e-5, atol=0)
+    assert int(ot.n_nodes.min()) == B                      # the fixed-budget run is a whole budget sweep
+    curve = to_cpu(gt.theta_curve).numpy()
+    stop = O.build_tree(x, 6, B, **kw)
+    for b in range(8):                                     # Corollary 1: the rule stops at the curve's first maximum
+        assert int(stop.n_nodes[b]) == int(np.argmax(curve[b] >= curve[b].max() * (1 - 1e-12)))

@@ -457,3 +457,41 @@ def test_cross_depth_exact_tie_prefers_lower_depth():
     assert t.token_ids[0, 1:5].tolist() == [0, 1, 1, 1]
     assert t.parent_idx[0, 1:5].tolist() == [0, 0, 1, 2]
     np.testing.assert_allclose(t.node_logprob[0, 1:5].numpy(), math.log(0.5), rtol=1e-15)
+
+
+# ---------------- context interpolation of the cost tables (Eq. 13) ----------------
+def test_context_interpolated_cost():
+    from paper_2606_01813_b200 import synth
+    B = 96
+    tables, grid = synth.make_context_cost_tables(B)
+    assert np.all(np.diff(tables.numpy(), 2, axis=1) >= -1e-12) and np.all(np.diff(tables.numpy(), axis=1) > 0)
+    x = rand_logits(31, 6, 5, 400, dtype=torch.bfloat16, scale=3.0)
+    td = torch.full((6,), 0.3, dtype=torch.float64)
+    kw = dict(cost_kind=O.COST_TABLE_INTERP, cost_table=tables, ctx_grid=grid, t_draft=td)
+    # on a grid point, below and above the profiled range: exactly one table
+    ctx = torch.tensor([0, 2048, 8192, 20000, 3072, 1024], dtype=torch.int32)
+    ti = O.build_tree(x, 4, B, ctx_len=ctx, **kw)
+    tt = O.build_tree(x, 4, B, ctx_len=ctx, cost_kind=O.COST_TABLE, cost_table=tables, t_draft=td,
+                      table_idx=torch.tensor([0, 2, 8, 8, 3, 1], dtype=torch.int32))
+    assert torch.equal(ti.n_nodes, tt.n_nodes) and torch.equal(ti.token_ids, tt.token_ids)
+    np.testing.assert_allclose(ti.theta.numpy(), tt.theta.numpy(), rtol=1e-15)
+    # between two grid points: the blend is itself a table; it stays convex and increasing (the remark after Eq. 13)
+    ctx = torch.tensor([512, 1536, 2300, 5000, 7000, 8191], dtype=torch.int32)
+    blended = []
+    for l in ctx.tolist():
+        j = max(k for k in range(len(grid)) if int(grid[k]) <= l)
+        alpha = (l - int(grid[j])) / (int(grid[j + 1]) - int(grid[j]))
+        assert 0.0 <= alpha < 1.0
+        blended.append((1 - alpha) * tables[j] + alpha * tables[j + 1])
+    blended = torch.stack(blended)
+    assert np.all(np.diff(blended.numpy(), 2, axis=1) >= -1e-12) and np.all(np.diff(blended.numpy(), axis=1) > 0)
+    ti = O.build_tree(x, 4, B, ctx_len=ctx, **kw)
+    tt = O.build_tree(x, 4, B, ctx_len=ctx, cost_kind=O.COST_TABLE, cost_table=blended, t_draft=td,
+                      table_idx=torch.arange(6, dtype=torch.int32))
+    assert torch.equal(ti.n_nodes, tt.n_nodes) and torch.equal(ti.token_ids, tt.token_ids)
+    np.testing.assert_allclose(ti.theta.numpy(), tt.theta.numpy(), rtol=1e-14)
+    # a longer context costs more per node, so the chosen budget cannot grow (Section 5.3, third observation)
+    same = x[:1].expand(9, -1, -1).contiguous()
+    sweep = O.build_tree(same, 4, B, ctx_len=torch.tensor([0, 700, 1500, 2600, 4000, 5500, 6100, 7900, 9000], dtype=torch.int32),
+                         cost_kind=O.COST_TABLE_INTERP, cost_table=tables, ctx_grid=grid, t_draft=torch.full((9,), 0.3, dtype=torch.float64))
+    assert np.all(np.diff(sweep.n_nodes.numpy()) <= 0) and np.all(np.diff(sweep.theta.numpy()) < 0)
