@@ -19,6 +19,8 @@
  *   - Index arithmetic is 64-bit; strides are counted in ELEMENTS of the logits dtype; the
  *     vocabulary axis is contiguous.
  *   - There is no CPU fallback: a machine without a CUDA device gets CADD_ERR_LAUNCH.
+ *   - Finite logits are expected to satisfy |x| <= 1e6 (real logits are far smaller).  Larger finite values are
+ *     processed without fault, rankings stay exact, but the reported log-probabilities lose accuracy.
  *
  * Notation follows the paper: V vocabulary size, L draft block length (= maximum depth),
  * K candidates kept per position, n the number of DRAFT nodes of the tree (the root, i.e. the

@@ -231,3 +231,30 @@ def test_context_interpolated_cost_and_theta_curve():
     stop = O.build_tree(x, 6, B, **kw)
     for b in range(8):                                     # Corollary 1: the rule stops at the curve's first maximum
         assert int(stop.n_nodes[b]) == int(np.argmax(curve[b] >= curve[b].max() * (1 - 1e-12)))
+
+
+def test_adversarial_rows_full_vocabulary():
+    """Rows that defeat the streaming top-K heuristics at V = 151936: ascending (every element a new best: the
+    candidate ring overflows and the careful path takes over), descending, all equal, two values alternating,
+    large magnitudes, denormals, and a row whose mass sits in one token.  K = 64 is the largest list."""
+    V, L = 151936, 8
+    g = torch.Generator().manual_seed(123)
+    base = torch.randn(L, V, generator=g) * 2
+    x = torch.empty(1, L, V)
+    x[0, 0] = torch.sort(base[0]).values                           # ascending
+    x[0, 1] = torch.sort(base[1], descending=True).values          # descending
+    x[0, 2] = 1.5                                                   # all equal
+    x[0, 3] = torch.where(torch.arange(V) % 2 == 0, torch.tensor(0.25), torch.tensor(-0.25))
+    x[0, 4] = base[4] * 1e4                                         # large magnitudes (the documented range is |x| <= 1e6)
+    x[0, 5] = base[5] * 1e-40                                       # denormals in fp32, zeros in bf16
+    x[0, 6] = base[6]; x[0, 6, 77777] = 80.0                        # one dominant token
+    x[0, 7] = torch.round(base[7])                                  # a handful of distinct values, massive ties
+    coef = quad_coef(1, 0.3, 1.0, 0.002, 0.00002)
+    for dtype in (torch.bfloat16, torch.float32):
+        xs = x.to(dtype)
+        for K, B in ((64, 300), (3, 40)):
+            for flags in (0, G.FLAG_FIXED_BUDGET):
+                gt, ot = run_both_build(xs, K, B, cost_coef=coef, flags=flags)
+                diag = compare_build(gt, ot, K)
+                assert not diag["exempt"], diag
+                assert diag["max_logZ_err"] < 1e-6, diag
