@@ -37,7 +37,7 @@ UNIT = "rounds/s"
 KERNELS_PER_STEP = 4          # softmax_topk_partial, expand_emit, row_argmax, accept_walk
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one row_argmax launch as a multiple of its
-# algorithmic bytes, from the ncu capture of the config-2 launch summarised in profiles/row_argmax_config2.md
+# algorithmic bytes, from an ncu capture of the config-2 launch (summary kept under profiles/)
 # (2.5055 GB for 2.4990 GB).  Traffic grows in proportion to the rows read, so other workloads scale it.
 ARGMAX_TRAFFIC_RATIO = 1.0026
 

@@ -18,22 +18,24 @@
 // elements and one compare against the CTA's running KP-th best value; per element two FMAs
 // (x*log2e split in hi+lo, minus an integer reference exponent; issued as packed fma.rn.f32x2), one
 // ex2.approx, packed adds; the fp32 sum of the tile goes to an fp64 accumulator.  An element that reaches
-// the threshold is appended to a shared ring of candidate keys and replaced by -Inf in the register copy,
-// so that it is left out of the sum exactly.  Whenever KP new candidates have gathered, ONE warp (whichever
-// gets the lock) merges them into the sorted list of the KP best, folds the losers into its sums and
-// publishes the new threshold; the other warps keep streaming with the old one (a stale threshold only
-// means a few extra candidates).
+// the threshold is appended to a shared buffer of candidate keys and replaced by -Inf in the register copy,
+// so that it is left out of the sum exactly.  The buffer is append-only while the segment streams.  Whenever
+// 32 new candidates have gathered, one warp sorts that block in registers (bitonic network over the lanes)
+// and raises the threshold to the block's KP-th best key: every candidate already beat the old threshold,
+// so this is a valid lower bound on the segment's KP-th best, and it costs about a hundred instructions with
+// no lock and no list to maintain.  At the end of the segment the CTA selects the KP best of the buffer and
+// folds the rest back into the sums.
 //
-// If the candidate ring overflows (pathological inputs such as an ascending row) or a non-finite value
-// poisons the sums, the segment is redone by the careful path: element by element from global memory,
-// with a CTA-wide barrier protocol.  Slow, but correct for every input.
+// If the buffer overflows (pathological inputs such as an ascending row) or a non-finite value poisons the
+// sums, the segment is redone by the careful path: element by element from global memory, with a CTA-wide
+// barrier protocol that compacts the buffer as it goes.  Slow, but correct for every input.
 #pragma once
 #include "common.cuh"
 #include "tile_ring.cuh"
 
 namespace cadd {
 
-constexpr int kCandCap = 512;             // candidate ring entries per CTA (power of two)
+constexpr int kCandCap = 768;             // candidate buffer entries per CTA
 constexpr int kMaxKP = 64;
 
 constexpr uint32_t kPartNonfinite = 1u;   // NaN or +Inf seen
@@ -95,7 +97,7 @@ __device__ __forceinline__ void fold_scalar(ThreadSum& s, float x) {   // x fini
 
 // Shared state of one CTA.
 struct TopkShared {
-    uint64_t keys[kCandCap]; // fast path: ring of candidate keys (0 = not written yet); careful path: plain buffer
+    uint64_t keys[kCandCap]; // candidate keys; fast path: append-only, 0 = not written yet
     uint64_t win[kMaxKP];    // the KP best candidates so far, sorted, best first
     unsigned hist[256];
     unsigned count;          // careful path: entries in keys[]
@@ -105,8 +107,7 @@ struct TopkShared {
     uint64_t sel_prefix;
     unsigned sel_need;
     unsigned pushed;         // fast path: candidates appended so far
-    unsigned consumed;       // fast path: candidates merged so far (changed under the lock only)
-    unsigned lock;           // fast path: 1 while a warp merges
+    unsigned scanned;        // fast path: candidates already used for a threshold update (claimed in blocks)
     unsigned overflow;       // fast path: the ring was full at some push
     unsigned timeout;        // a bounded wait ran out
     double red_d[kThreads / 32];
@@ -171,67 +172,70 @@ __device__ __noinline__ uint32_t take_candidate(TopkShared& sh, float x, uint32_
     const uint64_t key = make_key(x, id);
     if (key <= thrk) return 0u;                            // equal value, higher id than the threshold key
     const unsigned pos = atomicAdd(&sh.pushed, 1u);
-    if (pos - *(volatile unsigned*)&sh.consumed >= (unsigned)kCandCap) {
+    if (pos >= (unsigned)kCandCap) {
         sh.overflow = 1;                                   // no room: the segment will be redone carefully
         return 0u;
     }
-    *(volatile uint64_t*)&sh.keys[pos & (kCandCap - 1)] = key;
+    *(volatile uint64_t*)&sh.keys[pos] = key;
     return kTakeExclude;
 }
 
-// One warp merges the candidates appended since the last merge (at most 32 per call) into the sorted list
-// of the KP best, folds the losers into its lanes' sums and raises the threshold.  The caller holds the lock.
-// ok = false if an entry that was announced never showed up within the spin limit.
-struct MergeResult { ThreadSum s; bool ok; };
-__device__ __noinline__ MergeResult warp_merge_candidates(TopkShared& sh, ThreadSum s, int KP) {
+// Candidates per threshold update: at least twice KP, so that the block's KP-th best is a sharp bound.
+__device__ __forceinline__ unsigned threshold_block(int KP) { return KP <= 16 ? 32u : (KP <= 32 ? 64u : 128u); }
+
+// One warp turns a block of freshly appended candidates, starting at entry c0, into a new threshold: the
+// block's KP-th best key.  Any KP distinct elements of the segment bound its KP-th best from below, so the
+// result is always valid.  Nothing is removed from the buffer.
+// Returns false if an announced entry never showed up within the spin limit.
+__device__ __noinline__ bool warp_block_threshold(TopkShared& sh, unsigned c0, int KP) {
     const int lane = threadIdx.x & 31;
-    const unsigned c0 = *(volatile unsigned*)&sh.consumed;
-    const unsigned avail = *(volatile unsigned*)&sh.pushed - c0;
-    const unsigned m = avail < 32u ? avail : 32u;
+    const int per_lane = (int)threshold_block(KP) / 32;    // 1, 2 or 4
+    uint64_t k[4] = {0ull, 0ull, 0ull, 0ull};
     bool ok = true;
-    uint64_t kn = 0;                                       // this lane's new candidate
-    if ((unsigned)lane < m) {
-        volatile uint64_t* slot = &sh.keys[(c0 + lane) & (kCandCap - 1)];
-        int spins = 0;
-        while ((kn = *slot) == 0ull && spins < kSpinLimit && !*(volatile unsigned*)&sh.overflow) ++spins;   // its writer is about to store it
-        if (kn == 0ull) ok = false;
-        *slot = 0ull;                                      // the ring entry is free again
-    }
-    ok = __all_sync(kFullMask, ok);
-    const int nold = (int)sh.nwin;
-    const uint64_t k0 = lane < nold ? sh.win[lane] : 0ull;  // the current list is sorted: win[i] has rank i
-    const uint64_t k1 = lane + 32 < nold ? sh.win[lane + 32] : 0ull;
-    // New rank of an old key = its old rank + the number of new keys above it; rank of a new key = the
-    // number of old and new keys above it.  Every new key is broadcast once (keys are unique; 0 = absent).
-    int r0 = lane, r1 = lane + 32, rn = 0;
-    for (int j = 0; j < (int)m; ++j) {
-        const uint64_t bn = __shfl_sync(kFullMask, kn, j);
-        r0 += bn > k0;
-        r1 += bn > k1;
-        int above = __popc(__ballot_sync(kFullMask, k0 > bn)) + __popc(__ballot_sync(kFullMask, kn > bn));
-        if (nold > 32) above += __popc(__ballot_sync(kFullMask, k1 > bn));
-        if (lane == j) rn = above;
-    }
-    __syncwarp();
-    if (k0) { if (r0 < KP) sh.win[r0] = k0; else fold_scalar(s, key_value(k0)); }
-    if (k1) { if (r1 < KP) sh.win[r1] = k1; else fold_scalar(s, key_value(k1)); }
-    if (kn) { if (rn < KP) sh.win[rn] = kn; else fold_scalar(s, key_value(kn)); }
-    __syncwarp();
-    if (lane == 0) {
-        const int total = nold + (int)m;
-        const int nw = total < KP ? total : KP;
-        sh.nwin = nw;
-        if (nw == KP) {
-            const uint64_t kth = sh.win[KP - 1];
-            if (kth > sh.thr_key) *(volatile uint64_t*)&sh.thr_key = kth;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        if (q < per_lane) {
+            volatile uint64_t* slot = &sh.keys[c0 + q * 32 + lane];
+            int spins = 0;
+            while ((k[q] = *slot) == 0ull && spins < kSpinLimit && !*(volatile unsigned*)&sh.overflow) ++spins;   // its writer is about to store it
+            if (k[q] == 0ull) ok = false;
         }
-        __threadfence_block();
-        *(volatile unsigned*)&sh.consumed = c0 + m;
     }
-    __syncwarp();
-    MergeResult res;
-    res.s = s; res.ok = ok;
-    return res;
+    if (!__all_sync(kFullMask, ok)) return false;
+    uint64_t kth;
+    if (per_lane == 1) {
+        uint64_t key = k[0];                               // bitonic sort over the lanes, best first
+#pragma unroll
+        for (int blk = 2; blk <= 32; blk <<= 1) {
+#pragma unroll
+            for (int j = blk >> 1; j > 0; j >>= 1) {
+                const uint64_t other = __shfl_xor_sync(kFullMask, key, j);
+                const bool take_max = ((lane & j) != 0) == ((lane & blk) != 0);
+                key = take_max ? max(key, other) : min(key, other);
+            }
+        }
+        kth = __shfl_sync(kFullMask, key, KP - 1);
+    } else {                                               // rank the keys by counting (they are unique)
+        int r[4] = {0, 0, 0, 0};
+        for (int j = 0; j < 32; ++j) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (q < per_lane) {
+                    const uint64_t bq = __shfl_sync(kFullMask, k[q], j);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) r[t] += (t < per_lane) && bq > k[t];
+                }
+            }
+        }
+        kth = 0ull;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const unsigned m = __ballot_sync(kFullMask, q < per_lane && r[q] == KP - 1);
+            if (m) kth = __shfl_sync(kFullMask, k[q], __ffs(m) - 1);
+        }
+    }
+    if (lane == 0) atomicMax((unsigned long long*)&sh.thr_key, (unsigned long long)kth);
+    return true;
 }
 
 // The thread's sum is passed and returned by value so that it stays in registers in the hot loop.
@@ -392,7 +396,6 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkParams p) {
     using E = Elem<DT>;
     static_assert(kTopkUnroll == 4, "the tile loop below is written for four chunks per thread");
-    static_assert((kCandCap & (kCandCap - 1)) == 0, "the candidate ring is indexed with a mask");
     extern __shared__ unsigned char topk_smem_raw[];
     TopkShared& sh = *reinterpret_cast<TopkShared*>(((uintptr_t)topk_smem_raw + 127) & ~(uintptr_t)127);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -416,7 +419,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
     for (int q = tid; q < kCandCap; q += kThreads) sh.keys[q] = 0ull;
     if (tid == 0) {
         for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
-        sh.timeout = 0; sh.overflow = 0; sh.lock = 0; sh.pushed = 0; sh.consumed = 0; sh.nwin = 0;
+        sh.timeout = 0; sh.overflow = 0; sh.pushed = 0; sh.scanned = 0; sh.nwin = 0;
         sh.count = 0; sh.thr_key = 0; sh.thr_val = -INFINITY;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -451,34 +454,59 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
         __syncthreads();
         if (tid == 0) { sh.pushed = sh.count; sh.count = 0; }
 
-        // Seed the threshold from tile 0: at least KP finite elements are >= the smallest of KP' group maxima
-        // (groups of 256/KP' consecutive threads, KP' = KP rounded up to a power of two), each thread
-        // contributing the maximum of its chunks of the tile.  Elements equal to the seed stay candidates.
+        // Seed the threshold from tile 0.  Every thread takes the maximum of its chunks of the tile: 256 distinct
+        // elements.  For KP <= 32 the seed is the exact KP-th largest of them: each warp sorts its 32 maxima over
+        // the lanes (bitonic network), then warp 0 folds the eight sorted lists together, keeping the 32 largest
+        // (elementwise max of one list with the other reversed, then one bitonic merge).  For larger KP it is the
+        // smallest of 64 group maxima.  At least KP finite elements are >= the seed either way; elements equal
+        // to it stay candidates.
         bool landed = true;
+        float* seeds = (float*)sh.hist;
+        float gm = -INFINITY;
         if (n_tiles > 0) {
             landed = mbar_wait_bounded(&sh.full[0], 0);
-            float gm = -INFINITY;
             if (landed) {
 #pragma unroll
                 for (int u = 0; u < kTopkUnroll; ++u)
                     if (c_begin + u * kThreads + tid < c_end) gm = fmaxf(gm, E::chunk_max(sh.ring[0][u * kThreads + tid]));
             }
             if (!(fabsf(gm) < INFINITY)) gm = -INFINITY;           // NaN or Inf: no help from this thread
-            const int gs = KP <= 16 ? 16 : (KP <= 32 ? 8 : 4);
-            for (int o = gs >> 1; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(kFullMask, gm, o));
-            float* seeds = (float*)sh.hist;
-            if ((tid & (gs - 1)) == 0) seeds[tid / gs] = gm;
+            if (KP <= 32) {
+#pragma unroll
+                for (int blk = 2; blk <= 32; blk <<= 1) {
+#pragma unroll
+                    for (int j = blk >> 1; j > 0; j >>= 1) {
+                        const float other = __shfl_xor_sync(kFullMask, gm, j);
+                        const bool take_max = ((lane & j) != 0) == ((lane & blk) != 0);
+                        gm = take_max ? fmaxf(gm, other) : fminf(gm, other);
+                    }
+                }
+                seeds[tid] = gm;                                   // lane q of a warp: its q-th largest
+            } else {
+                for (int o = 2; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(kFullMask, gm, o));
+                if ((tid & 3) == 0) seeds[tid >> 2] = gm;
+            }
             if (!landed) sh.timeout = 1;
         }
         __syncthreads();
-        if (tid < 32 && n_tiles > 0 && c_end - c_begin >= kThreads) {
-            const int gs = KP <= 16 ? 16 : (KP <= 32 ? 8 : 4);
-            const int ng = kThreads / gs;
-            const float* seeds = (const float*)sh.hist;
-            float v = INFINITY;
-            for (int q = tid; q < ng; q += 32) v = fminf(v, seeds[q]);
+        if (tid < 32 && n_tiles > 0) {
+            float v;
+            if (KP <= 32) {
+                v = gm;
+                for (int w = 1; w < kThreads / 32; ++w) {
+                    v = fmaxf(v, seeds[w * 32 + 31 - lane]);       // the 32 largest of both lists, as a bitonic sequence
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(kFullMask, v, o));
+                    for (int j = 16; j > 0; j >>= 1) {
+                        const float other = __shfl_xor_sync(kFullMask, v, j);
+                        v = (lane & j) == 0 ? fmaxf(v, other) : fminf(v, other);
+                    }
+                }
+                v = __shfl_sync(kFullMask, v, KP - 1);
+            } else {
+                v = fminf(seeds[tid], seeds[tid + 32]);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(kFullMask, v, o));
+            }
             if (tid == 0 && v > -INFINITY) sh.thr_key = make_key(v, 0xffffffffu);   // the lowest key carrying this value
         }
         __syncthreads();
@@ -545,27 +573,35 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
                     if (t + kStages < n_tiles) issue_tile(t + kStages);
                 }
             }
-            // enough new candidates: one warp merges them and raises the threshold
+            // a full block of new candidates: one warp claims it and raises the threshold
+            const unsigned blk = threshold_block(KP);
+            unsigned c0 = 0;
             int go = 0;
-            if (lane == 0 && *(volatile unsigned*)&sh.pushed - *(volatile unsigned*)&sh.consumed >= (unsigned)min(2 * KP, 32))
-                go = atomicCAS(&sh.lock, 0u, 1u) == 0u;
-            if (__shfl_sync(kFullMask, go, 0)) {
-                const MergeResult mr = warp_merge_candidates(sh, s, KP);
-                s = mr.s;
-                if (!mr.ok && !*(volatile unsigned*)&sh.overflow) sh.timeout = 1;
-                __syncwarp();
-                if (lane == 0) { __threadfence_block(); atomicExch(&sh.lock, 0u); }
+            if (lane == 0) {
+                c0 = *(volatile unsigned*)&sh.scanned;
+                const unsigned have = min(*(volatile unsigned*)&sh.pushed, (unsigned)kCandCap);
+                if (have >= c0 + blk) go = atomicCAS(&sh.scanned, c0, c0 + blk) == c0;
+            }
+            go = __shfl_sync(kFullMask, go, 0);
+            if (go) {
+                c0 = __shfl_sync(kFullMask, c0, 0);
+                if (!warp_block_threshold(sh, c0, KP) && !*(volatile unsigned*)&sh.overflow) sh.timeout = 1;
             }
         }
         __syncthreads();
-        // drain: warp 0 merges what is left (nobody appends any more)
-        if (warp == 0 && !sh.overflow && !sh.timeout) {
-            for (int guard = 0; guard < 4 * kCandCap; ++guard) {
-                if (*(volatile unsigned*)&sh.pushed == *(volatile unsigned*)&sh.consumed) break;
-                const MergeResult mr = warp_merge_candidates(sh, s, KP);
-                s = mr.s;
-                if (!mr.ok) { sh.timeout = 1; break; }
+        // keep the KP best of the buffer, fold the rest into the sums (CTA-wide), sort the survivors into win[]
+        if (tid == 0) sh.count = min(sh.pushed, (unsigned)kCandCap);
+        __syncthreads();
+        if (!sh.overflow && !sh.timeout) {
+            s = refresh_candidates(sh, s, KP);
+            const int cnt = (int)sh.count;
+            if (tid < cnt) {
+                const uint64_t k = sh.keys[tid];
+                int rank = 0;
+                for (int q = 0; q < cnt; ++q) rank += sh.keys[q] > k;
+                sh.win[rank] = k;
             }
+            if (tid == 0) sh.nwin = cnt;
         }
         __syncthreads();
     }
