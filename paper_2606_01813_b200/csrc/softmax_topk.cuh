@@ -165,18 +165,20 @@ __device__ __forceinline__ bool slow_element(TopkShared& sh, ThreadSum& s, uint3
 // the tile loop stays small.  Returns kTakeExclude when the element was appended to the candidate ring
 // (or is +-Inf) and must be kept out of the fast sum, plus partial flags shifted left by 8.
 constexpr uint32_t kTakeExclude = 1u;
-__device__ __noinline__ uint32_t take_candidate(TopkShared& sh, float x, uint32_t id, uint64_t thrk) {
+__device__ __noinline__ uint32_t take_candidate(uint32_t sh_addr, float x, uint32_t id, uint64_t thrk) {
     const uint32_t bits = __float_as_uint(x);
     if ((bits & 0x7f800000u) == 0x7f800000u)               // +Inf (-Inf only while no threshold is set)
         return kTakeExclude | (bits == 0x7f800000u ? (kPartNonfinite | kPartPosInf) << 8 : 0u);
     const uint64_t key = make_key(x, id);
     if (key <= thrk) return 0u;                            // equal value, higher id than the threshold key
-    const unsigned pos = atomicAdd(&sh.pushed, 1u);
+    // the function is not inlined, so it addresses the CTA's shared state by its shared-window address
+    unsigned pos;
+    asm volatile("atom.shared.add.u32 %0, [%1], 1;" : "=r"(pos) : "r"(sh_addr + (uint32_t)offsetof(TopkShared, pushed)) : "memory");
     if (pos >= (unsigned)kCandCap) {
-        sh.overflow = 1;                                   // no room: the segment will be redone carefully
-        return 0u;
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(sh_addr + (uint32_t)offsetof(TopkShared, overflow)), "r"(1u) : "memory");
+        return 0u;                                         // no room: the segment will be redone carefully
     }
-    *(volatile uint64_t*)&sh.keys[pos] = key;
+    asm volatile("st.shared.u64 [%0], %1;" ::"r"(sh_addr + (uint32_t)offsetof(TopkShared, keys) + pos * 8u), "l"(key) : "memory");
     return kTakeExclude;
 }
 
@@ -396,8 +398,11 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkParams p) {
     using E = Elem<DT>;
     static_assert(kTopkUnroll == 4, "the tile loop below is written for four chunks per thread");
-    extern __shared__ unsigned char topk_smem_raw[];
-    TopkShared& sh = *reinterpret_cast<TopkShared*>(((uintptr_t)topk_smem_raw + 127) & ~(uintptr_t)127);
+    extern __shared__ __align__(16) unsigned char topk_smem_raw[];
+    // aligned by pointer arithmetic on the shared array itself, so that every access below compiles to a
+    // shared-memory instruction rather than a generic one
+    TopkShared& sh = *reinterpret_cast<TopkShared*>(topk_smem_raw + ((128u - (smem_u32(topk_smem_raw) & 127u)) & 127u));
+    const uint32_t sh_addr = smem_u32(&sh);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int item = blockIdx.x;
     const int rowi = item / p.S;
@@ -530,7 +535,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
 #pragma unroll
                 for (int q = 0; q < E::EPC; ++q) {
                     if (f[q] >= thrv) {
-                        const uint32_t r = take_candidate(sh, f[q], id0 + q, thrk);
+                        const uint32_t r = take_candidate(sh_addr, f[q], id0 + q, thrk);
                         if (r & kTakeExclude) mask_out<DT>(w, q);
                         flags |= r >> 8;
                     }

@@ -34,8 +34,9 @@ inline size_t argmax_smem_bytes() { return sizeof(ArgmaxRing) + 128; }
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) row_argmax_kernel(ArgmaxParams p) {
     using E = Elem<DT>;
-    extern __shared__ unsigned char argmax_smem_raw[];
-    ArgmaxRing& sh = *reinterpret_cast<ArgmaxRing*>(((uintptr_t)argmax_smem_raw + 127) & ~(uintptr_t)127);
+    extern __shared__ __align__(16) unsigned char argmax_smem_raw[];
+    // aligned by pointer arithmetic on the shared array itself: accesses stay shared-memory instructions
+    ArgmaxRing& sh = *reinterpret_cast<ArgmaxRing*>(argmax_smem_raw + ((128u - (smem_u32(argmax_smem_raw) & 127u)) & 127u));
     const int b = blockIdx.x / p.R;
     const int j = blockIdx.x - b * p.R;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
