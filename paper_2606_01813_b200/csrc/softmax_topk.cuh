@@ -15,16 +15,17 @@
 // there is no CTA-wide barrier in the steady state.
 //
 // Hot loop per thread and tile (four 16-byte chunks = 32 bf16 / 16 fp32): one packed max over all
-// elements and one compare against the CTA's running KP-th best value; per element two FMAs
+// elements and one compare against the CTA's running threshold, voted across the warp; per element two FMAs
 // (x*log2e split in hi+lo, minus an integer reference exponent; issued as packed fma.rn.f32x2), one
-// ex2.approx, packed adds; the fp32 sum of the tile goes to an fp64 accumulator.  An element that reaches
-// the threshold is appended to a shared buffer of candidate keys and replaced by -Inf in the register copy,
-// so that it is left out of the sum exactly.  The buffer is append-only while the segment streams.  Whenever
-// 32 new candidates have gathered, one warp sorts that block in registers (bitonic network over the lanes)
-// and raises the threshold to the block's KP-th best key: every candidate already beat the old threshold,
-// so this is a valid lower bound on the segment's KP-th best, and it costs about a hundred instructions with
-// no lock and no list to maintain.  At the end of the segment the CTA selects the KP best of the buffer and
-// folds the rest back into the sums.
+// ex2.approx, packed adds; the fp32 sum of the tile goes to an fp64 accumulator.  When some lane holds an
+// element that reaches the threshold, the whole warp examines that lane's elements together, one element per
+// lane, straight from the tile in shared memory: candidates are appended to a shared buffer of keys (one atomic
+// per lane examined) and overwritten by -Inf in the tile, and the owner reloads its chunks, so that candidates
+// are left out of the sum exactly.  The buffer is append-only while the segment streams.  The append that
+// completes a block of 2*KP candidates makes its warp sort that block in registers (bitonic network over the
+// lanes) and raise the threshold to the block's KP-th best key: every candidate already beat the old
+// threshold, so this is a valid lower bound on the segment's KP-th best, with no lock and no list to maintain.
+// At the end of the segment the CTA selects the KP best of the buffer and folds the rest back into the sums.
 //
 // If the buffer overflows (pathological inputs such as an ascending row) or a non-finite value poisons the
 // sums, the segment is redone by the careful path: element by element from global memory, with a CTA-wide
@@ -107,7 +108,6 @@ struct TopkShared {
     uint64_t sel_prefix;
     unsigned sel_need;
     unsigned pushed;         // fast path: candidates appended so far
-    unsigned scanned;        // fast path: candidates already used for a threshold update (claimed in blocks)
     unsigned overflow;       // fast path: the ring was full at some push
     unsigned timeout;        // a bounded wait ran out
     double red_d[kThreads / 32];
@@ -159,27 +159,6 @@ __device__ __forceinline__ bool slow_element(TopkShared& sh, ThreadSum& s, uint3
     }
     fold_scalar(s, x);
     return false;
-}
-
-// Fast-path handling of one element whose value reached the threshold value.  Kept out of line so that
-// the tile loop stays small.  Returns kTakeExclude when the element was appended to the candidate ring
-// (or is +-Inf) and must be kept out of the fast sum, plus partial flags shifted left by 8.
-constexpr uint32_t kTakeExclude = 1u;
-__device__ __noinline__ uint32_t take_candidate(uint32_t sh_addr, float x, uint32_t id, uint64_t thrk) {
-    const uint32_t bits = __float_as_uint(x);
-    if ((bits & 0x7f800000u) == 0x7f800000u)               // +Inf (-Inf only while no threshold is set)
-        return kTakeExclude | (bits == 0x7f800000u ? (kPartNonfinite | kPartPosInf) << 8 : 0u);
-    const uint64_t key = make_key(x, id);
-    if (key <= thrk) return 0u;                            // equal value, higher id than the threshold key
-    // the function is not inlined, so it addresses the CTA's shared state by its shared-window address
-    unsigned pos;
-    asm volatile("atom.shared.add.u32 %0, [%1], 1;" : "=r"(pos) : "r"(sh_addr + (uint32_t)offsetof(TopkShared, pushed)) : "memory");
-    if (pos >= (unsigned)kCandCap) {
-        asm volatile("st.shared.u32 [%0], %1;" ::"r"(sh_addr + (uint32_t)offsetof(TopkShared, overflow)), "r"(1u) : "memory");
-        return 0u;                                         // no room: the segment will be redone carefully
-    }
-    asm volatile("st.shared.u64 [%0], %1;" ::"r"(sh_addr + (uint32_t)offsetof(TopkShared, keys) + pos * 8u), "l"(key) : "memory");
-    return kTakeExclude;
 }
 
 // Candidates per threshold update: at least twice KP, so that the block's KP-th best is a sharp bound.
@@ -242,49 +221,45 @@ __device__ __noinline__ bool warp_block_threshold(TopkShared& sh, unsigned c0, i
 
 // The thread's sum is passed and returned by value so that it stays in registers in the hot loop.
 // CTA-wide: keep the KP best candidates of the buffer, fold the rest into the callers' sums and raise
-// the threshold to the KP-th best key.  Small buffers are ranked by counting; larger ones go through
-// an MSB-first radix select.  Leaves the survivors sorted, best first.
+// the threshold to the KP-th best key.  Entries below the current threshold are dropped first; what is left is
+// ranked by counting, or goes through an MSB-first radix select if it is still large.  Leaves the survivors sorted, best first.
 __device__ __noinline__ ThreadSum refresh_candidates(TopkShared& sh, ThreadSum s, int KP) {
     const int tid = threadIdx.x;
     __syncthreads();
-    const int n = min(sh.count, (unsigned)kCandCap);
+    int n = min(sh.count, (unsigned)kCandCap);
     if (n <= KP) {
         if (tid == 0) sh.count = n;
         __syncthreads();
         return s;
     }
-    uint64_t kth;
-    if (n <= 64) {
-        // the common case: warp 0 ranks all entries in registers (two per lane), every entry is
-        // broadcast once and compared against both
-        if (tid < 32) {
-            const uint64_t k0 = tid < n ? sh.keys[tid] : 0ull;
-            const uint64_t k1 = tid + 32 < n ? sh.keys[tid + 32] : 0ull;
-            int r0 = 0, r1 = 0;
-            for (int j = 0; j < n; ++j) {
-                const uint64_t kj = __shfl_sync(kFullMask, j < 32 ? k0 : k1, j & 31);
-                r0 += kj > k0;
-                r1 += kj > k1;
-            }
-            if (tid < n) { if (r0 < KP) sh.win[r0] = k0; else fold_scalar(s, key_value(k0)); }
-            if (tid + 32 < n) { if (r1 < KP) sh.win[r1] = k1; else fold_scalar(s, key_value(k1)); }
+    if (n > 64) {
+        // The current threshold is the KP-th best of some subset of the buffer (or zero), so at least KP entries
+        // reach it: everything below it is folded into the sums right away and only the rest is ranked.
+        const uint64_t thr = sh.thr_key;
+        uint64_t mine[kCandCap / kThreads];
+#pragma unroll
+        for (int q = 0; q < kCandCap / kThreads; ++q) mine[q] = tid + q * kThreads < n ? sh.keys[tid + q * kThreads] : 0ull;
+        if (tid == 0) sh.nwin = 0;
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < kCandCap / kThreads; ++q) {
+            if (mine[q] == 0ull) continue;
+            if (mine[q] >= thr) sh.keys[atomicAdd(&sh.nwin, 1u)] = mine[q];
+            else fold_scalar(s, key_value(mine[q]));
         }
         __syncthreads();
-        kth = sh.win[KP - 1];
-    } else if (n <= kThreads) {
-        // rank by counting, one warp per entry: 32 comparisons per step, counted with a ballot
-        const int lane = tid & 31;
-        for (int i = tid >> 5; i < n; i += kThreads / 32) {
-            const uint64_t k = sh.keys[i];
+        n = (int)sh.nwin;
+        __syncthreads();
+    }
+    uint64_t kth;
+    if (n <= kThreads) {
+        // rank by counting, one thread per entry (keys are unique); every entry is read as a broadcast
+        if (tid < n) {
+            const uint64_t k = sh.keys[tid];
             int rank = 0;
-            for (int q0 = 0; q0 < n; q0 += 32) {
-                const uint64_t kk = (q0 + lane < n) ? sh.keys[q0 + lane] : 0ull;
-                rank += __popc(__ballot_sync(kFullMask, kk > k));
-            }
-            if (lane == 0) {
-                if (rank < KP) sh.win[rank] = k;
-                else fold_scalar(s, key_value(k));
-            }
+            for (int j = 0; j < n; ++j) rank += sh.keys[j] > k;
+            if (rank < KP) sh.win[rank] = k;
+            else fold_scalar(s, key_value(k));
         }
         __syncthreads();
         kth = sh.win[KP - 1];
@@ -382,18 +357,6 @@ __device__ __forceinline__ uint64_t chunk_exp_sum2(const uint4& w, uint64_t l2e_
     return r;
 }
 
-// Replace element q of a chunk by -Inf (its exponential is exactly zero afterwards).
-template <int DT>
-__device__ __forceinline__ void mask_out(uint4& w, int q) {
-    uint32_t* words = reinterpret_cast<uint32_t*>(&w);
-    if constexpr (DT == CADD_DTYPE_BF16) {
-        uint32_t& x = words[q >> 1];
-        x = (q & 1) ? ((x & 0x0000ffffu) | 0xff800000u) : ((x & 0xffff0000u) | 0x0000ff80u);
-    } else {
-        words[q] = 0xff800000u;
-    }
-}
-
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkParams p) {
     using E = Elem<DT>;
@@ -402,7 +365,6 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
     // aligned by pointer arithmetic on the shared array itself, so that every access below compiles to a
     // shared-memory instruction rather than a generic one
     TopkShared& sh = *reinterpret_cast<TopkShared*>(topk_smem_raw + ((128u - (smem_u32(topk_smem_raw) & 127u)) & 127u));
-    const uint32_t sh_addr = smem_u32(&sh);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int item = blockIdx.x;
     const int rowi = item / p.S;
@@ -424,7 +386,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
     for (int q = tid; q < kCandCap; q += kThreads) sh.keys[q] = 0ull;
     if (tid == 0) {
         for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
-        sh.timeout = 0; sh.overflow = 0; sh.pushed = 0; sh.scanned = 0; sh.nwin = 0;
+        sh.timeout = 0; sh.overflow = 0; sh.pushed = 0; sh.nwin = 0;
         sh.count = 0; sh.thr_key = 0; sh.thr_val = -INFINITY;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -527,29 +489,70 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
             const uint64_t negc2 = pack2(s.negc, s.negc);
             const int cbase = c_begin + t * kTileChunks;
             const uint4* tile = &sh.ring[st][tid];
-            // append the candidates of a chunk and replace them by -Inf in the register copy
-            auto extract_candidates = [&](uint4& w, int c) {
-                const uint32_t id0 = (uint32_t)(sp.head + (int64_t)c * E::EPC);
-                float f[E::EPC];
-                E::unpack(w, f);
-#pragma unroll
-                for (int q = 0; q < E::EPC; ++q) {
-                    if (f[q] >= thrv) {
-                        const uint32_t r = take_candidate(sh_addr, f[q], id0 + q, thrk);
-                        if (r & kTakeExclude) mask_out<DT>(w, q);
-                        flags |= r >> 8;
+            // this thread's chunks of the tile; chunks past the end of the segment read as -Inf (no mass, never
+            // a candidate), so that one code path serves whole and ragged tiles
+            const uint4 kNone = DT == CADD_DTYPE_BF16 ? make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u)
+                                                      : make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
+            const int nv = c_end - (cbase + tid);                        // > u * kThreads  <=>  chunk u is valid
+            uint4 w0 = nv > 0 ? tile[0] : kNone;
+            uint4 w1 = nv > kThreads ? tile[kThreads] : kNone;
+            uint4 w2 = nv > 2 * kThreads ? tile[2 * kThreads] : kNone;
+            uint4 w3 = nv > 3 * kThreads ? tile[3 * kThreads] : kNone;
+            const float mx = E::max4(w0, w1, w2, w3);
+            unsigned hits = __ballot_sync(kFullMask, mx >= thrv && mx > -INFINITY);
+            if (hits) {
+                // Some lane holds an element that reaches the threshold (about every second warp-tile, one or two
+                // lanes).  The whole warp looks at that lane's elements together, one element per lane, straight
+                // from the tile in shared memory: candidates are appended with one atomic per lane examined, and
+                // overwritten by -Inf in the tile so that the owner's reload leaves them out of the sum exactly.
+                constexpr int NE = kTopkUnroll * E::EPC;                 // elements per thread and tile: 32 or 16
+                const int u = lane / E::EPC, q = lane % E::EPC;
+                do {
+                    const int src = __ffs(hits) - 1;
+                    hits &= hits - 1;
+                    const int slot = u * kThreads + warp * 32 + src;     // chunk slot inside the tile
+                    const int c = cbase + slot;
+                    const bool valid = lane < NE && c < c_end;
+                    char* ep = (char*)&sh.ring[st][0] + (size_t)slot * 16 + q * E::ES;
+                    float x = -INFINITY;
+                    if (valid) x = E::load(ep, 0);
+                    const uint32_t bits = __float_as_uint(x);
+                    const bool ge = valid && x >= thrv;                  // false for NaN
+                    const bool inf = (bits & 0x7f800000u) == 0x7f800000u;
+                    const uint32_t id = (uint32_t)(sp.head + (int64_t)c * E::EPC + q);
+                    const uint64_t key = make_key(x, id);
+                    const bool cand = ge && !inf && key > thrk;          // equal value, higher id than the threshold key: stays in the sum
+                    if (ge && bits == 0x7f800000u) flags |= kPartNonfinite | kPartPosInf;
+                    const unsigned m = __ballot_sync(kFullMask, cand);
+                    if (m) {
+                        const unsigned cnt = __popc(m);
+                        unsigned base = 0;
+                        if (lane == 0) base = atomicAdd(&sh.pushed, cnt);
+                        base = __shfl_sync(kFullMask, base, 0);
+                        if (cand) {
+                            const unsigned pos = base + __popc(m & ((1u << lane) - 1u));
+                            if (pos < (unsigned)kCandCap) *(volatile uint64_t*)&sh.keys[pos] = key;
+                            else sh.overflow = 1;                        // no room: the segment will be redone carefully
+                        }
+                        // the append that completes a block of candidates turns that block into a new threshold
+                        const unsigned blk = threshold_block(KP), end = base + cnt;
+                        if (end / blk != base / blk && end <= (unsigned)kCandCap) {
+                            __syncwarp();
+                            if (!warp_block_threshold(sh, (end / blk - 1u) * blk, KP) && !*(volatile unsigned*)&sh.overflow) sh.timeout = 1;
+                        }
                     }
-                }
-            };
-            if (cbase + 3 * kThreads + tid < c_end) {
-                // whole tile for this thread: one test for all 32 (16) elements
-                uint4 w0 = tile[0], w1 = tile[kThreads], w2 = tile[2 * kThreads], w3 = tile[3 * kThreads];
-                if (E::max4(w0, w1, w2, w3) >= thrv) {              // rare: some element is a candidate
-                    if (E::chunk_max(w0) >= thrv) extract_candidates(w0, cbase + tid);
-                    if (E::chunk_max(w1) >= thrv) extract_candidates(w1, cbase + kThreads + tid);
-                    if (E::chunk_max(w2) >= thrv) extract_candidates(w2, cbase + 2 * kThreads + tid);
-                    if (E::chunk_max(w3) >= thrv) extract_candidates(w3, cbase + 3 * kThreads + tid);
-                }
+                    if (cand || (ge && inf)) {
+                        if constexpr (DT == CADD_DTYPE_BF16) *(volatile uint16_t*)ep = 0xff80u;
+                        else *(volatile uint32_t*)ep = 0xff800000u;
+                    }
+                } while (hits);
+                __syncwarp();
+                w0 = nv > 0 ? tile[0] : kNone;
+                w1 = nv > kThreads ? tile[kThreads] : kNone;
+                w2 = nv > 2 * kThreads ? tile[2 * kThreads] : kNone;
+                w3 = nv > 3 * kThreads ? tile[3 * kThreads] : kNone;
+            }
+            {
                 const uint64_t a = add2(chunk_exp_sum2<DT>(w0, l2e_hi2, l2e_lo2, negc2),
                                         chunk_exp_sum2<DT>(w1, l2e_hi2, l2e_lo2, negc2));
                 const uint64_t c2 = add2(chunk_exp_sum2<DT>(w2, l2e_hi2, l2e_lo2, negc2),
@@ -557,40 +560,17 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
                 float lo, hi;
                 unpack2(add2(a, c2), lo, hi);
                 s.acc += (double)(lo + hi);
-            } else {                                                // ragged last tile
-#pragma unroll 1
-                for (int u = 0; u < kTopkUnroll; ++u) {
-                    const int c = cbase + u * kThreads + tid;
-                    if (c >= c_end) break;
-                    uint4 w = tile[u * kThreads];
-                    if (E::chunk_max(w) >= thrv) extract_candidates(w, c);
-                    float lo, hi;
-                    unpack2(chunk_exp_sum2<DT>(w, l2e_hi2, l2e_lo2, negc2), lo, hi);
-                    s.acc += (double)(lo + hi);
-                }
             }
             __syncwarp();
-            // This warp is done with the stage (its loads from it have returned: their values were consumed
-            // above); the last warp to say so refills the stage at once.
+            // This warp is done with the stage: its loads from it have returned (their values were consumed above)
+            // and its stores to it are ordered before the release.  The last warp to say so refills the stage.
             if (lane == 0) {
+                __threadfence_block();
                 if (atomicAdd(&sh.released[st], 1u) == kThreads / 32 - 1) {
                     atomicExch(&sh.released[st], 0u);
+                    __threadfence_block();
                     if (t + kStages < n_tiles) issue_tile(t + kStages);
                 }
-            }
-            // a full block of new candidates: one warp claims it and raises the threshold
-            const unsigned blk = threshold_block(KP);
-            unsigned c0 = 0;
-            int go = 0;
-            if (lane == 0) {
-                c0 = *(volatile unsigned*)&sh.scanned;
-                const unsigned have = min(*(volatile unsigned*)&sh.pushed, (unsigned)kCandCap);
-                if (have >= c0 + blk) go = atomicCAS(&sh.scanned, c0, c0 + blk) == c0;
-            }
-            go = __shfl_sync(kFullMask, go, 0);
-            if (go) {
-                c0 = __shfl_sync(kFullMask, c0, 0);
-                if (!warp_block_threshold(sh, c0, KP) && !*(volatile unsigned*)&sh.overflow) sh.timeout = 1;
             }
         }
         __syncthreads();
