@@ -17,9 +17,7 @@ static inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) 
 
 struct BuildPlan {
     int KP;          // candidates kept per (row, segment)
-    int S;           // record slots per row
-    int tpr, min_tiles, slots;
-    unsigned G;      // CTAs of the softmax/top-K kernel
+    int S;           // segments per row
     size_t partial_bytes;
     ExpandLayout lay;
 };
@@ -43,44 +41,29 @@ static int check_build_shape(const cadd_build_args* a) {
     return CADD_OK;
 }
 
-// How the softmax/top-K kernel is cut.  All tiles of all rows form one sequence and every CTA takes an equal
-// contiguous share of it, so a row may be shared by several CTAs, each leaving one partial record.
-//   tpr        tiles per row
-//   min_tiles  shortest share a CTA may get = the share when every row is live; never so short that a row would
-//              be shared by more than kMaxSegments CTAs (a share needs a few tiles to learn a sharp threshold)
-//   G          CTAs: one per resident-CTA slot, in as many equal waves as it takes to keep the rows one CTA
-//              touches within kMaxPieces; fewer when the whole job is small
-//   S          record slots per row = the most CTAs that can share a row under this cut
+// Segments per row.  Whole rows are cheapest per element (one threshold warm-up per CTA), but the
+// grid must fill the resident-CTA slots of the machine evenly: take the smallest cut whose last wave
+// is at least 85 % full (else the fullest), never making a segment shorter than 4 iterations.
 constexpr int kMaxSegments = 8;
 static BuildPlan plan_build(const cadd_build_args* a, int slots) {
     BuildPlan pl;
     pl.KP = a->K > kPreciseMin ? a->K : kPreciseMin;
     const int epc = a->logits_dtype == CADD_DTYPE_BF16 ? 8 : 4;
     const int64_t rows = (int64_t)a->batch * a->L;
-    int64_t tpr = ((a->V / epc) + kTileChunks - 1) / kTileChunks;
-    if (tpr < 1) tpr = 1;
-    const int64_t T = rows * tpr;                               // upper bound: every row live
-    int64_t m = tpr >= 2 ? (tpr - 2 + kMaxSegments - 3) / (kMaxSegments - 2) : 1;   // ceil((tpr - 2) / (kMaxSegments - 2))
-    const int64_t want = tpr < 4 ? tpr : 4;
-    if (m < want) m = want;
-    // tiles one CTA may take: half of what kMaxPieces rows allow, because the device may round the CTA count
-    // down to a whole number of waves when rows are masked, which at most doubles a share
-    const int64_t per_cta_cap = (int64_t)(kMaxPieces - 2) * tpr / 2 > 0 ? (int64_t)(kMaxPieces - 2) * tpr / 2 : 1;
-    int64_t waves = (T + (int64_t)slots * per_cta_cap - 1) / ((int64_t)slots * per_cta_cap);
-    if (waves < 1) waves = 1;
-    int64_t G = (int64_t)slots * waves;
-    if (G > T / m) G = T / m;
-    if (G < 1) G = 1;
-    const int64_t share = T / G;                                // shortest share with every row live
-    pl.tpr = (int)tpr;
-    pl.min_tiles = (int)(share < 1 ? 1 : share);                // the device never makes a share shorter than this
-    pl.slots = slots;
-    pl.G = (unsigned)G;
-    // CTAs that can overlap one row: the one holding its first tile, then one per further share start inside it.
-    // With fewer live rows the device shrinks the CTA count so that shares never get shorter than min_tiles.
-    const int64_t lo = pl.min_tiles;
-    pl.S = tpr >= 2 ? (int)((tpr - 2) / lo + 2) : 1;
-    if (pl.S > kMaxSegments) pl.S = kMaxSegments;               // unreachable by the choice of m
+    const int64_t chunks = a->V / epc;
+    int64_t cap = chunks / (4 * kTopkUnroll * kThreads);
+    if (cap > kMaxSegments) cap = kMaxSegments;
+    if (cap < 1) cap = 1;
+    int best = 1;
+    double best_eff = 0.0;
+    for (int S = 1; S <= (int)cap; ++S) {
+        const int64_t items = rows * S;
+        const int64_t waves = (items + slots - 1) / slots;
+        const double eff = (double)items / (double)(waves * slots);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = S; }
+        if (eff >= 0.85) { best = S; break; }
+    }
+    pl.S = best;
     pl.partial_bytes = (size_t)rows * pl.S * seg_partial_stride(pl.KP);
     pl.lay = expand_layout(a->L, a->K, pl.KP, pl.S, a->B_max);
     return pl;
@@ -169,9 +152,8 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
 
     TopkParams tp;
     tp.logits = a->draft_logits; tp.V = a->V; tp.stride_b = a->stride_b; tp.stride_l = a->stride_l;
-    tp.batch = a->batch; tp.L = a->L; tp.S = pl.S; tp.KP = pl.KP; tp.tpr = pl.tpr; tp.min_tiles = pl.min_tiles; tp.slots = pl.slots; tp.G = pl.G;
-    tp.l_eff = a->l_eff; tp.partials = (unsigned char*)a->workspace;
-    const unsigned items = pl.G;
+    tp.L = a->L; tp.S = pl.S; tp.KP = pl.KP; tp.l_eff = a->l_eff; tp.partials = (unsigned char*)a->workspace;
+    const unsigned items = (unsigned)((int64_t)a->batch * a->L * pl.S);
     if (a->logits_dtype == CADD_DTYPE_BF16) softmax_topk_partial_kernel<CADD_DTYPE_BF16><<<items, kThreads, topk_smem_bytes(), st>>>(tp);
     else softmax_topk_partial_kernel<CADD_DTYPE_FP32><<<items, kThreads, topk_smem_bytes(), st>>>(tp);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;

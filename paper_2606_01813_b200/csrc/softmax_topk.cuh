@@ -36,7 +36,7 @@
 
 namespace cadd {
 
-constexpr int kCandCap = 720;             // candidate buffer entries per CTA
+constexpr int kCandCap = 768;             // candidate buffer entries per CTA
 constexpr int kMaxKP = 64;
 
 constexpr uint32_t kPartNonfinite = 1u;   // NaN or +Inf seen
@@ -58,26 +58,9 @@ __host__ __device__ inline size_t seg_partial_stride(int KP) { return sizeof(Seg
 struct TopkParams {
     const void* logits;          // [batch, L, V]
     int64_t V, stride_b, stride_l;
-    int batch, L, S, KP;
-    int tpr;                     // tiles per row used for cutting: max(1, ceil((V / elements per chunk) / kTileChunks))
-    int min_tiles;               // no CTA gets fewer tiles than this (unless the whole job is smaller)
-    int slots;                   // CTAs resident on the device at once
-    unsigned G;                  // CTAs launched
+    int L, S, KP;
     const int32_t* l_eff;
     unsigned char* partials;     // [batch*L*S] records of seg_partial_stride(KP) bytes
-};
-
-// The piece of one row that one CTA handles: a run of whole tiles of the row, or all of it.
-constexpr int kMaxPieces = 8;
-struct Piece {
-    const char* row;             // first element of the row
-    int head, tail;              // the row's scalar head / tail elements (split_row)
-    int first, last;             // this piece starts / ends the row (it then takes the head / tail elements)
-    int c_begin, c_end;          // 16-byte chunks of the row in this piece
-    int n_tiles;                 // tiles with data
-    int q0;                      // index of its first tile in the CTA's own tile sequence
-    int rec;                     // record index: row * S + slot
-    int empties;                 // empty records to write behind it (the row's last piece fills the unused slots)
 };
 
 constexpr float kLog2eHi = 1.44269502162933349609375f;     // float(log2 e)
@@ -127,9 +110,6 @@ struct TopkShared {
     unsigned pushed;         // fast path: candidates appended so far
     unsigned overflow;       // fast path: the ring was full at some push
     unsigned timeout;        // a bounded wait ran out
-    int n_pieces, q_total;   // this CTA's pieces and tiles
-    int row_bi[kMaxPieces][2];   // (request, position) of the rows this CTA touches
-    Piece pieces[kMaxPieces];
     double red_d[kThreads / 32];
     float red_f[kThreads / 32];
     unsigned red_u[kThreads / 32];
@@ -256,13 +236,13 @@ __device__ __noinline__ ThreadSum refresh_candidates(TopkShared& sh, ThreadSum s
         // The current threshold is the KP-th best of some subset of the buffer (or zero), so at least KP entries
         // reach it: everything below it is folded into the sums right away and only the rest is ranked.
         const uint64_t thr = sh.thr_key;
-        uint64_t mine[(kCandCap + kThreads - 1) / kThreads];
+        uint64_t mine[kCandCap / kThreads];
 #pragma unroll
-        for (int q = 0; q < (kCandCap + kThreads - 1) / kThreads; ++q) mine[q] = tid + q * kThreads < n ? sh.keys[tid + q * kThreads] : 0ull;
+        for (int q = 0; q < kCandCap / kThreads; ++q) mine[q] = tid + q * kThreads < n ? sh.keys[tid + q * kThreads] : 0ull;
         if (tid == 0) sh.nwin = 0;
         __syncthreads();
 #pragma unroll
-        for (int q = 0; q < (kCandCap + kThreads - 1) / kThreads; ++q) {
+        for (int q = 0; q < kCandCap / kThreads; ++q) {
             if (mine[q] == 0ull) continue;
             if (mine[q] >= thr) sh.keys[atomicAdd(&sh.nwin, 1u)] = mine[q];
             else fold_scalar(s, key_value(mine[q]));
@@ -377,112 +357,6 @@ __device__ __forceinline__ uint64_t chunk_exp_sum2(const uint4& w, uint64_t l2e_
     return r;
 }
 
-// Number of position rows of request b that are read (l_eff clamped to [0, L]).
-__device__ __forceinline__ int live_rows_of(const TopkParams& p, int b) {
-    int clamped;
-    return clamp_l_eff(p.l_eff, b, p.L, &clamped);
-}
-
-// Work distribution.  All tiles of all live rows form one sequence (row-major, p.tpr tiles per row); CTA j of G'
-// takes the contiguous range [j*T/G', (j+1)*T/G'), so every CTA streams the same number of tiles (+-1) whatever
-// the number of rows, and a row is shared by at most S CTAs.  G' = min(G, T / min_tiles), rounded down to whole
-// waves, keeps ranges from getting shorter than planned when few rows are live.  Fills sh.pieces / sh.n_pieces / sh.q_total.
-// Returns false when this CTA has nothing to do.  CTA-wide (contains barriers).
-template <int DT>
-__device__ __forceinline__ bool plan_pieces(TopkShared& sh, const TopkParams& p) {
-    using E = Elem<DT>;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // ---- total number of live rows ----
-    int64_t n_live;
-    if (p.l_eff == nullptr) {
-        n_live = (int64_t)p.batch * p.L;
-    } else {
-        int mine = 0;
-        for (int b = tid; b < p.batch; b += kThreads) mine += live_rows_of(p, b);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(kFullMask, mine, o);
-        if (lane == 0) sh.red_u[warp] = (unsigned)mine;
-        __syncthreads();
-        n_live = 0;
-#pragma unroll
-        for (int q = 0; q < kThreads / 32; ++q) n_live += sh.red_u[q];
-        __syncthreads();
-    }
-    const int64_t T = n_live * p.tpr;
-    if (T == 0) return false;
-    int64_t Ge = T / p.min_tiles;
-    Ge = Ge < 1 ? 1 : (Ge > (int64_t)p.G ? (int64_t)p.G : Ge);
-    if (Ge > p.slots) Ge -= Ge % p.slots;                             // whole waves of equal CTAs
-    const int64_t j = blockIdx.x;
-    if (j >= Ge) return false;
-    const int64_t g0 = j * T / Ge, g1 = (j + 1) * T / Ge;             // this CTA's tiles
-    if (g1 <= g0) return false;
-    const int64_t lr0 = g0 / p.tpr, lr1 = (g1 - 1) / p.tpr;           // live rows touched
-    const int n_rows = (int)min(lr1 - lr0 + 1, (int64_t)kMaxPieces);  // more cannot happen by the launch plan
-
-    // ---- (request, position) of those rows ----
-    if (p.l_eff == nullptr) {
-        if (tid < n_rows) { sh.row_bi[tid][0] = (int)((lr0 + tid) / p.L); sh.row_bi[tid][1] = (int)((lr0 + tid) % p.L); }
-    } else {
-        int64_t running = 0;                                          // live rows of requests before the current block
-        for (int base = 0; base < p.batch && running <= lr1; base += kThreads) {
-            const int b = base + tid;
-            const int v = b < p.batch ? live_rows_of(p, b) : 0;
-            int incl = v;                                             // inclusive scan over the CTA
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int u = __shfl_up_sync(kFullMask, incl, o);
-                if (lane >= o) incl += u;
-            }
-            if (lane == 31) sh.red_u[warp] = (unsigned)incl;
-            __syncthreads();
-            int before = 0, total = 0;
-#pragma unroll
-            for (int q = 0; q < kThreads / 32; ++q) { const int w = (int)sh.red_u[q]; before += q < warp ? w : 0; total += w; }
-            const int64_t off = running + before + incl - v;          // first live-row index of request b
-            for (int64_t lr = max(off, lr0); lr < off + v && lr < lr0 + n_rows; ++lr) {
-                sh.row_bi[lr - lr0][0] = b;
-                sh.row_bi[lr - lr0][1] = (int)(lr - off);
-            }
-            running += total;
-            __syncthreads();
-        }
-    }
-    __syncthreads();
-
-    // ---- one thread per piece ----
-    if (tid < n_rows) {
-        Piece pc;
-        const int b = sh.row_bi[tid][0], i = sh.row_bi[tid][1];
-        const int64_t lr = lr0 + tid;
-        pc.row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)i * p.stride_l) * E::ES;
-        const RowSplit sp = split_row<DT>(pc.row, p.V);
-        const int64_t va = max(g0, lr * p.tpr) - lr * p.tpr, vb = min(g1, (lr + 1) * p.tpr) - lr * p.tpr;
-        pc.head = sp.head; pc.tail = sp.tail;
-        pc.first = va == 0; pc.last = vb == p.tpr;
-        pc.c_begin = (int)min(va * kTileChunks, (int64_t)sp.n_chunks);
-        pc.c_end = pc.last ? sp.n_chunks : (int)min(vb * kTileChunks, (int64_t)sp.n_chunks);
-        pc.n_tiles = (pc.c_end - pc.c_begin + kTileChunks - 1) / kTileChunks;
-        // the first CTA that touches this row: the largest j' with j'*T/Ge <= lr*tpr
-        const int64_t j_first = ((lr * p.tpr + 1) * Ge + T - 1) / T - 1;
-        int slot = (int)(j - j_first);
-        slot = slot < 0 ? 0 : (slot > p.S - 1 ? p.S - 1 : slot);     // cannot go out of range by the launch plan
-        pc.rec = (b * p.L + i) * p.S + slot;
-        pc.empties = pc.last ? p.S - 1 - slot : 0;
-        pc.q0 = 0;
-        sh.pieces[tid] = pc;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int q = 0;
-        for (int k = 0; k < n_rows; ++k) { sh.pieces[k].q0 = q; q += sh.pieces[k].n_tiles; }
-        sh.n_pieces = n_rows;
-        sh.q_total = q;
-    }
-    __syncthreads();
-    return true;
-}
-
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkParams p) {
     using E = Elem<DT>;
@@ -492,60 +366,54 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
     // shared-memory instruction rather than a generic one
     TopkShared& sh = *reinterpret_cast<TopkShared*>(topk_smem_raw + ((128u - (smem_u32(topk_smem_raw) & 127u)) & 127u));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int item = blockIdx.x;
+    const int rowi = item / p.S;
+    const int seg = item - rowi * p.S;
+    const int b = rowi / p.L;
+    const int i = rowi - b * p.L;
+    int clamped;
+    if (i >= clamp_l_eff(p.l_eff, b, p.L, &clamped)) return;      // masked position: never read
+
+    const char* row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)i * p.stride_l) * E::ES;
+    const RowSplit sp = split_row<DT>(row, p.V);
+    const int cps = (sp.n_chunks + p.S - 1) / p.S;                 // chunks per segment
+    const int c_begin = min(seg * cps, sp.n_chunks);
+    const int c_end = min(c_begin + cps, sp.n_chunks);
+    const uint4* body = (const uint4*)(row + (int64_t)sp.head * E::ES);
     const int KP = p.KP;
+    const int n_tiles = (c_end - c_begin + kTileChunks - 1) / kTileChunks;
 
-    if (!plan_pieces<DT>(sh, p)) return;
-    const int n_pieces = sh.n_pieces, q_total = sh.q_total;
-
+    for (int q = tid; q < kCandCap; q += kThreads) sh.keys[q] = 0ull;
     if (tid == 0) {
         for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
-        sh.timeout = 0;
+        sh.timeout = 0; sh.overflow = 0; sh.pushed = 0; sh.nwin = 0;
+        sh.count = 0; sh.thr_key = 0; sh.thr_val = -INFINITY;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    // One thread issues tile qq of the CTA's sequence into stage qq % kStages: thread 0 for the first kStages
-    // tiles, afterwards lane 0 of whichever warp is the last to finish with the tile that occupied the stage.
-    // The sequence runs across pieces, so the next row is already streaming while one row is being finished.
-    auto issue_tile = [&](int qq) {
-        int k = 0;
-        while (k + 1 < n_pieces && qq >= sh.pieces[k + 1].q0) ++k;
-        const Piece& pc = sh.pieces[k];
-        const int c0 = pc.c_begin + (qq - pc.q0) * kTileChunks;
-        const unsigned bytes = (unsigned)min(kTileChunks, pc.c_end - c0) * 16u;
-        const unsigned st = (unsigned)qq % kStages;
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic accesses to the stage are done
+    // one thread issues tile t into stage t % kStages: thread 0 for the first kStages tiles, afterwards
+    // lane 0 of whichever warp is the last to finish with the tile that occupied the stage
+    auto issue_tile = [&](int t) {
+        const int c0 = c_begin + t * kTileChunks;
+        const unsigned bytes = (unsigned)min(kTileChunks, c_end - c0) * 16u;
+        const unsigned st = (unsigned)t % kStages;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic reads of the stage are done
         mbar_arrive_expect_tx(&sh.full[st], bytes);
-        bulk_load(&sh.ring[st][0], pc.row + (int64_t)pc.head * E::ES + (int64_t)c0 * 16, bytes, &sh.full[st]);
+        bulk_load(&sh.ring[st][0], body + c0, bytes, &sh.full[st]);
     };
     if (tid == 0)
-        for (int qq = 0; qq < kStages && qq < q_total; ++qq) issue_tile(qq);
+        for (int t = 0; t < kStages && t < n_tiles; ++t) issue_tile(t);
 
     const uint64_t l2e_hi2 = pack2(kLog2eHi, kLog2eHi), l2e_lo2 = pack2(kLog2eLo, kLog2eLo);
-    unsigned st = 0, phase = 0;                                        // stage and parity of the next tile
-    int qcur = 0;                                                      // its index in the CTA's sequence
-    bool dead = false;                                                 // a bounded wait ran out earlier: only flag the rest
+    ThreadSum s{0.0, -INFINITY, 0.0f};
+    uint32_t flags = 0;
 
-    for (int pi = 0; pi < n_pieces; ++pi) {
-        const Piece& pc = sh.pieces[pi];                                // stays in shared memory: read where needed
-        const char* row = pc.row;
-        const int c_begin = pc.c_begin, c_end = pc.c_end;
-        const int n_tiles = dead ? 0 : pc.n_tiles;
-        RowSplit sp; sp.head = pc.head; sp.tail = pc.tail; sp.n_chunks = 0;
-
-        for (int q = tid; q < kCandCap; q += kThreads) sh.keys[q] = 0ull;
-        if (tid == 0) {
-            sh.overflow = 0; sh.pushed = 0; sh.nwin = 0;
-            sh.count = 0; sh.thr_key = 0; sh.thr_val = -INFINITY;
-        }
-        __syncthreads();
-        ThreadSum s{0.0, -INFINITY, 0.0f};
-        uint32_t flags = 0;
-
-        // ---------- fast path: warps advance through the piece's tiles on their own ----------
-        // ragged ends of the row, one element per thread (the row's first piece takes the head, its last one the tail)
+    // ================= fast path: warps advance on their own =================
+    {
+        // ragged ends of the row, one element per thread (segment 0 takes the head, the last one the tail)
         bool dummy = false;
-        if (!dead && pc.first && tid < sp.head) slow_element(sh, s, flags, dummy, E::load(row, tid), (uint32_t)tid);
-        if (!dead && pc.last && tid < sp.tail) {
+        if (seg == 0 && tid < sp.head) slow_element(sh, s, flags, dummy, E::load(row, tid), (uint32_t)tid);
+        if (seg == p.S - 1 && tid < sp.tail) {
             const int64_t e = p.V - sp.tail + tid;
             slow_element(sh, s, flags, dummy, E::load(row, e), (uint32_t)e);
         }
@@ -563,11 +431,11 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
         float* seeds = (float*)sh.hist;
         float gm = -INFINITY;
         if (n_tiles > 0) {
-            landed = mbar_wait_bounded(&sh.full[st], phase);
+            landed = mbar_wait_bounded(&sh.full[0], 0);
             if (landed) {
 #pragma unroll
                 for (int u = 0; u < kTopkUnroll; ++u)
-                    if (c_begin + u * kThreads + tid < c_end) gm = fmaxf(gm, E::chunk_max(sh.ring[st][u * kThreads + tid]));
+                    if (c_begin + u * kThreads + tid < c_end) gm = fmaxf(gm, E::chunk_max(sh.ring[0][u * kThreads + tid]));
             }
             if (!(fabsf(gm) < INFINITY)) gm = -INFINITY;           // NaN or Inf: no help from this thread
             if (KP <= 32) {
@@ -610,9 +478,9 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
         }
         __syncthreads();
 
-        int t = 0;
-        for (; t < n_tiles; ++t, ++qcur, st = (st + 1 == kStages ? 0u : st + 1), phase ^= (st == 0 ? 1u : 0u)) {
-            if (*(volatile unsigned*)&sh.timeout) break;
+        const bool timed_out = sh.timeout != 0;
+        unsigned st = 0, phase = 0;
+        for (int t = 0; t < n_tiles && !timed_out; ++t, st = (st + 1 == kStages ? 0u : st + 1), phase ^= (st == 0 ? 1u : 0u)) {
             const bool here = __all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase));
             if (!here) { sh.timeout = 1; break; }
             const uint64_t thrk = *(volatile uint64_t*)&sh.thr_key;          // only ever rises; stale is safe
@@ -707,7 +575,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
                 if (atomicAdd(&sh.released[st], 1u) == kThreads / 32 - 1) {
                     atomicExch(&sh.released[st], 0u);
                     __threadfence_block();
-                    if (qcur + kStages < q_total) issue_tile(qcur + kStages);
+                    if (t + kStages < n_tiles) issue_tile(t + kStages);
                 }
             }
         }
@@ -727,6 +595,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
             if (tid == 0) sh.nwin = cnt;
         }
         __syncthreads();
+    }
 
     // CTA combine: common reference C = max c_t, W = sum acc_t * 2^(c_t - C)
     double W, Cmax;
@@ -766,8 +635,8 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
         s = ThreadSum{0.0, -INFINITY, 0.0f};
         flags = 0;
         bool want_refresh = false;
-        if (pc.first && tid < sp.head) slow_element(sh, s, flags, want_refresh, E::load(row, tid), (uint32_t)tid);
-        if (pc.last && tid < sp.tail) {
+        if (seg == 0 && tid < sp.head) slow_element(sh, s, flags, want_refresh, E::load(row, tid), (uint32_t)tid);
+        if (seg == p.S - 1 && tid < sp.tail) {
             const int64_t e = p.V - sp.tail + tid;
             slow_element(sh, s, flags, want_refresh, E::load(row, e), (uint32_t)e);
         }
@@ -813,27 +682,16 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
     }
 
     // write the record: win[] is sorted, best first
-    {
-        unsigned char* rec = p.partials + (size_t)pc.rec * seg_partial_stride(KP);
-        uint64_t* out_keys = (uint64_t*)(rec + sizeof(SegPartial));
-        const int cnt = timed_out ? 0 : (int)sh.nwin;
-        if (tid < cnt) out_keys[tid] = sh.win[tid];
-        if (tid == 0) {
-            SegPartial h;
-            h.W = timed_out ? 0.0 : W * kEx2BiasFix; h.C = timed_out ? 0.0 : Cmax; h.cnt = cnt;
-            h.flags = flags | (timed_out ? kPartTimeout : 0u); h.pad[0] = h.pad[1] = 0;
-            *(SegPartial*)rec = h;
-        }
-        // the row's last piece marks the slots that no CTA fills as empty
-        if (tid >= 32 && tid < 32 + pc.empties) {
-            SegPartial h;
-            h.W = 0.0; h.C = 0.0; h.cnt = 0; h.flags = 0; h.pad[0] = h.pad[1] = 0;
-            *(SegPartial*)(rec + (size_t)(tid - 31) * seg_partial_stride(KP)) = h;
-        }
+    unsigned char* rec = p.partials + (size_t)item * seg_partial_stride(KP);
+    uint64_t* out_keys = (uint64_t*)(rec + sizeof(SegPartial));
+    const int cnt = timed_out ? 0 : (int)sh.nwin;
+    if (tid < cnt) out_keys[tid] = sh.win[tid];
+    if (tid == 0) {
+        SegPartial h;
+        h.W = timed_out ? 0.0 : W * kEx2BiasFix; h.C = timed_out ? 0.0 : Cmax; h.cnt = cnt;
+        h.flags = flags | (timed_out ? kPartTimeout : 0u); h.pad[0] = h.pad[1] = 0;
+        *(SegPartial*)rec = h;
     }
-    dead = timed_out;
-    __syncthreads();                                                   // win[] and the sums are free for the next piece
-    }   // pieces
 }
 
 }  // namespace cadd
