@@ -38,8 +38,8 @@ KERNELS_PER_STEP = 4          # softmax_topk_partial, expand_emit, row_argmax, a
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one row_argmax launch as a multiple of its
 # algorithmic bytes, from an ncu capture of the config-2 launch (summary kept under profiles/)
-# (2.5055 GB for 2.4990 GB).  Traffic grows in proportion to the rows read, so other workloads scale it.
-ARGMAX_TRAFFIC_RATIO = 1.0026
+# (2.5037 GB for 2.4990 GB).  Traffic grows in proportion to the rows read, so other workloads scale it.
+ARGMAX_TRAFFIC_RATIO = 1.0019
 
 
 def measured_peak_gbs():
