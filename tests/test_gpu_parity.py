@@ -211,6 +211,36 @@ def test_deterministic_and_reused_buffers():
         assert torch.equal(fin, torch.isfinite(b)) and torch.allclose(a[fin], b[fin], rtol=0, atol=2e-9), f
 
 
+def test_round_replays_from_a_cuda_graph():
+    """Both entry points only enqueue kernels on the given stream, so one round can be captured once and
+    replayed; a replay on fresh inputs of the same shape gives the oracle's answer."""
+    cfg = synth.scaled(synth.CONFIGS["c2"], batch=2, V=32000)
+    d0, d1 = synth.make_draft_inputs(cfg, 5), synth.make_draft_inputs(cfg, 6)
+    c = synth.make_cost_inputs(cfg, 5)
+    x = d0.logits.cuda()
+    y = torch.zeros(cfg.batch, cfg.R, cfg.V, dtype=x.dtype, device="cuda")
+    kw = dict(l_eff=d0.l_eff.cuda(), bonus_token=d0.bonus_token.cuda(), ctx_len=d0.ctx_len.cuda(), cost_coef=c.coef.cuda())
+    ws = torch.empty(G.cadd_build_workspace_bytes(cfg.batch, cfg.L, cfg.V, cfg.K, cfg.B_max, cfg.R, x.dtype),
+                     dtype=torch.uint8, device="cuda")
+    tree = G.cadd_build_tree(x, cfg.K, cfg.B_max, cfg.R, workspace=ws, **kw)            # first call outside capture
+    verdict = G.cadd_verify_tree(y, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, G.ROWS_LIVE)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        G.cadd_build_tree(x, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=tree, **kw)
+        G.cadd_verify_tree(y, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, G.ROWS_LIVE, out=verdict)
+    for d in (d1, d0):
+        x.copy_(d.logits)
+        ot = O.build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, l_eff=d0.l_eff, bonus_token=d0.bonus_token, ctx_len=d0.ctx_len,
+                          cost_coef=c.coef)
+        yy = synth.make_target_logits(cfg, 5, d, ot.depth)
+        y.copy_(yy)
+        g.replay()
+        torch.cuda.synchronize()
+        compare_build(tree, ot, cfg.K)
+        compare_verify(verdict, O.verify_tree(yy, cfg.L, ot.n_nodes, ot.token_ids, ot.parent_idx, rows_mode=G.ROWS_LIVE))
+
+
 def test_context_interpolated_cost_and_theta_curve():
     """Table cost blended by context length (Eq. 13) and the theta*(n) curve output, against the oracle."""
     B = 200
