@@ -37,7 +37,7 @@
 extern "C" {
 #endif
 
-#define CADD_ABI_VERSION 2
+#define CADD_ABI_VERSION 3
 
 /* ---- return codes (host side, synchronous) ---- */
 #define CADD_OK              0
@@ -160,6 +160,42 @@ typedef struct cadd_verify_args {
     size_t   workspace_bytes;
 } cadd_verify_args;
 
+/*
+ * Tree verification fused into the target's output projection (Section 3.1: "the target's prediction at every
+ * tree node" is argmax_v of h_j . W_v, with h_j the target's last hidden state at node j and W the output
+ * embedding; Section 3.3 for the walk).  cadd_verify_tree reads materialised logits [batch, R, V]; this entry
+ * point takes the hidden states and the weight instead and never writes the logits: the product is formed tile
+ * by tile on the tensor cores (bf16 inputs, fp32 accumulation) and reduced to one token per row on the fly.
+ * Outputs, tie rule (lowest token id), rows_mode and the walk are those of cadd_verify_tree.  A logit is the
+ * fp32-accumulated dot product; two tokens whose exact dot products differ by less than that accumulation's
+ * rounding error may be ranked either way.
+ * All pointers are DEVICE pointers owned by the caller.
+ */
+typedef struct cadd_head_args {
+    uint32_t struct_size;          /* = sizeof(cadd_head_args) */
+    uint32_t flags;                /* reserved, 0 */
+    int32_t  batch, L, R;
+    int32_t  hidden;               /* hidden size (the contraction length), >= 1 */
+    int32_t  rows_mode;            /* CADD_ROWS_*; in LIVE mode rows j > n_nodes[b] get node_argmax -1 */
+    int32_t  reserved0;
+    int64_t  V;
+    const void* hidden_states;     /* bf16 [batch, R, hidden]; element (b,j,k) at (b*R + j)*stride_row + k; 16-byte aligned */
+    int64_t  stride_row;           /* in elements, >= hidden, multiple of 8 */
+    const void* weight;            /* bf16 [V, hidden]; element (v,k) at v*stride_w + k; 16-byte aligned */
+    int64_t  stride_w;             /* in elements, >= hidden, multiple of 8 */
+    const int32_t* n_nodes;        /* [batch]   from cadd_build_tree */
+    const int32_t* token_ids;      /* [batch,R] from cadd_build_tree */
+    const int32_t* parent_idx;     /* [batch,R] from cadd_build_tree */
+    /* outputs, all required except status */
+    int32_t* node_argmax;          /* [batch,R] */
+    int32_t* accepted_len;         /* [batch] */
+    int32_t* accepted_nodes;       /* [batch,L], -1 padded */
+    int32_t* next_bonus;           /* [batch] */
+    int32_t* status;               /* [batch] CADD_STATUS_* bits, may be NULL */
+    void*    workspace;            /* >= cadd_head_workspace_bytes, 256-byte aligned; needs no initialisation */
+    size_t   workspace_bytes;
+} cadd_head_args;
+
 /* ABI version of the loaded library (CADD_ABI_VERSION it was built with). */
 int cadd_version(void);
 
@@ -176,6 +212,16 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream);
 
 /* Tree verification (Sections 3.1 and 3.3).  Asynchronous on `cuda_stream`. */
 int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream);
+
+/* Scratch size of cadd_verify_tree_fused_head: pure host arithmetic on batch and R. */
+int cadd_head_workspace_bytes(const cadd_head_args* a, size_t* out);
+
+/* Tree verification from hidden states and the output-projection weight (see cadd_head_args).  Asynchronous on
+ * `cuda_stream`: one memset of the workspace and three kernels.  Errors as for cadd_verify_tree; CADD_ERR_ALIGN
+ * if a base pointer is not 16-byte aligned or a stride is not a multiple of 8 elements; CADD_ERR_LAUNCH if the
+ * driver's tensor-map encoder is unavailable.  If an internal bounded wait runs out, every request reports
+ * CADD_STATUS_INTERNAL_TIMEOUT. */
+int cadd_verify_tree_fused_head(const cadd_head_args* a, void* cuda_stream);
 
 /*
  * cadd_build_tree for callers that cannot provide scratch memory.  (The paper has no counterpart to

@@ -416,3 +416,26 @@ int cadd_oracle_verify_tree(
     }
     return 0;
 }
+
+/*
+ * Target logits from the target's last hidden states and its output-projection weight (Section 3.1:
+ * the target's prediction at tree node j is argmax_v of  y_{j,v} = sum_k h_{j,k} W_{v,k}):
+ *   out[r*V + v] = sum_{k < hidden} h[r*stride_row + k] * w[v*stride_w + k]      (ascending k, fp64)
+ * h and w are bf16, widened exactly; a product of two bf16 values is exact in double.
+ */
+int cadd_oracle_head_logits(int64_t rows, int64_t V, int hidden,
+                            const void *h, int64_t stride_row, const void *w, int64_t stride_w,
+                            double *out)
+{
+    if (rows < 1 || V < 1 || hidden < 1) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t v = 0; v < V; ++v) {
+            double acc = 0.0;
+            for (int k = 0; k < hidden; ++k)
+                acc += logit_at(h, ORC_BF16, r * stride_row + k) * logit_at(w, ORC_BF16, v * stride_w + k);
+            out[r * V + v] = acc;
+        }
+    }
+    return 0;
+}

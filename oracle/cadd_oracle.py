@@ -179,3 +179,28 @@ def verify_tree(target_logits: torch.Tensor, L: int, n_nodes, token_ids, parent_
     if rc != 0:
         raise ValueError(f"cadd_oracle_verify_tree rejected its arguments (rc={rc})")
     return out
+
+
+def head_logits(hidden_states: torch.Tensor, weight: torch.Tensor) -> torch.Tensor:
+    """fp64 logits [batch, R, V] = hidden_states [batch, R, hidden] . weight [V, hidden]^T (Section 3.1), both bf16 on CPU."""
+    h, w = hidden_states, weight
+    assert h.device.type == "cpu" and w.device.type == "cpu" and h.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
+    assert h.dim() == 3 and w.dim() == 2 and h.shape[2] == w.shape[1]
+    h, w = h.contiguous(), w.contiguous()
+    batch, R, hidden = h.shape
+    V = w.shape[0]
+    out = torch.empty(batch, R, V, dtype=torch.float64)
+    rc = lib().cadd_oracle_head_logits(C.c_int64(batch * R), C.c_int64(V), hidden, _p(h), C.c_int64(hidden), _p(w),
+                                       C.c_int64(hidden), _p(out))
+    if rc != 0:
+        raise ValueError(f"cadd_oracle_head_logits rejected its arguments (rc={rc})")
+    return out
+
+
+def verify_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor, L: int, n_nodes, token_ids, parent_idx,
+                           rows_mode: int = ROWS_LIVE):
+    """O5+O6 on logits formed from hidden states and the output projection.  The decision is taken in the
+    precision the GPU path reports its logits in (fp32): the exact fp64 dot products are rounded once to fp32,
+    then the plain argmax (lowest id among equals) and the walk follow.  Returns (OracleVerify, fp64 logits)."""
+    y64 = head_logits(hidden_states, weight)
+    return verify_tree(y64.to(torch.float32), L, n_nodes, token_ids, parent_idx, rows_mode), y64

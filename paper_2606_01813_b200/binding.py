@@ -26,7 +26,8 @@ FLAG_EMIT_DENSE_MASK, FLAG_EMIT_TOPK, FLAG_FIXED_BUDGET = 1, 2, 4
 ROWS_LIVE, ROWS_DENSE = 0, 1
 
 EXPORTS = ("cadd_version", "cadd_status_string", "cadd_build_workspace_bytes", "cadd_verify_workspace_bytes",
-           "cadd_build_tree", "cadd_verify_tree", "cadd_build_tree_static_scratch")
+           "cadd_build_tree", "cadd_verify_tree", "cadd_build_tree_static_scratch",
+           "cadd_head_workspace_bytes", "cadd_verify_tree_fused_head")
 ERR_STATIC_SCRATCH = -8
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -63,6 +64,20 @@ class VerifyArgs(C.Structure):
     ]
 
 
+class HeadArgs(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("flags", C.c_uint32),
+        ("batch", C.c_int32), ("L", C.c_int32), ("R", C.c_int32), ("hidden", C.c_int32),
+        ("rows_mode", C.c_int32), ("reserved0", C.c_int32), ("V", C.c_int64),
+        ("hidden_states", C.c_void_p), ("stride_row", C.c_int64),
+        ("weight", C.c_void_p), ("stride_w", C.c_int64),
+        ("n_nodes", C.c_void_p), ("token_ids", C.c_void_p), ("parent_idx", C.c_void_p),
+        ("node_argmax", C.c_void_p), ("accepted_len", C.c_void_p), ("accepted_nodes", C.c_void_p),
+        ("next_bonus", C.c_void_p), ("status", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+    ]
+
+
 _lib = None
 
 
@@ -81,6 +96,8 @@ def lib() -> C.CDLL:
         l.cadd_verify_workspace_bytes.argtypes = [C.POINTER(VerifyArgs), C.POINTER(C.c_size_t)]
         l.cadd_build_tree.argtypes = [C.POINTER(BuildArgs), C.c_void_p]
         l.cadd_verify_tree.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
+        l.cadd_head_workspace_bytes.argtypes = [C.POINTER(HeadArgs), C.POINTER(C.c_size_t)]
+        l.cadd_verify_tree_fused_head.argtypes = [C.POINTER(HeadArgs), C.c_void_p]
         l.cadd_build_tree_static_scratch.argtypes = [C.POINTER(BuildArgs), C.c_void_p]
         _lib = l
     return _lib
@@ -269,6 +286,63 @@ def cadd_verify_tree(target_logits: torch.Tensor, L: int, n_nodes: torch.Tensor,
         rc = lib().cadd_verify_tree(C.byref(a), _stream_ptr(stream))
     if rc != OK:
         raise CaddError(rc)
+    return out
+
+
+def cadd_head_workspace_bytes(batch: int, R: int, hidden: int, V: int, L: int = 1) -> int:
+    a = HeadArgs()
+    a.struct_size = C.sizeof(HeadArgs)
+    a.batch, a.L, a.R, a.hidden, a.V = batch, L, R, hidden, V
+    n = C.c_size_t(0)
+    rc = lib().cadd_head_workspace_bytes(C.byref(a), C.byref(n))
+    if rc != OK:
+        raise CaddError(rc)
+    return int(n.value)
+
+
+def cadd_verify_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor, L: int, n_nodes: torch.Tensor,
+                                token_ids: torch.Tensor, parent_idx: torch.Tensor, rows_mode: int = ROWS_LIVE, *,
+                                out: Optional[Verdict] = None, workspace: Optional[torch.Tensor] = None,
+                                stream: Optional[torch.cuda.Stream] = None) -> Verdict:
+    """Greedy tree verification from the target's last hidden states [batch, R, hidden] and its output-projection
+    weight [V, hidden] (both bf16): the logits h . W^T are formed on the tensor cores and reduced to the per-node
+    argmax without being written to memory (Section 3.1), then the accepted path is walked (Section 3.3)."""
+    h, w = hidden_states, weight
+    if not (h.is_cuda and w.is_cuda):
+        raise ValueError("hidden_states and weight must be CUDA tensors (there is no CPU path)")
+    if h.dtype != torch.bfloat16 or w.dtype != torch.bfloat16:
+        raise ValueError("hidden_states and weight must be bfloat16")
+    if h.dim() != 3 or h.stride(2) != 1 or h.stride(0) != h.shape[1] * h.stride(1):
+        raise ValueError("hidden_states must be [batch, R, hidden] with contiguous rows of equal stride")
+    if w.dim() != 2 or w.stride(1) != 1 or w.shape[1] != h.shape[2]:
+        raise ValueError("weight must be [V, hidden] with a contiguous hidden axis")
+    dev = h.device
+    batch, R, hidden = h.shape
+    V = w.shape[0]
+    for t in (n_nodes, token_ids, parent_idx):
+        if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()):
+            raise ValueError("tree arrays must be contiguous int32 CUDA tensors")
+    a = HeadArgs()
+    a.struct_size = C.sizeof(HeadArgs)
+    a.batch, a.L, a.R, a.hidden, a.V = batch, L, R, hidden, V
+    a.rows_mode = rows_mode
+    a.hidden_states, a.stride_row = h.data_ptr(), h.stride(1)
+    a.weight, a.stride_w = w.data_ptr(), w.stride(0)
+    a.n_nodes, a.token_ids, a.parent_idx = n_nodes.data_ptr(), token_ids.data_ptr(), parent_idx.data_ptr()
+    if out is None:
+        i32 = lambda *s: torch.empty(*s, dtype=torch.int32, device=dev)
+        out = Verdict(node_argmax=i32(batch, R), accepted_len=i32(batch), accepted_nodes=i32(batch, L),
+                      next_bonus=i32(batch), status=i32(batch))
+    a.node_argmax, a.accepted_len, a.accepted_nodes = _ptr(out.node_argmax), _ptr(out.accepted_len), _ptr(out.accepted_nodes)
+    a.next_bonus, a.status = _ptr(out.next_bonus), _ptr(out.status)
+    if workspace is None:
+        workspace = torch.empty(cadd_head_workspace_bytes(batch, R, hidden, V, L), dtype=torch.uint8, device=dev)
+    a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    with torch.cuda.device(dev):
+        rc = lib().cadd_verify_tree_fused_head(C.byref(a), _stream_ptr(stream))
+    if rc != OK:
+        raise CaddError(rc)
+    workspace.record_stream(torch.cuda.current_stream() if stream is None else stream)
     return out
 
 

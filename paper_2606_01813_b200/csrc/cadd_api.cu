@@ -8,6 +8,7 @@
 #include "expand_emit.cuh"
 #include "softmax_topk.cuh"
 #include "verify.cuh"
+#include "head_argmax.cuh"
 
 namespace cadd {
 
@@ -224,6 +225,108 @@ int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream) {
     }
     if (a->logits_dtype == CADD_DTYPE_BF16) row_argmax_kernel<CADD_DTYPE_BF16><<<rows, kThreads, argmax_smem_bytes(), st>>>(ap);
     else row_argmax_kernel<CADD_DTYPE_FP32><<<rows, kThreads, argmax_smem_bytes(), st>>>(ap);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+
+    WalkParams wp;
+    wp.batch = a->batch; wp.L = a->L; wp.R = a->R; wp.n_nodes = a->n_nodes; wp.token_ids = a->token_ids;
+    wp.parent_idx = a->parent_idx; wp.node_argmax = a->node_argmax; wp.accepted_len = a->accepted_len;
+    wp.accepted_nodes = a->accepted_nodes; wp.next_bonus = a->next_bonus; wp.status = a->status;
+    const int wpb = 4;
+    accept_walk_kernel<<<(a->batch + wpb - 1) / wpb, wpb * 32, 0, st>>>(wp);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    return CADD_OK;
+}
+
+// ---------------- verification fused into the output projection ----------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+// The driver's tensor-map encoder, looked up through the runtime (the library does not link the driver directly).
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            return (EncodeTiledFn) nullptr;
+        }
+        return (EncodeTiledFn)f;
+    }();
+    return fn;
+}
+// 2-D map of a row-major bf16 matrix [rows, cols] (row stride in elements); boxes of box_rows x 64 columns, 128-byte
+// swizzle, out-of-range elements read as zero (ragged rows, columns and hidden sizes need no special casing).
+static bool make_map_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t stride, int box_rows) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)stride * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kHeadBK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int check_head_shape(const cadd_head_args* a) {
+    if (!a) return CADD_ERR_NULL;
+    if (a->struct_size != sizeof(cadd_head_args)) return CADD_ERR_STRUCT_SIZE;
+    if (a->batch < 1 || a->L < 1 || a->L > 64 || a->R < 1 || a->V < 1 || a->V >= ((int64_t)1 << 31) || a->hidden < 1 ||
+        a->hidden > (1 << 20) || (int64_t)a->batch * a->R >= ((int64_t)1 << 31))
+        return CADD_ERR_SHAPE;
+    if (a->rows_mode != CADD_ROWS_LIVE && a->rows_mode != CADD_ROWS_DENSE) return CADD_ERR_DTYPE;
+    return CADD_OK;
+}
+
+int cadd_head_workspace_bytes(const cadd_head_args* a, size_t* out) {
+    int rc = check_head_shape(a);
+    if (rc != CADD_OK) return rc;
+    if (!out) return CADD_ERR_NULL;
+    *out = (((size_t)a->batch * a->R * 8 + 255) & ~(size_t)255) + 256;    // packed row maxima + the error word
+    return CADD_OK;
+}
+
+int cadd_verify_tree_fused_head(const cadd_head_args* a, void* cuda_stream) {
+    int rc = check_head_shape(a);
+    if (rc != CADD_OK) return rc;
+    if (!a->hidden_states || !a->weight || !a->n_nodes || !a->token_ids || !a->parent_idx || !a->node_argmax || !a->accepted_len ||
+        !a->accepted_nodes || !a->next_bonus)
+        return CADD_ERR_NULL;
+    // the tiled bulk copies need 16-byte aligned bases and row strides
+    if (!aligned(a->hidden_states, 16) || !aligned(a->weight, 16) || a->stride_row % 8 != 0 || a->stride_w % 8 != 0) return CADD_ERR_ALIGN;
+    if (!aligned(a->n_nodes, 4) || !aligned(a->token_ids, 4) || !aligned(a->parent_idx, 4) || !aligned(a->node_argmax, 4) ||
+        !aligned(a->accepted_len, 4) || !aligned(a->accepted_nodes, 4) || !aligned(a->next_bonus, 4) || !aligned(a->status, 4))
+        return CADD_ERR_ALIGN;
+    if (a->stride_row < a->hidden || a->stride_w < a->hidden) return CADD_ERR_SHAPE;
+    size_t need = 0;
+    cadd_head_workspace_bytes(a, &need);
+    if (!a->workspace || !aligned(a->workspace, 256) || a->workspace_bytes < need) return CADD_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    const int64_t M = (int64_t)a->batch * a->R;
+    CUtensorMap map_h, map_w;
+    if (!make_map_bf16(&map_h, a->hidden_states, M, a->hidden, a->stride_row, kHeadBM) ||
+        !make_map_bf16(&map_w, a->weight, a->V, a->hidden, a->stride_w, kHeadBN))
+        return CADD_ERR_LAUNCH;
+
+    HeadParams hp;
+    hp.M = M; hp.V = a->V; hp.Kdim = a->hidden;
+    hp.m_tiles = (int)((M + kHeadBM - 1) / kHeadBM);
+    hp.n_tiles = (int)((a->V + kHeadBN - 1) / kHeadBN);
+    hp.R = a->R; hp.rows_mode = a->rows_mode; hp.n_nodes = a->n_nodes;
+    hp.row_best = (unsigned long long*)a->workspace;
+    hp.error = (int32_t*)((unsigned char*)a->workspace + (need - 256));
+    if (cudaMemsetAsync(a->workspace, 0, need, st) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+    if (cudaFuncSetAttribute(head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem_bytes()) != cudaSuccess) {
+        cudaGetLastError();
+        return CADD_ERR_LAUNCH;
+    }
+    const int64_t work = (int64_t)hp.m_tiles * hp.n_tiles;
+    const int sms = sm_count();
+    const unsigned grid = (unsigned)(work < sms ? work : sms);
+    head_argmax_kernel<<<grid, kHeadThreads, head_smem_bytes(), st>>>(map_h, map_w, hp);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    head_decode_kernel<<<(unsigned)((M + 255) / 256), 256, 0, st>>>(hp.row_best, a->n_nodes, hp.error, M, a->R, a->rows_mode, a->node_argmax);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
 
     WalkParams wp;

@@ -1,0 +1,257 @@
+// Verification argmax fused into the output projection (the step right before the path: Section 3.1 takes the
+// target's prediction at every tree node, i.e. argmax over v of  h_j . W_v  with h the target's last hidden state at
+// node j and W the output embedding).  The logits [rows, V] are never written to memory: a bf16 x bf16 -> fp32 GEMM
+// on the 5th-generation tensor cores keeps each 128 x 256 tile of logits in tensor memory, and the epilogue reduces it
+// to one (value, token) pair per row, merged across tiles by a 64-bit atomic max.
+//
+// One CTA per SM, 192 threads, three roles:
+//   warp 0      producer: 2-D tiled bulk tensor copies (TMA, 128-byte swizzle, no multicast) of a 128 x 64 tile of
+//               hidden states and a 256 x 64 tile of W into a 4-stage shared-memory ring, completion on mbarriers;
+//   warp 1      one elected thread issues tcgen05.mma (M 128, N 256, K 16 per instruction, operands described by
+//               shared-memory matrix descriptors, accumulator in tensor memory), tcgen05.commit frees the stage and,
+//               after the last k-step, hands the accumulator to the epilogue; the warp also owns the tensor-memory
+//               allocation (all 512 columns = two accumulators, so the epilogue of one tile overlaps the next);
+//   warps 2-5   epilogue: each thread owns one row of the tile (one tensor-memory lane), reads it 32 columns at a time
+//               with tcgen05.ld and keeps the running maximum and its first column.
+// Tiles are walked in the order (column tile outer, row tile inner), CTA c taking tiles c, c + grid, ...: at any time
+// the CTAs work on neighbouring column tiles of W, which then come from L2 after their first use, and the hidden
+// states (tens of MB) stay L2-resident.
+//
+// Every wait on an mbarrier has an iteration limit; a role that gives up sets an error word, all roles then leave
+// their loops, the CTA meets at a barrier and the tensor memory is released before it exits.
+#pragma once
+#include <cuda.h>
+#include "common.cuh"
+#include "tile_ring.cuh"
+
+namespace cadd {
+
+constexpr int kHeadBM = 128;              // rows per tile (tensor-memory lanes)
+constexpr int kHeadBN = 256;              // columns (tokens) per tile
+constexpr int kHeadBK = 64;               // bf16 elements per k-step: one 128-byte swizzle row
+constexpr int kHeadStages = 4;
+constexpr int kHeadThreads = 192;
+constexpr int kHeadTmemCols = 512;        // two fp32 accumulators of kHeadBN columns
+constexpr uint32_t kHeadABytes = kHeadBM * kHeadBK * 2;   // 16 KB
+constexpr uint32_t kHeadBBytes = kHeadBN * kHeadBK * 2;   // 32 KB
+
+struct HeadShared {
+    alignas(1024) unsigned char a[kHeadStages][kHeadABytes];
+    alignas(1024) unsigned char b[kHeadStages][kHeadBBytes];
+    alignas(8) uint64_t full[kHeadStages];     // tile pair landed (producer -> MMA)
+    uint64_t empty[kHeadStages];               // MMAs that read the stage are done (MMA -> producer)
+    uint64_t acc_full[2];                      // accumulator complete (MMA -> epilogue)
+    uint64_t acc_empty[2];                     // accumulator read out (epilogue -> MMA)
+    uint32_t tmem_base;
+    uint32_t error;
+};
+inline size_t head_smem_bytes() { return sizeof(HeadShared) + 1024; }
+
+struct HeadParams {
+    int64_t M;                 // rows = batch * R
+    int64_t V;                 // tokens
+    int Kdim;                  // hidden size
+    int m_tiles, n_tiles;
+    int R, rows_mode;
+    const int32_t* n_nodes;    // [batch] (LIVE mode: row tiles without a live row are skipped)
+    unsigned long long* row_best;   // [M] packed (ordered logit << 32 | ~token), zeroed before the launch
+    int32_t* error;            // device word, set non-zero when a bounded wait ran out
+};
+
+// Bounded wait without a sleep between tries: the roles of this kernel are single threads or warps that own their
+// issue slots (one CTA per SM), and a late wake-up of the MMA thread would leave the tensor cores idle.
+constexpr int kHeadSpinLimit = 1 << 20;
+__device__ __forceinline__ bool head_wait(uint64_t* bar, unsigned parity) {
+    for (int it = 0; it < kHeadSpinLimit; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// ---- tcgen05 / TMA wrappers ----
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {      // whole warp
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {         // whole warp
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; one thread issues.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier gets one arrival when all tcgen05.mma issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {         // whole warp: 32 lanes x 32 columns
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements) under the 128-byte
+// swizzle, rows packed densely: 8-row groups are 1024 bytes apart (stride byte offset), the leading byte offset is
+// unused for swizzled K-major operands (1), descriptor version 1 (sm_100), layout type 2 = 128-byte swizzle.
+// A k-step of 16 elements inside the 128-byte row advances the start address by 32 bytes.
+__device__ __forceinline__ uint64_t umma_desc_k_sw128(const void* tile, int k16) {
+    const uint32_t addr = smem_u32(tile) + (uint32_t)k16 * 32u;
+    return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)1 << 16) | ((uint64_t)(1024u >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+// Instruction descriptor: fp32 accumulator (bits 4-5 = 1), A and B bf16 (bits 7-9 and 10-12 = 1), both K-major
+// (bits 15, 16 = 0), N / 8 in bits 17-22, M / 16 in bits 24-28.
+constexpr uint32_t kHeadIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kHeadBN >> 3) << 17) | ((uint32_t)(kHeadBM >> 4) << 24);
+
+// True if row tile mt holds a row that is read: always in DENSE mode; in LIVE mode rows j <= n_nodes[b] of a request.
+__device__ __forceinline__ bool head_tile_live(const HeadParams& p, int mt) {
+    if (p.rows_mode != CADD_ROWS_LIVE) return true;
+    const int64_t r0 = (int64_t)mt * kHeadBM;
+    const int64_t r1 = min(r0 + kHeadBM, p.M) - 1;
+    for (int64_t b = r0 / p.R; b <= r1 / p.R; ++b) {
+        int n = p.n_nodes[b];
+        n = n < 0 ? 0 : (n > p.R - 1 ? p.R - 1 : n);
+        const int64_t lo = max(r0, b * p.R), hi = min(r1, b * p.R + n);   // live rows of request b inside the tile
+        if (lo <= hi) return true;
+    }
+    return false;
+}
+
+__global__ void __launch_bounds__(kHeadThreads, 1)
+head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, HeadParams p) {
+    extern __shared__ __align__(16) unsigned char head_smem_raw[];
+    HeadShared& sh = *reinterpret_cast<HeadShared*>(head_smem_raw + ((1024u - (smem_u32(head_smem_raw) & 1023u)) & 1023u));
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int k_steps = (p.Kdim + kHeadBK - 1) / kHeadBK;
+    const int64_t n_work = (int64_t)p.m_tiles * p.n_tiles;
+
+    if (tid == 0) {
+        for (int s = 0; s < kHeadStages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sh.acc_full[s], 1); mbar_init(&sh.acc_empty[s], 4); }
+        sh.error = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(&sh.tmem_base, kHeadTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *(volatile uint32_t*)&sh.tmem_base;
+
+    if (warp == 0) {
+        // ---------------- producer ----------------
+        if (lane == 0) {
+            unsigned s = 0, ph = 0;
+            for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
+                const int nt = (int)(w / p.m_tiles), mt = (int)(w - (int64_t)nt * p.m_tiles);
+                if (!head_tile_live(p, mt)) continue;
+                for (int k = 0; k < k_steps; ++k) {
+                    if (!head_wait(&sh.empty[s], ph ^ 1u)) { sh.error = 1; break; }   // first pass: free at once
+                    mbar_arrive_expect_tx(&sh.full[s], kHeadABytes + kHeadBBytes);
+                    tma_load_2d(&sh.a[s][0], &map_h, k * kHeadBK, mt * kHeadBM, &sh.full[s]);
+                    tma_load_2d(&sh.b[s][0], &map_w, k * kHeadBK, nt * kHeadBN, &sh.full[s]);
+                    if (++s == kHeadStages) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            unsigned s = 0, ph = 0, buf = 0, aph = 0;
+            for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
+                const int nt = (int)(w / p.m_tiles), mt = (int)(w - (int64_t)nt * p.m_tiles);
+                if (!head_tile_live(p, mt)) continue;
+                if (!head_wait(&sh.acc_empty[buf], aph ^ 1u)) { sh.error = 2; break; }   // epilogue has drained it
+                tc_fence_after();
+                const uint32_t d = tmem_base + buf * kHeadBN;
+                bool ok = true;
+                for (int k = 0; k < k_steps; ++k) {
+                    if (!head_wait(&sh.full[s], ph)) { sh.error = 3; ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < kHeadBK / 16; ++kk)
+                        umma_bf16(d, umma_desc_k_sw128(&sh.a[s][0], kk), umma_desc_k_sw128(&sh.b[s][0], kk), kHeadIdesc,
+                                  (k | kk) != 0 ? 1u : 0u);
+                    umma_commit(&sh.empty[s]);                       // the stage is free once these MMAs have read it
+                    if (++s == kHeadStages) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(&sh.acc_full[buf]);                       // accumulator complete
+                if (++buf == 2) { buf = 0; aph ^= 1u; }
+            }
+        }
+    } else {
+        // ---------------- epilogue: warps 2..5, tensor-memory lane quarter = warp % 4 ----------------
+        const int quarter = warp & 3;
+        unsigned buf = 0, aph = 0;
+        for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
+            const int nt = (int)(w / p.m_tiles), mt = (int)(w - (int64_t)nt * p.m_tiles);
+            if (!head_tile_live(p, mt)) continue;
+            if (!__all_sync(kFullMask, head_wait(&sh.acc_full[buf], aph))) { sh.error = 4; break; }
+            tc_fence_after();
+            const int64_t row = (int64_t)mt * kHeadBM + quarter * 32 + lane;
+            const int64_t col0 = (int64_t)nt * kHeadBN;
+            float best = -INFINITY;
+            int64_t best_col = -1;
+#pragma unroll 1
+            for (int c = 0; c < kHeadBN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kHeadBN + c * 32, r);
+                tmem_ld_wait();
+                const int64_t cb = col0 + c * 32;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float v = __uint_as_float(r[i]);
+                    if (v > best && cb + i < p.V) { best = v; best_col = cb + i; }     // strict: the first column wins ties
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.acc_empty[buf]);
+            if (row < p.M && best_col >= 0)
+                atomicMax(&p.row_best[row], (unsigned long long)make_key(best, (uint32_t)best_col));
+            if (++buf == 2) { buf = 0; aph ^= 1u; }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kHeadTmemCols);
+    }
+    if (tid == 0 && sh.error) atomicExch(p.error, (int32_t)sh.error);
+}
+
+// Turns the packed per-row maxima into token ids.  Rows not read in LIVE mode get -1; a row whose logits were all
+// -Inf or NaN gets 0, like the plain argmax kernel; -2 marks every row when the GEMM gave up on a wait.
+__global__ void head_decode_kernel(const unsigned long long* row_best, const int32_t* n_nodes, const int32_t* error, int64_t M, int R,
+                                   int rows_mode, int32_t* node_argmax) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= M) return;
+    const int64_t b = r / R;
+    const int j = (int)(r - b * R);
+    int32_t ans;
+    if (rows_mode == CADD_ROWS_LIVE) {
+        int n = n_nodes[b];
+        n = n < 0 ? 0 : (n > R - 1 ? R - 1 : n);
+        if (j > n) { node_argmax[r] = -1; return; }
+    }
+    const unsigned long long k = row_best[r];
+    ans = k ? (int32_t)key_id((uint64_t)k) : 0;
+    if (*error) ans = -2;
+    node_argmax[r] = ans;
+}
+
+}  // namespace cadd

@@ -1,0 +1,111 @@
+"""GPU parity of the verification fused into the output projection (tensor-core path) against the CPU oracle."""
+import pytest
+import torch
+
+from oracle import cadd_oracle as O
+from paper_2606_01813_b200 import binding as G
+from paper_2606_01813_b200 import synth
+from parity_util import to_cpu
+
+pytestmark = pytest.mark.gpu
+
+
+def planted_head_inputs(tree: O.OracleTree, L: int, hidden: int, V: int, seed: int, agreement: float = 0.6):
+    """Hidden states and weight such that the target's argmax at a node is, with probability `agreement`, the token
+    of one of its children (so that walks of several steps occur), else some other token."""
+    g = torch.Generator().manual_seed(seed)
+    batch, R = tree.token_ids.shape
+    w = torch.randn(V, hidden, generator=g)
+    h = 0.3 * torch.randn(batch, R, hidden, generator=g)
+    for b in range(batch):
+        n = int(tree.n_nodes[b])
+        for j in range(R):
+            kids = [c for c in range(1, n + 1) if int(tree.parent_idx[b, c]) == j] if j <= n else []
+            if kids and (j == 0 or torch.rand((), generator=g) < agreement):     # the root always agrees
+                t = int(tree.token_ids[b, kids[int(torch.randint(len(kids), (), generator=g))]])
+            else:
+                t = int(torch.randint(V, (), generator=g))
+            h[b, j] += 4.0 * w[t] / w[t].norm()
+    return h.bfloat16(), w.bfloat16()
+
+
+def check_head(h, w, tree, L, rows_mode):
+    ov, y64 = O.verify_tree_fused_head(h, w, L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode=rows_mode)
+    dev = lambda t: t.cuda()
+    gv = G.cadd_verify_tree_fused_head(h.cuda(), w.cuda(), L, dev(tree.n_nodes), dev(tree.token_ids), dev(tree.parent_idx), rows_mode)
+    torch.cuda.synchronize()
+    ga, oa = to_cpu(gv.node_argmax), ov.node_argmax
+    assert int(to_cpu(gv.status).max()) & G.STATUS_INTERNAL_TIMEOUT == 0
+    # fp32 accumulation of `hidden` products in an order the hardware chooses: |error| <= hidden * 2^-24 * sum |terms|
+    # in the worst case; a differing pick is admissible only inside that bound (and then nothing downstream is compared)
+    absdot = h.double().abs().reshape(-1, h.shape[2]) @ w.double().abs().T
+    batch, R, V = y64.shape
+    exempt = 0
+    for b in range(batch):
+        for j in range(R):
+            if ga[b, j] == oa[b, j]:
+                continue
+            assert ga[b, j] >= 0 and oa[b, j] >= 0, (b, j, int(ga[b, j]), int(oa[b, j]))
+            tol = h.shape[2] * 2.0 ** -24 * float(absdot[b * R + j, [int(ga[b, j]), int(oa[b, j])]].max())
+            gap = float(y64[b, j, int(oa[b, j])] - y64[b, j, int(ga[b, j])])
+            assert abs(gap) <= tol, (b, j, int(ga[b, j]), int(oa[b, j]), gap, tol)
+            exempt += 1
+    if exempt == 0:
+        assert torch.equal(to_cpu(gv.accepted_len), ov.accepted_len)
+        assert torch.equal(to_cpu(gv.accepted_nodes), ov.accepted_nodes)
+        assert torch.equal(to_cpu(gv.next_bonus), ov.next_bonus)
+    return exempt, ov
+
+
+@pytest.mark.parametrize("shape", [
+    # batch, hidden, V      (R comes from the tree; ragged row tiles, column tiles and k-steps on purpose)
+    (1, 64, 300),
+    (2, 256, 4099),
+    (3, 200, 1000),
+    (2, 1032, 2500),
+])
+@pytest.mark.parametrize("rows_mode", [G.ROWS_LIVE, G.ROWS_DENSE])
+def test_fused_head_small(shape, rows_mode):
+    batch, hidden, V = shape
+    cfg = synth.scaled(synth.CONFIGS["c2"], batch=batch, V=max(V, 64))
+    d = synth.make_draft_inputs(cfg, 11)
+    c = synth.make_cost_inputs(cfg, 11)
+    tree = O.build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, l_eff=d.l_eff, bonus_token=d.bonus_token, ctx_len=d.ctx_len,
+                        cost_coef=c.coef, flags=O.FLAG_FIXED_BUDGET)        # fixed budget: trees with many nodes
+    h, w = planted_head_inputs(tree, cfg.L, hidden, V, seed=5)
+    exempt, ov = check_head(h, w, tree, cfg.L, rows_mode)
+    assert exempt <= 2
+    assert int(ov.accepted_len.max()) >= 1                                  # the walk has something to follow
+
+
+def test_fused_head_matches_materialised_logits():
+    """Same answer as forming the logits with a library GEMM and calling cadd_verify_tree on them (up to the two
+    GEMMs' own rounding: rows whose top two logits are closer than that are skipped)."""
+    cfg = synth.scaled(synth.CONFIGS["c2"], batch=2, V=5000)
+    d = synth.make_draft_inputs(cfg, 12)
+    c = synth.make_cost_inputs(cfg, 12)
+    tree = O.build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, l_eff=d.l_eff, bonus_token=d.bonus_token, ctx_len=d.ctx_len,
+                        cost_coef=c.coef, flags=O.FLAG_FIXED_BUDGET)
+    h, w = planted_head_inputs(tree, cfg.L, 512, 5000, seed=6)
+    hc, wc = h.cuda(), w.cuda()
+    dev = lambda t: t.cuda()
+    y = (hc.float() @ wc.float().T)
+    top2 = y.topk(2, dim=-1).values
+    clear = (top2[..., 0] - top2[..., 1]) > 1e-3
+    g1 = G.cadd_verify_tree_fused_head(hc, wc, cfg.L, dev(tree.n_nodes), dev(tree.token_ids), dev(tree.parent_idx), G.ROWS_DENSE)
+    g2 = G.cadd_verify_tree(y.contiguous(), cfg.L, dev(tree.n_nodes), dev(tree.token_ids), dev(tree.parent_idx), G.ROWS_DENSE)
+    torch.cuda.synchronize()
+    assert clear.float().mean() > 0.9
+    assert torch.equal(g1.node_argmax[clear], g2.node_argmax[clear])
+
+
+def test_fused_head_rejects_bad_arguments():
+    h = torch.zeros(1, 3, 64, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(10, 64, dtype=torch.bfloat16, device="cuda")
+    z = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t = torch.zeros(1, 3, dtype=torch.int32, device="cuda")
+    with pytest.raises(ValueError):
+        G.cadd_verify_tree_fused_head(h.float(), w, 4, z, t, t)
+    with pytest.raises(G.CaddError):                                       # stride not a multiple of 8 elements
+        G.cadd_verify_tree_fused_head(torch.zeros(1, 3, 68, dtype=torch.bfloat16, device="cuda")[:, :, :60],
+                                      torch.zeros(10, 60, dtype=torch.bfloat16, device="cuda"), 4, z, t, t)

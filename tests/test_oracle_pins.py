@@ -495,3 +495,50 @@ def test_context_interpolated_cost():
     sweep = O.build_tree(same, 4, B, ctx_len=torch.tensor([0, 700, 1500, 2600, 4000, 5500, 6100, 7900, 9000], dtype=torch.int32),
                          cost_kind=O.COST_TABLE_INTERP, cost_table=tables, ctx_grid=grid, t_draft=torch.full((9,), 0.3, dtype=torch.float64))
     assert np.all(np.diff(sweep.n_nodes.numpy()) <= 0) and np.all(np.diff(sweep.theta.numpy()) < 0)
+
+
+# ---- logits from hidden states and the output projection (Section 3.1) ----
+
+def test_head_logits_against_library_matmul_and_loops():
+    g = torch.Generator().manual_seed(3)
+    h = torch.randn(2, 3, 24, generator=g).bfloat16()
+    w = torch.randn(7, 24, generator=g).bfloat16()
+    y = O.head_logits(h, w)
+    ref = torch.einsum("brk,vk->brv", h.double(), w.double())              # library contraction
+    assert torch.allclose(y, ref, rtol=1e-14, atol=1e-14)
+    for (b, r, v) in [(0, 0, 0), (1, 2, 6), (0, 1, 3)]:                      # plain loops
+        acc = 0.0
+        for k in range(24):
+            acc += float(h[b, r, k]) * float(w[v, k])
+        assert abs(float(y[b, r, v]) - acc) < 1e-12
+
+
+def test_head_logits_closed_forms():
+    hidden, V = 16, 5
+    w = (torch.arange(V * hidden, dtype=torch.float32).reshape(V, hidden) % 7 - 3).bfloat16()
+    h = torch.zeros(1, hidden, hidden)
+    h[0] = torch.eye(hidden)                                                # row j selects column j of W
+    y = O.head_logits(h.bfloat16(), w)
+    assert torch.equal(y[0], w.double().T)
+    # a transposed operand or a wrong stride would fail here: W rows are not symmetric
+    h2 = torch.ones(1, 1, hidden).bfloat16()
+    assert torch.equal(O.head_logits(h2, w)[0, 0], w.double().sum(dim=1))
+
+
+def test_fused_head_verdict_on_a_hand_made_tree():
+    # root (token 9) with children tokens 1 and 2; node 1 has child token 3.  W = identity rows scaled, so the
+    # argmax at a node is the index of the largest coordinate of its hidden state.
+    V = hidden = 8
+    w = torch.eye(V).bfloat16()
+    n_nodes = torch.tensor([3], dtype=torch.int32)
+    token_ids = torch.tensor([[9, 1, 2, 3, -1]], dtype=torch.int32)
+    parent_idx = torch.tensor([[-1, 0, 0, 1, -1]], dtype=torch.int32)
+    h = torch.zeros(1, 5, hidden)
+    h[0, 0, 1] = 2.0      # root predicts token 1 -> accept node 1
+    h[0, 1, 3] = 1.0      # node 1 predicts token 3 -> accept node 3
+    h[0, 3, 5] = 1.0      # node 3 predicts token 5 -> no such child: stop, bonus 5
+    h[0, 2, 2] = 1.0
+    h[0, 1, 6] = 1.0      # tie at node 1 between tokens 3 and 6: the lower id wins
+    ov, y64 = O.verify_tree_fused_head(h.bfloat16(), w, 4, n_nodes, token_ids, parent_idx, rows_mode=O.ROWS_LIVE)
+    assert ov.node_argmax[0].tolist() == [1, 3, 2, 5, -1]
+    assert int(ov.accepted_len[0]) == 2 and ov.accepted_nodes[0].tolist() == [1, 3, -1, -1] and int(ov.next_bonus[0]) == 5
