@@ -248,6 +248,14 @@ def run_ours(args, rank, world):
         except Exception as ex:  # capture is an extra measurement: report why it is missing, keep the main line
             graph = {"error": str(ex)[:200]}
 
+    # ---- verification fused into the output projection (tensor-core path), next to library GEMM + argmax ----
+    fused_head = None
+    if args.head_hidden > 0:
+        try:
+            fused_head = head_block(G, cfg, tree, verdict, y, rows_mode, args.head_hidden, dev, min(K, 10))
+        except Exception as ex:
+            fused_head = {"error": str(ex)[:200]}
+
     # ---- the oracle timed on this machine's host cores, on a bounded sample (rank 0, N = 1 only) ----
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -263,11 +271,57 @@ def run_ours(args, rank, world):
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": f"replicas x{world}",
                        "n_star_mean": round(float(n_star.float().mean()), 2), "n_star_max": int(n_star.max()),
                        "accepted_mean": round(float(verdict.accepted_len.float().mean().item()), 2)},
-            "roofline": roofline, "build": build_info, "cuda_graph": graph, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "e2e": e2e, "cpu_baseline": cpu_baseline,
             "gpu_launches": KERNELS_PER_STEP * K, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
     replicas.shutdown()
+
+
+def measured_peak_tflops():
+    try:
+        with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured (burst)"
+    except Exception:
+        return 1590.0, "fallback"
+
+
+def head_block(G, cfg, tree, verdict, y, rows_mode, hidden, dev, iters):
+    """cadd_verify_tree_fused_head on synthetic hidden states / weight of the workload's shape, timed alone with CUDA
+    events, beside the same work done as a library GEMM that writes the logits plus cadd_verify_tree."""
+    g = torch.Generator(device=dev).manual_seed(1234)
+    M = cfg.batch * cfg.R
+    h = torch.randn(cfg.batch, cfg.R, hidden, device=dev, dtype=torch.bfloat16, generator=g)
+    w = torch.randn(cfg.V, hidden, device=dev, dtype=torch.bfloat16, generator=g)
+    ws = torch.empty(G.cadd_head_workspace_bytes(cfg.batch, cfg.R, hidden, cfg.V, cfg.L), dtype=torch.uint8, device=dev)
+    out = G.cadd_verify_tree_fused_head(h, w, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, workspace=ws)
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    t_fused = timed(lambda: G.cadd_verify_tree_fused_head(h, w, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode,
+                                                          workspace=ws, out=out))
+    y2 = torch.empty(cfg.batch, cfg.R, cfg.V, device=dev, dtype=torch.bfloat16)   # own buffer: the step's logits stay intact
+    t_gemm = timed(lambda: torch.matmul(h.view(M, hidden), w.T, out=y2.view(M, cfg.V)))   # library GEMM, logits written in bf16
+    v2 = G.cadd_verify_tree(y2, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode)
+    t_arg = timed(lambda: G.cadd_verify_tree(y2, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, out=v2))
+    flops = 2.0 * M * hidden * cfg.V
+    peak, kind = measured_peak_tflops()
+    ach = flops / (t_fused * 1e-3) / 1e12
+    return {"hidden": hidden, "rows": M, "ms": round(t_fused, 4), "flops": flops,
+            "roofline": {"bound": "tensor", "achieved": round(ach, 1), "peak": peak, "peak_kind": f"of {kind}", "unit": "TFLOP/s",
+                         "frac": round(ach / peak, 4)},
+            "library_gemm_ms": round(t_gemm, 4), "argmax_on_logits_ms": round(t_arg, 4),
+            "status_bits": int(out.status.max().item()), "iters": iters}
 
 
 def oracle_sample(cfg, d, c, y, tree, dense, n_req, target_cpu_seconds=15.0):
@@ -358,6 +412,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
+    ap.add_argument("--head-hidden", type=int, default=4096,
+                    help="hidden size for the fused output-projection verification measurement (0 = skip)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))

@@ -313,6 +313,11 @@ int cadd_verify_tree_fused_head(const cadd_head_args* a, void* cuda_stream) {
     hp.M = M; hp.V = a->V; hp.Kdim = a->hidden;
     hp.m_tiles = (int)((M + kHeadBM - 1) / kHeadBM);
     hp.n_tiles = (int)((a->V + kHeadBN - 1) / kHeadBN);
+    {
+        // row tiles per group: about 24 MB of hidden states, so that they stay L2-resident while W streams by
+        int64_t g = ((int64_t)24 << 20) / ((int64_t)kHeadBM * a->hidden * 2);
+        hp.group_m = (int)(g < 1 ? 1 : (g > hp.m_tiles ? hp.m_tiles : g));
+    }
     hp.R = a->R; hp.rows_mode = a->rows_mode; hp.n_nodes = a->n_nodes;
     hp.row_best = (unsigned long long*)a->workspace;
     hp.error = (int32_t*)((unsigned char*)a->workspace + (need - 256));

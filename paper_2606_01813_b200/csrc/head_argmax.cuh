@@ -13,9 +13,10 @@
 //               allocation (all 512 columns = two accumulators, so the epilogue of one tile overlaps the next);
 //   warps 2-5   epilogue: each thread owns one row of the tile (one tensor-memory lane), reads it 32 columns at a time
 //               with tcgen05.ld and keeps the running maximum and its first column.
-// Tiles are walked in the order (column tile outer, row tile inner), CTA c taking tiles c, c + grid, ...: at any time
-// the CTAs work on neighbouring column tiles of W, which then come from L2 after their first use, and the hidden
-// states (tens of MB) stay L2-resident.
+// Tiles are walked in groups of row tiles whose hidden states fit in L2 (about 24 MB); inside a group the order is
+// (column tile outer, row tile inner), CTA c taking tiles c, c + grid, ...: at any time the CTAs work on neighbouring
+// column tiles of W, which come from L2 after their first use, the group's hidden states stay L2-resident, and W is
+// streamed from HBM once per group.
 //
 // Every wait on an mbarrier has an iteration limit; a role that gives up sets an error word, all roles then leave
 // their loops, the CTA meets at a barrier and the tensor memory is released before it exits.
@@ -52,18 +53,21 @@ struct HeadParams {
     int64_t V;                 // tokens
     int Kdim;                  // hidden size
     int m_tiles, n_tiles;
+    int group_m;               // row tiles per group: a group's hidden states stay L2-resident while all of W streams by
     int R, rows_mode;
     const int32_t* n_nodes;    // [batch] (LIVE mode: row tiles without a live row are skipped)
     unsigned long long* row_best;   // [M] packed (ordered logit << 32 | ~token), zeroed before the launch
     int32_t* error;            // device word, set non-zero when a bounded wait ran out
 };
 
-// Bounded wait without a sleep between tries: the roles of this kernel are single threads or warps that own their
-// issue slots (one CTA per SM), and a late wake-up of the MMA thread would leave the tensor cores idle.
+// Bounded wait.  The MMA thread polls without a sleep between tries: a late wake-up would leave the tensor cores
+// idle.
 constexpr int kHeadSpinLimit = 1 << 20;
-__device__ __forceinline__ bool head_wait(uint64_t* bar, unsigned parity) {
-    for (int it = 0; it < kHeadSpinLimit; ++it)
+__device__ __forceinline__ bool head_wait(uint64_t* bar, unsigned parity, unsigned sleep_ns = 0) {
+    for (int it = 0; it < kHeadSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (sleep_ns) __nanosleep(sleep_ns);      // roles off the critical path back off: spinning costs power the tensor cores need
+    }
     return false;
 }
 
@@ -116,6 +120,17 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(const void* tile, int k16)
 // (bits 15, 16 = 0), N / 8 in bits 17-22, M / 16 in bits 24-28.
 constexpr uint32_t kHeadIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kHeadBN >> 3) << 17) | ((uint32_t)(kHeadBM >> 4) << 24);
 
+// Tile order: groups of group_m row tiles; inside a group the column tile is the outer index and the row tile the
+// inner one.  Work item w (CTA c takes w = c, c + grid, ...) -> (row tile, column tile).
+__device__ __forceinline__ void head_tile_of(const HeadParams& p, int64_t w, int& mt, int& nt) {
+    const int64_t per_group = (int64_t)p.group_m * p.n_tiles;
+    const int g = (int)(w / per_group);
+    const int64_t rem = w - (int64_t)g * per_group;
+    const int gsz = min(p.group_m, p.m_tiles - g * p.group_m);
+    nt = (int)(rem / gsz);
+    mt = g * p.group_m + (int)(rem - (int64_t)nt * gsz);
+}
+
 // True if row tile mt holds a row that is read: always in DENSE mode; in LIVE mode rows j <= n_nodes[b] of a request.
 __device__ __forceinline__ bool head_tile_live(const HeadParams& p, int mt) {
     if (p.rows_mode != CADD_ROWS_LIVE) return true;
@@ -155,10 +170,11 @@ head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
         if (lane == 0) {
             unsigned s = 0, ph = 0;
             for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
-                const int nt = (int)(w / p.m_tiles), mt = (int)(w - (int64_t)nt * p.m_tiles);
+                int mt, nt;
+                head_tile_of(p, w, mt, nt);
                 if (!head_tile_live(p, mt)) continue;
                 for (int k = 0; k < k_steps; ++k) {
-                    if (!head_wait(&sh.empty[s], ph ^ 1u)) { sh.error = 1; break; }   // first pass: free at once
+                    if (!head_wait(&sh.empty[s], ph ^ 1u, 64)) { sh.error = 1; break; }   // first pass: free at once
                     mbar_arrive_expect_tx(&sh.full[s], kHeadABytes + kHeadBBytes);
                     tma_load_2d(&sh.a[s][0], &map_h, k * kHeadBK, mt * kHeadBM, &sh.full[s]);
                     tma_load_2d(&sh.b[s][0], &map_w, k * kHeadBK, nt * kHeadBN, &sh.full[s]);
@@ -171,7 +187,8 @@ head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
         if (lane == 0) {
             unsigned s = 0, ph = 0, buf = 0, aph = 0;
             for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
-                const int nt = (int)(w / p.m_tiles), mt = (int)(w - (int64_t)nt * p.m_tiles);
+                int mt, nt;
+                head_tile_of(p, w, mt, nt);
                 if (!head_tile_live(p, mt)) continue;
                 if (!head_wait(&sh.acc_empty[buf], aph ^ 1u)) { sh.error = 2; break; }   // epilogue has drained it
                 tc_fence_after();
@@ -197,9 +214,10 @@ head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
         const int quarter = warp & 3;
         unsigned buf = 0, aph = 0;
         for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
-            const int nt = (int)(w / p.m_tiles), mt = (int)(w - (int64_t)nt * p.m_tiles);
+            int mt, nt;
+            head_tile_of(p, w, mt, nt);
             if (!head_tile_live(p, mt)) continue;
-            if (!__all_sync(kFullMask, head_wait(&sh.acc_full[buf], aph))) { sh.error = 4; break; }
+            if (!__all_sync(kFullMask, head_wait(&sh.acc_full[buf], aph, 256))) { sh.error = 4; break; }
             tc_fence_after();
             const int64_t row = (int64_t)mt * kHeadBM + quarter * 32 + lane;
             const int64_t col0 = (int64_t)nt * kHeadBN;
