@@ -116,6 +116,8 @@ def run_ours(args, rank, world):
     torch.cuda.set_device(dev)
     replicas.init_replicas("nccl", dev)
     cfg = synth.CONFIGS[args.workload]
+    if args.batch:
+        cfg = synth.scaled(cfg, batch=args.batch)        # reduced case of the same workload (profiling captures)
     seed = replicas.replica_seed(synth.config_seed(cfg), rank)
     rows_mode = G.ROWS_DENSE if args.rows_mode == "dense" else G.ROWS_LIVE
     flags = G.FLAG_FIXED_BUDGET if cfg.fixed_budget else 0
@@ -411,6 +413,7 @@ def main():
     ap.add_argument("--cpu-requests", type=int, default=32)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (0 = as defined)")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
     ap.add_argument("--head-hidden", type=int, default=4096,
                     help="hidden size for the fused output-projection verification measurement (0 = skip)")

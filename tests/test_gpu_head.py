@@ -109,3 +109,32 @@ def test_fused_head_rejects_bad_arguments():
     with pytest.raises(G.CaddError):                                       # stride not a multiple of 8 elements
         G.cadd_verify_tree_fused_head(torch.zeros(1, 3, 68, dtype=torch.bfloat16, device="cuda")[:, :, :60],
                                       torch.zeros(10, 60, dtype=torch.bfloat16, device="cuda"), 4, z, t, t)
+
+
+def test_fused_head_full_size_sampled_rows():
+    """Config 2's verification shape (8224 rows, V = 151936) with hidden size 4096, in the launch configuration the
+    bench times; the oracle recomputes a seeded sample of rows (one row costs V x hidden fp64 products)."""
+    cfg = synth.CONFIGS["c2"]
+    hidden = 4096
+    g = torch.Generator(device="cuda").manual_seed(77)
+    h = torch.randn(cfg.batch, cfg.R, hidden, device="cuda", dtype=torch.bfloat16, generator=g)
+    w = torch.randn(cfg.V, hidden, device="cuda", dtype=torch.bfloat16, generator=g)
+    n_nodes = torch.full((cfg.batch,), 7, dtype=torch.int32, device="cuda")
+    tok = torch.zeros(cfg.batch, cfg.R, dtype=torch.int32, device="cuda")
+    par = torch.zeros(cfg.batch, cfg.R, dtype=torch.int32, device="cuda")
+    out = G.cadd_verify_tree_fused_head(h, w, cfg.L, n_nodes, tok, par, G.ROWS_DENSE)
+    torch.cuda.synchronize()
+    assert int(out.status.max()) == 0
+    ga = to_cpu(out.node_argmax).reshape(-1)
+    assert int(ga.min()) >= 0 and int(ga.max()) < cfg.V
+    rows = torch.randint(0, cfg.batch * cfg.R, (12,), generator=torch.Generator().manual_seed(5)).tolist() + [0, cfg.batch * cfg.R - 1]
+    hs = h.reshape(-1, hidden)[rows].cpu().unsqueeze(0)
+    wc = w.cpu()
+    y64 = O.head_logits(hs, wc)[0]
+    absw = wc.double().abs()
+    for i, r in enumerate(rows):
+        o = int(y64[i].to(torch.float32).argmax())          # decision in the precision the GPU reports its logits in
+        gpick = int(ga[r])
+        if o != gpick:
+            tol = hidden * 2.0 ** -24 * float((hs[0, i].double().abs() * absw[[o, gpick]]).sum(dim=1).max())
+            assert abs(float(y64[i, o] - y64[i, gpick])) <= tol, (r, o, gpick)
