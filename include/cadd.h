@@ -196,6 +196,27 @@ typedef struct cadd_head_args {
     size_t   workspace_bytes;
 } cadd_head_args;
 
+/*
+ * Offline cost fitting (Section "Offline Cost Profiling", Eq. 12): for each of n_tables profiled context lengths,
+ * the least-squares fit to N measured verification latencies (node counts equally spaced, e.g. n = 1..N) among
+ * all convex, non-decreasing sequences.  The fitted rows can be passed to cadd_build_tree as cost_table (with
+ * CADD_COST_TABLE or CADD_COST_TABLE_INTERP); the caller decides what C_v(0) is.
+ * All pointers are DEVICE pointers owned by the caller; the call needs no workspace.
+ */
+#define CADD_FIT_MAX_N 2048
+#define CADD_FIT_STATUS_ITERATION_CAP 1   /* the active-set iteration was cut off; the row is its last iterate */
+#define CADD_FIT_STATUS_KNOT_CAP      2   /* reserved (the slope-change capacity equals CADD_FIT_MAX_N) */
+typedef struct cadd_fit_args {
+    uint32_t struct_size;          /* = sizeof(cadd_fit_args) */
+    uint32_t flags;                /* reserved, 0 */
+    int32_t  n_tables;             /* independent problems, >= 1 */
+    int32_t  N;                    /* points per problem, 1 .. CADD_FIT_MAX_N */
+    const double* y;               /* [n_tables, N] measurements */
+    double*  fit;                  /* [n_tables, N] out: fitted values (convex, non-decreasing along N) */
+    int32_t* n_breaks;             /* [n_tables] out: number of slope changes of the fit (first slope included), may be NULL */
+    int32_t* status;               /* [n_tables] out: CADD_FIT_STATUS_* bits, 0 = optimal; may be NULL */
+} cadd_fit_args;
+
 /* ABI version of the loaded library (CADD_ABI_VERSION it was built with). */
 int cadd_version(void);
 
@@ -222,6 +243,10 @@ int cadd_head_workspace_bytes(const cadd_head_args* a, size_t* out);
  * driver's tensor-map encoder is unavailable.  If an internal bounded wait runs out, every request reports
  * CADD_STATUS_INTERNAL_TIMEOUT. */
 int cadd_verify_tree_fused_head(const cadd_head_args* a, void* cuda_stream);
+
+/* Convex, non-decreasing least-squares fit of every row (see cadd_fit_args).  Asynchronous on `cuda_stream`: one
+ * kernel, one CTA per row, fp64.  CADD_ERR_SHAPE if N > CADD_FIT_MAX_N. */
+int cadd_fit_cost_tables(const cadd_fit_args* a, void* cuda_stream);
 
 /*
  * cadd_build_tree for callers that cannot provide scratch memory.  (The paper has no counterpart to

@@ -204,3 +204,26 @@ def verify_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor, L:
     then the plain argmax (lowest id among equals) and the walk follow.  Returns (OracleVerify, fp64 logits)."""
     y64 = head_logits(hidden_states, weight)
     return verify_tree(y64.to(torch.float32), L, n_nodes, token_ids, parent_idx, rows_mode), y64
+
+
+def fit_convex_nondecreasing(y) -> "torch.Tensor":
+    """Offline cost fitting (Eq. 12): for each row of y [n_tables, N] (latencies measured at N equally spaced node
+    counts) the least-squares fit among all convex, non-decreasing sequences.
+
+    Written out as the definition: a sequence f on points 0..N-1 is convex and non-decreasing iff
+    f_i = a + sum_k beta_k * max(0, i - k) with beta_k >= 0 for k = 0..N-2 (beta_0 is the first slope, beta_k the
+    slope increase at point k) and a free; the fit is therefore a non-negative least-squares problem in
+    (a+, a-, beta), handed to the library's NNLS routine.  fp64 throughout."""
+    import numpy as np
+    from scipy.optimize import nnls
+    y = torch.as_tensor(y, dtype=torch.float64)
+    assert y.dim() == 2
+    T, N = y.shape
+    i = np.arange(N, dtype=np.float64)[:, None]
+    k = np.arange(max(N - 1, 0), dtype=np.float64)[None, :]
+    A = np.concatenate([np.ones((N, 1)), -np.ones((N, 1)), np.maximum(0.0, i - k)], axis=1)
+    out = torch.empty_like(y)
+    for t in range(T):
+        coef, _ = nnls(A, y[t].numpy(), maxiter=50 * A.shape[1])
+        out[t] = torch.from_numpy(A @ coef)
+    return out

@@ -27,7 +27,7 @@ ROWS_LIVE, ROWS_DENSE = 0, 1
 
 EXPORTS = ("cadd_version", "cadd_status_string", "cadd_build_workspace_bytes", "cadd_verify_workspace_bytes",
            "cadd_build_tree", "cadd_verify_tree", "cadd_build_tree_static_scratch",
-           "cadd_head_workspace_bytes", "cadd_verify_tree_fused_head")
+           "cadd_head_workspace_bytes", "cadd_verify_tree_fused_head", "cadd_fit_cost_tables")
 ERR_STATIC_SCRATCH = -8
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -78,6 +78,13 @@ class HeadArgs(C.Structure):
     ]
 
 
+class FitArgs(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("flags", C.c_uint32), ("n_tables", C.c_int32), ("N", C.c_int32),
+        ("y", C.c_void_p), ("fit", C.c_void_p), ("n_breaks", C.c_void_p), ("status", C.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -98,6 +105,7 @@ def lib() -> C.CDLL:
         l.cadd_verify_tree.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
         l.cadd_head_workspace_bytes.argtypes = [C.POINTER(HeadArgs), C.POINTER(C.c_size_t)]
         l.cadd_verify_tree_fused_head.argtypes = [C.POINTER(HeadArgs), C.c_void_p]
+        l.cadd_fit_cost_tables.argtypes = [C.POINTER(FitArgs), C.c_void_p]
         l.cadd_build_tree_static_scratch.argtypes = [C.POINTER(BuildArgs), C.c_void_p]
         _lib = l
     return _lib
@@ -344,6 +352,27 @@ def cadd_verify_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tenso
         raise CaddError(rc)
     workspace.record_stream(torch.cuda.current_stream() if stream is None else stream)
     return out
+
+
+def cadd_fit_cost_tables(y: torch.Tensor, *, stream: Optional[torch.cuda.Stream] = None):
+    """Offline cost fitting (Eq. 12): the convex, non-decreasing least-squares fit of every row of y [n_tables, N]
+    (fp64, CUDA).  Returns (fit [n_tables, N] fp64, n_breaks [n_tables] int32, status [n_tables] int32)."""
+    if not y.is_cuda:
+        raise ValueError("y must be a CUDA tensor (there is no CPU path)")
+    if y.dtype != torch.float64 or y.dim() != 2 or not y.is_contiguous():
+        raise ValueError("y must be a contiguous float64 tensor [n_tables, N]")
+    a = FitArgs()
+    a.struct_size = C.sizeof(FitArgs)
+    a.n_tables, a.N = y.shape
+    fit = torch.empty_like(y)
+    nb = torch.empty(y.shape[0], dtype=torch.int32, device=y.device)
+    st = torch.empty(y.shape[0], dtype=torch.int32, device=y.device)
+    a.y, a.fit, a.n_breaks, a.status = y.data_ptr(), fit.data_ptr(), nb.data_ptr(), st.data_ptr()
+    with torch.cuda.device(y.device):
+        rc = lib().cadd_fit_cost_tables(C.byref(a), _stream_ptr(stream))
+    if rc != OK:
+        raise CaddError(rc)
+    return fit, nb, st
 
 
 def cadd_build_tree_static_scratch(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[int] = None, *,

@@ -9,6 +9,7 @@
 #include "softmax_topk.cuh"
 #include "verify.cuh"
 #include "head_argmax.cuh"
+#include "fit_cost.cuh"
 
 namespace cadd {
 
@@ -340,6 +341,25 @@ int cadd_verify_tree_fused_head(const cadd_head_args* a, void* cuda_stream) {
     wp.accepted_nodes = a->accepted_nodes; wp.next_bonus = a->next_bonus; wp.status = a->status;
     const int wpb = 4;
     accept_walk_kernel<<<(a->batch + wpb - 1) / wpb, wpb * 32, 0, st>>>(wp);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    return CADD_OK;
+}
+
+// ---------------- offline cost fitting (Eq. 12) ----------------
+
+int cadd_fit_cost_tables(const cadd_fit_args* a, void* cuda_stream) {
+    if (!a) return CADD_ERR_NULL;
+    if (a->struct_size != sizeof(cadd_fit_args)) return CADD_ERR_STRUCT_SIZE;
+    if (a->n_tables < 1 || a->n_tables > 65535 || a->N < 1 || a->N > kFitMaxN) return CADD_ERR_SHAPE;
+    if (!a->y || !a->fit) return CADD_ERR_NULL;
+    if (!aligned(a->y, 8) || !aligned(a->fit, 8) || !aligned(a->n_breaks, 4) || !aligned(a->status, 4)) return CADD_ERR_ALIGN;
+    if (cudaFuncSetAttribute(fit_cost_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fit_smem_bytes()) != cudaSuccess) {
+        cudaGetLastError();
+        return CADD_ERR_LAUNCH;
+    }
+    FitParams fp;
+    fp.n_tables = a->n_tables; fp.N = a->N; fp.y = a->y; fp.fit = a->fit; fp.n_breaks = a->n_breaks; fp.status = a->status;
+    fit_cost_kernel<<<a->n_tables, kFitThreads, fit_smem_bytes(), (cudaStream_t)cuda_stream>>>(fp);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
     return CADD_OK;
 }

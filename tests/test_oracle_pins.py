@@ -542,3 +542,75 @@ def test_fused_head_verdict_on_a_hand_made_tree():
     ov, y64 = O.verify_tree_fused_head(h.bfloat16(), w, 4, n_nodes, token_ids, parent_idx, rows_mode=O.ROWS_LIVE)
     assert ov.node_argmax[0].tolist() == [1, 3, 2, 5, -1]
     assert int(ov.accepted_len[0]) == 2 and ov.accepted_nodes[0].tolist() == [1, 3, -1, -1] and int(ov.next_bonus[0]) == 5
+
+
+# ---- offline cost fitting: convex, non-decreasing least squares (Eq. 12) ----
+
+def _kkt_violation(y, f):
+    """Optimality of f over the cone of convex non-decreasing sequences, checked from the definition with plain
+    numpy: feasibility; residual orthogonal to constants; <r, hinge_k> <= 0 for every hinge max(0, i - k), with
+    equality wherever the fit actually bends (or rises, for k = 0)."""
+    import numpy as np
+    y, f = np.asarray(y, dtype=np.float64), np.asarray(f, dtype=np.float64)
+    N = len(y)
+    scale = max(1.0, float(np.abs(y).max()))
+    r = y - f
+    slopes = np.diff(f)
+    bends = np.concatenate([slopes[:1], np.diff(slopes)])          # beta_k, k = 0..N-2
+    worst = max(0.0, float(-bends.min()) / scale) if N > 1 else 0.0   # feasibility
+    worst = max(worst, abs(float(r.sum())) / (scale * N))
+    i = np.arange(N)
+    for k in range(N - 1):
+        g = float((np.maximum(0, i - k) * r).sum()) / (scale * N * N)
+        worst = max(worst, g)                                       # dual feasibility
+        if bends[k] > 1e-9 * scale:
+            worst = max(worst, abs(g))                              # complementary slackness
+    return worst
+
+
+def test_convex_fit_satisfies_kkt_on_noisy_data():
+    g = torch.Generator().manual_seed(8)
+    n = torch.arange(200, dtype=torch.float64)
+    clean = torch.stack([2.0 + 0.01 * n + 2e-4 * n * n, 5.0 + 0.03 * n + torch.clamp(n - 120, min=0) * 0.2])
+    y = clean + 0.3 * torch.randn(2, 200, generator=g, dtype=torch.float64)
+    f = O.fit_convex_nondecreasing(y)
+    for t in range(2):
+        assert _kkt_violation(y[t].numpy(), f[t].numpy()) < 1e-8
+        assert float(((f[t] - clean[t]) ** 2).mean()) < float(((y[t] - clean[t]) ** 2).mean())   # it denoises
+
+
+def test_convex_fit_closed_forms():
+    n = torch.arange(50, dtype=torch.float64)
+    convex = 1.0 + 0.5 * n + 0.02 * n * n
+    assert torch.allclose(O.fit_convex_nondecreasing(convex[None])[0], convex, rtol=0, atol=1e-9)   # exact recovery
+    falling = 10.0 - 0.3 * n
+    assert torch.allclose(O.fit_convex_nondecreasing(falling[None])[0], torch.full_like(n, float(falling.mean())), atol=1e-9)
+    concave = torch.sqrt(n + 1.0)                                    # best convex fit of a concave rise: its regression line
+    X = torch.stack([torch.ones_like(n), n], dim=1)
+    line = X @ torch.linalg.lstsq(X, concave[:, None]).solution[:, 0]
+    assert torch.allclose(O.fit_convex_nondecreasing(concave[None])[0], line, atol=1e-9)
+
+
+def test_convex_fit_brute_force_over_active_sets():
+    """N = 6: the solution is the feasible least-squares fit with the smallest error over all 2^5 choices of which
+    hinges may be non-zero."""
+    import itertools
+    import numpy as np
+    rng = np.random.default_rng(4)
+    N = 6
+    i = np.arange(N, dtype=np.float64)
+    for trial in range(20):
+        y = np.cumsum(rng.normal(0.3, 1.0, N))
+        best, best_f = None, None
+        for mask in itertools.product([0, 1], repeat=N - 1):
+            cols = [np.ones(N)] + [np.maximum(0, i - k) for k in range(N - 1) if mask[k]]
+            A = np.stack(cols, axis=1)
+            coef = np.linalg.lstsq(A, y, rcond=None)[0]
+            if (coef[1:] < -1e-12).any():
+                continue
+            f = A @ coef
+            sse = float(((y - f) ** 2).sum())
+            if best is None or sse < best - 1e-12:
+                best, best_f = sse, f
+        f = O.fit_convex_nondecreasing(torch.from_numpy(y)[None])[0].numpy()
+        assert abs(float(((y - f) ** 2).sum()) - best) < 1e-9 and np.allclose(f, best_f, atol=1e-7)
