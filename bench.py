@@ -258,6 +258,14 @@ def run_ours(args, rank, world):
         except Exception as ex:
             fused_head = {"error": str(ex)[:200]}
 
+    # ---- offline cost fitting on a synthetic 9 x 1024 latency grid (the paper's profiling shape) ----
+    cost_fit = None
+    if not args.no_fit:
+        try:
+            cost_fit = fit_block(G, dev)
+        except Exception as ex:
+            cost_fit = {"error": str(ex)[:200]}
+
     # ---- the oracle timed on this machine's host cores, on a bounded sample (rank 0, N = 1 only) ----
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -273,7 +281,7 @@ def run_ours(args, rank, world):
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": f"replicas x{world}",
                        "n_star_mean": round(float(n_star.float().mean()), 2), "n_star_max": int(n_star.max()),
                        "accepted_mean": round(float(verdict.accepted_len.float().mean().item()), 2)},
-            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
             "gpu_launches": KERNELS_PER_STEP * K, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
@@ -324,6 +332,25 @@ def head_block(G, cfg, tree, verdict, y, rows_mode, hidden, dev, iters):
                          "frac": round(ach / peak, 4)},
             "library_gemm_ms": round(t_gemm, 4), "argmax_on_logits_ms": round(t_arg, 4),
             "status_bits": int(out.status.max().item()), "iters": iters}
+
+
+def fit_block(G, dev, iters=5):
+    """cadd_fit_cost_tables on nine noisy convex latency curves of 1024 points each; absolute time (a small,
+    latency-bound problem: one CTA per curve), not a roofline figure."""
+    g = torch.Generator(device="cpu").manual_seed(21)
+    n = torch.arange(1, 1025, dtype=torch.float64)
+    y = torch.stack([18.0 + 2.0 * j + (0.010 + 0.002 * j) * n + (2e-5 + 2e-6 * j) * n * n + 0.004 * torch.clamp(n - 256, min=0)
+                     + (0.2 + 0.05 * j) * torch.randn(1024, generator=g, dtype=torch.float64) for j in range(9)]).to(dev)
+    fit, nb, st = G.cadd_fit_cost_tables(y)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        G.cadd_fit_cost_tables(y)
+    e1.record()
+    torch.cuda.synchronize()
+    return {"tables": 9, "points": 1024, "ms": round(e0.elapsed_time(e1) / iters, 4), "slope_changes_max": int(nb.max().item()),
+            "status_bits": int(st.max().item()), "rmse": round(float(((fit - y) ** 2).mean().sqrt().item()), 5)}
 
 
 def oracle_sample(cfg, d, c, y, tree, dense, n_req, target_cpu_seconds=15.0):
@@ -415,6 +442,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (0 = as defined)")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
+    ap.add_argument("--no-fit", action="store_true", help="skip the offline cost-fitting measurement")
     ap.add_argument("--head-hidden", type=int, default=4096,
                     help="hidden size for the fused output-projection verification measurement (0 = skip)")
     args = ap.parse_args()
