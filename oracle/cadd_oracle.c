@@ -14,6 +14,9 @@
  *   O4  draft-tree arrays and the ancestor ("tree attention") mask       (Section 3.3)
  *   O5  greedy verification: argmax of the target logits at every node   (Section 3.1)
  *   O6  walk along the longest accepted path, next bonus token           (Sections 3.1, 3.3)
+ *   O7  target logits from hidden states and the output projection      (Section 3.1; feeds O5)
+ * The convex regression of the cost tables (Eq. 12) lives in the Python wrapper, written as a
+ * non-negative least-squares problem for the library's NNLS routine.
  *
  * All floating point is double.  bf16 / fp32 inputs are widened exactly.  No blocking, fusion
  * or reordering: sums run in ascending token order, the heap H of Algorithm 1 is an unordered
