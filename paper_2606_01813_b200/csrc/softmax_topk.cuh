@@ -10,8 +10,8 @@
 // only ever cover the part of the mass that is spread over many small terms.
 //
 // Data path: one elected thread streams the segment into a ring of shared-memory tiles with bulk
-// asynchronous copies (cp.async.bulk, completion on an mbarrier; no multicast); a second set of mbarriers
-// tells it when all eight warps are done with a stage.  Warps advance through the tiles on their own:
+// asynchronous copies (cp.async.bulk, completion on an mbarrier; no multicast); a per-stage counter tells when
+// all eight warps are done with a stage, and the last of them refills it.  Warps advance through the tiles on their own:
 // there is no CTA-wide barrier in the steady state.
 //
 // Hot loop per thread and tile (four 16-byte chunks = 32 bf16 / 16 fp32): one packed max over all
@@ -108,7 +108,7 @@ struct TopkShared {
     uint64_t sel_prefix;
     unsigned sel_need;
     unsigned pushed;         // fast path: candidates appended so far
-    unsigned overflow;       // fast path: the ring was full at some push
+    unsigned overflow;       // fast path: the candidate buffer was full at some push
     unsigned timeout;        // a bounded wait ran out
     double red_d[kThreads / 32];
     float red_f[kThreads / 32];
@@ -417,7 +417,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
             const int64_t e = p.V - sp.tail + tid;
             slow_element(sh, s, flags, dummy, E::load(row, e), (uint32_t)e);
         }
-        // (slow_element appends to keys[0..count): at most 14 entries, moved into the ring below)
+        // (slow_element appends to keys[0..count): at most 14 entries; they become the first candidates)
         __syncthreads();
         if (tid == 0) { sh.pushed = sh.count; sh.count = 0; }
 
