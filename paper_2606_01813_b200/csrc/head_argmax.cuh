@@ -5,7 +5,7 @@
 // to one (value, token) pair per row, merged across tiles by a 64-bit atomic max.
 //
 // One CTA per SM, 192 threads, three roles:
-//   warp 0      producer: 2-D tiled bulk tensor copies (TMA, 128-byte swizzle, no multicast) of a 128 x 64 tile of
+//   warp 0      producer: 2-D tiled bulk tensor copies (TMA, 128-byte swizzle, each into this CTA's own shared memory) of a 128 x 64 tile of
 //               hidden states and a 256 x 64 tile of W into a 4-stage shared-memory ring, completion on mbarriers;
 //   warp 1      one elected thread issues tcgen05.mma (M 128, N 256, K 16 per instruction, operands described by
 //               shared-memory matrix descriptors, accumulator in tensor memory), tcgen05.commit frees the stage and,

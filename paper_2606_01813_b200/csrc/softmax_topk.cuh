@@ -10,7 +10,7 @@
 // only ever cover the part of the mass that is spread over many small terms.
 //
 // Data path: one elected thread streams the segment into a ring of shared-memory tiles with bulk
-// asynchronous copies (cp.async.bulk, completion on an mbarrier; no multicast); a per-stage counter tells when
+// asynchronous copies (cp.async.bulk into this CTA's own shared memory, completion on an mbarrier); a per-stage counter tells when
 // all eight warps are done with a stage, and the last of them refills it.  Warps advance through the tiles on their own:
 // there is no CTA-wide barrier in the steady state.
 //

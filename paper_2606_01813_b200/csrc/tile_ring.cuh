@@ -1,6 +1,6 @@
 // Building blocks of the shared-memory tile ring used by the streaming kernels: a thread issues 1-D bulk
 // asynchronous copies (cp.async.bulk) of 16 KB tiles into a small ring of stages; each stage has an mbarrier
-// that completes when the tile's bytes have landed (complete_tx).  No cluster, no multicast: every copy goes
+// that completes when the tile's bytes have landed (complete_tx).  No cluster: every copy goes
 // into the issuing CTA's own shared memory.  Every wait is bounded.
 #pragma once
 #include "common.cuh"

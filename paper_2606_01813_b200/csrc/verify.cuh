@@ -26,7 +26,7 @@ struct ArgmaxRing {
 inline size_t argmax_smem_bytes() { return sizeof(ArgmaxRing) + 128; }
 
 // One CTA per (request, row).  One thread streams the row's 16-byte chunks into a ring of 16 KB
-// shared-memory tiles with cp.async.bulk + mbarrier (no multicast); the last warp to finish a tile refills
+// shared-memory tiles with cp.async.bulk + mbarrier (own shared memory only); the last warp to finish a tile refills
 // its stage, so (kStages - 1) x 16 KB stay in flight per CTA (4 CTAs per SM) without living in registers.
 // Each thread keeps the running maximum (packed bf16 max, NaN ignored) and the first position (chunk start or
 // scalar element) where it was reached; the CTA reduces (value descending, position ascending) and one warp
