@@ -283,7 +283,9 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         int n = 0, popped = 0;
         bool stopped = false;
         while (ok && !stopped) {
-            const int G = popped < 16 ? 8 : 32;
+            // group sizes grow with the tree: a stop is usually found within the group that contains it, and what a
+            // group pops beyond the stop is wasted (a pop costs about four group evaluations)
+            const int G = popped < 8 ? 4 : (popped < 32 ? 8 : (popped < 64 ? 16 : 32));
             int g = 0;
             while (g < G && popped < B_max && fsize > 0) {
                 // ---- arg-max of the 128-bit keys cached per lane, 32 bits at a time ----
