@@ -197,6 +197,28 @@ typedef struct cadd_head_args {
 } cadd_head_args;
 
 /*
+ * Tree construction fused into the drafter's output projection (Eq. 1 with l_i = h_i . W^T; Algorithm 1).
+ * cadd_build_tree reads materialised draft logits [batch, L, V]; this entry point takes the drafter's last hidden
+ * states and the output-projection weight instead and never writes the logits: they are formed tile by tile on the
+ * tensor cores (bf16 inputs, fp32 accumulation) and consumed at once by the softmax statistics and the top-K
+ * selection.  Everything after that (expansion, stopping rule, emission, outputs, status bits) is cadd_build_tree's.
+ * A logit is the fp32-accumulated dot product.  `build` carries all other arguments: its draft_logits, stride_b,
+ * stride_l and logits_dtype are ignored, its V is the number of tokens, its workspace must hold
+ * cadd_build_head_workspace_bytes.  K <= 32 on this path.
+ */
+typedef struct cadd_build_head_args {
+    uint32_t struct_size;          /* = sizeof(cadd_build_head_args) */
+    uint32_t flags;                /* reserved, 0 */
+    int32_t  hidden;               /* hidden size (the contraction length) */
+    int32_t  reserved0;
+    const void* hidden_states;     /* bf16 [batch, L, hidden]; element (b,i,k) at (b*L + i)*stride_row + k; 16-byte aligned */
+    int64_t  stride_row;           /* in elements, >= hidden, multiple of 8 */
+    const void* weight;            /* bf16 [V, hidden]; element (v,k) at v*stride_w + k; 16-byte aligned */
+    int64_t  stride_w;             /* in elements, >= hidden, multiple of 8 */
+    cadd_build_args build;         /* struct_size = sizeof(cadd_build_args) */
+} cadd_build_head_args;
+
+/*
  * Offline cost fitting (Section "Offline Cost Profiling", Eq. 12): for each of n_tables profiled context lengths,
  * the least-squares fit to N measured verification latencies (node counts equally spaced, e.g. n = 1..N) among
  * all convex, non-decreasing sequences.  The fitted rows can be passed to cadd_build_tree as cost_table (with
@@ -243,6 +265,14 @@ int cadd_head_workspace_bytes(const cadd_head_args* a, size_t* out);
  * driver's tensor-map encoder is unavailable.  If an internal bounded wait runs out, every request reports
  * CADD_STATUS_INTERNAL_TIMEOUT. */
 int cadd_verify_tree_fused_head(const cadd_head_args* a, void* cuda_stream);
+
+/* Scratch size of cadd_build_tree_fused_head: pure host arithmetic on batch, L and K. */
+int cadd_build_head_workspace_bytes(const cadd_build_head_args* a, size_t* out);
+
+/* Tree construction from hidden states and the output-projection weight (see cadd_build_head_args).  Asynchronous on
+ * `cuda_stream`: one small memset and three kernels.  Errors as for cadd_build_tree, plus CADD_ERR_SHAPE for K > 32,
+ * CADD_ERR_ALIGN for a base pointer that is not 16-byte aligned or a stride that is not a multiple of 8 elements. */
+int cadd_build_tree_fused_head(const cadd_build_head_args* a, void* cuda_stream);
 
 /* Convex, non-decreasing least-squares fit of every row (see cadd_fit_args).  Asynchronous on `cuda_stream`: one
  * kernel, one CTA per row, fp64.  CADD_ERR_SHAPE if N > CADD_FIT_MAX_N. */

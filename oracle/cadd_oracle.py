@@ -206,6 +206,14 @@ def verify_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor, L:
     return verify_tree(y64.to(torch.float32), L, n_nodes, token_ids, parent_idx, rows_mode), y64
 
 
+def build_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor, K: int, B_max: int, R: Optional[int] = None, **kw):
+    """O1-O4 on draft logits formed from the drafter's hidden states [batch, L, hidden] and its output projection
+    [V, hidden] (Eq. 1 with l_i = h_i . W^T).  The exact fp64 dot products are rounded once to fp32, the precision the
+    GPU path holds its logits in, and handed to build_tree.  Returns (OracleTree, fp64 logits)."""
+    y64 = head_logits(hidden_states, weight)
+    return build_tree(y64.to(torch.float32), K, B_max, R, **kw), y64
+
+
 def fit_convex_nondecreasing(y) -> "torch.Tensor":
     """Offline cost fitting (Eq. 12): for each row of y [n_tables, N] (latencies measured at N equally spaced node
     counts) the least-squares fit among all convex, non-decreasing sequences.

@@ -27,7 +27,8 @@ ROWS_LIVE, ROWS_DENSE = 0, 1
 
 EXPORTS = ("cadd_version", "cadd_status_string", "cadd_build_workspace_bytes", "cadd_verify_workspace_bytes",
            "cadd_build_tree", "cadd_verify_tree", "cadd_build_tree_static_scratch",
-           "cadd_head_workspace_bytes", "cadd_verify_tree_fused_head", "cadd_fit_cost_tables")
+           "cadd_head_workspace_bytes", "cadd_verify_tree_fused_head", "cadd_fit_cost_tables",
+           "cadd_build_head_workspace_bytes", "cadd_build_tree_fused_head")
 ERR_STATIC_SCRATCH = -8
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -78,6 +79,14 @@ class HeadArgs(C.Structure):
     ]
 
 
+class BuildHeadArgs(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("flags", C.c_uint32), ("hidden", C.c_int32), ("reserved0", C.c_int32),
+        ("hidden_states", C.c_void_p), ("stride_row", C.c_int64), ("weight", C.c_void_p), ("stride_w", C.c_int64),
+        ("build", BuildArgs),
+    ]
+
+
 class FitArgs(C.Structure):
     _fields_ = [
         ("struct_size", C.c_uint32), ("flags", C.c_uint32), ("n_tables", C.c_int32), ("N", C.c_int32),
@@ -106,6 +115,8 @@ def lib() -> C.CDLL:
         l.cadd_head_workspace_bytes.argtypes = [C.POINTER(HeadArgs), C.POINTER(C.c_size_t)]
         l.cadd_verify_tree_fused_head.argtypes = [C.POINTER(HeadArgs), C.c_void_p]
         l.cadd_fit_cost_tables.argtypes = [C.POINTER(FitArgs), C.c_void_p]
+        l.cadd_build_head_workspace_bytes.argtypes = [C.POINTER(BuildHeadArgs), C.POINTER(C.c_size_t)]
+        l.cadd_build_tree_fused_head.argtypes = [C.POINTER(BuildHeadArgs), C.c_void_p]
         l.cadd_build_tree_static_scratch.argtypes = [C.POINTER(BuildArgs), C.c_void_p]
         _lib = l
     return _lib
@@ -188,6 +199,35 @@ def _build_args(x, K, B_max, R, flags, cost_kind) -> BuildArgs:
     return a
 
 
+def _marshal_build(a: BuildArgs, dev, batch, L, K, R, flags, theta_curve, out, l_eff, bonus_token, ctx_len, cost_coef,
+                   cost_table, table_idx, t_draft, ctx_grid):
+    """Fills the per-request inputs and the output pointers of a BuildArgs; returns (out, tensors to keep alive)."""
+    keep = [_dev(l_eff, dev, torch.int32), _dev(bonus_token, dev, torch.int32), _dev(ctx_len, dev, torch.int32),
+            _dev(cost_coef, dev, torch.float64), _dev(cost_table, dev, torch.float64),
+            _dev(table_idx, dev, torch.int32), _dev(t_draft, dev, torch.float64), _dev(ctx_grid, dev, torch.int32)]
+    a.l_eff, a.bonus_token, a.ctx_len = _ptr(keep[0]), _ptr(keep[1]), _ptr(keep[2])
+    a.cost_coef, a.cost_table, a.table_idx, a.t_draft = _ptr(keep[3]), _ptr(keep[4]), _ptr(keep[5]), _ptr(keep[6])
+    a.ctx_grid = _ptr(keep[7])
+    a.n_tables = 0 if keep[4] is None else keep[4].shape[0]
+    if out is None:
+        W = (R + 31) // 32
+        i32 = lambda *s: torch.empty(*s, dtype=torch.int32, device=dev)
+        f64 = lambda *s: torch.empty(*s, dtype=torch.float64, device=dev)
+        out = Tree(n_nodes=i32(batch), token_ids=i32(batch, R), parent_idx=i32(batch, R), depth=i32(batch, R),
+                   position_ids=i32(batch, R), node_logprob=f64(batch, R), phi=f64(batch), theta=f64(batch),
+                   mask_bits=i32(batch, R, W),
+                   mask_dense=torch.empty(batch, R, R, dtype=torch.uint8, device=dev) if flags & FLAG_EMIT_DENSE_MASK else None,
+                   topk_token=i32(batch, L, K) if flags & FLAG_EMIT_TOPK else None,
+                   topk_logprob=f64(batch, L, K) if flags & FLAG_EMIT_TOPK else None,
+                   status=i32(batch), theta_curve=f64(batch, R) if theta_curve else None)
+    a.n_nodes, a.token_ids, a.parent_idx, a.depth = _ptr(out.n_nodes), _ptr(out.token_ids), _ptr(out.parent_idx), _ptr(out.depth)
+    a.position_ids, a.node_logprob, a.phi, a.theta = _ptr(out.position_ids), _ptr(out.node_logprob), _ptr(out.phi), _ptr(out.theta)
+    a.theta_curve = _ptr(out.theta_curve)
+    a.mask_bits, a.mask_dense = _ptr(out.mask_bits), _ptr(out.mask_dense)
+    a.topk_token, a.topk_logprob, a.status = _ptr(out.topk_token), _ptr(out.topk_logprob), _ptr(out.status)
+    return out, keep
+
+
 def cadd_build_workspace_bytes(batch: int, L: int, V: int, K: int, B_max: int, R: int, dtype: torch.dtype) -> int:
     a = BuildArgs()
     a.struct_size = C.sizeof(BuildArgs)
@@ -223,29 +263,8 @@ def cadd_build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[
     a = _build_args(x, K, B_max, R, flags, cost_kind)
     a.draft_logits = x.data_ptr()
     a.stride_b, a.stride_l = x.stride(0), x.stride(1)
-    keep = [_dev(l_eff, dev, torch.int32), _dev(bonus_token, dev, torch.int32), _dev(ctx_len, dev, torch.int32),
-            _dev(cost_coef, dev, torch.float64), _dev(cost_table, dev, torch.float64),
-            _dev(table_idx, dev, torch.int32), _dev(t_draft, dev, torch.float64), _dev(ctx_grid, dev, torch.int32)]
-    a.l_eff, a.bonus_token, a.ctx_len = _ptr(keep[0]), _ptr(keep[1]), _ptr(keep[2])
-    a.cost_coef, a.cost_table, a.table_idx, a.t_draft = _ptr(keep[3]), _ptr(keep[4]), _ptr(keep[5]), _ptr(keep[6])
-    a.ctx_grid = _ptr(keep[7])
-    a.n_tables = 0 if keep[4] is None else keep[4].shape[0]
-    if out is None:
-        W = (R + 31) // 32
-        i32 = lambda *s: torch.empty(*s, dtype=torch.int32, device=dev)
-        f64 = lambda *s: torch.empty(*s, dtype=torch.float64, device=dev)
-        out = Tree(n_nodes=i32(batch), token_ids=i32(batch, R), parent_idx=i32(batch, R), depth=i32(batch, R),
-                   position_ids=i32(batch, R), node_logprob=f64(batch, R), phi=f64(batch), theta=f64(batch),
-                   mask_bits=i32(batch, R, W),
-                   mask_dense=torch.empty(batch, R, R, dtype=torch.uint8, device=dev) if flags & FLAG_EMIT_DENSE_MASK else None,
-                   topk_token=i32(batch, L, K) if flags & FLAG_EMIT_TOPK else None,
-                   topk_logprob=f64(batch, L, K) if flags & FLAG_EMIT_TOPK else None,
-                   status=i32(batch), theta_curve=f64(batch, R) if theta_curve else None)
-    a.n_nodes, a.token_ids, a.parent_idx, a.depth = _ptr(out.n_nodes), _ptr(out.token_ids), _ptr(out.parent_idx), _ptr(out.depth)
-    a.position_ids, a.node_logprob, a.phi, a.theta = _ptr(out.position_ids), _ptr(out.node_logprob), _ptr(out.phi), _ptr(out.theta)
-    a.theta_curve = _ptr(out.theta_curve)
-    a.mask_bits, a.mask_dense = _ptr(out.mask_bits), _ptr(out.mask_dense)
-    a.topk_token, a.topk_logprob, a.status = _ptr(out.topk_token), _ptr(out.topk_logprob), _ptr(out.status)
+    out, keep = _marshal_build(a, dev, batch, L, K, R, flags, theta_curve, out, l_eff, bonus_token, ctx_len, cost_coef,
+                               cost_table, table_idx, t_draft, ctx_grid)
     if workspace is None:
         nbytes = cadd_build_workspace_bytes(batch, L, V, K, B_max, R, x.dtype)
         workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=dev)
@@ -351,6 +370,69 @@ def cadd_verify_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tenso
     if rc != OK:
         raise CaddError(rc)
     workspace.record_stream(torch.cuda.current_stream() if stream is None else stream)
+    return out
+
+
+def _build_head_args(batch, L, V, hidden, K, B_max, R, flags, cost_kind) -> BuildHeadArgs:
+    h = BuildHeadArgs()
+    h.struct_size = C.sizeof(BuildHeadArgs)
+    h.hidden = hidden
+    a = h.build
+    a.struct_size = C.sizeof(BuildArgs)
+    a.flags = flags
+    a.batch, a.L, a.V = batch, L, V
+    a.K, a.B_max, a.R = K, B_max, R
+    a.logits_dtype = DTYPE_FP32
+    a.cost_kind = cost_kind
+    return h
+
+
+def cadd_build_head_workspace_bytes(batch: int, L: int, V: int, hidden: int, K: int, B_max: int, R: int) -> int:
+    h = _build_head_args(batch, L, V, hidden, K, B_max, R, 0, COST_QUADRATIC)
+    n = C.c_size_t(0)
+    rc = lib().cadd_build_head_workspace_bytes(C.byref(h), C.byref(n))
+    if rc != OK:
+        raise CaddError(rc)
+    return int(n.value)
+
+
+def cadd_build_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor, K: int, B_max: int, R: Optional[int] = None, *,
+                               l_eff=None, bonus_token=None, ctx_len=None,
+                               cost_kind: int = COST_QUADRATIC, cost_coef=None, cost_table=None, table_idx=None,
+                               t_draft=None, ctx_grid=None, theta_curve: bool = False, flags: int = 0,
+                               out: Optional[Tree] = None, workspace: Optional[torch.Tensor] = None,
+                               stream: Optional[torch.cuda.Stream] = None) -> Tree:
+    """cadd_build_tree from the drafter's last hidden states [batch, L, hidden] and its output-projection weight
+    [V, hidden] (both bf16): the draft logits are formed on the tensor cores and consumed by the softmax statistics
+    and the top-K selection without being written to memory (Eq. 1, Algorithm 1)."""
+    hs, w = hidden_states, weight
+    if not (hs.is_cuda and w.is_cuda):
+        raise ValueError("hidden_states and weight must be CUDA tensors (there is no CPU path)")
+    if hs.dtype != torch.bfloat16 or w.dtype != torch.bfloat16:
+        raise ValueError("hidden_states and weight must be bfloat16")
+    if hs.dim() != 3 or hs.stride(2) != 1 or hs.stride(0) != hs.shape[1] * hs.stride(1):
+        raise ValueError("hidden_states must be [batch, L, hidden] with contiguous rows of equal stride")
+    if w.dim() != 2 or w.stride(1) != 1 or w.shape[1] != hs.shape[2]:
+        raise ValueError("weight must be [V, hidden] with a contiguous hidden axis")
+    dev = hs.device
+    batch, L, hidden = hs.shape
+    V = w.shape[0]
+    R = B_max + 1 if R is None else R
+    h = _build_head_args(batch, L, V, hidden, K, B_max, R, flags, cost_kind)
+    h.hidden_states, h.stride_row = hs.data_ptr(), hs.stride(1)
+    h.weight, h.stride_w = w.data_ptr(), w.stride(0)
+    out, keep = _marshal_build(h.build, dev, batch, L, K, R, flags, theta_curve, out, l_eff, bonus_token, ctx_len, cost_coef,
+                               cost_table, table_idx, t_draft, ctx_grid)
+    if workspace is None:
+        workspace = torch.empty(cadd_build_head_workspace_bytes(batch, L, V, hidden, K, B_max, R), dtype=torch.uint8, device=dev)
+    h.build.workspace, h.build.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    with torch.cuda.device(dev):
+        rc = lib().cadd_build_tree_fused_head(C.byref(h), _stream_ptr(stream))
+    if rc != OK:
+        raise CaddError(rc)
+    for t in keep + [workspace]:
+        if t is not None:
+            t.record_stream(torch.cuda.current_stream() if stream is None else stream)
     return out
 
 

@@ -10,6 +10,7 @@
 #include "verify.cuh"
 #include "head_argmax.cuh"
 #include "fit_cost.cuh"
+#include "head_softmax_topk.cuh"
 
 namespace cadd {
 
@@ -93,6 +94,30 @@ static size_t build_workspace_bytes(const BuildPlan& pl) { return (pl.partial_by
 
 using namespace cadd;
 
+// Launches the expansion + emission kernel on the per-row partial records at `partials` (S records per row).
+static int launch_expand(const cadd_build_args* a, int KP, int S, const unsigned char* partials, cudaStream_t st) {
+    const ExpandLayout lay = expand_layout(a->L, a->K, KP, S, a->B_max);
+    ExpandParams ep;
+    ep.batch = a->batch; ep.L = a->L; ep.K = a->K; ep.KP = KP; ep.S = S; ep.B_max = a->B_max; ep.R = a->R;
+    ep.flags = a->flags; ep.partials = partials;
+    ep.l_eff = a->l_eff; ep.bonus_token = a->bonus_token; ep.ctx_len = a->ctx_len;
+    ep.cost_kind = a->cost_kind; ep.cost_coef = a->cost_coef; ep.cost_table = a->cost_table;
+    ep.table_idx = a->table_idx; ep.t_draft = a->t_draft; ep.ctx_grid = a->ctx_grid; ep.n_tables = a->n_tables;
+    ep.n_nodes = a->n_nodes; ep.token_ids = a->token_ids; ep.parent_idx = a->parent_idx; ep.depth = a->depth;
+    ep.position_ids = a->position_ids; ep.node_logprob = a->node_logprob; ep.phi = a->phi; ep.theta = a->theta; ep.theta_curve = a->theta_curve;
+    ep.mask_bits = a->mask_bits; ep.mask_dense = a->mask_dense; ep.topk_token = a->topk_token;
+    ep.topk_logprob = a->topk_logprob; ep.status = a->status;
+    if (lay.total > 48 * 1024) {
+        if (cudaFuncSetAttribute(expand_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lay.total) != cudaSuccess) {
+            cudaGetLastError();
+            return CADD_ERR_LAUNCH;
+        }
+    }
+    expand_emit_kernel<<<a->batch, kThreads, lay.total, st>>>(ep);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    return CADD_OK;
+}
+
 extern "C" {
 
 int cadd_version(void) { return CADD_ABI_VERSION; }
@@ -160,25 +185,7 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
     else softmax_topk_partial_kernel<CADD_DTYPE_FP32><<<items, kThreads, topk_smem_bytes(), st>>>(tp);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
 
-    ExpandParams ep;
-    ep.batch = a->batch; ep.L = a->L; ep.K = a->K; ep.KP = pl.KP; ep.S = pl.S; ep.B_max = a->B_max; ep.R = a->R;
-    ep.flags = a->flags; ep.partials = (const unsigned char*)a->workspace;
-    ep.l_eff = a->l_eff; ep.bonus_token = a->bonus_token; ep.ctx_len = a->ctx_len;
-    ep.cost_kind = a->cost_kind; ep.cost_coef = a->cost_coef; ep.cost_table = a->cost_table;
-    ep.table_idx = a->table_idx; ep.t_draft = a->t_draft; ep.ctx_grid = a->ctx_grid; ep.n_tables = a->n_tables;
-    ep.n_nodes = a->n_nodes; ep.token_ids = a->token_ids; ep.parent_idx = a->parent_idx; ep.depth = a->depth;
-    ep.position_ids = a->position_ids; ep.node_logprob = a->node_logprob; ep.phi = a->phi; ep.theta = a->theta; ep.theta_curve = a->theta_curve;
-    ep.mask_bits = a->mask_bits; ep.mask_dense = a->mask_dense; ep.topk_token = a->topk_token;
-    ep.topk_logprob = a->topk_logprob; ep.status = a->status;
-    if (pl.lay.total > 48 * 1024) {
-        if (cudaFuncSetAttribute(expand_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.lay.total) != cudaSuccess) {
-            cudaGetLastError();
-            return CADD_ERR_LAUNCH;
-        }
-    }
-    expand_emit_kernel<<<a->batch, kThreads, pl.lay.total, st>>>(ep);
-    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
-    return CADD_OK;
+    return launch_expand(a, pl.KP, pl.S, (const unsigned char*)a->workspace, st);
 }
 
 static int check_verify_shape(const cadd_verify_args* a) {
@@ -362,6 +369,113 @@ int cadd_fit_cost_tables(const cadd_fit_args* a, void* cuda_stream) {
     fit_cost_kernel<<<a->n_tables, kFitThreads, fit_smem_bytes(), (cudaStream_t)cuda_stream>>>(fp);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
     return CADD_OK;
+}
+
+// ---------------- tree construction fused into the drafter's output projection ----------------
+
+struct DraftPlan {
+    int KP, m_tiles, n_tiles, chunk_tiles, n_chunks;
+    size_t chunk_bytes, merged_bytes, total_bytes;
+};
+// Chunks of column tiles per row: at most 64 (the merge kernel walks two lists per lane), chosen so that the number
+// of work items (row tiles x chunks) fills whole waves of one CTA per SM as evenly as possible.
+static DraftPlan plan_draft_head(const cadd_build_args* a, int sms) {
+    DraftPlan pl;
+    pl.KP = a->K > kPreciseMin ? a->K : kPreciseMin;
+    const int64_t M = (int64_t)a->batch * a->L;
+    pl.m_tiles = (int)((M + kHeadBM - 1) / kHeadBM);
+    pl.n_tiles = (int)((a->V + kHeadBN - 1) / kHeadBN);
+    int best = 1;
+    double best_eff = -1.0;
+    const int cap = pl.n_tiles < 64 ? pl.n_tiles : 64;
+    for (int nc = 1; nc <= cap; ++nc) {
+        const int ct = (pl.n_tiles + nc - 1) / nc;
+        const int real = (pl.n_tiles + ct - 1) / ct;                       // chunks that actually exist with this size
+        const int64_t items = (int64_t)pl.m_tiles * real;
+        const int64_t waves = (items + sms - 1) / sms;
+        const double eff = (double)items / (double)(waves * sms);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = real; }
+    }
+    pl.chunk_tiles = (pl.n_tiles + best - 1) / best;
+    pl.n_chunks = (pl.n_tiles + pl.chunk_tiles - 1) / pl.chunk_tiles;
+    const size_t stride = seg_partial_stride(pl.KP);
+    pl.chunk_bytes = (((size_t)M * pl.n_chunks * stride) + 255) & ~(size_t)255;
+    pl.merged_bytes = (((size_t)M * stride) + 255) & ~(size_t)255;
+    pl.total_bytes = pl.chunk_bytes + pl.merged_bytes + 256;
+    return pl;
+}
+
+static int check_build_head(const cadd_build_head_args* h) {
+    if (!h) return CADD_ERR_NULL;
+    if (h->struct_size != sizeof(cadd_build_head_args)) return CADD_ERR_STRUCT_SIZE;
+    int rc = check_build_shape(&h->build);
+    if (rc != CADD_OK) return rc;
+    if (h->hidden < 1 || h->hidden > (1 << 20) || h->build.K > kDraftMaxKP) return CADD_ERR_SHAPE;
+    return CADD_OK;
+}
+
+int cadd_build_head_workspace_bytes(const cadd_build_head_args* h, size_t* out) {
+    int rc = check_build_head(h);
+    if (rc != CADD_OK) return rc;
+    if (!out) return CADD_ERR_NULL;
+    // sized for the largest cut (64 chunks per row), so the answer does not depend on the device
+    const size_t stride = seg_partial_stride(h->build.K > kPreciseMin ? h->build.K : kPreciseMin);
+    const size_t M = (size_t)h->build.batch * h->build.L;
+    *out = ((M * 64 * stride + 255) & ~(size_t)255) + ((M * stride + 255) & ~(size_t)255) + 256;
+    return CADD_OK;
+}
+
+int cadd_build_tree_fused_head(const cadd_build_head_args* h, void* cuda_stream) {
+    int rc = check_build_head(h);
+    if (rc != CADD_OK) return rc;
+    const cadd_build_args* a = &h->build;
+    if (!h->hidden_states || !h->weight || !a->n_nodes || !a->token_ids || !a->parent_idx || !a->depth) return CADD_ERR_NULL;
+    if (a->cost_kind == CADD_COST_QUADRATIC && !a->cost_coef) return CADD_ERR_NULL;
+    if (a->cost_kind == CADD_COST_TABLE && (!a->cost_table || !a->table_idx || !a->t_draft || a->n_tables < 1)) return CADD_ERR_NULL;
+    if (a->cost_kind == CADD_COST_TABLE_INTERP && (!a->cost_table || !a->ctx_grid || !a->t_draft || a->n_tables < 1)) return CADD_ERR_NULL;
+    if ((a->flags & CADD_FLAG_EMIT_DENSE_MASK) && !a->mask_dense) return CADD_ERR_NULL;
+    if ((a->flags & CADD_FLAG_EMIT_TOPK) && !a->topk_token && !a->topk_logprob) return CADD_ERR_NULL;
+    if (!aligned(h->hidden_states, 16) || !aligned(h->weight, 16) || h->stride_row % 8 != 0 || h->stride_w % 8 != 0) return CADD_ERR_ALIGN;
+    if (h->stride_row < h->hidden || h->stride_w < h->hidden) return CADD_ERR_SHAPE;
+    if (!aligned(a->cost_coef, 8) || !aligned(a->cost_table, 8) || !aligned(a->t_draft, 8) || !aligned(a->node_logprob, 8) ||
+        !aligned(a->phi, 8) || !aligned(a->theta, 8) || !aligned(a->theta_curve, 8) || !aligned(a->topk_logprob, 8))
+        return CADD_ERR_ALIGN;
+    if (!aligned(a->n_nodes, 4) || !aligned(a->token_ids, 4) || !aligned(a->parent_idx, 4) || !aligned(a->depth, 4) ||
+        !aligned(a->position_ids, 4) || !aligned(a->mask_bits, 4) || !aligned(a->topk_token, 4) || !aligned(a->status, 4) ||
+        !aligned(a->l_eff, 4) || !aligned(a->bonus_token, 4) || !aligned(a->ctx_len, 4) || !aligned(a->table_idx, 4) ||
+        !aligned(a->ctx_grid, 4))
+        return CADD_ERR_ALIGN;
+    const int sms = sm_count();
+    const DraftPlan pl = plan_draft_head(a, sms);
+    size_t need = 0;
+    cadd_build_head_workspace_bytes(h, &need);
+    if (!a->workspace || !aligned(a->workspace, 256) || a->workspace_bytes < need) return CADD_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    const int64_t M = (int64_t)a->batch * a->L;
+    CUtensorMap map_h, map_w;
+    if (!make_map_bf16(&map_h, h->hidden_states, M, h->hidden, h->stride_row, kHeadBM) ||
+        !make_map_bf16(&map_w, h->weight, a->V, h->hidden, h->stride_w, kHeadBN))
+        return CADD_ERR_LAUNCH;
+    unsigned char* ws = (unsigned char*)a->workspace;
+    unsigned char* merged = ws + pl.chunk_bytes;
+    int32_t* err = (int32_t*)(ws + pl.chunk_bytes + pl.merged_bytes);
+    if (cudaMemsetAsync(err, 0, 256, st) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+
+    DraftHeadParams dp;
+    dp.M = M; dp.V = a->V; dp.Kdim = h->hidden; dp.m_tiles = pl.m_tiles; dp.n_tiles = pl.n_tiles;
+    dp.chunk_tiles = pl.chunk_tiles; dp.n_chunks = pl.n_chunks; dp.L = a->L; dp.KP = pl.KP; dp.l_eff = a->l_eff;
+    dp.chunk_partials = ws; dp.error = err;
+    if (cudaFuncSetAttribute(head_softmax_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)draft_head_smem_bytes()) != cudaSuccess) {
+        cudaGetLastError();
+        return CADD_ERR_LAUNCH;
+    }
+    const int64_t items = (int64_t)pl.m_tiles * pl.n_chunks;
+    head_softmax_topk_kernel<<<(unsigned)(items < sms ? items : sms), kHeadThreads, draft_head_smem_bytes(), st>>>(map_h, map_w, dp);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    draft_merge_kernel<<<(unsigned)((M + 3) / 4), 128, 0, st>>>(dp, merged);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    return launch_expand(a, pl.KP, 1, merged, st);
 }
 
 }  // extern "C"

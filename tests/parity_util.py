@@ -23,8 +23,11 @@ def to_cpu(t):
     return None if t is None else t.detach().cpu()
 
 
-def compare_build(gt: G.Tree, ot: O.OracleTree, K: int, check_topk: bool = True):
-    """Returns a dict of diagnostics; raises AssertionError on a parity failure."""
+def compare_build(gt: G.Tree, ot: O.OracleTree, K: int, check_topk: bool = True, rel_tol: float = None, near_tie: float = None):
+    """Returns a dict of diagnostics; raises AssertionError on a parity failure.  rel_tol / near_tie override the
+    module's bars for paths whose logits themselves carry a stated rounding error (the fused output projection)."""
+    REL_TOL_ = REL_TOL if rel_tol is None else rel_tol
+    NEAR_TIE_ = NEAR_TIE if near_tie is None else near_tie
     n_g, n_o = to_cpu(gt.n_nodes).numpy(), ot.n_nodes.numpy()
     batch, R = ot.token_ids.shape
     tok_g, par_g, dep_g = to_cpu(gt.token_ids).numpy(), to_cpu(gt.parent_idx).numpy(), to_cpu(gt.depth).numpy()
@@ -46,7 +49,7 @@ def compare_build(gt: G.Tree, ot: O.OracleTree, K: int, check_topk: bool = True)
             assert st_g[b] == st_o[b], f"status differs (request {b}): gpu {st_g[b]} oracle {st_o[b]}"
             assert np.array_equal(pos_g[b], pos_o[b]), f"position ids differ (request {b})"
             assert np.array_equal(mb_g[b], mb_o[b]), f"mask differs (request {b})"
-            np.testing.assert_allclose(np.exp(lp_g[b]), np.exp(lp_o[b]), rtol=REL_TOL, err_msg=f"node prob (request {b})")
+            np.testing.assert_allclose(np.exp(lp_g[b]), np.exp(lp_o[b]), rtol=REL_TOL_, err_msg=f"node prob (request {b})")
         else:
             # admissible only if the oracle's own decision at the first difference was a near-tie
             if not same_rows:
@@ -56,11 +59,11 @@ def compare_build(gt: G.Tree, ot: O.OracleTree, K: int, check_topk: bool = True)
             else:
                 margin = float(ot.stop_gap[b])
                 what = "stop test"
-            assert margin < NEAR_TIE, (f"request {b}: trees differ at {what} but the oracle's margin there is "
-                                       f"{margin:.3e} >= {NEAR_TIE}")
+            assert margin < NEAR_TIE_, (f"request {b}: trees differ at {what} but the oracle's margin there is "
+                                       f"{margin:.3e} >= {NEAR_TIE_}")
             exempt.append((b, what, margin))
-        np.testing.assert_allclose(phi_g[b], phi_o[b], rtol=REL_TOL, err_msg=f"Phi (request {b})")
-        np.testing.assert_allclose(th_g[b], th_o[b], rtol=REL_TOL, err_msg=f"theta (request {b})")
+        np.testing.assert_allclose(phi_g[b], phi_o[b], rtol=REL_TOL_, err_msg=f"Phi (request {b})")
+        np.testing.assert_allclose(th_g[b], th_o[b], rtol=REL_TOL_, err_msg=f"theta (request {b})")
     diag = {"exempt": exempt, "max_logprob_err": float(np.max(np.abs(np.where(tok_o >= 0, lp_g - lp_o, 0.0)))) if not exempt else None}
     if check_topk and gt.topk_token is not None:
         tt_g, tt_o = to_cpu(gt.topk_token).numpy(), ot.topk_token.numpy()
@@ -70,7 +73,7 @@ def compare_build(gt: G.Tree, ot: O.OracleTree, K: int, check_topk: bool = True)
         assert np.array_equal(np.isfinite(tl_g), fin)
         err = np.abs(tl_g[fin] - tl_o[fin])
         diag["max_logZ_err"] = float(err.max()) if err.size else 0.0
-        np.testing.assert_allclose(np.exp(tl_g[fin]), np.exp(tl_o[fin]), rtol=REL_TOL)
+        np.testing.assert_allclose(np.exp(tl_g[fin]), np.exp(tl_o[fin]), rtol=REL_TOL_)
     return diag
 
 

@@ -5,7 +5,7 @@ import torch
 from oracle import cadd_oracle as O
 from paper_2606_01813_b200 import binding as G
 from paper_2606_01813_b200 import synth
-from parity_util import to_cpu
+from parity_util import compare_build, to_cpu
 
 pytestmark = pytest.mark.gpu
 
@@ -138,3 +138,72 @@ def test_fused_head_full_size_sampled_rows():
         if o != gpick:
             tol = hidden * 2.0 ** -24 * float((hs[0, i].double().abs() * absw[[o, gpick]]).sum(dim=1).max())
             assert abs(float(y64[i, o] - y64[i, gpick])) <= tol, (r, o, gpick)
+
+
+# ---------------- tree construction fused into the drafter's output projection ----------------
+
+def planted_draft_inputs(batch, L, hidden, V, seed, sigma=1.5):
+    """Hidden states whose logits h . W^T are N(0, sigma^2) noise plus one boosted token per position."""
+    g = torch.Generator().manual_seed(seed)
+    w = torch.randn(V, hidden, generator=g)
+    h = torch.randn(batch, L, hidden, generator=g) * (sigma / hidden ** 0.5)
+    for b in range(batch):
+        for i in range(L):
+            t = int(torch.randint(V, (), generator=g))
+            boost = float(4.0 + 6.0 * torch.rand((), generator=g)) * 0.9 ** i
+            h[b, i] += boost * w[t] / float(w[t] @ w[t])
+    return h.bfloat16(), w.bfloat16()
+
+
+def check_fused_build(h, w, cfg, seed, **extra):
+    c = synth.make_cost_inputs(cfg, seed)
+    fixed = extra.pop("flags", 0)
+    kw = dict(cost_coef=c.coef, **extra)
+    ot, y64 = O.build_tree_fused_head(h, w, cfg.K, cfg.B_max, cfg.R, flags=fixed, **kw)
+    gt = G.cadd_build_tree_fused_head(h.cuda(), w.cuda(), cfg.K, cfg.B_max, cfg.R, flags=G.FLAG_EMIT_TOPK | fixed,
+                                      **{k: (v.cuda() if torch.is_tensor(v) else v) for k, v in kw.items()})
+    torch.cuda.synchronize()
+    # a logit is an fp32 accumulation of `hidden` products: |error| <= e = hidden * 2^-24 * sum_k |h_k W_vk| in the
+    # worst case; a log-prob (logit - log Z) then carries at most 2e, a score over L depths at most 2 L e
+    absdot = h.double().abs().reshape(-1, h.shape[2]) @ w.double().abs().T
+    e = h.shape[2] * 2.0 ** -24 * float(absdot.max())
+    diag = compare_build(gt, ot, cfg.K, check_topk=False, rel_tol=1e-5 + 2 * cfg.L * 2 * e, near_tie=max(1e-6, 2 * cfg.L * 2 * e))
+    # top-K: token ids equal unless the oracle's own gap at the K-th place is inside the bound
+    tt_g, tt_o = gt.topk_token.cpu(), ot.topk_token
+    mism = (tt_g != tt_o).any(dim=-1)
+    y = y64.reshape(-1, y64.shape[-1])
+    for r in torch.nonzero(mism.reshape(-1)).flatten().tolist():
+        top = torch.sort(y[r], descending=True).values[: cfg.K + 1]
+        assert float((top[:-1] - top[1:]).min()) <= 2 * e, f"row {r}: top-K differs without a near-tie"
+    lg, lo = gt.topk_logprob.cpu()[~mism], ot.topk_logprob[~mism]
+    fin = torch.isfinite(lo)                                   # masked positions and short lists carry no log-probs
+    assert torch.equal(torch.isfinite(lg), fin)
+    if fin.any():
+        assert float((lg[fin] - lo[fin]).abs().max()) <= 2 * e + 1e-7
+    return diag, int(mism.sum()), ot
+
+
+@pytest.mark.parametrize("shape", [
+    # batch, L, hidden, V, K
+    (1, 4, 64, 300, 4),
+    (2, 16, 256, 4099, 8),
+    (3, 16, 200, 20000, 16),
+    (9, 16, 512, 2500, 32),      # 144 rows: two row tiles, the second ragged
+])
+def test_fused_draft_head_small(shape):
+    batch, L, hidden, V, K = shape
+    cfg = synth.scaled(synth.CONFIGS["c2"], batch=batch, L=L, V=V, K=K, B_max=64)
+    h, w = planted_draft_inputs(batch, L, hidden, V, seed=hidden)
+    diag, mism, ot = check_fused_build(h, w, cfg, 3)
+    assert len(diag["exempt"]) <= 1 and mism <= 1
+    assert int(ot.n_nodes.max()) >= 2
+
+
+def test_fused_draft_head_masked_positions_and_fixed_budget():
+    batch, L, hidden, V = 5, 16, 128, 3000
+    cfg = synth.scaled(synth.CONFIGS["c5"], batch=batch, L=L, V=V, K=8, B_max=96)
+    h, w = planted_draft_inputs(batch, L, hidden, V, seed=31)
+    l_eff = torch.tensor([4, 16, 0, 9, 1], dtype=torch.int32)
+    bonus = torch.arange(batch, dtype=torch.int32)
+    diag, mism, ot = check_fused_build(h, w, cfg, 4, l_eff=l_eff, bonus_token=bonus, flags=O.FLAG_FIXED_BUDGET)
+    assert int(ot.n_nodes[2]) == 0 and int(ot.n_nodes.max()) == 96
