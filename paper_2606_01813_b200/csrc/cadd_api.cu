@@ -377,7 +377,7 @@ struct DraftPlan {
     int KP, m_tiles, n_tiles, chunk_tiles, n_chunks;
     size_t chunk_bytes, merged_bytes, total_bytes;
 };
-// Chunks of column tiles per row: at most 64 (the merge kernel walks two lists per lane), chosen so that the number
+// Chunks of column tiles per row: at most 32 (two records each; the merge kernel walks two lists per lane), chosen so that the number
 // of work items (row tiles x chunks) fills whole waves of one CTA per SM as evenly as possible.
 static DraftPlan plan_draft_head(const cadd_build_args* a, int sms) {
     DraftPlan pl;
@@ -387,7 +387,7 @@ static DraftPlan plan_draft_head(const cadd_build_args* a, int sms) {
     pl.n_tiles = (int)((a->V + kHeadBN - 1) / kHeadBN);
     int best = 1;
     double best_eff = -1.0;
-    const int cap = pl.n_tiles < 64 ? pl.n_tiles : 64;
+    const int cap = pl.n_tiles < 32 ? pl.n_tiles : 32;               // two records per chunk, at most 64 per row
     for (int nc = 1; nc <= cap; ++nc) {
         const int ct = (pl.n_tiles + nc - 1) / nc;
         const int real = (pl.n_tiles + ct - 1) / ct;                       // chunks that actually exist with this size
@@ -399,7 +399,7 @@ static DraftPlan plan_draft_head(const cadd_build_args* a, int sms) {
     pl.chunk_tiles = (pl.n_tiles + best - 1) / best;
     pl.n_chunks = (pl.n_tiles + pl.chunk_tiles - 1) / pl.chunk_tiles;
     const size_t stride = seg_partial_stride(pl.KP);
-    pl.chunk_bytes = (((size_t)M * pl.n_chunks * stride) + 255) & ~(size_t)255;
+    pl.chunk_bytes = (((size_t)M * pl.n_chunks * 2 * stride) + 255) & ~(size_t)255;
     pl.merged_bytes = (((size_t)M * stride) + 255) & ~(size_t)255;
     pl.total_bytes = pl.chunk_bytes + pl.merged_bytes + 256;
     return pl;
@@ -418,7 +418,7 @@ int cadd_build_head_workspace_bytes(const cadd_build_head_args* h, size_t* out) 
     int rc = check_build_head(h);
     if (rc != CADD_OK) return rc;
     if (!out) return CADD_ERR_NULL;
-    // sized for the largest cut (64 chunks per row), so the answer does not depend on the device
+    // sized for the largest cut (32 chunks = 64 records per row), so the answer does not depend on the device
     const size_t stride = seg_partial_stride(h->build.K > kPreciseMin ? h->build.K : kPreciseMin);
     const size_t M = (size_t)h->build.batch * h->build.L;
     *out = ((M * 64 * stride + 255) & ~(size_t)255) + ((M * stride + 255) & ~(size_t)255) + 256;
@@ -471,7 +471,7 @@ int cadd_build_tree_fused_head(const cadd_build_head_args* h, void* cuda_stream)
         return CADD_ERR_LAUNCH;
     }
     const int64_t items = (int64_t)pl.m_tiles * pl.n_chunks;
-    head_softmax_topk_kernel<<<(unsigned)(items < sms ? items : sms), kHeadThreads, draft_head_smem_bytes(), st>>>(map_h, map_w, dp);
+    head_softmax_topk_kernel<<<(unsigned)(items < sms ? items : sms), kDraftThreads, draft_head_smem_bytes(), st>>>(map_h, map_w, dp);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
     draft_merge_kernel<<<(unsigned)((M + 3) / 4), 128, 0, st>>>(dp, merged);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;

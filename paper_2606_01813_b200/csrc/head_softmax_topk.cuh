@@ -3,7 +3,9 @@
 // The logits l_i = h_i . W^T are formed tile by tile on the tensor cores exactly as in head_argmax.cuh (same TMA
 // ring, same tcgen05.mma issue, accumulators in tensor memory); the epilogue turns every row of a tile into running
 // softmax / top-K state instead of a single maximum:
-//   - the KP best (logit, token) pairs of the row so far, a sorted list per row in shared memory;
+//   - the KP best (logit, token) pairs of the row so far, a small unsorted list per row in shared memory with its
+//     smallest entry cached; elements that reach the threshold are queued per row and folded into the list by the
+//     whole warp at once, so the rare list update does not split the warp element by element;
 //   - W = sum over all other elements of 2^(x*log2e - C) with an integer reference exponent C, accumulated in fp64
 //     from fp32 exponentials (ex2.approx), the same split as in softmax_topk.cuh: the KP best are never put through
 //     the fp32 exponential.
@@ -18,9 +20,23 @@ namespace cadd {
 
 constexpr int kDraftMaxKP = 32;           // list capacity per row that fits beside the operand ring in shared memory
 
+constexpr int kDraftStages = 3;           // operand ring: one stage fewer than head_argmax.cuh, the room goes to the row state
+constexpr int kDraftPending = 8;          // queued candidates per row and column half between two list updates
+constexpr int kDraftThreads = 320;        // producer warp, MMA warp, eight epilogue warps
+
 struct DraftHeadShared {
-    HeadShared g;                                          // operand ring, barriers (head_argmax.cuh)
-    uint64_t list[kDraftMaxKP][kHeadBM];                   // list[k][row of the tile]: k-th best key of the row so far
+    alignas(1024) unsigned char a[kDraftStages][kHeadABytes];
+    alignas(1024) unsigned char b[kDraftStages][kHeadBBytes];
+    // Two epilogue warps share each group of 32 rows and split the tile's columns in halves; each half keeps its own
+    // row state and leaves its own record.
+    uint64_t list[2][kDraftMaxKP][kHeadBM];                // list[half][k][row of the tile]: the row's KP best keys so far, unsorted
+    uint64_t pend[2][kDraftPending][kHeadBM];              // candidates waiting for the next list update
+    alignas(8) uint64_t full[kDraftStages];
+    uint64_t empty[kDraftStages];
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint32_t tmem_base;
+    uint32_t error;
 };
 inline size_t draft_head_smem_bytes() { return sizeof(DraftHeadShared) + 1024; }
 
@@ -33,7 +49,7 @@ struct DraftHeadParams {
     int n_chunks;              // chunks per row = ceil(n_tiles / chunk_tiles)
     int L, KP;
     const int32_t* l_eff;      // [batch] or NULL
-    unsigned char* chunk_partials;   // [M * n_chunks] records of seg_partial_stride(KP) bytes
+    unsigned char* chunk_partials;   // [M * n_chunks * 2] records of seg_partial_stride(KP) bytes (two column halves per chunk)
     int32_t* error;
 };
 
@@ -53,19 +69,18 @@ __device__ __forceinline__ bool draft_tile_live(const DraftHeadParams& p, int mt
     return false;
 }
 
-__global__ void __launch_bounds__(kHeadThreads, 1)
+__global__ void __launch_bounds__(kDraftThreads, 1)
 head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, DraftHeadParams p) {
     extern __shared__ __align__(16) unsigned char head_smem_raw[];
-    DraftHeadShared& dsh = *reinterpret_cast<DraftHeadShared*>(head_smem_raw + ((1024u - (smem_u32(head_smem_raw) & 1023u)) & 1023u));
-    HeadShared& sh = dsh.g;
+    DraftHeadShared& sh = *reinterpret_cast<DraftHeadShared*>(head_smem_raw + ((1024u - (smem_u32(head_smem_raw) & 1023u)) & 1023u));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int k_steps = (p.Kdim + kHeadBK - 1) / kHeadBK;
     const int64_t n_items = (int64_t)p.m_tiles * p.n_chunks;      // item w -> (chunk = w / m_tiles, row tile = w % m_tiles)
     const int KP = p.KP;
 
     if (tid == 0) {
-        for (int s = 0; s < kHeadStages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&sh.acc_full[s], 1); mbar_init(&sh.acc_empty[s], 4); }
+        for (int s = 0; s < kDraftStages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sh.acc_full[s], 1); mbar_init(&sh.acc_empty[s], 8); }
         sh.error = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -89,7 +104,7 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
                         mbar_arrive_expect_tx(&sh.full[s], kHeadABytes + kHeadBBytes);
                         tma_load_2d(&sh.a[s][0], &map_h, k * kHeadBK, mt * kHeadBM, &sh.full[s]);
                         tma_load_2d(&sh.b[s][0], &map_w, k * kHeadBK, nt * kHeadBN, &sh.full[s]);
-                        if (++s == kHeadStages) { s = 0; ph ^= 1u; }
+                        if (++s == kDraftStages) { s = 0; ph ^= 1u; }
                     }
             }
         }
@@ -114,7 +129,7 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
                             umma_bf16(d, umma_desc_k_sw128(&sh.a[s][0], kk), umma_desc_k_sw128(&sh.b[s][0], kk), kHeadIdesc,
                                       (k | kk) != 0 ? 1u : 0u);
                         umma_commit(&sh.empty[s]);
-                        if (++s == kHeadStages) { s = 0; ph ^= 1u; }
+                        if (++s == kDraftStages) { s = 0; ph ^= 1u; }
                     }
                     if (!ok) break;
                     umma_commit(&sh.acc_full[buf]);
@@ -123,8 +138,9 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
             }
         }
     } else {
-        // ---------------- epilogue: warps 2..5; thread = one row of the tile ----------------
-        const int quarter = warp & 3;
+        // ---------------- epilogue: warps 2..9; thread = one row of the tile, one half of its columns ----------------
+        const int quarter = warp & 3;                            // tensor-memory lane quarter this warp may read
+        const int half = (warp - 2) >> 2;                        // columns [half * 128, half * 128 + 128) of every tile
         const int trow = quarter * 32 + lane;                    // row inside the tile = tensor-memory lane
         unsigned buf = 0, aph = 0;
         for (int64_t w = blockIdx.x; w < n_items && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
@@ -136,55 +152,103 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
             ThreadSum s{0.0, -INFINITY, 0.0f};
             uint32_t flags = 0;
             int cnt = 0;                                          // entries in the row's list
-            float thr = -INFINITY;                                // value of the list's last entry once it is full
-            uint64_t thr_key = 0;
+            float thr = -INFINITY;                                // hit test: value of the list's smallest entry at the last update
+            uint64_t thr_key = 0;                                 // the smallest entry itself (list full), at slot min_pos
+            int min_pos = 0;
+            int np = 0;                                           // queued candidates
+            // Folds the queue into the list.  It runs once per tile for all lanes together (lanes with fewer entries
+            // idle), and otherwise only when a lane's queue is full, so the rare, expensive list update does not split
+            // the warp element by element.  The list is unsorted with its smallest entry cached: a better key
+            // overwrites that slot and one scan finds the next smallest; whatever drops out, or never makes it in,
+            // joins the sum.
+            auto drain = [&]() {
+                for (int j = 0; j < np; ++j) {
+                    const uint64_t key = sh.pend[half][j][trow];
+                    if (cnt < KP) {
+                        sh.list[half][cnt][trow] = key;
+                        ++cnt;
+                        if (cnt < KP) continue;
+                    } else if (key > thr_key) {
+                        s.acc += (double)exp2_term(key_value(thr_key), s.negc);
+                        sh.list[half][min_pos][trow] = key;
+                    } else {
+                        s.acc += (double)exp2_term(key_value(key), s.negc);
+                        continue;
+                    }
+                    uint64_t mk = ~0ull;
+                    int mp = 0;
+#pragma unroll 4
+                    for (int k = 0; k < KP; ++k) {
+                        const uint64_t v = sh.list[half][k][trow];
+                        if (v < mk) { mk = v; mp = k; }
+                    }
+                    thr_key = mk; min_pos = mp;
+                    const float tv = key_value(mk);
+                    if (tv > s.tmax + 60.0f || s.tmax == -INFINITY) raise_reference(s, tv);   // keeps 2^(x*log2e - c) in range below tv
+                }
+                np = 0;
+                if (cnt == KP) thr = key_value(thr_key);
+            };
             const int nt1 = min((ch + 1) * p.chunk_tiles, p.n_tiles);
             bool ok = true;
             for (int nt = ch * p.chunk_tiles; nt < nt1 && ok; ++nt) {
                 if (!__all_sync(kFullMask, head_wait(&sh.acc_full[buf], aph, 256))) { sh.error = 4; ok = false; break; }
                 tc_fence_after();
-                const int64_t col0 = (int64_t)nt * kHeadBN;
+                const int64_t col0 = (int64_t)nt * kHeadBN + half * (kHeadBN / 2);
+                // 32 columns per tensor-memory load (narrow loads have the same latency, about 2 k cycles while the
+                // tensor cores run the next tile), the next 32 already on their way.  Pass 1 is branch-free: every
+                // element below the threshold adds its exponential, the others set a bit.  Pass 2 runs only while
+                // some lane has bits left: it queues them (or sums them, if a list update has raised the threshold
+                // meanwhile); when a lane's queue is full the whole warp folds its queues into the lists and pass 2
+                // repeats.
+                const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kHeadBN + half * (kHeadBN / 2);
+                uint32_t r[32], rn[32];
+                tmem_ld32(tbase, r);
+                tmem_ld_wait();
 #pragma unroll 1
-                for (int c = 0; c < kHeadBN / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kHeadBN + c * 32, r);
-                    tmem_ld_wait();
+                for (int c = 0; c < kHeadBN / 64; ++c) {
+                    if (c + 1 < kHeadBN / 64) tmem_ld32(tbase + (c + 1) * 32, rn);
                     const int64_t cb = col0 + c * 32;
                     float part = 0.0f;                            // fp32 sum of this run of 32 columns
+                    unsigned hit = 0;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {                 // fully unrolled: r[] must stay in registers
+                    for (int i = 0; i < 32; ++i) {
                         const float x = __uint_as_float(r[i]);
-                        if (cb + i >= p.V || !live) continue;
-                        if (x < thr) { part += exp2_term(x, s.negc); continue; }      // the common case
-                        const uint32_t bits = __float_as_uint(x);
-                        if ((bits & 0x7f800000u) == 0x7f800000u) {                    // Inf or NaN: no mass, never a candidate
-                            if (bits != 0xff800000u) flags |= kPartNonfinite;
-                            if (bits == 0x7f800000u) flags |= kPartPosInf;
-                            continue;
-                        }
-                        const uint64_t key = make_key(x, (uint32_t)(cb + i));
-                        if (cnt == KP && key < thr_key) { part += exp2_term(x, s.negc); continue; }   // ties with the last entry
-                        // insert into the sorted list; when it is full the last entry drops out and joins the sum
-                        if (cnt == KP) {
-                            s.acc += (double)part; part = 0.0f;
-                            fold_scalar(s, key_value(dsh.list[KP - 1][trow]));
-                        } else {
-                            ++cnt;
-                        }
-                        int k = cnt - 1;
-                        while (k > 0 && dsh.list[k - 1][trow] < key) { dsh.list[k][trow] = dsh.list[k - 1][trow]; --k; }
-                        dsh.list[k][trow] = key;
-                        if (cnt == KP) {
-                            thr_key = dsh.list[KP - 1][trow];
-                            thr = key_value(thr_key);
-                            if (thr > s.tmax + 60.0f || s.tmax == -INFINITY) {       // keep 2^(x*log2e - c) in range for x < thr
-                                s.acc += (double)part; part = 0.0f;
-                                raise_reference(s, thr);
-                            }
-                        }
+                        const bool valid = live && cb + i < p.V;
+                        const bool fast = valid && x < thr;
+                        part += exp2_term(fast ? x : -INFINITY, s.negc);              // 2^-inf = 0
+                        hit |= (valid && !fast) ? (1u << i) : 0u;
                     }
                     s.acc += (double)part;
+                    while (__any_sync(kFullMask, hit != 0)) {
+                        float part2 = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            if (hit & (1u << i)) {
+                                const float x = __uint_as_float(r[i]);
+                                const uint32_t bits = __float_as_uint(x);
+                                if ((bits & 0x7f800000u) == 0x7f800000u) {            // Inf or NaN: no mass, never a candidate
+                                    if (bits != 0xff800000u) flags |= kPartNonfinite;
+                                    if (bits == 0x7f800000u) flags |= kPartPosInf;
+                                    hit &= ~(1u << i);
+                                } else if (x < thr) {                                 // the threshold has risen since pass 1
+                                    part2 += exp2_term(x, s.negc);
+                                    hit &= ~(1u << i);
+                                } else if (np < kDraftPending) {
+                                    sh.pend[half][np][trow] = make_key(x, (uint32_t)(cb + i));
+                                    ++np;
+                                    hit &= ~(1u << i);
+                                }
+                            }
+                        }
+                        s.acc += (double)part2;
+                        if (__any_sync(kFullMask, hit != 0)) drain();                 // a queue is full: fold, then go on
+                    }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = rn[i];
                 }
+                drain();                                          // the accumulator's last candidates, then release it
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.acc_empty[buf]);
@@ -192,9 +256,14 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
             }
             if (!ok) break;
             if (live) {
-                unsigned char* rec = p.chunk_partials + ((size_t)row * p.n_chunks + ch) * seg_partial_stride(KP);
+                unsigned char* rec = p.chunk_partials + (((size_t)row * p.n_chunks + ch) * 2 + half) * seg_partial_stride(KP);
                 uint64_t* out_keys = (uint64_t*)(rec + sizeof(SegPartial));
-                for (int k = 0; k < cnt; ++k) out_keys[k] = dsh.list[k][trow];
+                for (int k = 0; k < cnt; ++k) {                     // rank by counting (keys are unique): sorted, best first
+                    const uint64_t v = sh.list[half][k][trow];
+                    int rank = 0;
+                    for (int j = 0; j < cnt; ++j) rank += sh.list[half][j][trow] > v;
+                    out_keys[rank] = v;
+                }
                 SegPartial h;
                 h.W = s.acc * kEx2BiasFix; h.C = s.acc != 0.0 ? (double)(-s.negc) : 0.0; h.cnt = cnt;
                 h.flags = flags; h.pad[0] = h.pad[1] = 0;
@@ -222,7 +291,7 @@ __global__ void __launch_bounds__(128) draft_merge_kernel(DraftHeadParams p, uns
     const int KP = p.KP;
     const size_t stride = seg_partial_stride(KP);
     const double kLog2e = 1.4426950408889634;
-    // lane owns chunks lane and lane + 32
+    // lane owns records lane and lane + 32 (at most 64 per row)
     const SegPartial* hdr[2];
     const uint64_t* keys[2];
     int cnt[2], cur[2] = {0, 0};
@@ -230,9 +299,9 @@ __global__ void __launch_bounds__(128) draft_merge_kernel(DraftHeadParams p, uns
     uint32_t flags = 0;
     int total = 0;
     for (int q = 0; q < 2; ++q) {
-        const int ch = lane + 32 * q;
-        if (ch < p.n_chunks) {
-            const unsigned char* rec = p.chunk_partials + ((size_t)row * p.n_chunks + ch) * stride;
+        const int ch = lane + 32 * q;                            // record index: chunk * 2 + column half
+        if (ch < 2 * p.n_chunks) {
+            const unsigned char* rec = p.chunk_partials + ((size_t)row * p.n_chunks * 2 + ch) * stride;
             hdr[q] = (const SegPartial*)rec;
             keys[q] = (const uint64_t*)(rec + sizeof(SegPartial));
             cnt[q] = hdr[q]->cnt;
