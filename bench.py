@@ -258,6 +258,14 @@ def run_ours(args, rank, world):
         except Exception as ex:
             fused_head = {"error": str(ex)[:200]}
 
+    # ---- tree construction fused into the drafter's output projection, next to library GEMM + cadd_build_tree ----
+    fused_draft = None
+    if args.head_hidden > 0:
+        try:
+            fused_draft = draft_head_block(G, cfg, kw, ck, args.head_hidden, dev, min(K, 10))
+        except Exception as ex:
+            fused_draft = {"error": str(ex)[:200]}
+
     # ---- offline cost fitting on a synthetic 9 x 1024 latency grid (the paper's profiling shape) ----
     cost_fit = None
     if not args.no_fit:
@@ -281,7 +289,7 @@ def run_ours(args, rank, world):
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": f"replicas x{world}",
                        "n_star_mean": round(float(n_star.float().mean()), 2), "n_star_max": int(n_star.max()),
                        "accepted_mean": round(float(verdict.accepted_len.float().mean().item()), 2)},
-            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "fused_draft_head": fused_draft, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
             "gpu_launches": KERNELS_PER_STEP * K, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
@@ -331,6 +339,46 @@ def head_block(G, cfg, tree, verdict, y, rows_mode, hidden, dev, iters):
             "roofline": {"bound": "tensor", "achieved": round(ach, 1), "peak": peak, "peak_kind": f"of {kind}", "unit": "TFLOP/s",
                          "frac": round(ach / peak, 4)},
             "library_gemm_ms": round(t_gemm, 4), "argmax_on_logits_ms": round(t_arg, 4),
+            "status_bits": int(out.status.max().item()), "iters": iters}
+
+
+def draft_head_block(G, cfg, kw, ck, hidden, dev, iters):
+    """cadd_build_tree_fused_head on synthetic drafter hidden states / weight of the workload's shape (logits of
+    standard deviation 1.5), timed alone, beside a library GEMM that writes bf16 logits plus cadd_build_tree."""
+    if cfg.K > 32:
+        return {"skipped": "K > 32"}
+    g = torch.Generator(device=dev).manual_seed(4321)
+    M = cfg.batch * cfg.L
+    h = (torch.randn(cfg.batch, cfg.L, hidden, device=dev, generator=g) * (1.5 / hidden ** 0.5)).to(torch.bfloat16)
+    w = torch.randn(cfg.V, hidden, device=dev, dtype=torch.bfloat16, generator=g)
+    ws = torch.empty(G.cadd_build_head_workspace_bytes(cfg.batch, cfg.L, cfg.V, hidden, cfg.K, cfg.B_max, cfg.R), dtype=torch.uint8, device=dev)
+    out = G.cadd_build_tree_fused_head(h, w, cfg.K, cfg.B_max, cfg.R, workspace=ws, **kw, **ck)
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    t_fused = timed(lambda: G.cadd_build_tree_fused_head(h, w, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=out, **kw, **ck))
+    x2 = torch.empty(cfg.batch, cfg.L, cfg.V, device=dev, dtype=torch.bfloat16)
+    t_gemm = timed(lambda: torch.matmul(h.view(M, hidden), w.T, out=x2.view(M, cfg.V)))
+    ws2 = torch.empty(G.cadd_build_workspace_bytes(cfg.batch, cfg.L, cfg.V, cfg.K, cfg.B_max, cfg.R, torch.bfloat16), dtype=torch.uint8, device=dev)
+    o2 = G.cadd_build_tree(x2, cfg.K, cfg.B_max, cfg.R, workspace=ws2, **kw, **ck)
+    t_build = timed(lambda: G.cadd_build_tree(x2, cfg.K, cfg.B_max, cfg.R, workspace=ws2, out=o2, **kw, **ck))
+    flops = 2.0 * M * hidden * cfg.V
+    peak, kind = measured_peak_tflops()
+    ach = flops / (t_fused * 1e-3) / 1e12
+    return {"hidden": hidden, "rows": M, "ms": round(t_fused, 4), "flops": flops,
+            "roofline": {"bound": "tensor", "achieved": round(ach, 1), "peak": peak, "peak_kind": f"of {kind}", "unit": "TFLOP/s",
+                         "frac": round(ach / peak, 4)},
+            "library_gemm_ms": round(t_gemm, 4), "build_on_logits_ms": round(t_build, 4),
             "status_bits": int(out.status.max().item()), "iters": iters}
 
 

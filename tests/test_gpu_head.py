@@ -207,3 +207,28 @@ def test_fused_draft_head_masked_positions_and_fixed_budget():
     bonus = torch.arange(batch, dtype=torch.int32)
     diag, mism, ot = check_fused_build(h, w, cfg, 4, l_eff=l_eff, bonus_token=bonus, flags=O.FLAG_FIXED_BUDGET)
     assert int(ot.n_nodes[2]) == 0 and int(ot.n_nodes.max()) == 96
+
+
+def test_fused_draft_head_full_size_sampled_rows():
+    """Config 2's draft shape (512 rows, V = 151936, K = 8) with hidden size 4096, in the launch configuration the
+    bench times.  The oracle recomputes the logits of a seeded sample of requests' rows; their top-K lists and
+    log-probabilities must agree (near-ties inside the accumulation bound excepted), and the whole tree of every
+    sampled request must be the oracle's."""
+    cfg = synth.CONFIGS["c2"]
+    hidden = 4096
+    h, w = planted_draft_inputs(cfg.batch, cfg.L, hidden, cfg.V, seed=99)
+    c = synth.make_cost_inputs(cfg, 3)
+    gt = G.cadd_build_tree_fused_head(h.cuda(), w.cuda(), cfg.K, cfg.B_max, cfg.R, cost_coef=c.coef.cuda(), flags=G.FLAG_EMIT_TOPK)
+    torch.cuda.synchronize()
+    assert int(gt.status.max()) & G.STATUS_INTERNAL_TIMEOUT == 0
+    sample = [0, 13, 31]
+    ot, y64 = O.build_tree_fused_head(h[sample], w, cfg.K, cfg.B_max, cfg.R, cost_coef=c.coef[sample])
+    absdot = h[sample].double().abs().reshape(-1, hidden) @ w.double().abs().T
+    e = hidden * 2.0 ** -24 * float(absdot.max())
+    sub = G.Tree(**{f: (getattr(gt, f)[sample] if getattr(gt, f) is not None else None) for f in gt.__dataclass_fields__})
+    diag = compare_build(sub, ot, cfg.K, check_topk=False, rel_tol=1e-5 + 2 * cfg.L * 2 * e, near_tie=max(1e-6, 2 * cfg.L * 2 * e))
+    assert len(diag["exempt"]) <= 1
+    mism = (sub.topk_token.cpu() != ot.topk_token).any(dim=-1)
+    assert int(mism.sum()) <= 1
+    lg, lo = sub.topk_logprob.cpu()[~mism], ot.topk_logprob[~mism]
+    assert float((lg - lo).abs().max()) <= 2 * e + 1e-7
