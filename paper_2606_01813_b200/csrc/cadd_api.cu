@@ -373,9 +373,10 @@ int cadd_fit_cost_tables(const cadd_fit_args* a, void* cuda_stream) {
 
 // ---------------- tree construction fused into the drafter's output projection ----------------
 
+constexpr int kDraftMaxCtas = 256;        // CTAs of the fused draft kernel (one per SM); sizes its list scratch
 struct DraftPlan {
-    int KP, m_tiles, n_tiles, chunk_tiles, n_chunks;
-    size_t chunk_bytes, merged_bytes, total_bytes;
+    int KP, m_tiles, n_tiles, chunk_tiles, n_chunks, halves;
+    size_t chunk_bytes, merged_bytes, list_bytes, total_bytes;
 };
 // Chunks of column tiles per row: at most 32 (two records each; the merge kernel walks two lists per lane), chosen so that the number
 // of work items (row tiles x chunks) fills whole waves of one CTA per SM as evenly as possible.
@@ -387,7 +388,9 @@ static DraftPlan plan_draft_head(const cadd_build_args* a, int sms) {
     pl.n_tiles = (int)((a->V + kHeadBN - 1) / kHeadBN);
     int best = 1;
     double best_eff = -1.0;
-    const int cap = pl.n_tiles < 32 ? pl.n_tiles : 32;               // two records per chunk, at most 64 per row
+    pl.halves = pl.KP <= 16 ? 2 : 1;                                  // epilogue warps per group of 32 rows (see DraftHeadShared)
+    const int max_chunks = 64 / pl.halves;                            // at most 64 records per row for the merge kernel
+    const int cap = pl.n_tiles < max_chunks ? pl.n_tiles : max_chunks;
     for (int nc = 1; nc <= cap; ++nc) {
         const int ct = (pl.n_tiles + nc - 1) / nc;
         const int real = (pl.n_tiles + ct - 1) / ct;                       // chunks that actually exist with this size
@@ -399,9 +402,10 @@ static DraftPlan plan_draft_head(const cadd_build_args* a, int sms) {
     pl.chunk_tiles = (pl.n_tiles + best - 1) / best;
     pl.n_chunks = (pl.n_tiles + pl.chunk_tiles - 1) / pl.chunk_tiles;
     const size_t stride = seg_partial_stride(pl.KP);
-    pl.chunk_bytes = (((size_t)M * pl.n_chunks * 2 * stride) + 255) & ~(size_t)255;
+    pl.chunk_bytes = (((size_t)M * pl.n_chunks * pl.halves * stride) + 255) & ~(size_t)255;
     pl.merged_bytes = (((size_t)M * stride) + 255) & ~(size_t)255;
-    pl.total_bytes = pl.chunk_bytes + pl.merged_bytes + 256;
+    pl.list_bytes = (size_t)kDraftMaxCtas * 2 * kDraftPending * kHeadBM * 8;   // the queues' scratch
+    pl.total_bytes = pl.chunk_bytes + pl.merged_bytes + pl.list_bytes + 256;
     return pl;
 }
 
@@ -421,7 +425,7 @@ int cadd_build_head_workspace_bytes(const cadd_build_head_args* h, size_t* out) 
     // sized for the largest cut (32 chunks = 64 records per row), so the answer does not depend on the device
     const size_t stride = seg_partial_stride(h->build.K > kPreciseMin ? h->build.K : kPreciseMin);
     const size_t M = (size_t)h->build.batch * h->build.L;
-    *out = ((M * 64 * stride + 255) & ~(size_t)255) + ((M * stride + 255) & ~(size_t)255) + 256;
+    *out = ((M * 64 * stride + 255) & ~(size_t)255) + ((M * stride + 255) & ~(size_t)255) + (size_t)kDraftMaxCtas * 2 * kDraftPending * kHeadBM * 8 + 256;
     return CADD_OK;
 }
 
@@ -459,19 +463,21 @@ int cadd_build_tree_fused_head(const cadd_build_head_args* h, void* cuda_stream)
         return CADD_ERR_LAUNCH;
     unsigned char* ws = (unsigned char*)a->workspace;
     unsigned char* merged = ws + pl.chunk_bytes;
-    int32_t* err = (int32_t*)(ws + pl.chunk_bytes + pl.merged_bytes);
+    uint64_t* pend = (uint64_t*)(ws + pl.chunk_bytes + pl.merged_bytes);
+    int32_t* err = (int32_t*)(ws + pl.chunk_bytes + pl.merged_bytes + pl.list_bytes);
     if (cudaMemsetAsync(err, 0, 256, st) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
 
     DraftHeadParams dp;
     dp.M = M; dp.V = a->V; dp.Kdim = h->hidden; dp.m_tiles = pl.m_tiles; dp.n_tiles = pl.n_tiles;
     dp.chunk_tiles = pl.chunk_tiles; dp.n_chunks = pl.n_chunks; dp.L = a->L; dp.KP = pl.KP; dp.l_eff = a->l_eff;
-    dp.chunk_partials = ws; dp.error = err;
+    dp.chunk_partials = ws; dp.pend = pend; dp.halves = pl.halves; dp.error = err;
     if (cudaFuncSetAttribute(head_softmax_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)draft_head_smem_bytes()) != cudaSuccess) {
         cudaGetLastError();
         return CADD_ERR_LAUNCH;
     }
     const int64_t items = (int64_t)pl.m_tiles * pl.n_chunks;
-    head_softmax_topk_kernel<<<(unsigned)(items < sms ? items : sms), kDraftThreads, draft_head_smem_bytes(), st>>>(map_h, map_w, dp);
+    const int ctas = sms < kDraftMaxCtas ? sms : kDraftMaxCtas;
+    head_softmax_topk_kernel<<<(unsigned)(items < ctas ? items : ctas), kDraftThreads, draft_head_smem_bytes(), st>>>(map_h, map_w, dp);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
     draft_merge_kernel<<<(unsigned)((M + 3) / 4), 128, 0, st>>>(dp, merged);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;

@@ -20,17 +20,17 @@ namespace cadd {
 
 constexpr int kDraftMaxKP = 32;           // list capacity per row that fits beside the operand ring in shared memory
 
-constexpr int kDraftStages = 3;           // operand ring: one stage fewer than head_argmax.cuh, the room goes to the row state
+constexpr int kDraftStages = 4;           // operand ring as in head_argmax.cuh: about 190 KB in flight cover the TMA latency
 constexpr int kDraftPending = 8;          // queued candidates per row and column half between two list updates
 constexpr int kDraftThreads = 320;        // producer warp, MMA warp, eight epilogue warps
 
 struct DraftHeadShared {
     alignas(1024) unsigned char a[kDraftStages][kHeadABytes];
     alignas(1024) unsigned char b[kDraftStages][kHeadBBytes];
-    // Two epilogue warps share each group of 32 rows and split the tile's columns in halves; each half keeps its own
-    // row state and leaves its own record.
-    uint64_t list[2][kDraftMaxKP][kHeadBM];                // list[half][k][row of the tile]: the row's KP best keys so far, unsorted
-    uint64_t pend[2][kDraftPending][kHeadBM];              // candidates waiting for the next list update
+    // The rows' lists of best keys, unsorted: list[(half * KP + k) * 128 + row of the tile].  32 KB is what is left
+    // beside four operand stages: for KP <= 16 two epilogue warps share each group of 32 rows and split the tile's
+    // columns in halves, each half with its own row state and its own record; for KP <= 32 one warp takes all columns.
+    uint64_t list[2 * 16 * kHeadBM];
     alignas(8) uint64_t full[kDraftStages];
     uint64_t empty[kDraftStages];
     uint64_t acc_full[2];
@@ -49,9 +49,25 @@ struct DraftHeadParams {
     int n_chunks;              // chunks per row = ceil(n_tiles / chunk_tiles)
     int L, KP;
     const int32_t* l_eff;      // [batch] or NULL
-    unsigned char* chunk_partials;   // [M * n_chunks * 2] records of seg_partial_stride(KP) bytes (two column halves per chunk)
+    uint64_t* pend;            // [gridDim][2][kDraftPending][128] scratch: candidates waiting for the next list update
+                               // (global memory: written on a hit, read back once per tile; L1/L2-resident)
+    int halves;                // column halves per tile handled by separate epilogue warps: 2 (KP <= 16) or 1
+    unsigned char* chunk_partials;   // [M * n_chunks * halves] records of seg_partial_stride(KP) bytes
     int32_t* error;
 };
+
+// r[i] for a run-time i, without spilling the array: a binary tree of selects (31 of them).
+__device__ __forceinline__ uint32_t pick32(const uint32_t (&r)[32], int i) {
+    uint32_t a[16], b[8], c[4];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) a[j] = (i & 1) ? r[2 * j + 1] : r[2 * j];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) b[j] = (i & 2) ? a[2 * j + 1] : a[2 * j];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) c[j] = (i & 4) ? b[2 * j + 1] : b[2 * j];
+    const uint32_t d0 = (i & 8) ? c[1] : c[0], d1 = (i & 8) ? c[3] : c[2];
+    return (i & 16) ? d1 : d0;
+}
 
 // Row r = b * L + i is read iff i < l_eff[b].
 __device__ __forceinline__ bool draft_row_live(const DraftHeadParams& p, int64_t r) {
@@ -80,7 +96,7 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
 
     if (tid == 0) {
         for (int s = 0; s < kDraftStages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&sh.acc_full[s], 1); mbar_init(&sh.acc_empty[s], 8); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sh.acc_full[s], 1); mbar_init(&sh.acc_empty[s], 4 * p.halves); }
         sh.error = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -142,8 +158,11 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
         const int quarter = warp & 3;                            // tensor-memory lane quarter this warp may read
         const int half = (warp - 2) >> 2;                        // columns [half * 128, half * 128 + 128) of every tile
         const int trow = quarter * 32 + lane;                    // row inside the tile = tensor-memory lane
+        uint64_t* list = &sh.list[(size_t)half * KP * kHeadBM + trow];                        // this thread's column of the list
+        uint64_t* pend = p.pend + (((size_t)blockIdx.x * 2 + half) * kDraftPending) * kHeadBM + trow;
+        const int width = kHeadBN / p.halves;                    // columns of a tile this warp handles
         unsigned buf = 0, aph = 0;
-        for (int64_t w = blockIdx.x; w < n_items && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
+        for (int64_t w = blockIdx.x; w < n_items && half < p.halves && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
             const int ch = (int)(w / p.m_tiles), mt = (int)(w - (int64_t)ch * p.m_tiles);
             if (!draft_tile_live(p, mt)) continue;
             const int64_t row = (int64_t)mt * kHeadBM + trow;
@@ -163,14 +182,14 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
             // joins the sum.
             auto drain = [&]() {
                 for (int j = 0; j < np; ++j) {
-                    const uint64_t key = sh.pend[half][j][trow];
+                    const uint64_t key = pend[(size_t)j * kHeadBM];
                     if (cnt < KP) {
-                        sh.list[half][cnt][trow] = key;
+                        list[(size_t)cnt * kHeadBM] = key;
                         ++cnt;
                         if (cnt < KP) continue;
                     } else if (key > thr_key) {
                         s.acc += (double)exp2_term(key_value(thr_key), s.negc);
-                        sh.list[half][min_pos][trow] = key;
+                        list[(size_t)min_pos * kHeadBM] = key;
                     } else {
                         s.acc += (double)exp2_term(key_value(key), s.negc);
                         continue;
@@ -179,7 +198,7 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
                     int mp = 0;
 #pragma unroll 4
                     for (int k = 0; k < KP; ++k) {
-                        const uint64_t v = sh.list[half][k][trow];
+                        const uint64_t v = list[(size_t)k * kHeadBM];
                         if (v < mk) { mk = v; mp = k; }
                     }
                     thr_key = mk; min_pos = mp;
@@ -194,55 +213,56 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
             for (int nt = ch * p.chunk_tiles; nt < nt1 && ok; ++nt) {
                 if (!__all_sync(kFullMask, head_wait(&sh.acc_full[buf], aph, 256))) { sh.error = 4; ok = false; break; }
                 tc_fence_after();
-                const int64_t col0 = (int64_t)nt * kHeadBN + half * (kHeadBN / 2);
+                const int64_t col0 = (int64_t)nt * kHeadBN + half * width;
+                const bool inside = col0 + width <= p.V;          // no column of this warp's share is past the vocabulary
                 // 32 columns per tensor-memory load (narrow loads have the same latency, about 2 k cycles while the
                 // tensor cores run the next tile), the next 32 already on their way.  Pass 1 is branch-free: every
                 // element below the threshold adds its exponential, the others set a bit.  Pass 2 runs only while
-                // some lane has bits left: it queues them (or sums them, if a list update has raised the threshold
-                // meanwhile); when a lane's queue is full the whole warp folds its queues into the lists and pass 2
-                // repeats.
-                const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kHeadBN + half * (kHeadBN / 2);
+                // some lane has bits left: each lane takes one of its marked elements per turn and queues it (or sums
+                // it, if a list update has raised the threshold meanwhile); when a lane's queue is full the whole warp
+                // folds its queues into the lists and pass 2 goes on.
+                const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kHeadBN + half * width;
                 uint32_t r[32], rn[32];
                 tmem_ld32(tbase, r);
                 tmem_ld_wait();
 #pragma unroll 1
-                for (int c = 0; c < kHeadBN / 64; ++c) {
-                    if (c + 1 < kHeadBN / 64) tmem_ld32(tbase + (c + 1) * 32, rn);
+                for (int c = 0; c < width / 32; ++c) {
+                    if (c + 1 < width / 32) tmem_ld32(tbase + (c + 1) * 32, rn);
                     const int64_t cb = col0 + c * 32;
                     float part = 0.0f;                            // fp32 sum of this run of 32 columns
                     unsigned hit = 0;
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const float x = __uint_as_float(r[i]);
-                        const bool valid = live && cb + i < p.V;
+                        const bool valid = live && (inside || cb + i < p.V);
                         const bool fast = valid && x < thr;
                         part += exp2_term(fast ? x : -INFINITY, s.negc);              // 2^-inf = 0
                         hit |= (valid && !fast) ? (1u << i) : 0u;
                     }
                     s.acc += (double)part;
                     while (__any_sync(kFullMask, hit != 0)) {
-                        float part2 = 0.0f;
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            if (hit & (1u << i)) {
-                                const float x = __uint_as_float(r[i]);
-                                const uint32_t bits = __float_as_uint(x);
-                                if ((bits & 0x7f800000u) == 0x7f800000u) {            // Inf or NaN: no mass, never a candidate
-                                    if (bits != 0xff800000u) flags |= kPartNonfinite;
-                                    if (bits == 0x7f800000u) flags |= kPartPosInf;
-                                    hit &= ~(1u << i);
-                                } else if (x < thr) {                                 // the threshold has risen since pass 1
-                                    part2 += exp2_term(x, s.negc);
-                                    hit &= ~(1u << i);
-                                } else if (np < kDraftPending) {
-                                    sh.pend[half][np][trow] = make_key(x, (uint32_t)(cb + i));
-                                    ++np;
-                                    hit &= ~(1u << i);
-                                }
+                        // one marked element per lane and turn, fetched from the register file by a select tree
+                        bool blocked = false;
+                        if (hit) {
+                            const int i = __ffs(hit) - 1;
+                            const float x = __uint_as_float(pick32(r, i));
+                            const uint32_t bits = __float_as_uint(x);
+                            if ((bits & 0x7f800000u) == 0x7f800000u) {                // Inf or NaN: no mass, never a candidate
+                                if (bits != 0xff800000u) flags |= kPartNonfinite;
+                                if (bits == 0x7f800000u) flags |= kPartPosInf;
+                                hit &= hit - 1;
+                            } else if (x < thr) {                                     // the threshold has risen since pass 1
+                                s.acc += (double)exp2_term(x, s.negc);
+                                hit &= hit - 1;
+                            } else if (np < kDraftPending) {
+                                pend[(size_t)np * kHeadBM] = make_key(x, (uint32_t)(cb + i));
+                                ++np;
+                                hit &= hit - 1;
+                            } else {
+                                blocked = true;
                             }
                         }
-                        s.acc += (double)part2;
-                        if (__any_sync(kFullMask, hit != 0)) drain();                 // a queue is full: fold, then go on
+                        if (__any_sync(kFullMask, blocked)) drain();                  // a queue is full: fold, then go on
                     }
                     tmem_ld_wait();
 #pragma unroll
@@ -256,12 +276,12 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
             }
             if (!ok) break;
             if (live) {
-                unsigned char* rec = p.chunk_partials + (((size_t)row * p.n_chunks + ch) * 2 + half) * seg_partial_stride(KP);
+                unsigned char* rec = p.chunk_partials + (((size_t)row * p.n_chunks + ch) * p.halves + half) * seg_partial_stride(KP);
                 uint64_t* out_keys = (uint64_t*)(rec + sizeof(SegPartial));
                 for (int k = 0; k < cnt; ++k) {                     // rank by counting (keys are unique): sorted, best first
-                    const uint64_t v = sh.list[half][k][trow];
+                    const uint64_t v = list[(size_t)k * kHeadBM];
                     int rank = 0;
-                    for (int j = 0; j < cnt; ++j) rank += sh.list[half][j][trow] > v;
+                    for (int j = 0; j < cnt; ++j) rank += list[(size_t)j * kHeadBM] > v;
                     out_keys[rank] = v;
                 }
                 SegPartial h;
@@ -299,9 +319,9 @@ __global__ void __launch_bounds__(128) draft_merge_kernel(DraftHeadParams p, uns
     uint32_t flags = 0;
     int total = 0;
     for (int q = 0; q < 2; ++q) {
-        const int ch = lane + 32 * q;                            // record index: chunk * 2 + column half
-        if (ch < 2 * p.n_chunks) {
-            const unsigned char* rec = p.chunk_partials + ((size_t)row * p.n_chunks * 2 + ch) * stride;
+        const int ch = lane + 32 * q;                            // record index: chunk * halves + column half
+        if (ch < p.halves * p.n_chunks) {
+            const unsigned char* rec = p.chunk_partials + ((size_t)row * p.n_chunks * p.halves + ch) * stride;
             hdr[q] = (const SegPartial*)rec;
             keys[q] = (const uint64_t*)(rec + sizeof(SegPartial));
             cnt[q] = hdr[q]->cnt;
