@@ -332,10 +332,18 @@ def head_block(G, cfg, tree, verdict, y, rows_mode, hidden, dev, iters):
     t_gemm = timed(lambda: torch.matmul(h.view(M, hidden), w.T, out=y2.view(M, cfg.V)))   # library GEMM, logits written in bf16
     v2 = G.cadd_verify_tree(y2, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode)
     t_arg = timed(lambda: G.cadd_verify_tree(y2, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, out=v2))
+    # LIVE mode: only rows j <= n*[b] are projected (packed first); with trees of a few nodes the weights' one pass
+    # over HBM sets the time
+    ws_l = torch.empty(G.cadd_head_workspace_bytes(cfg.batch, cfg.R, hidden, cfg.V, cfg.L, G.ROWS_LIVE), dtype=torch.uint8, device=dev)
+    out_l = G.cadd_verify_tree_fused_head(h, w, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, G.ROWS_LIVE, workspace=ws_l)
+    t_live = timed(lambda: G.cadd_verify_tree_fused_head(h, w, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, G.ROWS_LIVE,
+                                                         workspace=ws_l, out=out_l))
+    live_rows = int((tree.n_nodes.clamp(0, cfg.R - 1) + 1).sum().item())
     flops = 2.0 * M * hidden * cfg.V
     peak, kind = measured_peak_tflops()
     ach = flops / (t_fused * 1e-3) / 1e12
     return {"hidden": hidden, "rows": M, "ms": round(t_fused, 4), "flops": flops,
+            "live_rows": live_rows, "live_ms": round(t_live, 4), "weight_bytes": cfg.V * hidden * 2,
             "roofline": {"bound": "tensor", "achieved": round(ach, 1), "peak": peak, "peak_kind": f"of {kind}", "unit": "TFLOP/s",
                          "frac": round(ach / peak, 4)},
             "library_gemm_ms": round(t_gemm, 4), "argmax_on_logits_ms": round(t_arg, 4),

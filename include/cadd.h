@@ -176,7 +176,8 @@ typedef struct cadd_head_args {
     uint32_t flags;                /* reserved, 0 */
     int32_t  batch, L, R;
     int32_t  hidden;               /* hidden size (the contraction length), >= 1 */
-    int32_t  rows_mode;            /* CADD_ROWS_*; in LIVE mode rows j > n_nodes[b] get node_argmax -1 */
+    int32_t  rows_mode;            /* CADD_ROWS_*; in LIVE mode rows j > n_nodes[b] get node_argmax -1, and the product is
+                                      formed for the live rows only (they are copied next to one another first) */
     int32_t  reserved0;
     int64_t  V;
     const void* hidden_states;     /* bf16 [batch, R, hidden]; element (b,j,k) at (b*R + j)*stride_row + k; 16-byte aligned */
@@ -256,7 +257,8 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream);
 /* Tree verification (Sections 3.1 and 3.3).  Asynchronous on `cuda_stream`. */
 int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream);
 
-/* Scratch size of cadd_verify_tree_fused_head: pure host arithmetic on batch and R. */
+/* Scratch size of cadd_verify_tree_fused_head: pure host arithmetic on batch, R, hidden and rows_mode (LIVE mode
+ * needs room for a packed copy of the hidden states). */
 int cadd_head_workspace_bytes(const cadd_head_args* a, size_t* out);
 
 /* Tree verification from hidden states and the output-projection weight (see cadd_head_args).  Asynchronous on

@@ -316,10 +316,13 @@ def cadd_verify_tree(target_logits: torch.Tensor, L: int, n_nodes: torch.Tensor,
     return out
 
 
-def cadd_head_workspace_bytes(batch: int, R: int, hidden: int, V: int, L: int = 1) -> int:
+def cadd_head_workspace_bytes(batch: int, R: int, hidden: int, V: int, L: int = 1, rows_mode: int = ROWS_LIVE) -> int:
+    """Scratch bytes of cadd_verify_tree_fused_head; LIVE mode (the default here) needs room for a packed copy of the
+    live hidden states and is therefore the larger of the two."""
     a = HeadArgs()
     a.struct_size = C.sizeof(HeadArgs)
     a.batch, a.L, a.R, a.hidden, a.V = batch, L, R, hidden, V
+    a.rows_mode = rows_mode
     n = C.c_size_t(0)
     rc = lib().cadd_head_workspace_bytes(C.byref(a), C.byref(n))
     if rc != OK:
@@ -363,7 +366,7 @@ def cadd_verify_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tenso
     a.node_argmax, a.accepted_len, a.accepted_nodes = _ptr(out.node_argmax), _ptr(out.accepted_len), _ptr(out.accepted_nodes)
     a.next_bonus, a.status = _ptr(out.next_bonus), _ptr(out.status)
     if workspace is None:
-        workspace = torch.empty(cadd_head_workspace_bytes(batch, R, hidden, V, L), dtype=torch.uint8, device=dev)
+        workspace = torch.empty(cadd_head_workspace_bytes(batch, R, hidden, V, L, rows_mode), dtype=torch.uint8, device=dev)
     a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
     with torch.cuda.device(dev):
         rc = lib().cadd_verify_tree_fused_head(C.byref(a), _stream_ptr(stream))

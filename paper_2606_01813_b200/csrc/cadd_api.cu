@@ -286,11 +286,24 @@ static int check_head_shape(const cadd_head_args* a) {
     return CADD_OK;
 }
 
+// Workspace of the fused verification: packed row maxima [M] u64 | error word (256 B) | LIVE mode only: row offsets
+// [batch + 1] int32 and the packed copy of the live hidden states [M, hidden] bf16 (sized for every row live).
+struct HeadLayout { size_t best_bytes, off_bytes, pack_bytes, total; };
+static HeadLayout head_layout(const cadd_head_args* a) {
+    HeadLayout l;
+    const size_t M = (size_t)a->batch * a->R;
+    l.best_bytes = (M * 8 + 255) & ~(size_t)255;
+    l.off_bytes = a->rows_mode == CADD_ROWS_LIVE ? ((((size_t)a->batch + 1) * 4 + 255) & ~(size_t)255) : 0;
+    l.pack_bytes = a->rows_mode == CADD_ROWS_LIVE ? ((M * (size_t)a->hidden * 2 + 255) & ~(size_t)255) : 0;
+    l.total = l.best_bytes + 256 + l.off_bytes + l.pack_bytes;
+    return l;
+}
+
 int cadd_head_workspace_bytes(const cadd_head_args* a, size_t* out) {
     int rc = check_head_shape(a);
     if (rc != CADD_OK) return rc;
     if (!out) return CADD_ERR_NULL;
-    *out = (((size_t)a->batch * a->R * 8 + 255) & ~(size_t)255) + 256;    // packed row maxima + the error word
+    *out = head_layout(a).total;
     return CADD_OK;
 }
 
@@ -306,14 +319,29 @@ int cadd_verify_tree_fused_head(const cadd_head_args* a, void* cuda_stream) {
         !aligned(a->accepted_len, 4) || !aligned(a->accepted_nodes, 4) || !aligned(a->next_bonus, 4) || !aligned(a->status, 4))
         return CADD_ERR_ALIGN;
     if (a->stride_row < a->hidden || a->stride_w < a->hidden) return CADD_ERR_SHAPE;
-    size_t need = 0;
-    cadd_head_workspace_bytes(a, &need);
-    if (!a->workspace || !aligned(a->workspace, 256) || a->workspace_bytes < need) return CADD_ERR_WORKSPACE;
+    const bool live = a->rows_mode == CADD_ROWS_LIVE;
+    if (live && a->hidden % 8 != 0) return CADD_ERR_ALIGN;        // packed rows must keep 16-byte alignment
+    const HeadLayout lay = head_layout(a);
+    if (!a->workspace || !aligned(a->workspace, 256) || a->workspace_bytes < lay.total) return CADD_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
     const int64_t M = (int64_t)a->batch * a->R;
+    unsigned char* ws = (unsigned char*)a->workspace;
+    int32_t* err = (int32_t*)(ws + lay.best_bytes);
+    int32_t* row_off = live ? (int32_t*)(ws + lay.best_bytes + 256) : nullptr;
+    __nv_bfloat16* packed = live ? (__nv_bfloat16*)(ws + lay.best_bytes + 256 + lay.off_bytes) : nullptr;
+    if (cudaMemsetAsync(ws, 0, lay.best_bytes + 256, st) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+    if (live) {
+        // LIVE mode: the GEMM runs on the live rows only, copied next to one another first (a few MB at most for trees
+        // of tens of nodes); the row count stays on the device
+        head_live_offsets_kernel<<<1, 1024, 0, st>>>(a->n_nodes, a->batch, a->R, row_off);
+        head_pack_rows_kernel<<<dim3((unsigned)a->R, (unsigned)a->batch), 128, 0, st>>>((const __nv_bfloat16*)a->hidden_states, a->stride_row,
+                                                                                           a->hidden, a->R, a->n_nodes, row_off, packed);
+        if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    }
     CUtensorMap map_h, map_w;
-    if (!make_map_bf16(&map_h, a->hidden_states, M, a->hidden, a->stride_row, kHeadBM) ||
+    if (!(live ? make_map_bf16(&map_h, packed, M, a->hidden, a->hidden, kHeadBM)
+               : make_map_bf16(&map_h, a->hidden_states, M, a->hidden, a->stride_row, kHeadBM)) ||
         !make_map_bf16(&map_w, a->weight, a->V, a->hidden, a->stride_w, kHeadBN))
         return CADD_ERR_LAUNCH;
 
@@ -327,9 +355,9 @@ int cadd_verify_tree_fused_head(const cadd_head_args* a, void* cuda_stream) {
         hp.group_m = (int)(g < 1 ? 1 : (g > hp.m_tiles ? hp.m_tiles : g));
     }
     hp.R = a->R; hp.rows_mode = a->rows_mode; hp.n_nodes = a->n_nodes;
-    hp.row_best = (unsigned long long*)a->workspace;
-    hp.error = (int32_t*)((unsigned char*)a->workspace + (need - 256));
-    if (cudaMemsetAsync(a->workspace, 0, need, st) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+    hp.m_live = live ? row_off + a->batch : nullptr;
+    hp.row_best = (unsigned long long*)ws;
+    hp.error = err;
     if (cudaFuncSetAttribute(head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem_bytes()) != cudaSuccess) {
         cudaGetLastError();
         return CADD_ERR_LAUNCH;
@@ -339,7 +367,7 @@ int cadd_verify_tree_fused_head(const cadd_head_args* a, void* cuda_stream) {
     const unsigned grid = (unsigned)(work < sms ? work : sms);
     head_argmax_kernel<<<grid, kHeadThreads, head_smem_bytes(), st>>>(map_h, map_w, hp);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
-    head_decode_kernel<<<(unsigned)((M + 255) / 256), 256, 0, st>>>(hp.row_best, a->n_nodes, hp.error, M, a->R, a->rows_mode, a->node_argmax);
+    head_decode_kernel<<<(unsigned)((M + 255) / 256), 256, 0, st>>>(hp.row_best, a->n_nodes, row_off, hp.error, M, a->R, a->rows_mode, a->node_argmax);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
 
     WalkParams wp;

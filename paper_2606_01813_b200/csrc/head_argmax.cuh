@@ -55,7 +55,9 @@ struct HeadParams {
     int m_tiles, n_tiles;
     int group_m;               // row tiles per group: a group's hidden states stay L2-resident while all of W streams by
     int R, rows_mode;
-    const int32_t* n_nodes;    // [batch] (LIVE mode: row tiles without a live row are skipped)
+    const int32_t* n_nodes;    // [batch]
+    const int32_t* m_live;     // LIVE mode: device word holding the number of packed rows (the GEMM runs on the packed copy
+                               // of the live rows only); NULL in DENSE mode
     unsigned long long* row_best;   // [M] packed (ordered logit << 32 | ~token), zeroed before the launch
     int32_t* error;            // device word, set non-zero when a bounded wait ran out
 };
@@ -136,26 +138,17 @@ __device__ __forceinline__ void head_tile_of(const HeadParams& p, int64_t w, int
     mt = g * p.group_m + (int)(rem - (int64_t)nt * gsz);
 }
 
-// True if row tile mt holds a row that is read: always in DENSE mode; in LIVE mode rows j <= n_nodes[b] of a request.
-__device__ __forceinline__ bool head_tile_live(const HeadParams& p, int mt) {
-    if (p.rows_mode != CADD_ROWS_LIVE) return true;
-    const int64_t r0 = (int64_t)mt * kHeadBM;
-    const int64_t r1 = min(r0 + kHeadBM, p.M) - 1;
-    for (int64_t b = r0 / p.R; b <= r1 / p.R; ++b) {
-        int n = p.n_nodes[b];
-        n = n < 0 ? 0 : (n > p.R - 1 ? p.R - 1 : n);
-        const int64_t lo = max(r0, b * p.R), hi = min(r1, b * p.R + n);   // live rows of request b inside the tile
-        if (lo <= hi) return true;
-    }
-    return false;
-}
-
 __global__ void __launch_bounds__(kHeadThreads, 1)
 head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, HeadParams p) {
     extern __shared__ __align__(16) unsigned char head_smem_raw[];
     HeadShared& sh = *reinterpret_cast<HeadShared*>(head_smem_raw + ((1024u - (smem_u32(head_smem_raw) & 1023u)) & 1023u));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int k_steps = (p.Kdim + kHeadBK - 1) / kHeadBK;
+    if (p.m_live) {                                               // LIVE mode: only the packed live rows exist
+        p.M = *p.m_live;
+        p.m_tiles = (int)((p.M + kHeadBM - 1) / kHeadBM);
+        if (p.group_m > p.m_tiles) p.group_m = p.m_tiles > 0 ? p.m_tiles : 1;
+    }
     const int64_t n_work = (int64_t)p.m_tiles * p.n_tiles;
 
     if (tid == 0) {
@@ -177,7 +170,6 @@ head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
             for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
                 int mt, nt;
                 head_tile_of(p, w, mt, nt);
-                if (!head_tile_live(p, mt)) continue;
                 for (int k = 0; k < k_steps; ++k) {
                     if (!head_wait(&sh.empty[s], ph ^ 1u, 64)) { sh.error = 1; break; }   // first pass: free at once
                     mbar_arrive_expect_tx(&sh.full[s], kHeadABytes + kHeadBBytes);
@@ -194,7 +186,6 @@ head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
             for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
                 int mt, nt;
                 head_tile_of(p, w, mt, nt);
-                if (!head_tile_live(p, mt)) continue;
                 if (!head_wait(&sh.acc_empty[buf], aph ^ 1u)) { sh.error = 2; break; }   // epilogue has drained it
                 tc_fence_after();
                 const uint32_t d = tmem_base + buf * kHeadBN;
@@ -221,7 +212,6 @@ head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
         for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
             int mt, nt;
             head_tile_of(p, w, mt, nt);
-            if (!head_tile_live(p, mt)) continue;
             if (!__all_sync(kFullMask, head_wait(&sh.acc_full[buf], aph, 256))) { sh.error = 4; break; }
             tc_fence_after();
             const int64_t row = (int64_t)mt * kHeadBM + quarter * 32 + lane;
@@ -257,22 +247,67 @@ head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
     if (tid == 0 && sh.error) atomicExch(p.error, (int32_t)sh.error);
 }
 
+// LIVE mode, step 1: row_off[b] = number of live rows (j <= n_nodes[b]) of the requests before b; row_off[batch] is
+// the packed row count.  One CTA.
+__global__ void __launch_bounds__(1024) head_live_offsets_kernel(const int32_t* n_nodes, int batch, int R, int32_t* row_off) {
+    __shared__ int part[1024];
+    const int tid = threadIdx.x;
+    const int per = (batch + 1023) / 1024;
+    int run = 0;
+    for (int b = tid * per; b < min(batch, (tid + 1) * per); ++b) {
+        int n = n_nodes[b];
+        n = n < 0 ? 0 : (n > R - 1 ? R - 1 : n);
+        run += n + 1;
+    }
+    part[tid] = run;
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        for (int t = 0; t < 1024; ++t) { const int x = part[t]; part[t] = acc; acc += x; }
+        row_off[batch] = acc;
+    }
+    __syncthreads();
+    int acc = part[tid];
+    for (int b = tid * per; b < min(batch, (tid + 1) * per); ++b) {
+        row_off[b] = acc;
+        int n = n_nodes[b];
+        n = n < 0 ? 0 : (n > R - 1 ? R - 1 : n);
+        acc += n + 1;
+    }
+}
+
+// LIVE mode, step 2: copies the live rows of the hidden states next to one another (one CTA per (request, row)).
+__global__ void __launch_bounds__(128) head_pack_rows_kernel(const __nv_bfloat16* hidden_states, int64_t stride_row, int hidden, int R,
+                                                             const int32_t* n_nodes, const int32_t* row_off, __nv_bfloat16* packed) {
+    const int b = blockIdx.y, j = blockIdx.x;
+    int n = n_nodes[b];
+    n = n < 0 ? 0 : (n > R - 1 ? R - 1 : n);
+    if (j > n) return;
+    const uint4* src = (const uint4*)(hidden_states + ((int64_t)b * R + j) * stride_row);      // 16-byte aligned rows
+    uint4* dst = (uint4*)(packed + (int64_t)(row_off[b] + j) * hidden);
+    for (int c = threadIdx.x; c < hidden / 8; c += blockDim.x) dst[c] = src[c];
+    for (int k = (hidden / 8) * 8 + threadIdx.x; k < hidden; k += blockDim.x)                 // hidden % 8 != 0 cannot pass the
+        packed[(int64_t)(row_off[b] + j) * hidden + k] = hidden_states[((int64_t)b * R + j) * stride_row + k];   // stride check
+}
+
 // Turns the packed per-row maxima into token ids.  Rows not read in LIVE mode get -1; a row whose logits were all
-// -Inf or NaN gets 0, like the plain argmax kernel; -2 marks every row when the GEMM gave up on a wait.
-__global__ void head_decode_kernel(const unsigned long long* row_best, const int32_t* n_nodes, const int32_t* error, int64_t M, int R,
-                                   int rows_mode, int32_t* node_argmax) {
+// -Inf or NaN gets 0, like the plain argmax kernel; -2 marks every row when the GEMM gave up on a wait.  In LIVE
+// mode row (b, j) of the output is packed row row_off[b] + j of the GEMM.
+__global__ void head_decode_kernel(const unsigned long long* row_best, const int32_t* n_nodes, const int32_t* row_off,
+                                   const int32_t* error, int64_t M, int R, int rows_mode, int32_t* node_argmax) {
     const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= M) return;
     const int64_t b = r / R;
     const int j = (int)(r - b * R);
-    int32_t ans;
+    int64_t src = r;
     if (rows_mode == CADD_ROWS_LIVE) {
         int n = n_nodes[b];
         n = n < 0 ? 0 : (n > R - 1 ? R - 1 : n);
         if (j > n) { node_argmax[r] = -1; return; }
+        src = (int64_t)row_off[b] + j;
     }
-    const unsigned long long k = row_best[r];
-    ans = k ? (int32_t)key_id((uint64_t)k) : 0;
+    const unsigned long long k = row_best[src];
+    int32_t ans = k ? (int32_t)key_id((uint64_t)k) : 0;
     if (*error) ans = -2;
     node_argmax[r] = ans;
 }
