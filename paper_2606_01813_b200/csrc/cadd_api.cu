@@ -406,26 +406,28 @@ struct DraftPlan {
     int KP, m_tiles, n_tiles, chunk_tiles, n_chunks, halves;
     size_t chunk_bytes, merged_bytes, list_bytes, total_bytes;
 };
-// Chunks of column tiles per row: at most 32 (two records each; the merge kernel walks two lists per lane), chosen so that the number
-// of work items (row tiles x chunks) fills whole waves of one CTA per SM as evenly as possible.
+// Chunks of column tiles per row: at most kDraftMaxRecords records per row (one or two per chunk), chosen so that the number
+// of work items (row tiles x chunks) fills whole waves of one CTA per SM without making chunks needlessly short.
 static DraftPlan plan_draft_head(const cadd_build_args* a, int sms) {
     DraftPlan pl;
     pl.KP = a->K > kPreciseMin ? a->K : kPreciseMin;
     const int64_t M = (int64_t)a->batch * a->L;
     pl.m_tiles = (int)((M + kHeadBM - 1) / kHeadBM);
     pl.n_tiles = (int)((a->V + kHeadBN - 1) / kHeadBN);
-    int best = 1;
-    double best_eff = -1.0;
+    // estimated duration in tile times: waves x (tiles per chunk + about three tiles' worth of threshold warm-up and
+    // pipeline fill per chunk); the smallest wins, ties go to fewer chunks
     pl.halves = pl.KP <= 16 ? 2 : 1;                                  // epilogue warps per group of 32 rows (see DraftHeadShared)
-    const int max_chunks = 64 / pl.halves;                            // at most 64 records per row for the merge kernel
+    const int max_chunks = kDraftMaxRecords / pl.halves;              // what the merge kernel folds per row
     const int cap = pl.n_tiles < max_chunks ? pl.n_tiles : max_chunks;
+    int best = 1;
+    int64_t best_cost = -1;
     for (int nc = 1; nc <= cap; ++nc) {
         const int ct = (pl.n_tiles + nc - 1) / nc;
         const int real = (pl.n_tiles + ct - 1) / ct;                       // chunks that actually exist with this size
         const int64_t items = (int64_t)pl.m_tiles * real;
         const int64_t waves = (items + sms - 1) / sms;
-        const double eff = (double)items / (double)(waves * sms);
-        if (eff > best_eff + 1e-9) { best_eff = eff; best = real; }
+        const int64_t cost = waves * (ct + 3);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = real; }
     }
     pl.chunk_tiles = (pl.n_tiles + best - 1) / best;
     pl.n_chunks = (pl.n_tiles + pl.chunk_tiles - 1) / pl.chunk_tiles;
@@ -450,10 +452,10 @@ int cadd_build_head_workspace_bytes(const cadd_build_head_args* h, size_t* out) 
     int rc = check_build_head(h);
     if (rc != CADD_OK) return rc;
     if (!out) return CADD_ERR_NULL;
-    // sized for the largest cut (32 chunks = 64 records per row), so the answer does not depend on the device
+    // sized for the largest cut (kDraftMaxRecords records per row), so the answer does not depend on the device
     const size_t stride = seg_partial_stride(h->build.K > kPreciseMin ? h->build.K : kPreciseMin);
     const size_t M = (size_t)h->build.batch * h->build.L;
-    *out = ((M * 64 * stride + 255) & ~(size_t)255) + ((M * stride + 255) & ~(size_t)255) + (size_t)kDraftMaxCtas * 2 * kDraftPending * kHeadBM * 8 + 256;
+    *out = ((M * kDraftMaxRecords * stride + 255) & ~(size_t)255) + ((M * stride + 255) & ~(size_t)255) + (size_t)kDraftMaxCtas * 2 * kDraftPending * kHeadBM * 8 + 256;
     return CADD_OK;
 }
 

@@ -18,6 +18,7 @@
 
 namespace cadd {
 
+constexpr int kDraftMaxRecords = 96;      // chunk records per row the merge kernel can fold (three lists per lane)
 constexpr int kDraftMaxKP = 32;           // list capacity per row that fits beside the operand ring in shared memory
 
 constexpr int kDraftStages = 4;           // operand ring as in head_argmax.cuh: about 190 KB in flight cover the TMA latency
@@ -311,14 +312,16 @@ __global__ void __launch_bounds__(128) draft_merge_kernel(DraftHeadParams p, uns
     const int KP = p.KP;
     const size_t stride = seg_partial_stride(KP);
     const double kLog2e = 1.4426950408889634;
-    // lane owns records lane and lane + 32 (at most 64 per row)
-    const SegPartial* hdr[2];
-    const uint64_t* keys[2];
-    int cnt[2], cur[2] = {0, 0};
+    // lane owns records lane, lane + 32 and lane + 64 (at most kDraftMaxRecords per row)
+    constexpr int NL = kDraftMaxRecords / 32;
+    const SegPartial* hdr[NL];
+    const uint64_t* keys[NL];
+    int cnt[NL], cur[NL];
     double Cmax = -1e300;
     uint32_t flags = 0;
     int total = 0;
-    for (int q = 0; q < 2; ++q) {
+    for (int q = 0; q < NL; ++q) {
+        cur[q] = 0;
         const int ch = lane + 32 * q;                            // record index: chunk * halves + column half
         if (ch < p.halves * p.n_chunks) {
             const unsigned char* rec = p.chunk_partials + ((size_t)row * p.n_chunks * p.halves + ch) * stride;
@@ -339,26 +342,32 @@ __global__ void __launch_bounds__(128) draft_merge_kernel(DraftHeadParams p, uns
     uint64_t* out_keys = (uint64_t*)(out + sizeof(SegPartial));
     const int n_out = min(KP, total);
     for (int k = 0; k < n_out; ++k) {
-        const uint64_t h0 = cur[0] < cnt[0] ? keys[0][cur[0]] : 0ull, h1 = cur[1] < cnt[1] ? keys[1][cur[1]] : 0ull;
-        const uint64_t mine = max(h0, h1);
+        uint64_t mine = 0ull;
+        int from = 0;
+#pragma unroll
+        for (int q = 0; q < NL; ++q) {
+            const uint64_t hq = cur[q] < cnt[q] ? keys[q][cur[q]] : 0ull;
+            if (hq > mine) { mine = hq; from = q; }
+        }
         uint64_t best = mine;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(kFullMask, best, o));
         if (mine == best && best != 0ull) {                      // keys are unique across chunks (distinct tokens)
-            if (h0 == best) ++cur[0]; else ++cur[1];
+#pragma unroll
+            for (int q = 0; q < NL; ++q) cur[q] += (q == from) ? 1 : 0;
             out_keys[k] = best;
         }
     }
     // what is left in the lists joins the sum; reference exponent: the largest of the chunks' and the leftovers' own
     double xmax = -1e300;
-    for (int q = 0; q < 2; ++q)
+    for (int q = 0; q < NL; ++q)
         if (cur[q] < cnt[q]) xmax = fmax(xmax, (double)key_value(keys[q][cur[q]]));     // lists are sorted: the first is the largest
     double Cg = fmax(Cmax, xmax > -1e299 ? ceil(xmax * kLog2e) + 1.0 : -1e300);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) Cg = fmax(Cg, __shfl_xor_sync(kFullMask, Cg, o));
     double W = 0.0;
     if (Cg > -1e299) {
-        for (int q = 0; q < 2; ++q) {
+        for (int q = 0; q < NL; ++q) {
             if (!hdr[q]) continue;
             if (hdr[q]->W != 0.0) W += hdr[q]->W * exp2(hdr[q]->C - Cg);
             for (int k = cur[q]; k < cnt[q]; ++k) W += exp2((double)key_value(keys[q][k]) * kLog2e - Cg);
