@@ -127,6 +127,38 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(const void* tile, int k16)
 // (bits 15, 16 = 0), N / 8 in bits 17-22, M / 16 in bits 24-28.
 constexpr uint32_t kHeadIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kHeadBN >> 3) << 17) | ((uint32_t)(kHeadBM >> 4) << 24);
 
+// ---- the two single-thread roles' inner loops, shared by the kernels that run this GEMM pipeline ----
+// Producer: streams the k_steps operand tile pairs of one output tile (row tile mt, column tile nt) into the ring.
+// `s` / `ph` are the ring position and its phase parity, carried across tiles.  Returns false on a wait that ran out.
+template <class Shared, int Stages>
+__device__ __forceinline__ bool head_produce_tile(Shared& sh, const CUtensorMap* map_h, const CUtensorMap* map_w, int mt, int nt,
+                                                  int k_steps, unsigned& s, unsigned& ph) {
+    for (int k = 0; k < k_steps; ++k) {
+        if (!head_wait(&sh.empty[s], ph ^ 1u, 64)) return false;             // first pass over the ring: free at once
+        mbar_arrive_expect_tx(&sh.full[s], kHeadABytes + kHeadBBytes);
+        tma_load_2d(&sh.a[s][0], map_h, k * kHeadBK, mt * kHeadBM, &sh.full[s]);
+        tma_load_2d(&sh.b[s][0], map_w, k * kHeadBK, nt * kHeadBN, &sh.full[s]);
+        if (++s == Stages) { s = 0; ph ^= 1u; }
+    }
+    return true;
+}
+// MMA issuer: accumulates one output tile into the tensor-memory accumulator at `d`; every stage is committed back to
+// the producer once its MMAs have read it, the finished accumulator is committed to `acc_full`.
+template <class Shared, int Stages>
+__device__ __forceinline__ bool head_mma_tile(Shared& sh, uint32_t d, uint64_t* acc_full, int k_steps, unsigned& s, unsigned& ph) {
+    for (int k = 0; k < k_steps; ++k) {
+        if (!head_wait(&sh.full[s], ph)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < kHeadBK / 16; ++kk)
+            umma_bf16(d, umma_desc_k_sw128(&sh.a[s][0], kk), umma_desc_k_sw128(&sh.b[s][0], kk), kHeadIdesc, (k | kk) != 0 ? 1u : 0u);
+        umma_commit(&sh.empty[s]);                                            // the stage is free once these MMAs have read it
+        if (++s == Stages) { s = 0; ph ^= 1u; }
+    }
+    umma_commit(acc_full);                                                    // accumulator complete
+    return true;
+}
+
 // Tile order: groups of group_m row tiles; inside a group the column tile is the outer index and the row tile the
 // inner one.  Work item w (CTA c takes w = c, c + grid, ...) -> (row tile, column tile).
 __device__ __forceinline__ void head_tile_of(const HeadParams& p, int64_t w, int& mt, int& nt) {
@@ -170,13 +202,7 @@ head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
             for (int64_t w = blockIdx.x; w < n_work && !*(volatile uint32_t*)&sh.error; w += gridDim.x) {
                 int mt, nt;
                 head_tile_of(p, w, mt, nt);
-                for (int k = 0; k < k_steps; ++k) {
-                    if (!head_wait(&sh.empty[s], ph ^ 1u, 64)) { sh.error = 1; break; }   // first pass: free at once
-                    mbar_arrive_expect_tx(&sh.full[s], kHeadABytes + kHeadBBytes);
-                    tma_load_2d(&sh.a[s][0], &map_h, k * kHeadBK, mt * kHeadBM, &sh.full[s]);
-                    tma_load_2d(&sh.b[s][0], &map_w, k * kHeadBK, nt * kHeadBN, &sh.full[s]);
-                    if (++s == kHeadStages) { s = 0; ph ^= 1u; }
-                }
+                if (!head_produce_tile<HeadShared, kHeadStages>(sh, &map_h, &map_w, mt, nt, k_steps, s, ph)) { sh.error = 1; break; }
             }
         }
     } else if (warp == 1) {
@@ -188,20 +214,7 @@ head_argmax_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
                 head_tile_of(p, w, mt, nt);
                 if (!head_wait(&sh.acc_empty[buf], aph ^ 1u)) { sh.error = 2; break; }   // epilogue has drained it
                 tc_fence_after();
-                const uint32_t d = tmem_base + buf * kHeadBN;
-                bool ok = true;
-                for (int k = 0; k < k_steps; ++k) {
-                    if (!head_wait(&sh.full[s], ph)) { sh.error = 3; ok = false; break; }
-                    tc_fence_after();
-#pragma unroll
-                    for (int kk = 0; kk < kHeadBK / 16; ++kk)
-                        umma_bf16(d, umma_desc_k_sw128(&sh.a[s][0], kk), umma_desc_k_sw128(&sh.b[s][0], kk), kHeadIdesc,
-                                  (k | kk) != 0 ? 1u : 0u);
-                    umma_commit(&sh.empty[s]);                       // the stage is free once these MMAs have read it
-                    if (++s == kHeadStages) { s = 0; ph ^= 1u; }
-                }
-                if (!ok) break;
-                umma_commit(&sh.acc_full[buf]);                       // accumulator complete
+                if (!head_mma_tile<HeadShared, kHeadStages>(sh, tmem_base + buf * kHeadBN, &sh.acc_full[buf], k_steps, s, ph)) { sh.error = 3; break; }
                 if (++buf == 2) { buf = 0; aph ^= 1u; }
             }
         }

@@ -116,13 +116,7 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
                 if (!draft_tile_live(p, mt)) continue;
                 const int nt1 = min((ch + 1) * p.chunk_tiles, p.n_tiles);
                 for (int nt = ch * p.chunk_tiles; nt < nt1 && !*(volatile uint32_t*)&sh.error; ++nt)
-                    for (int k = 0; k < k_steps; ++k) {
-                        if (!head_wait(&sh.empty[s], ph ^ 1u, 64)) { sh.error = 1; break; }
-                        mbar_arrive_expect_tx(&sh.full[s], kHeadABytes + kHeadBBytes);
-                        tma_load_2d(&sh.a[s][0], &map_h, k * kHeadBK, mt * kHeadBM, &sh.full[s]);
-                        tma_load_2d(&sh.b[s][0], &map_w, k * kHeadBK, nt * kHeadBN, &sh.full[s]);
-                        if (++s == kDraftStages) { s = 0; ph ^= 1u; }
-                    }
+                    if (!head_produce_tile<DraftHeadShared, kDraftStages>(sh, &map_h, &map_w, mt, nt, k_steps, s, ph)) { sh.error = 1; break; }
             }
         }
     } else if (warp == 1) {
@@ -136,20 +130,7 @@ head_softmax_topk_kernel(const __grid_constant__ CUtensorMap map_h, const __grid
                 for (int nt = ch * p.chunk_tiles; nt < nt1 && !*(volatile uint32_t*)&sh.error; ++nt) {
                     if (!head_wait(&sh.acc_empty[buf], aph ^ 1u)) { sh.error = 2; break; }
                     tc_fence_after();
-                    const uint32_t d = tmem_base + buf * kHeadBN;
-                    bool ok = true;
-                    for (int k = 0; k < k_steps; ++k) {
-                        if (!head_wait(&sh.full[s], ph)) { sh.error = 3; ok = false; break; }
-                        tc_fence_after();
-#pragma unroll
-                        for (int kk = 0; kk < kHeadBK / 16; ++kk)
-                            umma_bf16(d, umma_desc_k_sw128(&sh.a[s][0], kk), umma_desc_k_sw128(&sh.b[s][0], kk), kHeadIdesc,
-                                      (k | kk) != 0 ? 1u : 0u);
-                        umma_commit(&sh.empty[s]);
-                        if (++s == kDraftStages) { s = 0; ph ^= 1u; }
-                    }
-                    if (!ok) break;
-                    umma_commit(&sh.acc_full[buf]);
+                    if (!head_mma_tile<DraftHeadShared, kDraftStages>(sh, tmem_base + buf * kHeadBN, &sh.acc_full[buf], k_steps, s, ph)) { sh.error = 3; break; }
                     if (++buf == 2) { buf = 0; aph ^= 1u; }
                 }
             }
