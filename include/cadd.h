@@ -37,7 +37,7 @@
 extern "C" {
 #endif
 
-#define CADD_ABI_VERSION 3
+#define CADD_ABI_VERSION 4
 
 /* ---- return codes (host side, synchronous) ---- */
 #define CADD_OK              0
@@ -220,6 +220,40 @@ typedef struct cadd_build_head_args {
 } cadd_build_head_args;
 
 /*
+ * Tree verification under sampling (temperature T > 0; the paper's T = 1 tables use it but the text does not
+ * define the tree variant).  The reading built here is lossless for a tree of deterministic candidates: at the
+ * current node one token x is drawn from the target's distribution softmax(y / T); if a child of the node carries x
+ * the walk moves there and repeats, otherwise it stops; x is the next bonus token either way.  Replace the draw by
+ * the arg-max and this is cadd_verify_tree.  The random numbers are inputs: one uniform u in [0, 1) per (request,
+ * row); the draw is the inverse CDF in token order, the smallest v with
+ * sum_{w <= v} exp(y_w / T) > u * sum_w exp(y_w / T).  NaN and infinite logits carry no mass; a row without a finite
+ * logit gives token 0.
+ * All pointers are DEVICE pointers owned by the caller; no workspace is needed.
+ */
+typedef struct cadd_sample_args {
+    uint32_t struct_size;          /* = sizeof(cadd_sample_args) */
+    uint32_t flags;                /* reserved, 0 */
+    int32_t  batch, L, R;
+    int32_t  logits_dtype;         /* CADD_DTYPE_* */
+    int32_t  rows_mode;            /* CADD_ROWS_*: LIVE draws for rows 0..n_nodes[b] only (others -1), DENSE for all R rows */
+    int32_t  reserved0;
+    int64_t  V;                    /* at most about 10^6 (bf16) / 5 * 10^5 (fp32) elements per row */
+    double   temperature;          /* T > 0 */
+    const void* target_logits;     /* [batch, R, V]; element (b,j,v) at b*stride_b + j*stride_row + v */
+    int64_t  stride_b, stride_row; /* in elements */
+    const double* uniforms;        /* [batch, R] in [0, 1) */
+    const int32_t* n_nodes;        /* [batch]   from cadd_build_tree */
+    const int32_t* token_ids;      /* [batch,R] from cadd_build_tree */
+    const int32_t* parent_idx;     /* [batch,R] from cadd_build_tree */
+    /* outputs, all required except status */
+    int32_t* node_token;           /* [batch,R] the token drawn at every row read; -1 for rows not read */
+    int32_t* accepted_len;         /* [batch] */
+    int32_t* accepted_nodes;       /* [batch,L], -1 padded */
+    int32_t* next_bonus;           /* [batch] the token drawn at the last accepted node */
+    int32_t* status;               /* [batch] CADD_STATUS_* bits, may be NULL */
+} cadd_sample_args;
+
+/*
  * Offline cost fitting (Section "Offline Cost Profiling", Eq. 12): for each of n_tables profiled context lengths,
  * the least-squares fit to N measured verification latencies (node counts equally spaced, e.g. n = 1..N) among
  * all convex, non-decreasing sequences.  The fitted rows can be passed to cadd_build_tree as cost_table (with
@@ -275,6 +309,11 @@ int cadd_build_head_workspace_bytes(const cadd_build_head_args* a, size_t* out);
  * `cuda_stream`: one small memset and three kernels.  Errors as for cadd_build_tree, plus CADD_ERR_SHAPE for K > 32,
  * CADD_ERR_ALIGN for a base pointer that is not 16-byte aligned or a stride that is not a multiple of 8 elements. */
 int cadd_build_tree_fused_head(const cadd_build_head_args* a, void* cuda_stream);
+
+/* Tree verification with one draw per node from softmax(target logits / T) (see cadd_sample_args).  Asynchronous on
+ * `cuda_stream`: two kernels.  Errors as for cadd_verify_tree; CADD_ERR_SHAPE also for T <= 0 and for rows longer than
+ * the stated limit. */
+int cadd_verify_tree_sampled(const cadd_sample_args* a, void* cuda_stream);
 
 /* Convex, non-decreasing least-squares fit of every row (see cadd_fit_args).  Asynchronous on `cuda_stream`: one
  * kernel, one CTA per row, fp64.  CADD_ERR_SHAPE if N > CADD_FIT_MAX_N. */

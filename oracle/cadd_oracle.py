@@ -214,6 +214,73 @@ def build_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor, K: 
     return build_tree(y64.to(torch.float32), K, B_max, R, **kw), y64
 
 
+def row_sample(row, u: float, temperature: float = 1.0):
+    """One draw from softmax(row / temperature) by the inverse CDF in token order, given the uniform u in [0, 1):
+    the smallest token v with  sum_{w <= v} e_w  >  u * sum_w e_w,  e_w = exp((y_w - max y) / temperature); NaN and
+    infinite logits carry no mass; a row without a finite logit gives token 0.  Returns (token, margin): margin is
+    the distance from u to the nearer end of the token's interval of the CDF, as a fraction of the total (rows whose
+    margin is at rounding level may legitimately resolve to the neighbouring token in another summation order)."""
+    import numpy as np
+    y = torch.as_tensor(row).to(torch.float64).numpy()
+    fin = np.isfinite(y)
+    if not fin.any():
+        return 0, 1.0
+    e = np.where(fin, np.exp((np.where(fin, y, 0.0) - y[fin].max()) / float(temperature)), 0.0)
+    cdf = np.cumsum(e)                       # ascending token order, fp64
+    Z = float(cdf[-1])
+    t = float(u) * Z
+    v = int(np.searchsorted(cdf, t, side="right"))     # first index with cdf > t
+    if v >= len(y):                          # u so close to 1 that u * Z rounds to Z: the last token with mass
+        v = int(np.nonzero(e > 0)[0][-1])
+    below = float(cdf[v - 1]) if v > 0 else 0.0
+    margin = min(float(cdf[v]) - t, t - below if v > 0 and below > 0 else np.inf) / Z
+    return v, float(margin)
+
+
+def accept_walk(L: int, n: int, token_ids_b, parent_idx_b, node_token_b):
+    """O6 for one request with the per-node target tokens given: from the root follow, at each node, the child
+    (lowest row first) whose token equals the target's token at that node.  Returns (accepted rows, next token)."""
+    cur, acc = 0, []
+    while len(acc) < L:
+        g = int(node_token_b[cur])
+        child = next((c for c in range(1, n + 1) if int(parent_idx_b[c]) == cur and int(token_ids_b[c]) == g), -1)
+        if child < 0:
+            break
+        acc.append(child)
+        cur = child
+    return acc, int(node_token_b[cur])
+
+
+def verify_tree_sampled(target_logits: torch.Tensor, uniforms: torch.Tensor, L: int, n_nodes, token_ids, parent_idx,
+                        rows_mode: int = ROWS_LIVE, temperature: float = 1.0):
+    """Tree verification under sampling (the T > 0 setting of the paper's Section 5 tables; the tree variant is
+    this repository's reading): the target's token at node j is ONE draw from softmax(y_j / T) at the supplied uniform
+    uniforms[b, j] (row_sample); the walk is O6 with the drawn tokens in place of the arg-max.  The emitted tokens are
+    distributed as the target's own sampling whatever the tree.  Returns (OracleVerify, margins [batch, R])."""
+    y = target_logits
+    assert y.device.type == "cpu" and y.dim() == 3
+    batch, R, V = y.shape
+    out = OracleVerify(torch.full((batch, R), -1, dtype=torch.int32), torch.zeros(batch, dtype=torch.int32),
+                       torch.full((batch, L), -1, dtype=torch.int32), torch.zeros(batch, dtype=torch.int32),
+                       torch.zeros(batch, dtype=torch.int32))
+    margins = torch.full((batch, R), float("inf"), dtype=torch.float64)
+    for b in range(batch):
+        n = int(n_nodes[b])
+        if n < 0 or n > R - 1:
+            out.status[b] = ST_BAD_N_NODES
+            n = min(max(n, 0), R - 1)
+        for j in range(R):
+            if j <= n or rows_mode == ROWS_DENSE:
+                tok, mg = row_sample(y[b, j], float(uniforms[b, j]), temperature)
+                out.node_argmax[b, j], margins[b, j] = tok, mg
+        acc, nxt = accept_walk(L, n, token_ids[b], parent_idx[b], out.node_argmax[b])
+        out.accepted_len[b] = len(acc)
+        for i, c in enumerate(acc):
+            out.accepted_nodes[b, i] = c
+        out.next_bonus[b] = nxt
+    return out, margins
+
+
 def fit_convex_nondecreasing(y) -> "torch.Tensor":
     """Offline cost fitting (Eq. 12): for each row of y [n_tables, N] (latencies measured at N equally spaced node
     counts) the least-squares fit among all convex, non-decreasing sequences.

@@ -28,7 +28,7 @@ ROWS_LIVE, ROWS_DENSE = 0, 1
 EXPORTS = ("cadd_version", "cadd_status_string", "cadd_build_workspace_bytes", "cadd_verify_workspace_bytes",
            "cadd_build_tree", "cadd_verify_tree", "cadd_build_tree_static_scratch",
            "cadd_head_workspace_bytes", "cadd_verify_tree_fused_head", "cadd_fit_cost_tables",
-           "cadd_build_head_workspace_bytes", "cadd_build_tree_fused_head")
+           "cadd_build_head_workspace_bytes", "cadd_build_tree_fused_head", "cadd_verify_tree_sampled")
 ERR_STATIC_SCRATCH = -8
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -87,6 +87,20 @@ class BuildHeadArgs(C.Structure):
     ]
 
 
+class SampleArgs(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("flags", C.c_uint32),
+        ("batch", C.c_int32), ("L", C.c_int32), ("R", C.c_int32),
+        ("logits_dtype", C.c_int32), ("rows_mode", C.c_int32), ("reserved0", C.c_int32), ("V", C.c_int64),
+        ("temperature", C.c_double),
+        ("target_logits", C.c_void_p), ("stride_b", C.c_int64), ("stride_row", C.c_int64),
+        ("uniforms", C.c_void_p),
+        ("n_nodes", C.c_void_p), ("token_ids", C.c_void_p), ("parent_idx", C.c_void_p),
+        ("node_token", C.c_void_p), ("accepted_len", C.c_void_p), ("accepted_nodes", C.c_void_p),
+        ("next_bonus", C.c_void_p), ("status", C.c_void_p),
+    ]
+
+
 class FitArgs(C.Structure):
     _fields_ = [
         ("struct_size", C.c_uint32), ("flags", C.c_uint32), ("n_tables", C.c_int32), ("N", C.c_int32),
@@ -115,6 +129,7 @@ def lib() -> C.CDLL:
         l.cadd_head_workspace_bytes.argtypes = [C.POINTER(HeadArgs), C.POINTER(C.c_size_t)]
         l.cadd_verify_tree_fused_head.argtypes = [C.POINTER(HeadArgs), C.c_void_p]
         l.cadd_fit_cost_tables.argtypes = [C.POINTER(FitArgs), C.c_void_p]
+        l.cadd_verify_tree_sampled.argtypes = [C.POINTER(SampleArgs), C.c_void_p]
         l.cadd_build_head_workspace_bytes.argtypes = [C.POINTER(BuildHeadArgs), C.POINTER(C.c_size_t)]
         l.cadd_build_tree_fused_head.argtypes = [C.POINTER(BuildHeadArgs), C.c_void_p]
         l.cadd_build_tree_static_scratch.argtypes = [C.POINTER(BuildArgs), C.c_void_p]
@@ -436,6 +451,48 @@ def cadd_build_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor
     for t in keep + [workspace]:
         if t is not None:
             t.record_stream(torch.cuda.current_stream() if stream is None else stream)
+    return out
+
+
+def cadd_verify_tree_sampled(target_logits: torch.Tensor, uniforms: torch.Tensor, L: int, n_nodes: torch.Tensor,
+                             token_ids: torch.Tensor, parent_idx: torch.Tensor, rows_mode: int = ROWS_LIVE, *,
+                             temperature: float = 1.0, out: Optional[Verdict] = None,
+                             stream: Optional[torch.cuda.Stream] = None) -> Verdict:
+    """Tree verification under sampling: one token is drawn per node from softmax(target_logits / temperature) by the
+    inverse CDF at uniforms[b, j]; the walk follows the child that carries the drawn token.  Verdict.node_argmax holds
+    the drawn tokens."""
+    y = target_logits
+    if not (y.is_cuda and uniforms.is_cuda):
+        raise ValueError("target_logits and uniforms must be CUDA tensors (there is no CPU path)")
+    if y.dim() != 3 or y.stride(2) != 1:
+        raise ValueError("target_logits must be [batch, R, V] with a contiguous vocabulary axis")
+    dev = y.device
+    batch, R, V = y.shape
+    if uniforms.dtype != torch.float64 or tuple(uniforms.shape) != (batch, R) or not uniforms.is_contiguous():
+        raise ValueError("uniforms must be a contiguous float64 tensor [batch, R]")
+    for t in (n_nodes, token_ids, parent_idx):
+        if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()):
+            raise ValueError("tree arrays must be contiguous int32 CUDA tensors")
+    a = SampleArgs()
+    a.struct_size = C.sizeof(SampleArgs)
+    a.batch, a.L, a.R, a.V = batch, L, R, V
+    a.logits_dtype = _dtype_code(y)
+    a.rows_mode = rows_mode
+    a.temperature = float(temperature)
+    a.target_logits = y.data_ptr()
+    a.stride_b, a.stride_row = y.stride(0), y.stride(1)
+    a.uniforms = uniforms.data_ptr()
+    a.n_nodes, a.token_ids, a.parent_idx = n_nodes.data_ptr(), token_ids.data_ptr(), parent_idx.data_ptr()
+    if out is None:
+        i32 = lambda *s: torch.empty(*s, dtype=torch.int32, device=dev)
+        out = Verdict(node_argmax=i32(batch, R), accepted_len=i32(batch), accepted_nodes=i32(batch, L),
+                      next_bonus=i32(batch), status=i32(batch))
+    a.node_token, a.accepted_len, a.accepted_nodes = _ptr(out.node_argmax), _ptr(out.accepted_len), _ptr(out.accepted_nodes)
+    a.next_bonus, a.status = _ptr(out.next_bonus), _ptr(out.status)
+    with torch.cuda.device(dev):
+        rc = lib().cadd_verify_tree_sampled(C.byref(a), _stream_ptr(stream))
+    if rc != OK:
+        raise CaddError(rc)
     return out
 
 

@@ -11,6 +11,7 @@
 #include "head_argmax.cuh"
 #include "fit_cost.cuh"
 #include "head_softmax_topk.cuh"
+#include "sample_verify.cuh"
 
 namespace cadd {
 
@@ -512,6 +513,54 @@ int cadd_build_tree_fused_head(const cadd_build_head_args* h, void* cuda_stream)
     draft_merge_kernel<<<(unsigned)((M + 3) / 4), 128, 0, st>>>(dp, merged);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
     return launch_expand(a, pl.KP, 1, merged, st);
+}
+
+// ---------------- tree verification under sampling ----------------
+
+int cadd_verify_tree_sampled(const cadd_sample_args* a, void* cuda_stream) {
+    if (!a) return CADD_ERR_NULL;
+    if (a->struct_size != sizeof(cadd_sample_args)) return CADD_ERR_STRUCT_SIZE;
+    if (a->batch < 1 || a->L < 1 || a->L > 64 || a->R < 1 || a->V < 1 || a->V >= ((int64_t)1 << 31) ||
+        (int64_t)a->batch * a->R >= ((int64_t)1 << 31) || !(a->temperature > 0.0) || !(a->temperature < 1e30))
+        return CADD_ERR_SHAPE;
+    if (a->logits_dtype != CADD_DTYPE_BF16 && a->logits_dtype != CADD_DTYPE_FP32) return CADD_ERR_DTYPE;
+    if (a->rows_mode != CADD_ROWS_LIVE && a->rows_mode != CADD_ROWS_DENSE) return CADD_ERR_DTYPE;
+    const int epc = a->logits_dtype == CADD_DTYPE_BF16 ? 8 : 4;
+    if (a->V / epc / kRunChunks + 3 > kMaxRuns) return CADD_ERR_SHAPE;     // rows longer than the run table
+    if (!a->target_logits || !a->uniforms || !a->n_nodes || !a->token_ids || !a->parent_idx || !a->node_token || !a->accepted_len ||
+        !a->accepted_nodes || !a->next_bonus)
+        return CADD_ERR_NULL;
+    const size_t es = a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
+    if (!aligned(a->target_logits, es) || !aligned(a->uniforms, 8)) return CADD_ERR_ALIGN;
+    if (!aligned(a->n_nodes, 4) || !aligned(a->token_ids, 4) || !aligned(a->parent_idx, 4) || !aligned(a->node_token, 4) ||
+        !aligned(a->accepted_len, 4) || !aligned(a->accepted_nodes, 4) || !aligned(a->next_bonus, 4) || !aligned(a->status, 4))
+        return CADD_ERR_ALIGN;
+    if (a->stride_row < a->V || a->stride_b < 0) return CADD_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    SampleParams sp;
+    sp.logits = a->target_logits; sp.V = a->V; sp.stride_b = a->stride_b; sp.stride_row = a->stride_row;
+    sp.R = a->R; sp.rows_mode = a->rows_mode; sp.c = (float)(1.4426950408889634 / a->temperature);
+    sp.n_nodes = a->n_nodes; sp.uniforms = a->uniforms; sp.node_token = a->node_token;
+    const unsigned rows = (unsigned)((int64_t)a->batch * a->R);
+    const void* kfn = a->logits_dtype == CADD_DTYPE_BF16 ? (const void*)row_sample_kernel<CADD_DTYPE_BF16>
+                                                          : (const void*)row_sample_kernel<CADD_DTYPE_FP32>;
+    if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sample_smem_bytes()) != cudaSuccess) {
+        cudaGetLastError();
+        return CADD_ERR_LAUNCH;
+    }
+    if (a->logits_dtype == CADD_DTYPE_BF16) row_sample_kernel<CADD_DTYPE_BF16><<<rows, kThreads, sample_smem_bytes(), st>>>(sp);
+    else row_sample_kernel<CADD_DTYPE_FP32><<<rows, kThreads, sample_smem_bytes(), st>>>(sp);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+
+    WalkParams wp;                                           // the walk is the greedy one with the drawn tokens in place of the arg-max
+    wp.batch = a->batch; wp.L = a->L; wp.R = a->R; wp.n_nodes = a->n_nodes; wp.token_ids = a->token_ids;
+    wp.parent_idx = a->parent_idx; wp.node_argmax = a->node_token; wp.accepted_len = a->accepted_len;
+    wp.accepted_nodes = a->accepted_nodes; wp.next_bonus = a->next_bonus; wp.status = a->status;
+    const int wpb = 4;
+    accept_walk_kernel<<<(a->batch + wpb - 1) / wpb, wpb * 32, 0, st>>>(wp);
+    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    return CADD_OK;
 }
 
 }  // extern "C"

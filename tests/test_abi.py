@@ -66,7 +66,7 @@ def test_host_validation_codes(lib):
     v.rows_mode = 3
     assert lib.cadd_verify_tree(C.byref(v), None) == G.ERR_DTYPE
     assert G.cadd_status_string(G.ERR_WORKSPACE).startswith("workspace")
-    assert G.cadd_version() == 3
+    assert G.cadd_version() == 4
 
 
 def test_binding_refuses_cpu_tensors():

@@ -41,7 +41,7 @@ def round_trip(cfg, seed, rows_mode=G.ROWS_LIVE, dense_mask=False):
 
 
 def test_library_reports_version():
-    assert G.cadd_version() == 3
+    assert G.cadd_version() == 4
     assert G.cadd_status_string(0) == "ok"
 
 

@@ -614,3 +614,109 @@ def test_convex_fit_brute_force_over_active_sets():
                 best, best_f = sse, f
         f = O.fit_convex_nondecreasing(torch.from_numpy(y)[None])[0].numpy()
         assert abs(float(((y - f) ** 2).sum()) - best) < 1e-9 and np.allclose(f, best_f, atol=1e-7)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Sampling-mode verification: the inverse-CDF draw and the walk with drawn tokens
+# ---------------------------------------------------------------------------------------------------------
+def test_row_sample_closed_forms():
+    # all logits equal: the CDF is (v+1)/V, so the draw is floor(u * V)
+    for V in (1, 2, 10, 1000):
+        row = torch.full((V,), 1.25, dtype=torch.float32)
+        for u in (0.0, 0.049, 0.31, 0.5 + 1e-9, 0.999999):
+            assert O.row_sample(row, u)[0] == int(math.floor(u * V))
+    # two tokens with probabilities 1/4 and 3/4 at T = 1 ...
+    row = torch.tensor([0.0, math.log(3.0)], dtype=torch.float64)
+    assert [O.row_sample(row, u)[0] for u in (0.0, 0.2499, 0.2501, 0.99)] == [0, 0, 1, 1]
+    # ... and the same probabilities from logits twice as far apart at T = 2
+    row2 = torch.tensor([0.0, 2.0 * math.log(3.0)], dtype=torch.float64)
+    assert [O.row_sample(row2, u, 2.0)[0] for u in (0.0, 0.2499, 0.2501, 0.99)] == [0, 0, 1, 1]
+    # one token holds all the mass; a tiny temperature turns the draw into the arg-max
+    row = torch.zeros(50, dtype=torch.float32)
+    row[37] = 2000.0                                   # exp(-2000) underflows: the others carry no mass at all
+    assert all(O.row_sample(row, u)[0] == 37 for u in (0.0, 0.5, 0.999999999))
+    g = torch.Generator().manual_seed(4)
+    y = torch.randn(300, generator=g, dtype=torch.float64)
+    assert all(O.row_sample(y, u, 1e-4)[0] == int(y.argmax()) for u in (0.0, 0.3, 0.999))
+    # values without mass are never drawn; a row with nothing finite gives token 0
+    row = torch.tensor([float("-inf"), float("nan"), 0.0, float("inf"), 0.0], dtype=torch.float32)
+    assert [O.row_sample(row, u)[0] for u in (0.0, 0.49, 0.51, 0.999)] == [2, 2, 4, 4]
+    assert O.row_sample(torch.full((7,), float("nan")), 0.4)[0] == 0
+    # margin: distance of u to the nearer interval end
+    row = torch.zeros(4, dtype=torch.float64)
+    tok, margin = O.row_sample(row, 0.30)
+    assert tok == 1 and abs(margin - 0.05) < 1e-12
+
+
+@pytest.mark.parametrize("T", [0.7, 1.0, 1.6])
+def test_row_sample_frequencies_on_a_uniform_grid(T):
+    """Over the equispaced uniforms (i + 1/2) / N an inverse-CDF sampler returns token v exactly
+    N * p_v times up to one grid point per interval end, with p from the library softmax."""
+    from scipy.special import softmax
+    g = torch.Generator().manual_seed(8)
+    y = (torch.randn(40, generator=g, dtype=torch.float64) * 2.0)
+    p = softmax(y.numpy() / T)
+    N = 4000
+    counts = np.zeros(40, dtype=np.int64)
+    prev = -1
+    for i in range(N):
+        v, _ = O.row_sample(y, (i + 0.5) / N, T)
+        assert v >= prev                      # monotone in u: intervals lie in token order
+        prev = v
+        counts[v] += 1
+    assert np.abs(counts - N * p).max() <= 1.0 + 1e-9
+
+
+def test_accept_walk_with_given_tokens_matches_the_greedy_walk():
+    """Pins the Python walk to the C one: one-hot target logits make the arg-max equal to the given tokens."""
+    g = torch.Generator().manual_seed(12)
+    V, R, L = 12, 9, 4
+    for trial in range(40):
+        n = int(torch.randint(0, R, (1,), generator=g))
+        par = torch.zeros(1, R, dtype=torch.int32)
+        tok = torch.zeros(1, R, dtype=torch.int32)
+        for c in range(1, n + 1):
+            par[0, c] = int(torch.randint(0, c, (1,), generator=g))
+            tok[0, c] = int(torch.randint(0, 3, (1,), generator=g))       # few tokens: matches are frequent
+        given = torch.randint(0, 3, (1, R), generator=g, dtype=torch.int32)
+        y = torch.zeros(1, R, V, dtype=torch.float32)
+        y.scatter_(2, given.long().unsqueeze(-1), 5.0)
+        ref = O.verify_tree(y, L, torch.tensor([n], dtype=torch.int32), tok, par, O.ROWS_DENSE)
+        acc, nxt = O.accept_walk(L, n, tok[0], par[0], given[0])
+        assert len(acc) == int(ref.accepted_len[0]) and nxt == int(ref.next_bonus[0])
+        assert acc == [int(c) for c in ref.accepted_nodes[0, : len(acc)]]
+
+
+def test_sampled_verification_limits_and_losslessness():
+    g = torch.Generator().manual_seed(5)
+    batch, R, V, L = 3, 7, 30, 3
+    y = torch.randn(batch, R, V, generator=g, dtype=torch.float32) * 3.0
+    par = torch.tensor([[0, 0, 0, 1, 1, 3, 2]] * batch, dtype=torch.int32)
+    tok = torch.randint(0, V, (batch, R), generator=g, dtype=torch.int32)
+    n = torch.tensor([6, 4, 0], dtype=torch.int32)
+    u = torch.rand(batch, R, generator=g, dtype=torch.float64)
+    # T -> 0: the greedy verdict, whatever the uniforms
+    cold, _ = O.verify_tree_sampled(y, u, L, n, tok, par, O.ROWS_LIVE, 1e-4)
+    ref = O.verify_tree(y, L, n, tok, par, O.ROWS_LIVE)
+    for f in ("node_argmax", "accepted_len", "accepted_nodes", "next_bonus", "status"):
+        assert torch.equal(getattr(cold, f), getattr(ref, f)), f
+    # LIVE leaves the rows beyond n unread
+    warm, mg = O.verify_tree_sampled(y, u, L, n, tok, par, O.ROWS_LIVE, 1.0)
+    assert int(warm.node_argmax[1, 5]) == -1 and int(warm.node_argmax[2, 1]) == -1 and int(warm.accepted_len[2]) == 0
+    assert torch.isinf(mg[1, 5])
+    # losslessness at the root: over a grid of root uniforms the first emitted token (the accepted child's token, or
+    # the bonus when nothing is accepted) is distributed as softmax(y_root)
+    from scipy.special import softmax
+    p = softmax(y[0, 0].double().numpy())
+    N = 2000
+    counts = np.zeros(V)
+    accepted = 0
+    for i in range(N):
+        u[0, 0] = (i + 0.5) / N
+        v, _ = O.verify_tree_sampled(y[:1], u[:1], L, n[:1], tok[:1], par[:1], O.ROWS_LIVE, 1.0)
+        first = int(tok[0, int(v.accepted_nodes[0, 0])]) if int(v.accepted_len[0]) > 0 else int(v.next_bonus[0])
+        counts[first] += 1
+        accepted += int(v.accepted_len[0]) > 0
+    assert np.abs(counts - N * p).max() <= 1.0 + 1e-9
+    kids = {int(tok[0, c]) for c in (1, 2)}
+    assert abs(accepted - N * sum(p[t] for t in kids)) <= len(kids) + 1e-9
