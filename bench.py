@@ -266,6 +266,14 @@ def run_ours(args, rank, world):
         except Exception as ex:
             fused_draft = {"error": str(ex)[:200]}
 
+    # ---- verification under sampling (T = 1) over the same target logits: one draw per row instead of the arg-max ----
+    sampled = None
+    if not args.no_sampled:
+        try:
+            sampled = sampled_block(G, cfg, tree, y, rows_mode, verify_bytes, dev, min(K, 10))
+        except Exception as ex:
+            sampled = {"error": str(ex)[:200]}
+
     # ---- offline cost fitting on a synthetic 9 x 1024 latency grid (the paper's profiling shape) ----
     cost_fit = None
     if not args.no_fit:
@@ -289,7 +297,7 @@ def run_ours(args, rank, world):
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": f"replicas x{world}",
                        "n_star_mean": round(float(n_star.float().mean()), 2), "n_star_max": int(n_star.max()),
                        "accepted_mean": round(float(verdict.accepted_len.float().mean().item()), 2)},
-            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "fused_draft_head": fused_draft, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "fused_draft_head": fused_draft, "sampled_verify": sampled, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
             "gpu_launches": KERNELS_PER_STEP * K, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
@@ -388,6 +396,27 @@ def draft_head_block(G, cfg, kw, ck, hidden, dev, iters):
                          "frac": round(ach / peak, 4)},
             "library_gemm_ms": round(t_gemm, 4), "build_on_logits_ms": round(t_build, 4),
             "status_bits": int(out.status.max().item()), "iters": iters}
+
+
+def sampled_block(G, cfg, tree, y, rows_mode, verify_bytes, dev, iters):
+    """cadd_verify_tree_sampled at temperature 1 on the step's target logits (the same bytes the arg-max reads)."""
+    gu = torch.Generator(device="cpu").manual_seed(cfg.index + 99)
+    u = torch.rand(cfg.batch, cfg.R, generator=gu, dtype=torch.float64).to(dev)
+    out = G.cadd_verify_tree_sampled(y, u, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, temperature=1.0)
+    for _ in range(2):
+        G.cadd_verify_tree_sampled(y, u, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, temperature=1.0, out=out)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        G.cadd_verify_tree_sampled(y, u, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, temperature=1.0, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    peak, kind = measured_peak_gbs()
+    gbs = verify_bytes / (ms * 1e-3) / 1e9
+    return {"temperature": 1.0, "ms": round(ms, 4), "achieved_gbs": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak, 3),
+            "peak_kind": kind, "accepted_mean": round(float(out.accepted_len.float().mean().item()), 2)}
 
 
 def fit_block(G, dev, iters=5):
@@ -498,6 +527,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (0 = as defined)")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
+    ap.add_argument("--no-sampled", action="store_true", help="skip the sampling-mode verification measurement")
     ap.add_argument("--no-fit", action="store_true", help="skip the offline cost-fitting measurement")
     ap.add_argument("--head-hidden", type=int, default=4096,
                     help="hidden size for the fused output-projection verification measurement (0 = skip)")

@@ -237,7 +237,7 @@ typedef struct cadd_sample_args {
     int32_t  logits_dtype;         /* CADD_DTYPE_* */
     int32_t  rows_mode;            /* CADD_ROWS_*: LIVE draws for rows 0..n_nodes[b] only (others -1), DENSE for all R rows */
     int32_t  reserved0;
-    int64_t  V;                    /* at most about 10^6 (bf16) / 5 * 10^5 (fp32) elements per row */
+    int64_t  V;                    /* at most 650,000 (bf16) / 325,000 (fp32) elements per row */
     double   temperature;          /* T > 0 */
     const void* target_logits;     /* [batch, R, V]; element (b,j,v) at b*stride_b + j*stride_row + v */
     int64_t  stride_b, stride_row; /* in elements */

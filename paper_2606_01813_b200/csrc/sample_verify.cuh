@@ -17,11 +17,13 @@
 #include "common.cuh"
 #include "tile_ring.cuh"
 #include "verify.cuh"
+#include "softmax_topk.cuh"     // packed fp32x2 helpers, ex2_approx
 
 namespace cadd {
 
 constexpr int kRunChunks = kTileChunks / (kThreads / 32);     // 128 chunks = 2 KB per warp and tile
-constexpr int kMaxRuns = 1024;                                // runs per row kept in shared memory (V up to ~1M bf16 / 0.5M fp32 elements)
+constexpr int kMaxRuns = 640;                                 // runs per row kept in shared memory (V up to 650k bf16 / 325k fp32 elements);
+                                                              // sized so that four CTAs fit in an SM's shared memory
 
 struct SampleParams {
     const void* logits;        // [batch, R, V]
@@ -38,20 +40,14 @@ struct SampleShared {
     unsigned released[kStages];
     unsigned timeout;
     int n_runs;
-    float run_m[kMaxRuns];                // per run: maximum (finite elements; -Inf if none)
-    double run_s[kMaxRuns];               // per run: sum of exp((y - m) / T)
+    float run_ref[kMaxRuns];              // per run: reference exponent = fp32(max * log2(e) / T) over its finite elements; -Inf if none
+    double run_s[kMaxRuns];               // per run: sum of 2^(y * log2(e) / T - reference)
     alignas(128) uint4 ring[kStages][kTileChunks];
 };
 inline size_t sample_smem_bytes() { return sizeof(SampleShared) + 128; }
 
-__device__ __forceinline__ float ex2f(float t) {
-    float r;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
-    return r;
-}
-
 template <int DT>
-__global__ void __launch_bounds__(kThreads, 3) row_sample_kernel(SampleParams p) {
+__global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p) {
     using E = Elem<DT>;
     extern __shared__ __align__(16) unsigned char sample_smem_raw[];
     SampleShared& sh = *reinterpret_cast<SampleShared*>(sample_smem_raw + ((128u - (smem_u32(sample_smem_raw) & 127u)) & 127u));
@@ -103,13 +99,15 @@ __global__ void __launch_bounds__(kThreads, 3) row_sample_kernel(SampleParams p)
         float m = x;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, o));
-        double s = (lane < cnt && x > -INFINITY) ? (double)ex2f((x - m) * p.c) : 0.0;
+        const float ref = m * p.c;
+        double s = (lane < cnt && x > -INFINITY) ? (double)ex2_approx(fmaf(x, p.c, -ref)) : 0.0;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(kFullMask, s, o);
-        if (lane == 0) { const int r = warp == 0 ? 0 : n_runs - 1; sh.run_m[r] = m; sh.run_s[r] = s; }
+        if (lane == 0) { const int r = warp == 0 ? 0 : n_runs - 1; sh.run_ref[r] = ref; sh.run_s[r] = s; }
     }
 
     unsigned st = 0, phase = 0;
+    const uint64_t c2 = pack2(p.c, p.c);
     for (int t = 0; t < n_tiles; ++t) {
         if (!__all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase))) { sh.timeout = 1; break; }
         // this warp's run of the tile: chunks [c0, c0 + kRunChunks), four per lane
@@ -117,35 +115,71 @@ __global__ void __launch_bounds__(kThreads, 3) row_sample_kernel(SampleParams p)
         const int nvw = max(0, min(kRunChunks, nc - c0));
         if (nvw > 0) {
             const uint4* run = &sh.ring[st][warp * kRunChunks];
-            float f[4 * E::EPC];
-            float m = -INFINITY;
+            const uint32_t ninf = E::ES == 2 ? 0xff80ff80u : 0xff800000u;      // -Inf in every element of a word
+            uint4 w[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (u * 32 + lane < nvw) {
-                    E::unpack(run[u * 32 + lane], &f[u * E::EPC]);
+            for (int u = 0; u < 4; ++u) w[u] = u * 32 + lane < nvw ? run[u * 32 + lane] : make_uint4(ninf, ninf, ninf, ninf);
+            // fast path: packed maximum (NaN ignored), one packed FMA per two elements, one ex2 per element.
+            // A +Inf or a NaN in the run shows as an infinite maximum or a NaN sum and sends the warp to the
+            // element-by-element path below.
+            float m = E::max4(w[0], w[1], w[2], w[3]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, o));
+            float ref = m * p.c;                                                // reference exponent of the run
+            double s = 0.0;
+            bool careful = !(m < INFINITY);                                     // +Inf, or nothing but NaN
+            if (!careful && m > -INFINITY) {
+                const uint64_t nref2 = pack2(-ref, -ref);
+                uint64_t acc2 = 0ull;                                           // {0.0f, 0.0f}
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    float f[E::EPC];
+                    E::unpack(w[u], f);
+                    uint64_t pr[E::EPC / 2];
+#pragma unroll
+                    for (int q = 0; q < E::EPC; q += 2) {
+                        float t0, t1;
+                        unpack2(fma2(pack2(f[q], f[q + 1]), c2, nref2), t0, t1);
+                        pr[q / 2] = pack2(ex2_approx(t0), ex2_approx(t1));     // exp2(-Inf) = 0
+                    }
+                    uint64_t r2 = add2(pr[0], pr[1]);
+                    if constexpr (E::EPC == 8) r2 = add2(r2, add2(pr[2], pr[3]));
+                    acc2 = add2(acc2, r2);
+                }
+                float a0, a1;
+                unpack2(acc2, a0, a1);
+                s = (double)(a0 + a1);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(kFullMask, s, o);
+                careful = !(s == s);                                            // a NaN among the elements
+            }
+            if (careful) {                                                      // warp-uniform, rare
+                float f[4 * E::EPC];
+                m = -INFINITY;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    E::unpack(w[u], &f[u * E::EPC]);
 #pragma unroll
                     for (int q = 0; q < E::EPC; ++q) {
                         float& x = f[u * E::EPC + q];
-                        if (!(fabsf(x) < INFINITY)) x = -INFINITY;          // NaN and infinities carry no mass
+                        if (!(fabsf(x) < INFINITY)) x = -INFINITY;              // NaN and infinities carry no mass
                         m = fmaxf(m, x);
                     }
-                } else {
-#pragma unroll
-                    for (int q = 0; q < E::EPC; ++q) f[u * E::EPC + q] = -INFINITY;
                 }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, o));
+                ref = m * p.c;
+                float part = 0.0f;
+                if (m > -INFINITY) {
+#pragma unroll
+                    for (int q = 0; q < 4 * E::EPC; ++q) part += ex2_approx(fmaf(f[q], p.c, -ref));
+                }
+                s = (double)part;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(kFullMask, s, o);
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, o));
-            float part = 0.0f;
-            if (m > -INFINITY) {
-#pragma unroll
-                for (int q = 0; q < 4 * E::EPC; ++q) part += ex2f((f[q] - m) * p.c);   // exp2(-inf) = 0
-            }
-            double s = (double)part;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(kFullMask, s, o);
             const int r = 1 + c0 / kRunChunks;
-            if (lane == 0 && r < kMaxRuns) { sh.run_m[r] = m; sh.run_s[r] = s; }
+            if (lane == 0 && r < kMaxRuns) { sh.run_ref[r] = ref; sh.run_s[r] = s; }
         }
         __syncwarp();
         if (lane == 0 && atomicAdd(&sh.released[st], 1u) == kThreads / 32 - 1) {
@@ -156,35 +190,42 @@ __global__ void __launch_bounds__(kThreads, 3) row_sample_kernel(SampleParams p)
     }
     __syncthreads();
 
-    // ---- combine the runs (warp 0): global maximum, total, the run that holds the crossing ----
+    // ---- combine the runs (warp 0): common reference, total, the run that holds the crossing ----
+    // Everything below is in "run units": an element's mass inside run r is the very term the streaming pass summed,
+    // ex2(y * c - ref_r), and the run's weight in the row is s_r * 2^(ref_r - M) with M the largest reference.
     if (warp == 0) {
         const int nr = min(n_runs, kMaxRuns);
         float M = -INFINITY;
-        for (int r = lane; r < nr; r += 32) M = fmaxf(M, sh.run_m[r]);
+        for (int r = lane; r < nr; r += 32) M = fmaxf(M, sh.run_ref[r]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFullMask, M, o));
         int32_t ans = 0;                                           // no finite logit at all: token 0, as the arg-max does
         if (M > -INFINITY && !sh.timeout) {
-            // weights of the runs relative to M, in fp64; prefix over the runs in token order, 32 runs per step
+            // weights of the runs relative to M (kept in place of the sums); prefix in token order, 32 runs per step
             double Z = 0.0;
-            for (int r = lane; r < nr; r += 32)
-                if (sh.run_m[r] > -INFINITY) Z += sh.run_s[r] * exp2((double)(sh.run_m[r] - M) * (double)p.c);
+            for (int r = lane; r < nr; r += 32) {
+                const float ref = sh.run_ref[r];
+                const double wgt = ref > -INFINITY ? sh.run_s[r] * (double)ex2_approx((float)((double)ref - (double)M)) : 0.0;
+                sh.run_s[r] = wgt;
+                Z += wgt;
+            }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) Z += __shfl_xor_sync(kFullMask, Z, o);
+            __syncwarp();
             const double target = p.uniforms[(int64_t)b * p.R + j] * Z;
             double before = 0.0;                                   // mass of the runs before the current block of 32
             int hit_run = -1;
             double hit_before = 0.0;
             for (int r0 = 0; r0 < nr && hit_run < 0; r0 += 32) {
                 const int r = r0 + lane;
-                const double wgt = (r < nr && sh.run_m[r] > -INFINITY) ? sh.run_s[r] * exp2((double)(sh.run_m[r] - M) * (double)p.c) : 0.0;
+                const double wgt = r < nr ? sh.run_s[r] : 0.0;
                 double incl = wgt;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const double up = __shfl_up_sync(kFullMask, incl, o);
                     if (lane >= o) incl += up;
                 }
-                const unsigned cross = __ballot_sync(kFullMask, r < nr && wgt > 0.0 && before + incl > target);
+                const unsigned cross = __ballot_sync(kFullMask, wgt > 0.0 && before + incl > target);
                 if (cross) {
                     const int l = __ffs(cross) - 1;
                     hit_run = r0 + l;
@@ -192,47 +233,64 @@ __global__ void __launch_bounds__(kThreads, 3) row_sample_kernel(SampleParams p)
                 }
                 before += __shfl_sync(kFullMask, incl, 31);
             }
-            if (hit_run < 0) {                                     // rounding left the target a hair above the total: last run with mass
+            bool take_last = false;                                // rounding left the target a hair above the total:
+            if (hit_run < 0) {                                     // the last element with mass of the last run with mass
                 for (int r = nr - 1; r >= 0 && hit_run < 0; --r)
-                    if (sh.run_m[r] > -INFINITY && sh.run_s[r] > 0.0) hit_run = r;
-                hit_before = -1.0;                                 // marks "take the run's last element with mass"
+                    if (sh.run_s[r] > 0.0) hit_run = r;
+                take_last = true;
             }
-            // ---- scan the elements of that run in token order: 32 consecutive elements per lane ----
-            int64_t e0;
-            int ne;
-            if (hit_run == 0) { e0 = 0; ne = sp.head; }
-            else if (hit_run == n_runs - 1) { e0 = p.V - sp.tail; ne = sp.tail; }
-            else { e0 = sp.head + (int64_t)(hit_run - 1) * kRunChunks * E::EPC; ne = (int)min((int64_t)kRunChunks * E::EPC, sp.head + (int64_t)nc * E::EPC - e0); }
-            const int per = (ne + 31) / 32;
-            const int lo = lane * per, hi = min(ne, lo + per);
+            const float ref = sh.run_ref[hit_run];
+            // mass wanted inside the run, in the run's own units
+            const double need = take_last ? 1e300 : (target - hit_before) / (double)ex2_approx((float)((double)ref - (double)M));
+            // ---- the elements of that run in token order: consecutive elements per lane, the streaming pass's terms ----
+            constexpr int EPL = (kRunChunks / 32) * E::EPC;        // elements per lane in a body run: 32 (bf16) / 16 (fp32)
+            float tm[EPL];
+            int64_t e0;                                            // token of this lane's first element
+            if (hit_run == 0 || hit_run == n_runs - 1) {           // scalar head / tail: one element per lane
+                const int cnt = hit_run == 0 ? sp.head : sp.tail;
+                e0 = (hit_run == 0 ? 0 : p.V - sp.tail) + lane;
+#pragma unroll
+                for (int q = 0; q < EPL; ++q) tm[q] = 0.0f;
+                if (lane < cnt) {
+                    const float x = E::load(row, e0);
+                    if (fabsf(x) < INFINITY) tm[0] = ex2_approx(fmaf(x, p.c, -ref));
+                }
+            } else {
+                const int rc0 = (hit_run - 1) * kRunChunks;        // first chunk of the run
+                e0 = sp.head + ((int64_t)rc0 + lane * (kRunChunks / 32)) * E::EPC;
+#pragma unroll
+                for (int u = 0; u < kRunChunks / 32; ++u) {
+                    const int cidx = rc0 + lane * (kRunChunks / 32) + u;
+                    float f[E::EPC];
+                    if (cidx < nc) E::unpack(body[cidx], f);
+#pragma unroll
+                    for (int q = 0; q < E::EPC; ++q)
+                        tm[u * E::EPC + q] = (cidx < nc && fabsf(f[q]) < INFINITY) ? ex2_approx(fmaf(f[q], p.c, -ref)) : 0.0f;
+                }
+            }
             double mine = 0.0;
-            for (int q = lo; q < hi; ++q) {
-                const float x = E::load(row, e0 + q);
-                if (fabsf(x) < INFINITY) mine += exp2((double)(x - M) * (double)p.c);
-            }
+#pragma unroll
+            for (int q = 0; q < EPL; ++q) mine += (double)tm[q];
             double incl = mine;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const double up = __shfl_up_sync(kFullMask, incl, o);
                 if (lane >= o) incl += up;
             }
-            const double need = hit_before < 0.0 ? 1e300 : target - hit_before;      // mass wanted inside the run
             unsigned cross = __ballot_sync(kFullMask, mine > 0.0 && incl > need);
             if (!cross) cross = 0x80000000u >> __clz(__ballot_sync(kFullMask, mine > 0.0) | 1u);   // the last lane with mass
             const int l = __ffs(cross) - 1;
-            const double base = __shfl_sync(kFullMask, incl - mine, l);
-            if (lane == l) {
-                double acc = base;
-                int64_t pick = -1, last = -1;
-                for (int q = lo; q < hi; ++q) {
-                    const float x = E::load(row, e0 + q);
-                    if (!(fabsf(x) < INFINITY)) continue;
-                    acc += exp2((double)(x - M) * (double)p.c);
-                    last = e0 + q;
-                    if (acc > need) { pick = e0 + q; break; }
+            double acc = incl - mine;                              // mass before this lane's elements
+            int pick = -1, last = 0;
+#pragma unroll
+            for (int q = 0; q < EPL; ++q) {
+                acc += (double)tm[q];
+                if (tm[q] > 0.0f) {
+                    last = q;
+                    if (pick < 0 && acc > need) pick = q;
                 }
-                ans = (int32_t)(pick >= 0 ? pick : last);
             }
+            ans = (int32_t)(e0 + (pick >= 0 ? pick : last));
             ans = __shfl_sync(kFullMask, ans, l);
         }
         if (sh.timeout) ans = -2;
