@@ -46,6 +46,118 @@ struct SampleShared {
 };
 inline size_t sample_smem_bytes() { return sizeof(SampleShared) + 128; }
 
+// Combine step of row_sample_kernel, run by one warp once the row's runs are in shared memory.  Kept out of line so
+// that its registers (a lane's 32 terms of the crossing run) do not weigh on the streaming loop.
+// Everything is in "run units": an element's mass inside run r is the very term the streaming pass summed,
+// ex2(y * c - ref_r), and the run's weight in the row is s_r * 2^(ref_r - M) with M the largest reference.
+template <int DT>
+__device__ __noinline__ int32_t sample_combine(SampleShared& sh, int n_runs, float c, double u, const char* row, RowSplit sp,
+                                               const uint4* body, int64_t V) {
+    using E = Elem<DT>;
+    const int lane = threadIdx.x & 31;
+    const int nc = sp.n_chunks;
+    const int nr = min(n_runs, kMaxRuns);
+    float M = -INFINITY;
+    for (int r = lane; r < nr; r += 32) M = fmaxf(M, sh.run_ref[r]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFullMask, M, o));
+    int32_t ans = 0;                                           // no finite logit at all: token 0, as the arg-max does
+    if (M > -INFINITY) {
+        // weights of the runs relative to M (kept in place of the sums); prefix in token order, 32 runs per step
+        double Z = 0.0;
+        for (int r = lane; r < nr; r += 32) {
+            const float ref = sh.run_ref[r];
+            const double wgt = ref > -INFINITY ? sh.run_s[r] * (double)ex2_approx((float)((double)ref - (double)M)) : 0.0;
+            sh.run_s[r] = wgt;
+            Z += wgt;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) Z += __shfl_xor_sync(kFullMask, Z, o);
+        __syncwarp();
+        const double target = u * Z;
+        double before = 0.0;                                   // mass of the runs before the current block of 32
+        int hit_run = -1;
+        double hit_before = 0.0;
+        for (int r0 = 0; r0 < nr && hit_run < 0; r0 += 32) {
+            const int r = r0 + lane;
+            const double wgt = r < nr ? sh.run_s[r] : 0.0;
+            double incl = wgt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double up = __shfl_up_sync(kFullMask, incl, o);
+                if (lane >= o) incl += up;
+            }
+            const unsigned cross = __ballot_sync(kFullMask, wgt > 0.0 && before + incl > target);
+            if (cross) {
+                const int l = __ffs(cross) - 1;
+                hit_run = r0 + l;
+                hit_before = before + __shfl_sync(kFullMask, incl - wgt, l);
+            }
+            before += __shfl_sync(kFullMask, incl, 31);
+        }
+        bool take_last = false;                                // rounding left the target a hair above the total:
+        if (hit_run < 0) {                                     // the last element with mass of the last run with mass
+            for (int r = nr - 1; r >= 0 && hit_run < 0; --r)
+                if (sh.run_s[r] > 0.0) hit_run = r;
+            take_last = true;
+        }
+        const float ref = sh.run_ref[hit_run];
+        // mass wanted inside the run, in the run's own units
+        const double need = take_last ? 1e300 : (target - hit_before) / (double)ex2_approx((float)((double)ref - (double)M));
+        // ---- the elements of that run in token order: consecutive elements per lane, the streaming pass's terms ----
+        constexpr int EPL = (kRunChunks / 32) * E::EPC;        // elements per lane in a body run: 32 (bf16) / 16 (fp32)
+        float tm[EPL];
+        int64_t e0;                                            // token of this lane's first element
+        if (hit_run == 0 || hit_run == n_runs - 1) {           // scalar head / tail: one element per lane
+            const int cnt = hit_run == 0 ? sp.head : sp.tail;
+            e0 = (hit_run == 0 ? 0 : V - sp.tail) + lane;
+#pragma unroll
+            for (int q = 0; q < EPL; ++q) tm[q] = 0.0f;
+            if (lane < cnt) {
+                const float x = E::load(row, e0);
+                if (fabsf(x) < INFINITY) tm[0] = ex2_approx(fmaf(x, c, -ref));
+            }
+        } else {
+            const int rc0 = (hit_run - 1) * kRunChunks;        // first chunk of the run
+            e0 = sp.head + ((int64_t)rc0 + lane * (kRunChunks / 32)) * E::EPC;
+#pragma unroll
+            for (int u = 0; u < kRunChunks / 32; ++u) {
+                const int cidx = rc0 + lane * (kRunChunks / 32) + u;
+                float f[E::EPC];
+                if (cidx < nc) E::unpack(body[cidx], f);
+#pragma unroll
+                for (int q = 0; q < E::EPC; ++q)
+                    tm[u * E::EPC + q] = (cidx < nc && fabsf(f[q]) < INFINITY) ? ex2_approx(fmaf(f[q], c, -ref)) : 0.0f;
+            }
+        }
+        double mine = 0.0;
+#pragma unroll
+        for (int q = 0; q < EPL; ++q) mine += (double)tm[q];
+        double incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(kFullMask, incl, o);
+            if (lane >= o) incl += up;
+        }
+        unsigned cross = __ballot_sync(kFullMask, mine > 0.0 && incl > need);
+        if (!cross) cross = 0x80000000u >> __clz(__ballot_sync(kFullMask, mine > 0.0) | 1u);   // the last lane with mass
+        const int l = __ffs(cross) - 1;
+        double acc = incl - mine;                              // mass before this lane's elements
+        int pick = -1, last = 0;
+#pragma unroll
+        for (int q = 0; q < EPL; ++q) {
+            acc += (double)tm[q];
+            if (tm[q] > 0.0f) {
+                last = q;
+                if (pick < 0 && acc > need) pick = q;
+            }
+        }
+        ans = (int32_t)(e0 + (pick >= 0 ? pick : last));
+        ans = __shfl_sync(kFullMask, ans, l);
+    }
+    return ans;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p) {
     using E = Elem<DT>;
@@ -190,110 +302,10 @@ __global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p)
     }
     __syncthreads();
 
-    // ---- combine the runs (warp 0): common reference, total, the run that holds the crossing ----
-    // Everything below is in "run units": an element's mass inside run r is the very term the streaming pass summed,
-    // ex2(y * c - ref_r), and the run's weight in the row is s_r * 2^(ref_r - M) with M the largest reference.
+    // ---- combine the runs (warp 0): total, the run that holds the crossing, the token inside it ----
     if (warp == 0) {
-        const int nr = min(n_runs, kMaxRuns);
-        float M = -INFINITY;
-        for (int r = lane; r < nr; r += 32) M = fmaxf(M, sh.run_ref[r]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFullMask, M, o));
-        int32_t ans = 0;                                           // no finite logit at all: token 0, as the arg-max does
-        if (M > -INFINITY && !sh.timeout) {
-            // weights of the runs relative to M (kept in place of the sums); prefix in token order, 32 runs per step
-            double Z = 0.0;
-            for (int r = lane; r < nr; r += 32) {
-                const float ref = sh.run_ref[r];
-                const double wgt = ref > -INFINITY ? sh.run_s[r] * (double)ex2_approx((float)((double)ref - (double)M)) : 0.0;
-                sh.run_s[r] = wgt;
-                Z += wgt;
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) Z += __shfl_xor_sync(kFullMask, Z, o);
-            __syncwarp();
-            const double target = p.uniforms[(int64_t)b * p.R + j] * Z;
-            double before = 0.0;                                   // mass of the runs before the current block of 32
-            int hit_run = -1;
-            double hit_before = 0.0;
-            for (int r0 = 0; r0 < nr && hit_run < 0; r0 += 32) {
-                const int r = r0 + lane;
-                const double wgt = r < nr ? sh.run_s[r] : 0.0;
-                double incl = wgt;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const double up = __shfl_up_sync(kFullMask, incl, o);
-                    if (lane >= o) incl += up;
-                }
-                const unsigned cross = __ballot_sync(kFullMask, wgt > 0.0 && before + incl > target);
-                if (cross) {
-                    const int l = __ffs(cross) - 1;
-                    hit_run = r0 + l;
-                    hit_before = before + __shfl_sync(kFullMask, incl - wgt, l);
-                }
-                before += __shfl_sync(kFullMask, incl, 31);
-            }
-            bool take_last = false;                                // rounding left the target a hair above the total:
-            if (hit_run < 0) {                                     // the last element with mass of the last run with mass
-                for (int r = nr - 1; r >= 0 && hit_run < 0; --r)
-                    if (sh.run_s[r] > 0.0) hit_run = r;
-                take_last = true;
-            }
-            const float ref = sh.run_ref[hit_run];
-            // mass wanted inside the run, in the run's own units
-            const double need = take_last ? 1e300 : (target - hit_before) / (double)ex2_approx((float)((double)ref - (double)M));
-            // ---- the elements of that run in token order: consecutive elements per lane, the streaming pass's terms ----
-            constexpr int EPL = (kRunChunks / 32) * E::EPC;        // elements per lane in a body run: 32 (bf16) / 16 (fp32)
-            float tm[EPL];
-            int64_t e0;                                            // token of this lane's first element
-            if (hit_run == 0 || hit_run == n_runs - 1) {           // scalar head / tail: one element per lane
-                const int cnt = hit_run == 0 ? sp.head : sp.tail;
-                e0 = (hit_run == 0 ? 0 : p.V - sp.tail) + lane;
-#pragma unroll
-                for (int q = 0; q < EPL; ++q) tm[q] = 0.0f;
-                if (lane < cnt) {
-                    const float x = E::load(row, e0);
-                    if (fabsf(x) < INFINITY) tm[0] = ex2_approx(fmaf(x, p.c, -ref));
-                }
-            } else {
-                const int rc0 = (hit_run - 1) * kRunChunks;        // first chunk of the run
-                e0 = sp.head + ((int64_t)rc0 + lane * (kRunChunks / 32)) * E::EPC;
-#pragma unroll
-                for (int u = 0; u < kRunChunks / 32; ++u) {
-                    const int cidx = rc0 + lane * (kRunChunks / 32) + u;
-                    float f[E::EPC];
-                    if (cidx < nc) E::unpack(body[cidx], f);
-#pragma unroll
-                    for (int q = 0; q < E::EPC; ++q)
-                        tm[u * E::EPC + q] = (cidx < nc && fabsf(f[q]) < INFINITY) ? ex2_approx(fmaf(f[q], p.c, -ref)) : 0.0f;
-                }
-            }
-            double mine = 0.0;
-#pragma unroll
-            for (int q = 0; q < EPL; ++q) mine += (double)tm[q];
-            double incl = mine;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const double up = __shfl_up_sync(kFullMask, incl, o);
-                if (lane >= o) incl += up;
-            }
-            unsigned cross = __ballot_sync(kFullMask, mine > 0.0 && incl > need);
-            if (!cross) cross = 0x80000000u >> __clz(__ballot_sync(kFullMask, mine > 0.0) | 1u);   // the last lane with mass
-            const int l = __ffs(cross) - 1;
-            double acc = incl - mine;                              // mass before this lane's elements
-            int pick = -1, last = 0;
-#pragma unroll
-            for (int q = 0; q < EPL; ++q) {
-                acc += (double)tm[q];
-                if (tm[q] > 0.0f) {
-                    last = q;
-                    if (pick < 0 && acc > need) pick = q;
-                }
-            }
-            ans = (int32_t)(e0 + (pick >= 0 ? pick : last));
-            ans = __shfl_sync(kFullMask, ans, l);
-        }
-        if (sh.timeout) ans = -2;
+        int32_t ans = -2;                                          // a wait ran out: no draw
+        if (!sh.timeout) ans = sample_combine<DT>(sh, n_runs, p.c, p.uniforms[(int64_t)b * p.R + j], row, sp, body, p.V);
         if (lane == 0) *out = ans;
     }
 }
