@@ -357,6 +357,69 @@ __device__ __forceinline__ uint64_t chunk_exp_sum2(const uint4& w, uint64_t l2e_
     return r;
 }
 
+// Careful path of softmax_topk_partial_kernel: the segment element by element from global memory under a CTA-wide
+// protocol (taken when the candidate buffer overflowed or the sum came out non-finite).  Out of line: it is rare and
+// large, and the streaming loop's code should not carry it.  Leaves the winners sorted in win[].
+template <int DT>
+__device__ __noinline__ ThreadSum careful_segment(TopkShared& sh, const char* row, RowSplit sp, int64_t V, int seg, int S,
+                                                  int c_begin, int c_end, int KP, uint32_t* flags_out) {
+    using E = Elem<DT>;
+    const int tid = threadIdx.x;
+    ThreadSum s;
+    uint32_t flags;
+    __syncthreads();
+    if (tid == 0) { sh.count = 0; sh.nwin = 0; sh.thr_key = 0; sh.thr_val = -INFINITY; }
+    __syncthreads();
+    s = ThreadSum{0.0, -INFINITY, 0.0f};
+    flags = 0;
+    bool want_refresh = false;
+    if (seg == 0 && tid < sp.head) slow_element(sh, s, flags, want_refresh, E::load(row, tid), (uint32_t)tid);
+    if (seg == S - 1 && tid < sp.tail) {
+        const int64_t e = V - sp.tail + tid;
+        slow_element(sh, s, flags, want_refresh, E::load(row, e), (uint32_t)e);
+    }
+    for (int cbase = c_begin; cbase < c_end; cbase += kThreads) {
+        const int c = cbase + tid;
+        uint32_t dropped = 0;
+        if (c < c_end) {
+            const int64_t e0 = sp.head + (int64_t)c * E::EPC;
+#pragma unroll 1
+            for (int q = 0; q < E::EPC; ++q)
+                if (slow_element(sh, s, flags, want_refresh, E::load(row, e0 + q), (uint32_t)(e0 + q))) dropped |= 1u << q;
+        }
+        if (__syncthreads_or(want_refresh || dropped != 0)) {
+            want_refresh = false;
+            for (;;) {
+                s = refresh_candidates(sh, s, KP);
+                uint32_t again = 0;
+                while (dropped) {                               // retry what did not fit
+                    const int q = __ffs(dropped) - 1;
+                    dropped &= dropped - 1;
+                    const int64_t e = sp.head + (int64_t)c * E::EPC + q;
+                    if (slow_element(sh, s, flags, want_refresh, E::load(row, e), (uint32_t)e)) again |= 1u << q;
+                }
+                dropped = again;
+                if (!__syncthreads_or(dropped != 0 || want_refresh)) break;
+                want_refresh = false;
+            }
+        }
+    }
+    s = refresh_candidates(sh, s, KP);                          // leaves min(KP, candidates) keys in keys[]
+    __syncthreads();
+    // sort them into win[] by counting
+    const int cnt = (int)sh.count;
+    if (tid < cnt) {
+        const uint64_t k = sh.keys[tid];
+        int rank = 0;
+        for (int q = 0; q < cnt; ++q) rank += sh.keys[q] > k;
+        sh.win[rank] = k;
+    }
+    if (tid == 0) sh.nwin = cnt;
+    __syncthreads();
+    *flags_out = flags;
+    return s;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkParams p) {
     using E = Elem<DT>;
@@ -629,55 +692,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
 
     // ================= careful path: element by element from global memory, CTA-wide protocol =================
     if (redo) {
-        __syncthreads();
-        if (tid == 0) { sh.count = 0; sh.nwin = 0; sh.thr_key = 0; sh.thr_val = -INFINITY; }
-        __syncthreads();
-        s = ThreadSum{0.0, -INFINITY, 0.0f};
-        flags = 0;
-        bool want_refresh = false;
-        if (seg == 0 && tid < sp.head) slow_element(sh, s, flags, want_refresh, E::load(row, tid), (uint32_t)tid);
-        if (seg == p.S - 1 && tid < sp.tail) {
-            const int64_t e = p.V - sp.tail + tid;
-            slow_element(sh, s, flags, want_refresh, E::load(row, e), (uint32_t)e);
-        }
-        for (int cbase = c_begin; cbase < c_end; cbase += kThreads) {
-            const int c = cbase + tid;
-            uint32_t dropped = 0;
-            if (c < c_end) {
-                const int64_t e0 = sp.head + (int64_t)c * E::EPC;
-#pragma unroll 1
-                for (int q = 0; q < E::EPC; ++q)
-                    if (slow_element(sh, s, flags, want_refresh, E::load(row, e0 + q), (uint32_t)(e0 + q))) dropped |= 1u << q;
-            }
-            if (__syncthreads_or(want_refresh || dropped != 0)) {
-                want_refresh = false;
-                for (;;) {
-                    s = refresh_candidates(sh, s, KP);
-                    uint32_t again = 0;
-                    while (dropped) {                               // retry what did not fit
-                        const int q = __ffs(dropped) - 1;
-                        dropped &= dropped - 1;
-                        const int64_t e = sp.head + (int64_t)c * E::EPC + q;
-                        if (slow_element(sh, s, flags, want_refresh, E::load(row, e), (uint32_t)e)) again |= 1u << q;
-                    }
-                    dropped = again;
-                    if (!__syncthreads_or(dropped != 0 || want_refresh)) break;
-                    want_refresh = false;
-                }
-            }
-        }
-        s = refresh_candidates(sh, s, KP);                          // leaves min(KP, candidates) keys in keys[]
-        __syncthreads();
-        // sort them into win[] by counting
-        const int cnt = (int)sh.count;
-        if (tid < cnt) {
-            const uint64_t k = sh.keys[tid];
-            int rank = 0;
-            for (int q = 0; q < cnt; ++q) rank += sh.keys[q] > k;
-            sh.win[rank] = k;
-        }
-        if (tid == 0) sh.nwin = cnt;
-        __syncthreads();
+        s = careful_segment<DT>(sh, row, sp, p.V, seg, p.S, c_begin, c_end, KP, &flags);
         combine();
     }
 
