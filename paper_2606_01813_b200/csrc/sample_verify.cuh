@@ -21,7 +21,6 @@
 
 namespace cadd {
 
-constexpr int kRunChunks = kTileChunks / (kThreads / 32);     // 128 chunks = 2 KB per warp and tile
 constexpr int kMaxRuns = 640;                                 // runs per row kept in shared memory (V up to 650k bf16 / 325k fp32 elements);
                                                               // sized so that four CTAs fit in an SM's shared memory
 

@@ -10,6 +10,7 @@ namespace cadd {
 constexpr int kTopkUnroll = 4;            // chunks per thread per tile
 constexpr int kTileChunks = kTopkUnroll * kThreads;   // 16-byte chunks per tile (16 KB)
 constexpr int kStages = 3;                // tiles in flight per CTA
+constexpr int kRunChunks = kTileChunks / (kThreads / 32);   // a warp's share of a tile when each warp takes a contiguous run: 128 chunks = 2 KB
 constexpr int kSpinLimit = 1 << 16;       // bounded waits: tries of up to ~2 us each (mbarrier), or plain polls
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
