@@ -301,3 +301,37 @@ def test_adversarial_rows_full_vocabulary():
                 diag = compare_build(gt, ot, K)
                 assert not diag["exempt"], diag
                 assert diag["max_logZ_err"] < 1e-6, diag
+
+
+def scaled_cost_kwargs(c, cd_scale: float, cv_scale: float):
+    """The cost inputs with the draft cost C_d and the verification cost C_v(.) multiplied by constants."""
+    if c.kind == synth.COST_TABLE:
+        return dict(cost_kind=G.COST_TABLE, cost_table=c.table * cv_scale, table_idx=c.table_idx, t_draft=c.t_draft * cd_scale)
+    coef = c.coef.clone()
+    coef[:, 0] *= cd_scale
+    coef[:, 1:] *= cv_scale
+    return dict(cost_kind=G.COST_QUADRATIC, cost_coef=coef)
+
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c5"])
+def test_cost_sensitivity_analogue(name):
+    """Synthetic analogue of the paper's sensitivity ablation (Section 5, Table "Sensitivity ... to cost parameter
+    perturbations"): the builder is run with C_d and C_v each scaled by 0.5 and 2.  Parity with the oracle at every
+    setting, plus what Eq. 11 implies: the stop test compares delta/(1+Phi) with (C_v(n+1)-C_v(n))/(C_d+C_v(n)), whose
+    right side falls when C_d grows and rises when C_v is scaled up, so n* is non-decreasing in the C_d scale and
+    non-increasing in the C_v scale, request by request."""
+    cfg = synth.scaled(synth.CONFIGS[name], **SMALL[name])
+    seed = synth.config_seed(cfg)
+    d = synth.make_draft_inputs(cfg, seed)
+    c = synth.make_cost_inputs(cfg, seed)
+    n_star = {}
+    for cd, cv in ((1.0, 1.0), (0.5, 1.0), (2.0, 1.0), (1.0, 0.5), (1.0, 2.0)):
+        gt, ot = run_both_build(d.logits, cfg.K, cfg.B_max, cfg.R, l_eff=d.l_eff, bonus_token=d.bonus_token,
+                                ctx_len=d.ctx_len, **scaled_cost_kwargs(c, cd, cv))
+        diag = compare_build(gt, ot, cfg.K)
+        assert len(diag["exempt"]) <= 1, diag
+        n_star[(cd, cv)] = to_cpu(gt.n_nodes)
+    assert bool((n_star[(0.5, 1.0)] <= n_star[(1.0, 1.0)]).all()) and bool((n_star[(1.0, 1.0)] <= n_star[(2.0, 1.0)]).all())
+    assert bool((n_star[(1.0, 0.5)] >= n_star[(1.0, 1.0)]).all()) and bool((n_star[(1.0, 1.0)] >= n_star[(1.0, 2.0)]).all())
+    if name == "c3":                                                              # large enough trees: the perturbation does move them
+        assert int(n_star[(1.0, 0.5)].sum()) > int(n_star[(1.0, 2.0)].sum())
