@@ -95,8 +95,30 @@ static size_t build_workspace_bytes(const BuildPlan& pl) { return (pl.partial_by
 
 using namespace cadd;
 
+// Problems that stream at least this many bytes of logits are launched with programmatic stream serialization.
+constexpr int64_t kOverlapMinBytes = 16ll << 20;
+
+// Launch with programmatic stream serialization: the grid may be set up and its CTAs dispatched while the previous
+// kernel of the stream drains; every kernel launched this way starts with griddepcontrol.wait, which returns once the
+// previous kernel has completed and its writes are visible (and at once when there is no such dependency).
+// Costs a few microseconds more on the host than a plain launch, so launch-bound (small) problems ask for `overlap` = false.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_dependent(bool overlap, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    if (!overlap) {
+        kernel<<<grid, block, smem, st>>>(args...);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // Launches the expansion + emission kernel on the per-row partial records at `partials` (S records per row).
-static int launch_expand(const cadd_build_args* a, int KP, int S, const unsigned char* partials, cudaStream_t st) {
+static int launch_expand(const cadd_build_args* a, int KP, int S, const unsigned char* partials, cudaStream_t st, bool overlap) {
     const ExpandLayout lay = expand_layout(a->L, a->K, KP, S, a->B_max);
     ExpandParams ep;
     ep.batch = a->batch; ep.L = a->L; ep.K = a->K; ep.KP = KP; ep.S = S; ep.B_max = a->B_max; ep.R = a->R;
@@ -114,8 +136,7 @@ static int launch_expand(const cadd_build_args* a, int KP, int S, const unsigned
             return CADD_ERR_LAUNCH;
         }
     }
-    expand_emit_kernel<<<a->batch, kThreads, lay.total, st>>>(ep);
-    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    if (launch_dependent(overlap, expand_emit_kernel, dim3((unsigned)a->batch), dim3(kThreads), lay.total, st, ep) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
     return CADD_OK;
 }
 
@@ -182,11 +203,13 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
     tp.logits = a->draft_logits; tp.V = a->V; tp.stride_b = a->stride_b; tp.stride_l = a->stride_l;
     tp.L = a->L; tp.S = pl.S; tp.KP = pl.KP; tp.l_eff = a->l_eff; tp.partials = (unsigned char*)a->workspace;
     const unsigned items = (unsigned)((int64_t)a->batch * a->L * pl.S);
-    if (a->logits_dtype == CADD_DTYPE_BF16) softmax_topk_partial_kernel<CADD_DTYPE_BF16><<<items, kThreads, topk_smem_bytes(), st>>>(tp);
-    else softmax_topk_partial_kernel<CADD_DTYPE_FP32><<<items, kThreads, topk_smem_bytes(), st>>>(tp);
-    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    const bool overlap = (int64_t)a->batch * a->L * a->V * (int64_t)es >= kOverlapMinBytes;
+    const cudaError_t le = a->logits_dtype == CADD_DTYPE_BF16
+        ? launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, dim3(items), dim3(kThreads), topk_smem_bytes(), st, tp)
+        : launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, dim3(items), dim3(kThreads), topk_smem_bytes(), st, tp);
+    if (le != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
 
-    return launch_expand(a, pl.KP, pl.S, (const unsigned char*)a->workspace, st);
+    return launch_expand(a, pl.KP, pl.S, (const unsigned char*)a->workspace, st, overlap);
 }
 
 static int check_verify_shape(const cadd_verify_args* a) {
@@ -226,23 +249,27 @@ int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream) {
     ap.logits = a->target_logits; ap.V = a->V; ap.stride_b = a->stride_b; ap.stride_row = a->stride_row;
     ap.R = a->R; ap.rows_mode = a->rows_mode; ap.n_nodes = a->n_nodes; ap.node_argmax = a->node_argmax;
     const unsigned rows = (unsigned)((int64_t)a->batch * a->R);
+    const bool overlap = (int64_t)rows * a->V * (a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4) >= kOverlapMinBytes;
     const void* kfn = a->logits_dtype == CADD_DTYPE_BF16 ? (const void*)row_argmax_kernel<CADD_DTYPE_BF16>
                                                           : (const void*)row_argmax_kernel<CADD_DTYPE_FP32>;
     if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)argmax_smem_bytes()) != cudaSuccess) {
         cudaGetLastError();
         return CADD_ERR_LAUNCH;
     }
-    if (a->logits_dtype == CADD_DTYPE_BF16) row_argmax_kernel<CADD_DTYPE_BF16><<<rows, kThreads, argmax_smem_bytes(), st>>>(ap);
-    else row_argmax_kernel<CADD_DTYPE_FP32><<<rows, kThreads, argmax_smem_bytes(), st>>>(ap);
-    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    const cudaError_t le = a->logits_dtype == CADD_DTYPE_BF16
+        ? launch_dependent(overlap, row_argmax_kernel<CADD_DTYPE_BF16>, dim3(rows), dim3(kThreads), argmax_smem_bytes(), st, ap)
+        : launch_dependent(overlap, row_argmax_kernel<CADD_DTYPE_FP32>, dim3(rows), dim3(kThreads), argmax_smem_bytes(), st, ap);
+    if (le != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
 
     WalkParams wp;
     wp.batch = a->batch; wp.L = a->L; wp.R = a->R; wp.n_nodes = a->n_nodes; wp.token_ids = a->token_ids;
     wp.parent_idx = a->parent_idx; wp.node_argmax = a->node_argmax; wp.accepted_len = a->accepted_len;
     wp.accepted_nodes = a->accepted_nodes; wp.next_bonus = a->next_bonus; wp.status = a->status;
     const int wpb = 4;
-    accept_walk_kernel<<<(a->batch + wpb - 1) / wpb, wpb * 32, 0, st>>>(wp);
-    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    if (launch_dependent(overlap, accept_walk_kernel, dim3((unsigned)((a->batch + wpb - 1) / wpb)), dim3(wpb * 32), 0, st, wp) != cudaSuccess) {
+        cudaGetLastError();
+        return CADD_ERR_LAUNCH;
+    }
     return CADD_OK;
 }
 
@@ -512,7 +539,7 @@ int cadd_build_tree_fused_head(const cadd_build_head_args* h, void* cuda_stream)
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
     draft_merge_kernel<<<(unsigned)((M + 3) / 4), 128, 0, st>>>(dp, merged);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
-    return launch_expand(a, pl.KP, 1, merged, st);
+    return launch_expand(a, pl.KP, 1, merged, st, false);
 }
 
 // ---------------- tree verification under sampling ----------------

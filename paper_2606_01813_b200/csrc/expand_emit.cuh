@@ -110,6 +110,7 @@ __device__ __forceinline__ double cost_verify(const CostModel& cm, int n) {
 }
 
 __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
+    grid_dependency_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     const ExpandLayout lay = expand_layout(p.L, p.K, p.KP, p.S, p.B_max);
     double* a_list = (double*)(smem + lay.a_list);

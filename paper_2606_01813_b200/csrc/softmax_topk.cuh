@@ -424,6 +424,7 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkParams p) {
     using E = Elem<DT>;
     static_assert(kTopkUnroll == 4, "the tile loop below is written for four chunks per thread");
+    grid_dependency_wait();
     extern __shared__ __align__(16) unsigned char topk_smem_raw[];
     // aligned by pointer arithmetic on the shared array itself, so that every access below compiles to a
     // shared-memory instruction rather than a generic one

@@ -13,6 +13,12 @@ constexpr int kStages = 3;                // tiles in flight per CTA
 constexpr int kRunChunks = kTileChunks / (kThreads / 32);   // a warp's share of a tile when each warp takes a contiguous run: 128 chunks = 2 KB
 constexpr int kSpinLimit = 1 << 16;       // bounded waits: tries of up to ~2 us each (mbarrier), or plain polls
 
+// First statement of a kernel that may be launched while the previous kernel of its stream still runs (programmatic
+// stream serialization): returns when that kernel has completed and its writes are visible; a no-op otherwise.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream be dispatched from now on (it still waits, in its own first statement, for this
+// kernel to complete).  Only worth calling where the next kernel is tiny: its CTAs hold their resources while they wait.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");

@@ -34,6 +34,8 @@ inline size_t argmax_smem_bytes() { return sizeof(ArgmaxRing) + 128; }
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) row_argmax_kernel(ArgmaxParams p) {
     using E = Elem<DT>;
+    grid_dependency_wait();
+    grid_launch_dependents();                            // the walk kernel that follows is a handful of warps
     extern __shared__ __align__(16) unsigned char argmax_smem_raw[];
     // aligned by pointer arithmetic on the shared array itself: accesses stay shared-memory instructions
     ArgmaxRing& sh = *reinterpret_cast<ArgmaxRing*>(argmax_smem_raw + ((128u - (smem_u32(argmax_smem_raw) & 127u)) & 127u));
@@ -151,6 +153,7 @@ struct WalkParams {
 // One warp per request: from the root, move to the child whose token equals the target's argmax at
 // the current node (children always have a larger row index than their parent); stop at the first miss.
 __global__ void __launch_bounds__(128) accept_walk_kernel(WalkParams p) {
+    grid_dependency_wait();
     const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (b >= p.batch) return;
