@@ -576,17 +576,21 @@ int cadd_verify_tree_sampled(const cadd_sample_args* a, void* cuda_stream) {
         cudaGetLastError();
         return CADD_ERR_LAUNCH;
     }
-    if (a->logits_dtype == CADD_DTYPE_BF16) row_sample_kernel<CADD_DTYPE_BF16><<<rows, kThreads, sample_smem_bytes(), st>>>(sp);
-    else row_sample_kernel<CADD_DTYPE_FP32><<<rows, kThreads, sample_smem_bytes(), st>>>(sp);
-    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    const bool overlap = (int64_t)rows * a->V * (int64_t)es >= kOverlapMinBytes;
+    const cudaError_t le = a->logits_dtype == CADD_DTYPE_BF16
+        ? launch_dependent(overlap, row_sample_kernel<CADD_DTYPE_BF16>, dim3(rows), dim3(kThreads), sample_smem_bytes(), st, sp)
+        : launch_dependent(overlap, row_sample_kernel<CADD_DTYPE_FP32>, dim3(rows), dim3(kThreads), sample_smem_bytes(), st, sp);
+    if (le != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
 
     WalkParams wp;                                           // the walk is the greedy one with the drawn tokens in place of the arg-max
     wp.batch = a->batch; wp.L = a->L; wp.R = a->R; wp.n_nodes = a->n_nodes; wp.token_ids = a->token_ids;
     wp.parent_idx = a->parent_idx; wp.node_argmax = a->node_token; wp.accepted_len = a->accepted_len;
     wp.accepted_nodes = a->accepted_nodes; wp.next_bonus = a->next_bonus; wp.status = a->status;
     const int wpb = 4;
-    accept_walk_kernel<<<(a->batch + wpb - 1) / wpb, wpb * 32, 0, st>>>(wp);
-    if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+    if (launch_dependent(overlap, accept_walk_kernel, dim3((unsigned)((a->batch + wpb - 1) / wpb)), dim3(wpb * 32), 0, st, wp) != cudaSuccess) {
+        cudaGetLastError();
+        return CADD_ERR_LAUNCH;
+    }
     return CADD_OK;
 }
 

@@ -160,6 +160,8 @@ __device__ __noinline__ int32_t sample_combine(SampleShared& sh, int n_runs, flo
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p) {
     using E = Elem<DT>;
+    grid_dependency_wait();
+    grid_launch_dependents();                            // the walk kernel that follows is a handful of warps
     extern __shared__ __align__(16) unsigned char sample_smem_raw[];
     SampleShared& sh = *reinterpret_cast<SampleShared*>(sample_smem_raw + ((128u - (smem_u32(sample_smem_raw) & 127u)) & 127u));
     const int b = blockIdx.x / p.R;
