@@ -179,6 +179,8 @@ def run_ours(args, rank, world):
         torch.cuda.synchronize()
     clocks = sampler.stop() if sampler is not None else None
     instrumented_ms = ev[0].elapsed_time(ev[3 * K - 1]) / K
+    per_step = sorted(ev[3 * i].elapsed_time(ev[3 * i + 2]) for i in range(K))
+    step_median_ms, step_min_ms = per_step[K // 2], per_step[0]
     build_ms = sum(ev[3 * i].elapsed_time(ev[3 * i + 1]) for i in range(K)) / K
     verify_ms = sum(ev[3 * i + 1].elapsed_time(ev[3 * i + 2]) for i in range(K)) / K
     total_ms = replicas.max_over_ranks(total_ms, dev)
@@ -307,20 +309,31 @@ def run_ours(args, rank, world):
     if rank == 0:
         line = {
             "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-            "ms_per_step": round(total_ms / K, 5), "instrumented_ms_per_step": round(instrumented_ms, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": round(total_ms / K, 5), "instrumented_ms_per_step": round(instrumented_ms, 5), "instrumented_step_median_ms": round(step_median_ms, 5), "instrumented_step_min_ms": round(step_min_ms, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": cfg.dtype, "data": "synthetic",
             "config": {"workload": f"config {cfg.index} ({cfg.name}): batch={cfg.batch} L={cfg.L} V={cfg.V} {cfg.dtype} "
                                    f"K={cfg.K} B_max={cfg.B_max} R={cfg.R}, verify rows_mode={args.rows_mode}",
                        "l2": ("inputs larger than L2 (no flush needed)" if build_bytes + verify_bytes > (126 << 20)
                               else "inputs fit in L2 and are not flushed between steps (a launch-bound case, not the headline workload)"),
                        "timing": "value: K steps between one pair of CUDA events; roofline/build: a second pass of K steps with events around every call (instrumented_ms_per_step)", "parallelism": f"replicas x{world}",
-                       "n_star_mean": round(float(n_star.float().mean()), 2), "n_star_max": int(n_star.max()),
+                       "n_star_mean": round(float(n_star.float().mean()), 2), "n_star_max": int(n_star.max()), "n_star_hist": n_star_histogram(n_star),
                        "accepted_mean": round(float(verdict.accepted_len.float().mean().item()), 2)},
             "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "fused_draft_head": fused_draft, "sampled_verify": sampled, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
             "gpu_launches": KERNELS_PER_STEP * K, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
     replicas.shutdown()
+
+
+def n_star_histogram(n_star):
+    """Requests per tree-size bin: 0, 1-3, 4-7, 8-15, ... (powers of two)."""
+    edges = [0, 1, 4, 8, 16, 32, 64, 128, 256, 512, 1024, 2049]
+    out = {}
+    for lo, hi in zip(edges[:-1], edges[1:]):
+        cnt = int(((n_star >= lo) & (n_star < hi)).sum())
+        if cnt:
+            out[str(lo) if hi == lo + 1 else f"{lo}-{hi - 1}"] = cnt
+    return out
 
 
 def measured_peak_tflops():
