@@ -301,6 +301,14 @@ def run_ours(args, rank, world):
         except Exception as ex:
             cost_fit = {"error": str(ex)[:200]}
 
+    # ---- rounds with a fresh seed each (configuration 5 is defined that way): inputs regenerated outside the timing ----
+    fresh = None
+    if args.fresh_rounds > 0:
+        try:
+            fresh = fresh_rounds_block(G, cfg, rank, rows_mode, flags, ws, tree, verdict, y, dev, args.fresh_rounds)
+        except Exception as ex:
+            fresh = {"error": str(ex)[:200]}
+
     # ---- the oracle timed on this machine's host cores, on a bounded sample (rank 0, N = 1 only) ----
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -318,7 +326,7 @@ def run_ours(args, rank, world):
                        "timing": "value: K steps between one pair of CUDA events; roofline/build: a second pass of K steps with events around every call (instrumented_ms_per_step)", "parallelism": f"replicas x{world}",
                        "n_star_mean": round(float(n_star.float().mean()), 2), "n_star_max": int(n_star.max()), "n_star_hist": n_star_histogram(n_star),
                        "accepted_mean": round(float(verdict.accepted_len.float().mean().item()), 2)},
-            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "fused_draft_head": fused_draft, "sampled_verify": sampled, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "fused_draft_head": fused_draft, "sampled_verify": sampled, "fresh_seed_rounds": fresh, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
             "gpu_launches": KERNELS_PER_STEP * K, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
@@ -451,6 +459,38 @@ def sampled_block(G, cfg, tree, y, rows_mode, verify_bytes, dev, iters):
             "peak_kind": kind, "accepted_mean": round(float(out.accepted_len.float().mean().item()), 2)}
 
 
+def fresh_rounds_block(G, cfg, rank, rows_mode, flags, ws, tree, verdict, y, dev, n_rounds):
+    """n_rounds rounds, each on inputs drawn from its own seed (1000 * config + round): draft logits and costs are
+    regenerated, the tree is built once untimed so that the target logits can be drawn for it (as the target's forward
+    pass would produce them), then one build + verify is timed with CUDA events."""
+    times, n_mean, acc_mean = [], [], []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for r in range(n_rounds):
+        seed = replicas.replica_seed(synth.config_seed(cfg, r), rank)
+        d = synth.make_draft_inputs(cfg, seed, device=str(dev))
+        c = synth.make_cost_inputs(cfg, seed)
+        kw = dict(l_eff=d.l_eff.to(dev), bonus_token=d.bonus_token.to(dev), ctx_len=d.ctx_len.to(dev), flags=flags)
+        ck = {k: (v.to(dev) if torch.is_tensor(v) else v) for k, v in cost_kwargs(G, c).items()}
+        G.cadd_build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=tree, **kw, **ck)
+        torch.cuda.synchronize()
+        synth.make_target_logits(cfg, seed, d, tree.depth.cpu(), device=str(dev), out=y)
+        torch.cuda.synchronize()
+        e0.record()
+        G.cadd_build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=tree, **kw, **ck)
+        G.cadd_verify_tree(y, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, out=verdict)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+        n_mean.append(float(tree.n_nodes.float().mean().item()))
+        acc_mean.append(float(verdict.accepted_len.float().mean().item()))
+        del d
+    ts = sorted(times)
+    return {"rounds": n_rounds, "value": round(n_rounds / (sum(times) * 1e-3), 3), "unit": UNIT,
+            "ms_mean": round(sum(times) / n_rounds, 4), "ms_median": round(ts[n_rounds // 2], 4), "ms_min": round(ts[0], 4),
+            "ms_max": round(ts[-1], 4), "n_star_mean": round(sum(n_mean) / n_rounds, 2),
+            "accepted_mean": round(sum(acc_mean) / n_rounds, 2)}
+
+
 def fit_block(G, dev, iters=5):
     """cadd_fit_cost_tables on nine noisy convex latency curves of 1024 points each; absolute time (a small,
     latency-bound problem: one CTA per curve), not a roofline figure."""
@@ -560,6 +600,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (0 = as defined)")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
     ap.add_argument("--no-sampled", action="store_true", help="skip the sampling-mode verification measurement")
+    ap.add_argument("--fresh-rounds", type=int, default=0,
+                    help="also time this many rounds with a fresh seed each (inputs regenerated outside the timed calls)")
     ap.add_argument("--no-fit", action="store_true", help="skip the offline cost-fitting measurement")
     ap.add_argument("--head-hidden", type=int, default=4096,
                     help="hidden size for the fused output-projection verification measurement (0 = skip)")
