@@ -97,6 +97,8 @@ using namespace cadd;
 
 // Problems that stream at least this many bytes of logits are launched with programmatic stream serialization.
 constexpr int64_t kOverlapMinBytes = 16ll << 20;
+// LIVE verification shares a CTA between eight rows up to this row capacity (node cap 512).
+constexpr int kLiveSharedRowsMaxR = 513;
 
 // Launch with programmatic stream serialization: the grid may be set up and its CTAs dispatched while the previous
 // kernel of the stream drains; every kernel launched this way starts with griddepcontrol.wait, which returns once the
@@ -248,8 +250,12 @@ int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream) {
     ArgmaxParams ap;
     ap.logits = a->target_logits; ap.V = a->V; ap.stride_b = a->stride_b; ap.stride_row = a->stride_row;
     ap.R = a->R; ap.rows_mode = a->rows_mode; ap.n_nodes = a->n_nodes; ap.node_argmax = a->node_argmax;
-    const unsigned rows = (unsigned)((int64_t)a->batch * a->R);
-    const bool overlap = (int64_t)rows * a->V * (a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4) >= kOverlapMinBytes;
+    // LIVE with a small node cap: most rows are padding on typical trees, so eight rows share a CTA (interleaved, so
+    // that a request's live rows, which come first, still spread over its CTAs) and few CTAs are launched only to exit.
+    // Large caps and DENSE keep one row per CTA: every row is work there and short CTAs keep the last wave short.
+    ap.ctas_per_request = (a->rows_mode == CADD_ROWS_LIVE && a->R <= kLiveSharedRowsMaxR) ? (a->R + 7) / 8 : a->R;
+    const unsigned rows = (unsigned)((int64_t)a->batch * ap.ctas_per_request);
+    const bool overlap = (int64_t)a->batch * a->R * a->V * (a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4) >= kOverlapMinBytes;
     const void* kfn = a->logits_dtype == CADD_DTYPE_BF16 ? (const void*)row_argmax_kernel<CADD_DTYPE_BF16>
                                                           : (const void*)row_argmax_kernel<CADD_DTYPE_FP32>;
     if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)argmax_smem_bytes()) != cudaSuccess) {

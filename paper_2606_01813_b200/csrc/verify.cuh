@@ -10,6 +10,7 @@ struct ArgmaxParams {
     const void* logits;        // [batch, R, V]
     int64_t V, stride_b, stride_row;
     int R, rows_mode;
+    int ctas_per_request;      // CTA g of a request reads rows g, g + ctas_per_request, ... (= R: one row per CTA)
     const int32_t* n_nodes;    // [batch]
     int32_t* node_argmax;      // [batch, R]
 };
@@ -25,7 +26,7 @@ struct ArgmaxRing {
 };
 inline size_t argmax_smem_bytes() { return sizeof(ArgmaxRing) + 128; }
 
-// One CTA per (request, row).  One thread streams the row's 16-byte chunks into a ring of 16 KB
+// One CTA per (request, row) (or per few rows of a request, see ctas_per_request).  One thread streams the row's 16-byte chunks into a ring of 16 KB
 // shared-memory tiles with cp.async.bulk + mbarrier (own shared memory only); the last warp to finish a tile refills
 // its stage, so (kStages - 1) x 16 KB stay in flight per CTA (4 CTAs per SM) without living in registers.
 // Each thread keeps the running maximum (packed bf16 max, NaN ignored) and the first position (chunk start or
@@ -39,102 +40,121 @@ __global__ void __launch_bounds__(kThreads, 4) row_argmax_kernel(ArgmaxParams p)
     extern __shared__ __align__(16) unsigned char argmax_smem_raw[];
     // aligned by pointer arithmetic on the shared array itself: accesses stay shared-memory instructions
     ArgmaxRing& sh = *reinterpret_cast<ArgmaxRing*>(argmax_smem_raw + ((128u - (smem_u32(argmax_smem_raw) & 127u)) & 127u));
-    const int b = blockIdx.x / p.R;
-    const int j = blockIdx.x - b * p.R;
+    // CTA g of request b takes rows g, g + ctas_per_request, ...: one row each when every row is read (DENSE), several
+    // when most rows are expected to be padding (LIVE with a small node cap), so that few CTAs are launched only to exit.
+    const int b = blockIdx.x / p.ctas_per_request;
+    const int g = blockIdx.x - b * p.ctas_per_request;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int32_t* out = p.node_argmax + (int64_t)b * p.R + j;
+    int n = p.R - 1;
     if (p.rows_mode == CADD_ROWS_LIVE) {
-        int n = p.n_nodes[b];
+        n = p.n_nodes[b];
         n = n < 0 ? 0 : (n > p.R - 1 ? p.R - 1 : n);
-        if (j > n) {
-            if (tid == 0) *out = -1;
+        if (g > n) {                                     // nothing to read for this CTA: mark its rows and leave
+            for (int j = g + tid * p.ctas_per_request; j < p.R; j += kThreads * p.ctas_per_request)
+                p.node_argmax[(int64_t)b * p.R + j] = -1;
             return;
         }
     }
-    const char* row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)j * p.stride_row) * E::ES;
-    const RowSplit sp = split_row<DT>(row, p.V);
-    const uint4* body = (const uint4*)(row + (int64_t)sp.head * E::ES);
-    const int nc = sp.n_chunks;
-    const int n_tiles = (nc + kTileChunks - 1) / kTileChunks;
-
     if (tid == 0) {
         for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
         sh.timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    auto issue_tile = [&](int t) {
-        const int c0 = t * kTileChunks;
-        const unsigned bytes = (unsigned)min(kTileChunks, nc - c0) * 16u;
-        const unsigned st = (unsigned)t % kStages;
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive_expect_tx(&sh.full[st], bytes);
-        bulk_load(&sh.ring[st][0], body + c0, bytes, &sh.full[st]);
-    };
-    if (tid == 0)
-        for (int t = 0; t < kStages && t < n_tiles; ++t) issue_tile(t);
+    unsigned st = 0, phase = 0;                          // ring position: carries on from row to row
+    unsigned issued = 0;                                 // tiles issued so far (thread-uniform by construction)
+    for (int j = g; j < p.R; j += p.ctas_per_request) {
+        int32_t* out = p.node_argmax + (int64_t)b * p.R + j;
+        if (j > n) {
+            if (tid == 0) *out = -1;
+            continue;
+        }
+        const char* row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)j * p.stride_row) * E::ES;
+        const RowSplit sp = split_row<DT>(row, p.V);
+        const uint4* body = (const uint4*)(row + (int64_t)sp.head * E::ES);
+        const int nc = sp.n_chunks;
+        const int n_tiles = (nc + kTileChunks - 1) / kTileChunks;
+        const unsigned base = issued;                    // stage of tile t of this row: (base + t) % kStages
+        auto issue_tile = [&](int t) {
+            const int c0 = t * kTileChunks;
+            const unsigned bytes = (unsigned)min(kTileChunks, nc - c0) * 16u;
+            const unsigned stg = (base + (unsigned)t) % kStages;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive_expect_tx(&sh.full[stg], bytes);
+            bulk_load(&sh.ring[stg][0], body + c0, bytes, &sh.full[stg]);
+        };
+        if (tid == 0)
+            for (int t = 0; t < kStages && t < n_tiles; ++t) issue_tile(t);
+        issued += (unsigned)n_tiles;
 
-    float rm = -INFINITY;            // running maximum (NaN never enters: only strict '>' updates it)
-    int64_t rpos = INT64_MAX;        // first position where rm was reached
-    if (tid < sp.head) {
-        float x = E::load(row, tid);
-        if (x > rm) { rm = x; rpos = tid; }
-    }
-    unsigned st = 0, phase = 0;
-    for (int t = 0; t < n_tiles; ++t) {
-        if (!__all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase))) { sh.timeout = 1; break; }
-        const uint4* tile = &sh.ring[st][tid];
-        const int cbase = t * kTileChunks + tid;
+        float rm = -INFINITY;            // running maximum (NaN never enters: only strict '>' updates it)
+        int64_t rpos = INT64_MAX;        // first position where rm was reached
+        if (tid < sp.head) {
+            float x = E::load(row, tid);
+            if (x > rm) { rm = x; rpos = tid; }
+        }
+        for (int t = 0; t < n_tiles; ++t) {
+            if (!__all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase))) { sh.timeout = 1; break; }
+            const uint4* tile = &sh.ring[st][tid];
+            const int cbase = t * kTileChunks + tid;
 #pragma unroll
-        for (int u = 0; u < kTopkUnroll; ++u) {
-            const int c = cbase + u * kThreads;
-            if (c < nc) {
-                const float cm = E::chunk_max(tile[u * kThreads]);
-                if (cm > rm) { rm = cm; rpos = sp.head + (int64_t)c * E::EPC; }
+            for (int u = 0; u < kTopkUnroll; ++u) {
+                const int c = cbase + u * kThreads;
+                if (c < nc) {
+                    const float cm = E::chunk_max(tile[u * kThreads]);
+                    if (cm > rm) { rm = cm; rpos = sp.head + (int64_t)c * E::EPC; }
+                }
             }
+            __syncwarp();
+            if (lane == 0 && atomicAdd(&sh.released[st], 1u) == kThreads / 32 - 1) {   // last warp refills the stage
+                atomicExch(&sh.released[st], 0u);
+                if (t + kStages < n_tiles) issue_tile(t + kStages);
+            }
+            if (++st == kStages) { st = 0; phase ^= 1u; }
         }
-        __syncwarp();
-        if (lane == 0 && atomicAdd(&sh.released[st], 1u) == kThreads / 32 - 1) {   // last warp refills the stage
-            atomicExch(&sh.released[st], 0u);
-            if (t + kStages < n_tiles) issue_tile(t + kStages);
+        if (tid < sp.tail) {
+            int64_t i = p.V - sp.tail + tid;
+            float x = E::load(row, i);
+            if (x > rm) { rm = x; rpos = i; }
         }
-        if (++st == kStages) { st = 0; phase ^= 1u; }
-    }
-    if (tid < sp.tail) {
-        int64_t i = p.V - sp.tail + tid;
-        float x = E::load(row, i);
-        if (x > rm) { rm = x; rpos = i; }
-    }
 
-    // CTA reduction of (value descending, position ascending)
+        // CTA reduction of (value descending, position ascending)
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        float om = __shfl_xor_sync(kFullMask, rm, o);
-        int64_t op = __shfl_xor_sync(kFullMask, rpos, o);
-        if (om > rm || (om == rm && op < rpos)) { rm = om; rpos = op; }
-    }
-    if (lane == 0) { sh.red_m[warp] = rm; sh.red_p[warp] = rpos; }
-    __syncthreads();
-    if (tid < 32) {
-        rm = tid < kThreads / 32 ? sh.red_m[tid] : -INFINITY;
-        rpos = tid < kThreads / 32 ? sh.red_p[tid] : INT64_MAX;
-#pragma unroll
-        for (int o = 4; o > 0; o >>= 1) {
+        for (int o = 16; o > 0; o >>= 1) {
             float om = __shfl_xor_sync(kFullMask, rm, o);
             int64_t op = __shfl_xor_sync(kFullMask, rpos, o);
             if (om > rm || (om == rm && op < rpos)) { rm = om; rpos = op; }
         }
-        rm = __shfl_sync(kFullMask, rm, 0);
-        rpos = __shfl_sync(kFullMask, rpos, 0);
-        int32_t ans = 0;                                  // every logit is -Inf or NaN: lowest id
-        if (rpos != INT64_MAX) {
-            int64_t i = rpos + tid;
-            bool hit = tid < E::EPC && i < p.V && E::load(row, i) == rm;
-            unsigned m = __ballot_sync(kFullMask, hit);
-            ans = (int32_t)(rpos + (__ffs(m) - 1));
+        if (lane == 0) { sh.red_m[warp] = rm; sh.red_p[warp] = rpos; }
+        __syncthreads();
+        const bool timed_out = sh.timeout != 0;
+        if (tid < 32) {
+            rm = tid < kThreads / 32 ? sh.red_m[tid] : -INFINITY;
+            rpos = tid < kThreads / 32 ? sh.red_p[tid] : INT64_MAX;
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) {
+                float om = __shfl_xor_sync(kFullMask, rm, o);
+                int64_t op = __shfl_xor_sync(kFullMask, rpos, o);
+                if (om > rm || (om == rm && op < rpos)) { rm = om; rpos = op; }
+            }
+            rm = __shfl_sync(kFullMask, rm, 0);
+            rpos = __shfl_sync(kFullMask, rpos, 0);
+            int32_t ans = 0;                                  // every logit is -Inf or NaN: lowest id
+            if (rpos != INT64_MAX) {
+                int64_t i = rpos + tid;
+                bool hit = tid < E::EPC && i < p.V && E::load(row, i) == rm;
+                unsigned m = __ballot_sync(kFullMask, hit);
+                ans = (int32_t)(rpos + (__ffs(m) - 1));
+            }
+            if (timed_out) ans = -2;                          // a bulk copy never landed: the walk kernel flags the request
+            if (tid == 0) *out = ans;
         }
-        if (sh.timeout) ans = -2;                         // a bulk copy never landed: the walk kernel flags the request
-        if (tid == 0) *out = ans;
+        if (timed_out) {                                      // the ring's state is unknown: give up on this CTA's other rows too
+            for (int jj = j + p.ctas_per_request + tid * p.ctas_per_request; jj < p.R; jj += kThreads * p.ctas_per_request)
+                p.node_argmax[(int64_t)b * p.R + jj] = jj > n ? -1 : -2;
+            return;
+        }
+        __syncthreads();                                      // red_m / red_p and the ring are free for the next row
     }
 }
 

@@ -335,3 +335,39 @@ def test_cost_sensitivity_analogue(name):
     assert bool((n_star[(1.0, 0.5)] >= n_star[(1.0, 1.0)]).all()) and bool((n_star[(1.0, 1.0)] >= n_star[(1.0, 2.0)]).all())
     if name == "c3":                                                              # large enough trees: the perturbation does move them
         assert int(n_star[(1.0, 0.5)].sum()) > int(n_star[(1.0, 2.0)].sum())
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_live_verification_with_several_rows_per_cta(dtype):
+    """LIVE verification with a small node cap lets one CTA read several rows of a request one after the other
+    (its ring of tiles carries on from row to row): requests with 0, a few and all rows live, rows that start off a
+    16-byte boundary, against the oracle; the padding rows read -1 and DENSE agrees on the live rows."""
+    g = torch.Generator().manual_seed(44)
+    batch, R, V, L = 4, 201, 9001, 6
+    big = (torch.randn(batch, R, V + 5, generator=g) * 2.0).to(dtype)
+    y = big[:, :, 3: 3 + V]                                        # unaligned rows, odd row stride
+    n = torch.tensor([0, 5, 200, 37], dtype=torch.int32)
+    par = torch.zeros(batch, R, dtype=torch.int32)
+    for c in range(1, R):
+        par[:, c] = torch.randint(0, c, (batch,), generator=g, dtype=torch.int32)
+    tok = torch.randint(0, V, (batch, R), generator=g, dtype=torch.int32)
+    am = y.float().argmax(-1).to(torch.int32)
+    for b in range(batch):                                         # plant a chain so that the walk accepts a few nodes
+        cur = 0
+        for c in range(1, min(int(n[b]), 4) + 1):
+            par[b, c] = cur
+            tok[b, c] = am[b, cur]
+            cur = c
+    yd = big.cuda()[:, :, 3: 3 + V]
+    dev = lambda t: t.cuda()
+    live = G.cadd_verify_tree(yd, L, dev(n), dev(tok), dev(par), rows_mode=G.ROWS_LIVE)
+    dense = G.cadd_verify_tree(yd, L, dev(n), dev(tok), dev(par), rows_mode=G.ROWS_DENSE)
+    torch.cuda.synchronize()
+    ov = O.verify_tree(y.contiguous(), L, n, tok, par, rows_mode=O.ROWS_LIVE)
+    compare_verify(live, ov)
+    la, da = to_cpu(live.node_argmax), to_cpu(dense.node_argmax)
+    for b in range(batch):
+        nb = int(n[b])
+        assert torch.equal(la[b, : nb + 1], da[b, : nb + 1]) and bool((la[b, nb + 1:] == -1).all())
+    assert torch.equal(to_cpu(live.accepted_len), to_cpu(dense.accepted_len))
+    assert to_cpu(live.accepted_len).tolist() == [0, 4, 4, 4]
