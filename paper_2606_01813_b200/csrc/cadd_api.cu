@@ -138,7 +138,7 @@ static int launch_expand(const cadd_build_args* a, int KP, int S, const unsigned
             return CADD_ERR_LAUNCH;
         }
     }
-    if (launch_dependent(overlap, expand_emit_kernel, dim3((unsigned)a->batch), dim3(kThreads), lay.total, st, ep) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+    if (launch_dependent(overlap, expand_emit_kernel, dim3((unsigned)a->batch), dim3(kExpandThreads), lay.total, st, ep) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
     return CADD_OK;
 }
 

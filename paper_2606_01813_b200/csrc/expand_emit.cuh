@@ -53,7 +53,8 @@ struct ExpandParams {
     int32_t* status;
 };
 
-constexpr int kExpandWarps = kThreads / 32;
+constexpr int kExpandThreads = 512;        // sixteen warps: one per draft position in the merge phase for L <= 16
+constexpr int kExpandWarps = kExpandThreads / 32;
 
 // Tie-break half of a frontier / node key.  Smaller packed value = earlier in the pop order
 // (depth, then token id, then parent row); the rank within the position's top-K list rides along in
@@ -109,7 +110,7 @@ __device__ __forceinline__ double cost_verify(const CostModel& cm, int n) {
     return cm.q[1] + cm.q[2] * x + cm.q[3] * (x * x);
 }
 
-__global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
+__global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandParams p) {
     grid_dependency_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     const ExpandLayout lay = expand_layout(p.L, p.K, p.KP, p.S, p.B_max);
@@ -133,7 +134,7 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
     int clamped;
     const int Le = clamp_l_eff(p.l_eff, b, L, &clamped);
     if (tid == 0) { s_status = clamped ? CADD_STATUS_L_EFF_CLAMPED : 0; s_pinf = 0; }
-    for (int d = tid; d < L + 2; d += kThreads) keff[d] = 0;
+    for (int d = tid; d < L + 2; d += kExpandThreads) keff[d] = 0;
     __syncthreads();
 
     // ---------------- phase 0: merge partials, one warp per position ----------------
@@ -447,8 +448,8 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         if (p.theta_curve) p.theta_curve[(int64_t)b * R] = s_theta0;
     }
     if (p.theta_curve)
-        for (int j = n + 1 + tid; j < R; j += kThreads) p.theta_curve[(int64_t)b * R + j] = 0.0;
-    for (int j = tid; j < R; j += kThreads) {
+        for (int j = n + 1 + tid; j < R; j += kExpandThreads) p.theta_curve[(int64_t)b * R + j] = 0.0;
+    for (int j = tid; j < R; j += kExpandThreads) {
         const int64_t o = (int64_t)b * R + j;
         int t = -1, par = -1, d = 0, pos = 0;
         double lp = 0.0;
@@ -468,7 +469,7 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
     // all rows zero first (coalesced), then the few non-zero words / bytes of the live rows
     if (p.mask_bits) {
         uint32_t* base = p.mask_bits + (int64_t)b * R * W;
-        for (int64_t q = tid; q < (int64_t)R * W; q += kThreads) base[q] = 0u;
+        for (int64_t q = tid; q < (int64_t)R * W; q += kExpandThreads) base[q] = 0u;
     }
     if (dense) {
         uint8_t* base = p.mask_dense + (int64_t)b * R * R;
@@ -478,11 +479,11 @@ __global__ void __launch_bounds__(kThreads) expand_emit_kernel(ExpandParams p) {
         const int64_t words = (total - head) >> 2;
         if (tid < head) base[tid] = 0;
         uint32_t* mid = (uint32_t*)(base + head);
-        for (int64_t q = tid; q < words; q += kThreads) mid[q] = 0u;
-        for (int64_t q = head + words * 4 + tid; q < total; q += kThreads) base[q] = 0;
+        for (int64_t q = tid; q < words; q += kExpandThreads) mid[q] = 0u;
+        for (int64_t q = head + words * 4 + tid; q < total; q += kExpandThreads) base[q] = 0;
     }
     __syncthreads();
-    for (int j = tid; j <= n; j += kThreads) {              // self and ancestors: at most L+1 bits, rows descending
+    for (int j = tid; j <= n; j += kExpandThreads) {              // self and ancestors: at most L+1 bits, rows descending
         uint32_t* wrow = p.mask_bits ? p.mask_bits + ((int64_t)b * R + j) * W : nullptr;
         uint8_t* brow = dense ? p.mask_dense + ((int64_t)b * R + j) * R : nullptr;
         int cur = j, word = j >> 5;
