@@ -575,18 +575,22 @@ int cadd_verify_tree_sampled(const cadd_sample_args* a, void* cuda_stream) {
     sp.logits = a->target_logits; sp.V = a->V; sp.stride_b = a->stride_b; sp.stride_row = a->stride_row;
     sp.R = a->R; sp.rows_mode = a->rows_mode; sp.c = (float)(1.4426950408889634 / a->temperature);
     sp.n_nodes = a->n_nodes; sp.uniforms = a->uniforms; sp.node_token = a->node_token;
-    const unsigned rows = (unsigned)((int64_t)a->batch * a->R);
-    const void* kfn = a->logits_dtype == CADD_DTYPE_BF16 ? (const void*)row_sample_kernel<CADD_DTYPE_BF16>
-                                                          : (const void*)row_sample_kernel<CADD_DTYPE_FP32>;
-    if (cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sample_smem_bytes()) != cudaSuccess) {
+    // LIVE with a small node cap: eight rows of a request share a CTA (as in cadd_verify_tree)
+    const bool shared_rows = a->rows_mode == CADD_ROWS_LIVE && a->R <= kLiveSharedRowsMaxR;
+    sp.ctas_per_request = shared_rows ? (a->R + 7) / 8 : a->R;
+    const unsigned rows = (unsigned)((int64_t)a->batch * sp.ctas_per_request);
+    const bool bf16 = a->logits_dtype == CADD_DTYPE_BF16;
+    auto kfn = bf16 ? (shared_rows ? row_sample_shared_rows_kernel<CADD_DTYPE_BF16> : row_sample_kernel<CADD_DTYPE_BF16>)
+                    : (shared_rows ? row_sample_shared_rows_kernel<CADD_DTYPE_FP32> : row_sample_kernel<CADD_DTYPE_FP32>);
+    if (cudaFuncSetAttribute((const void*)kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sample_smem_bytes()) != cudaSuccess) {
         cudaGetLastError();
         return CADD_ERR_LAUNCH;
     }
-    const bool overlap = (int64_t)rows * a->V * (int64_t)es >= kOverlapMinBytes;
-    const cudaError_t le = a->logits_dtype == CADD_DTYPE_BF16
-        ? launch_dependent(overlap, row_sample_kernel<CADD_DTYPE_BF16>, dim3(rows), dim3(kThreads), sample_smem_bytes(), st, sp)
-        : launch_dependent(overlap, row_sample_kernel<CADD_DTYPE_FP32>, dim3(rows), dim3(kThreads), sample_smem_bytes(), st, sp);
-    if (le != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+    const bool overlap = (int64_t)a->batch * a->R * a->V * (int64_t)es >= kOverlapMinBytes;
+    if (launch_dependent(overlap, kfn, dim3(rows), dim3(kThreads), sample_smem_bytes(), st, sp) != cudaSuccess) {
+        cudaGetLastError();
+        return CADD_ERR_LAUNCH;
+    }
 
     WalkParams wp;                                           // the walk is the greedy one with the drawn tokens in place of the arg-max
     wp.batch = a->batch; wp.L = a->L; wp.R = a->R; wp.n_nodes = a->n_nodes; wp.token_ids = a->token_ids;

@@ -28,6 +28,7 @@ struct SampleParams {
     const void* logits;        // [batch, R, V]
     int64_t V, stride_b, stride_row;
     int R, rows_mode;
+    int ctas_per_request;      // row_sample_shared_rows_kernel: CTA g of a request reads rows g, g + ctas_per_request, ...
     float c;                   // log2(e) / T
     const int32_t* n_nodes;    // [batch]
     const double* uniforms;    // [batch, R]
@@ -157,25 +158,15 @@ __device__ __noinline__ int32_t sample_combine(SampleShared& sh, int n_runs, flo
     return ans;
 }
 
+// One row of row_sample_kernel: streams the row through the ring (whose position st / phase and tile count `issued`
+// carry on from the caller's previous row), leaves the runs in shared memory and lets warp 0 draw the token.
+// Returns false if a wait ran out (the row then reads -2 and the ring must not be used again).
 template <int DT>
-__global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p) {
+__device__ __forceinline__ bool sample_one_row(SampleShared& sh, const SampleParams& p, int b, int j, unsigned& st, unsigned& phase,
+                                               unsigned& issued) {
     using E = Elem<DT>;
-    grid_dependency_wait();
-    grid_launch_dependents();                            // the walk kernel that follows is a handful of warps
-    extern __shared__ __align__(16) unsigned char sample_smem_raw[];
-    SampleShared& sh = *reinterpret_cast<SampleShared*>(sample_smem_raw + ((128u - (smem_u32(sample_smem_raw) & 127u)) & 127u));
-    const int b = blockIdx.x / p.R;
-    const int j = blockIdx.x - b * p.R;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t* out = p.node_token + (int64_t)b * p.R + j;
-    if (p.rows_mode == CADD_ROWS_LIVE) {
-        int n = p.n_nodes[b];
-        n = n < 0 ? 0 : (n > p.R - 1 ? p.R - 1 : n);
-        if (j > n) {
-            if (tid == 0) *out = -1;
-            return;
-        }
-    }
     const char* row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)j * p.stride_row) * E::ES;
     const RowSplit sp = split_row<DT>(row, p.V);
     const uint4* body = (const uint4*)(row + (int64_t)sp.head * E::ES);
@@ -185,17 +176,12 @@ __global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p)
     const int body_runs = (nc + kRunChunks - 1) / kRunChunks;
     const int n_runs = 1 + body_runs + 1;
 
-    if (tid == 0) {
-        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
-        sh.timeout = 0;
-        sh.n_runs = n_runs;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
+    const unsigned base = issued;                        // stage of tile t of this row: (base + t) % kStages
+    issued += (unsigned)n_tiles;
     auto issue_tile = [&](int t) {
         const int c0 = t * kTileChunks;
         const unsigned bytes = (unsigned)min(kTileChunks, nc - c0) * 16u;
-        const unsigned st = (unsigned)t % kStages;
+        const unsigned st = (base + (unsigned)t) % kStages;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive_expect_tx(&sh.full[st], bytes);
         bulk_load(&sh.ring[st][0], body + c0, bytes, &sh.full[st]);
@@ -219,7 +205,6 @@ __global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p)
         if (lane == 0) { const int r = warp == 0 ? 0 : n_runs - 1; sh.run_ref[r] = ref; sh.run_s[r] = s; }
     }
 
-    unsigned st = 0, phase = 0;
     const uint64_t c2 = pack2(p.c, p.c);
     for (int t = 0; t < n_tiles; ++t) {
         if (!__all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase))) { sh.timeout = 1; break; }
@@ -304,10 +289,79 @@ __global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p)
     __syncthreads();
 
     // ---- combine the runs (warp 0): total, the run that holds the crossing, the token inside it ----
+    const bool ok = sh.timeout == 0;
     if (warp == 0) {
         int32_t ans = -2;                                          // a wait ran out: no draw
-        if (!sh.timeout) ans = sample_combine<DT>(sh, n_runs, p.c, p.uniforms[(int64_t)b * p.R + j], row, sp, body, p.V);
+        if (ok) ans = sample_combine<DT>(sh, n_runs, p.c, p.uniforms[(int64_t)b * p.R + j], row, sp, body, p.V);
         if (lane == 0) *out = ans;
+    }
+    return ok;
+}
+
+// One CTA per (request, row).
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p) {
+    grid_dependency_wait();
+    grid_launch_dependents();                            // the walk kernel that follows is a handful of warps
+    extern __shared__ __align__(16) unsigned char sample_smem_raw[];
+    SampleShared& sh = *reinterpret_cast<SampleShared*>(sample_smem_raw + ((128u - (smem_u32(sample_smem_raw) & 127u)) & 127u));
+    const int b = blockIdx.x / p.R;
+    const int j = blockIdx.x - b * p.R;
+    const int tid = threadIdx.x;
+    if (p.rows_mode == CADD_ROWS_LIVE) {
+        int n = p.n_nodes[b];
+        n = n < 0 ? 0 : (n > p.R - 1 ? p.R - 1 : n);
+        if (j > n) {
+            if (tid == 0) p.node_token[(int64_t)b * p.R + j] = -1;
+            return;
+        }
+    }
+    if (tid == 0) {
+        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
+        sh.timeout = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    unsigned st = 0, phase = 0, issued = 0;
+    sample_one_row<DT>(sh, p, b, j, st, phase, issued);
+}
+
+// LIVE with a small node cap: CTA g of request b takes rows g, g + ctas_per_request, ... one after the other (see
+// row_argmax_kernel), so that few CTAs are launched only to exit.
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 4) row_sample_shared_rows_kernel(SampleParams p) {
+    grid_dependency_wait();
+    grid_launch_dependents();
+    extern __shared__ __align__(16) unsigned char sample_smem_raw[];
+    SampleShared& sh = *reinterpret_cast<SampleShared*>(sample_smem_raw + ((128u - (smem_u32(sample_smem_raw) & 127u)) & 127u));
+    const int b = blockIdx.x / p.ctas_per_request;
+    const int g = blockIdx.x - b * p.ctas_per_request;
+    const int tid = threadIdx.x;
+    int n = p.n_nodes[b];
+    n = n < 0 ? 0 : (n > p.R - 1 ? p.R - 1 : n);
+    if (g > n) {                                         // nothing to read for this CTA: mark its rows and leave
+        for (int j = g + tid * p.ctas_per_request; j < p.R; j += kThreads * p.ctas_per_request)
+            p.node_token[(int64_t)b * p.R + j] = -1;
+        return;
+    }
+    if (tid == 0) {
+        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
+        sh.timeout = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    unsigned st = 0, phase = 0, issued = 0;
+    for (int j = g; j < p.R; j += p.ctas_per_request) {
+        if (j > n) {
+            if (tid == 0) p.node_token[(int64_t)b * p.R + j] = -1;
+            continue;
+        }
+        if (!sample_one_row<DT>(sh, p, b, j, st, phase, issued)) {   // give up on this CTA's other rows too
+            for (int jj = j + p.ctas_per_request + tid * p.ctas_per_request; jj < p.R; jj += kThreads * p.ctas_per_request)
+                p.node_token[(int64_t)b * p.R + jj] = jj > n ? -1 : -2;
+            return;
+        }
+        __syncthreads();                                 // the run table and the ring are free for the next row
     }
 }
 
