@@ -38,7 +38,9 @@
  * all nodes and of all prefix-closed trees on tiny (K, L); fp64 log-softmax and stable argsort
  * from numpy/scipy; closed forms (uniform logits, K=1 chain, near-one-hot marginals);
  * the invariants the paper proves (Lemma 1, Theorem 1, Corollaries 1 and 2); numpy argmax;
- * brute-force accepted-path search.  No function here is "parity unpinned".
+ * brute-force accepted-path search; the two diagnostic margins (pop_gap, stop_gap) by hand-worked
+ * rationals, by the heap contents rebuilt from the pop order, and by a constructed near-tie.
+ * No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>

@@ -1,7 +1,8 @@
 """The five benchmark configurations at their full sizes, in the launch configuration bench.py times
 (inputs generated on the device, buffers reused, dense verification).  Trees are compared with the
 oracle for every request; per-node argmax and the accepted path are compared on every live row and on
-a seeded sample (>= 1 %) of the padding rows, which the oracle computes one row at a time."""
+every padding row for configurations 1 and 2, a seeded sample (>= 1 %) of them for the larger ones; the oracle
+computes those one row at a time."""
 import numpy as np
 import pytest
 import torch
@@ -36,7 +37,7 @@ def test_full_size_round(name):
     n = ot.n_nodes
     print(f"{name}: n* mean {n.float().mean():.1f} max {int(n.max())}; exempt {diag['exempt']}; "
           f"max |dlogZ| {diag['max_logZ_err']:.2e}")
-    assert len(diag["exempt"]) <= max(1, cfg.batch // 50)
+    assert diag["exempt"] == [], f"requests decided inside the oracle's own rounding margin: {diag['exempt']}"
     assert diag["max_logZ_err"] < LOGZ_TOL
     if name == "c4_stress":
         assert int(n.min()) == cfg.B_max
@@ -56,10 +57,11 @@ def test_full_size_round(name):
         assert int(gv.accepted_len[b]) == int(ov.accepted_len[0]), f"accepted_len, request {b}"
         assert torch.equal(to_cpu(gv.accepted_nodes[b]), ov.accepted_nodes[0]), f"accepted path, request {b}"
         assert int(gv.next_bonus[b]) == int(ov.next_bonus[0]), f"next bonus, request {b}"
-    # a seeded sample of all rows (live or padding), one oracle argmax per row
+    # configurations 1 and 2: every row of the dense tensor, live or padding; the larger ones: a seeded sample of
+    # at least 1 % of all rows (one oracle argmax per row)
     rng = np.random.default_rng(seed)
     total = cfg.batch * cfg.R
-    k = min(total, max(64, total // 100))
+    k = total if name in ("c1", "c2") else min(total, max(64, total // 100))
     picks = rng.choice(total, size=k, replace=False)
     rows = torch.from_numpy(picks).to(dev)
     sample = y.view(total, cfg.V)[rows].cpu()

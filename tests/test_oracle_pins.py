@@ -79,6 +79,30 @@ def test_softmax_topk_nonfinite():
     assert nf == 1 and pinf == 1
 
 
+def test_softmax_topk_lists_of_a_row_with_positive_infinity():
+    """+Inf is invalid input: it is flagged and carries no mass, and the lists reported for the row are those of
+    its finite logits alone — the library log-softmax of the finite sub-row, with the original token ids."""
+    for dtype in (torch.float32, torch.bfloat16):
+        row = torch.tensor([0.0, float("nan"), float("inf"), 1.0, 1.0, -float("inf"), 0.5, float("inf"), -2.0], dtype=dtype)
+        m, lz, tok, a, lp, ke, nf, pinf = O.row_softmax_topk(row, 4)
+        keep = np.array([0, 3, 4, 6, 8])                       # ids of the finite logits
+        x = f64(row)[keep]
+        order = np.argsort(-x, kind="stable")[:4]
+        assert nf == 1 and pinf == 1 and ke == 4
+        assert tok.tolist() == keep[order].tolist() == [3, 4, 6, 0]
+        assert m == 1.0
+        np.testing.assert_allclose(lp.numpy(), log_softmax(x)[order], rtol=0, atol=1e-15)
+        np.testing.assert_allclose(a.numpy(), x[order] - 1.0, rtol=0, atol=0)
+        assert lz == pytest.approx(math.log(2 + math.exp(-0.5) + math.exp(-1.0) + math.exp(-3.0)), rel=1e-15)
+    # a request with such a row returns the empty tree, flagged, and still reports those lists
+    x = torch.zeros(1, 2, 9)
+    x[0, 0] = row.float()
+    t = O.build_tree(x, K=4, B_max=8, cost_coef=quad_coef(1, 1.0, 1.0, 0.01, 0.0))
+    assert int(t.n_nodes[0]) == 0 and int(t.status[0]) & O.ST_NONFINITE
+    assert t.topk_token[0, 0].tolist() == [3, 4, 6, 0]
+    assert t.topk_token[0, 1].tolist() == [0, 1, 2, 3]
+
+
 # ---------------------------------------------------------------- hand-worked example
 def _golden():
     d = {}
@@ -108,6 +132,118 @@ def test_hand_worked_example():
     assert full.token_ids[0, 1:13].tolist() == [int(v) for v in g["full_order_tokens"]]
     assert full.parent_idx[0, 1:13].tolist() == [int(v) for v in g["full_order_parents"]]
     np.testing.assert_allclose(full.node_logprob[0, 1:13].exp().numpy(), g["full_order_prob"], rtol=1e-6)
+
+
+# ---------------------------------------------------------------- the margins that gate parity exemptions
+def test_exemption_margins_on_the_hand_worked_example():
+    """pop_gap[j] = 1 - (best strictly smaller prefix probability in the heap) / (prefix probability of pop j),
+    1 when the heap holds nothing smaller; stop_gap = |theta_new - theta_prev| / theta_prev at the test that
+    stopped the loop.  On the two-position example every value is a rational worked out by hand from the heap
+    contents (Algorithm 1: the heap holds the next sibling and the first child of what was popped)."""
+    from fractions import Fraction as Fr
+    g = _golden()
+    logits = torch.tensor(np.log(np.array([[g["q1"], g["q2"]]])), dtype=torch.float32)
+    coef = torch.tensor([g["cost"]], dtype=torch.float64)
+    # heap when row j is popped (prefix probabilities), popped value first:
+    #  1: {1/2}                       2: {1/3, 1/4}            3: {1/4, 1/12}          4: {1/4, 1/6, 1/12}
+    #  5: {1/6, 1/6, 1/12}            6: {1/6, 1/12, 1/24}     7: {1/12, 1/24, 1/24}   8: {1/12, 1/24, 1/24}
+    #  9..12: only 1/24 entries left
+    # pops 5 and 6 tie exactly at 1/6 while both are in the heap: the margin is the one to 1/12, not 0
+    want = [Fr(1), 1 - Fr(1, 4) / Fr(1, 3), 1 - Fr(1, 12) / Fr(1, 4), 1 - Fr(1, 6) / Fr(1, 4),
+            1 - Fr(1, 12) / Fr(1, 6), 1 - Fr(1, 12) / Fr(1, 6), 1 - Fr(1, 24) / Fr(1, 12), 1 - Fr(1, 24) / Fr(1, 12),
+            Fr(1), Fr(1), Fr(1), Fr(1)]
+    assert [float(w) for w in want[:8]] == pytest.approx([1, 1 / 4, 2 / 3, 1 / 3, 1 / 2, 1 / 2, 1 / 2, 1 / 2])
+    full = O.build_tree(logits, K=3, B_max=12, cost_coef=coef, flags=O.FLAG_FIXED_BUDGET)
+    np.testing.assert_allclose(full.pop_gap[0, 1:13].numpy(), [float(w) for w in want], rtol=1e-5)
+    assert float(full.pop_gap[0, 0]) == 1.0                                  # the root is not a pop
+    stop = O.build_tree(logits, K=3, B_max=12, cost_coef=coef)
+    np.testing.assert_allclose(stop.pop_gap[0, 1:5].numpy(), [float(w) for w in want[:4]], rtol=1e-5)
+    assert bool((stop.pop_gap[0, 5:] == 1.0).all())                          # padding rows
+    # the loop stopped on theta(5) = 10/13 <= theta(4) = 7/9
+    assert float(stop.stop_gap[0]) == pytest.approx(float(abs(Fr(10, 13) - Fr(7, 9)) / Fr(7, 9)), rel=1e-4)
+    assert float(abs(Fr(10, 13) - Fr(7, 9)) / Fr(7, 9)) == pytest.approx(1 / 91)
+    # nothing stops a fixed-budget run: the smallest margin over the accepted nodes is reported
+    probs = [Fr(1, 2), Fr(1, 3), Fr(1, 4), Fr(1, 4), Fr(1, 6), Fr(1, 6), Fr(1, 12), Fr(1, 12)] + [Fr(1, 24)] * 4
+    theta, phi = [Fr(1, 2)], Fr(0)
+    for n, pr in enumerate(probs, 1):
+        phi += pr
+        theta.append((1 + phi) / (2 + Fr(n, 4)))
+    assert theta[4] == Fr(7, 9) and theta[5] == Fr(10, 13)
+    smallest = min(abs(theta[n] - theta[n - 1]) / theta[n - 1] for n in range(1, 13))
+    assert float(full.stop_gap[0]) == pytest.approx(float(smallest), rel=1e-4)
+
+
+def frontier_margins(x_row_major, K, paths, scores):
+    """Margins by the definition, from the pop order alone: when the j-th node is popped the heap holds exactly the
+    unpopped nodes whose parent (a prefix) and whose previous sibling (same prefix, rank - 1) were popped before.
+    Scores are library log-softmax sums; scores closer than 1e-12 count as equal."""
+    L, V = x_row_major.shape
+    lps, toks = [], []
+    for i in range(L):
+        lp = log_softmax(x_row_major[i])
+        order = np.argsort(-x_row_major[i], kind="stable")[:K]
+        lps.append(lp[order]); toks.append([int(t) for t in order])
+    score = lambda path: sum(lps[i][toks[i].index(t)] for i, t in enumerate(path))
+    popped, out = {()}, []
+    for j, path in enumerate(paths):
+        heap = []
+        for pre in popped:                                       # children of popped nodes
+            d = len(pre)
+            if d == L:
+                continue
+            for r, t in enumerate(toks[d]):
+                c = pre + (t,)
+                if c in popped:
+                    continue
+                if r == 0 or pre + (toks[d][r - 1],) in popped:
+                    heap.append(score(c))
+        assert abs(max(heap) - scores[j]) < 1e-12                # the popped node is the heap's maximum
+        smaller = [s for s in heap if s < scores[j] - 1e-12]
+        out.append(1.0 - math.exp(max(smaller) - scores[j]) if smaller else 1.0)
+        popped.add(path)
+    return out
+
+
+@pytest.mark.parametrize("K,L,V,seed,quant", [(2, 3, 5, 0, None), (3, 3, 6, 1, 2), (4, 3, 9, 2, 4), (2, 5, 4, 3, 1), (3, 2, 40, 4, None)])
+def test_pop_gap_equals_runner_up_margin_by_definition(K, L, V, seed, quant):
+    x = rand_logits(seed + 7, 1, L, V, quant=quant)
+    B = sum(min(K, V) ** d for d in range(1, L + 1))
+    t = O.build_tree(x, K, B_max=B, cost_coef=quad_coef(1, 1.0, 1.0, 0.0, 0.0), flags=O.FLAG_FIXED_BUDGET)
+    assert int(t.n_nodes[0]) == B
+    want = frontier_margins(f64(x[0]), K, tree_paths(t), t.node_logprob[0, 1:B + 1].numpy())
+    got = t.pop_gap[0, 1:B + 1].numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-9, atol=1e-12)
+    if quant:                                                    # quantised logits: exact ties occur and are skipped over
+        sig = t.node_logprob[0, 1:B + 1].numpy()
+        assert np.any(np.diff(sig) == 0.0) and np.all(got > 1e-3)
+
+
+def test_margins_of_a_constructed_near_tie():
+    """Depth-1 runner-up against the first child of the best token, 1e-9 apart in probability: the margin must come
+    out as that 1e-9 (not 0, not the gap to some farther score), and an exact tie beside it must be skipped."""
+    # position 2: p = softmax(0, -1, r); log p_0 moves by ~e^r per unit of r, so r near -20 tunes it in steps of
+    # ~1e-15; position 1: tokens 0 and 1 differ by d = fp32(log p_0) (so the sibling ties the child up to rounding)
+    d32 = np.float32(-math.log(1 + math.exp(-1.0)))
+    best = None
+    for r in np.arange(-21.0, -19.0, 1.0 / 1024, dtype=np.float32):
+        lp0 = log_softmax(np.array([0.0, -1.0, float(r)]))[0]
+        gap = 1.0 - math.exp(lp0 - float(d32)) if lp0 < float(d32) else None       # child just below the sibling
+        if gap is not None and (best is None or abs(gap - 1e-9) < abs(best[1] - 1e-9)):
+            best = (float(r), gap)
+    r, gap = best
+    assert 0.2e-9 < gap < 5e-9
+    x = torch.tensor([[[0.0, float(d32), float(d32), -30.0], [0.0, -1.0, r, -40.0]]], dtype=torch.float32)
+    t = O.build_tree(x, K=3, B_max=4, cost_coef=quad_coef(1, 1.0, 1.0, 0.0, 0.0), flags=O.FLAG_FIXED_BUDGET)
+    # pops: token 0; then its sibling token 1 (depth 1) against the child (0, 0), 1e-9 below it
+    assert t.token_ids[0, 1:4].tolist() == [0, 1, 2] and t.depth[0, 1:4].tolist() == [1, 1, 1]
+    assert float(t.pop_gap[0, 2]) == pytest.approx(gap, rel=1e-5)
+    # third pop: token 2 ties token 1 exactly (already popped, so not in the heap); the child (0, 0) is the nearest
+    # distinct score and the margin is again the constructed one
+    assert float(t.pop_gap[0, 3]) == pytest.approx(gap, rel=1e-5)
+    # fourth pop: the child (0, 0) itself; below it are (1, 0) and (2, 0), which tie each other exactly at
+    # p_1(1) p_2(0): margin 1 - p_1(1) / p_1(0) = 1 - e^d
+    assert t.depth[0, 4].item() == 2 and t.parent_idx[0, 4].item() == 1
+    assert float(t.pop_gap[0, 4]) == pytest.approx(1.0 - math.exp(float(d32)), rel=1e-9)
 
 
 # ---------------------------------------------------------------- O3: pop order = plain definition
