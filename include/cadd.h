@@ -58,6 +58,7 @@ extern "C" {
 #define CADD_STATUS_L_EFF_CLAMPED       16   /* l_eff[b] was outside [0, L] */
 #define CADD_STATUS_COST_NONPOSITIVE    32   /* C_d + C_v(n) <= 0 (or not finite) was met; expansion stopped there */
 #define CADD_STATUS_BAD_N_NODES         64   /* verify: n_nodes[b] was outside [0, R-1] and was clamped */
+#define CADD_STATUS_BAD_TABLE_IDX      256   /* build, CADD_COST_TABLE: table_idx[b] was outside [0, n_tables); the request returns the empty tree */
 #define CADD_STATUS_INTERNAL_TIMEOUT   128   /* a bounded wait on an asynchronous copy ran out; build returns the empty tree, verify leaves -2 in node_argmax */
 
 #define CADD_DTYPE_BF16 0
@@ -106,7 +107,7 @@ typedef struct cadd_build_args {
     int32_t  n_tables;             /* TABLE, TABLE_INTERP: number of rows of cost_table */
     const double*  cost_coef;      /* QUADRATIC: [batch,4] = (C_d, a, b, c) */
     const double*  cost_table;     /* TABLE: [n_tables, B_max+1] */
-    const int32_t* table_idx;      /* TABLE: [batch], each in [0, n_tables) */
+    const int32_t* table_idx;      /* TABLE: [batch], each in [0, n_tables); a value outside is never dereferenced: CADD_STATUS_BAD_TABLE_IDX, empty tree */
     const double*  t_draft;        /* TABLE, TABLE_INTERP: [batch] C_d */
     const int32_t* ctx_grid;       /* TABLE_INTERP: [n_tables] strictly ascending context lengths of the tables */
     /* outputs; n_nodes, token_ids, parent_idx, depth are required, the rest may be NULL */

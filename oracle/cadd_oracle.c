@@ -61,7 +61,8 @@ enum {
     ORC_ST_FRONTIER_EXHAUSTED = 8,
     ORC_ST_L_EFF_CLAMPED = 16,
     ORC_ST_COST_NONPOSITIVE = 32,
-    ORC_ST_BAD_N_NODES = 64
+    ORC_ST_BAD_N_NODES = 64,
+    ORC_ST_BAD_TABLE_IDX = 256
 };
 
 int cadd_oracle_num_threads(void)
@@ -242,9 +243,14 @@ int cadd_oracle_build_tree(
 
         /* ---- O3: Algorithm 1 ---- */
         cost_model_t cm = { cost_kind, NULL, NULL, NULL, 0.0 };
+        int bad_table = 0;
         if (cost_kind == ORC_COST_QUADRATIC) cm.coef4 = cost_coef + (size_t)b * 4;
-        else if (cost_kind == ORC_COST_TABLE) cm.row0 = cost_table + (size_t)table_idx[b] * (B_max + 1);
-        else {                                   /* Eq. 13: the two profiled context lengths around l */
+        else if (cost_kind == ORC_COST_TABLE) {
+            /* a table index outside [0, n_tables) names no cost model: flagged, empty tree */
+            int ti = table_idx[b];
+            if (ti < 0 || ti >= n_tables) { st |= ORC_ST_BAD_TABLE_IDX; bad_table = 1; ti = 0; }
+            cm.row0 = cost_table + (size_t)ti * (B_max + 1);
+        } else {                                   /* Eq. 13: the two profiled context lengths around l */
             const int l = ctx_len ? ctx_len[b] : 0;
             int jlo = 0;
             while (jlo + 1 < n_tables && ctx_grid[jlo + 1] <= l) ++jlo;      /* largest j with L_j <= l (or 0) */
@@ -265,8 +271,8 @@ int cadd_oracle_build_tree(
         double Phi = 0.0, theta_prev = 0.0;
         double min_margin = INFINITY, stop_margin = -1.0;
         double den0 = C_d + cost_verify(&cm, 0);
-        int ok = 1;
-        if (!(den0 > 0.0)) { st |= ORC_ST_COST_NONPOSITIVE; ok = 0; }
+        int ok = !bad_table;
+        if (ok && !(den0 > 0.0)) { st |= ORC_ST_COST_NONPOSITIVE; ok = 0; }
         else theta_prev = 1.0 / den0;
         if (any_pinf) ok = 0;
         if (theta_curve) theta_curve[(size_t)b * R] = theta_prev;

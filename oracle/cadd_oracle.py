@@ -24,6 +24,7 @@ FLAG_FIXED_BUDGET = 4
 ROWS_LIVE, ROWS_DENSE = 0, 1
 ST_NONFINITE, ST_FEWER_THAN_K, ST_CAP_HIT, ST_FRONTIER_EXHAUSTED = 1, 2, 4, 8
 ST_L_EFF_CLAMPED, ST_COST_NONPOSITIVE, ST_BAD_N_NODES = 16, 32, 64
+ST_BAD_TABLE_IDX = 256
 
 
 def build(force: bool = False) -> str:

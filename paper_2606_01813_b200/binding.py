@@ -20,6 +20,7 @@ OK = 0
 ERR_NULL, ERR_STRUCT_SIZE, ERR_SHAPE, ERR_DTYPE, ERR_ALIGN, ERR_WORKSPACE, ERR_LAUNCH = -1, -2, -3, -4, -5, -6, -7
 STATUS_NONFINITE_INPUT, STATUS_FEWER_THAN_K_FINITE, STATUS_CAP_HIT, STATUS_FRONTIER_EXHAUSTED = 1, 2, 4, 8
 STATUS_L_EFF_CLAMPED, STATUS_COST_NONPOSITIVE, STATUS_BAD_N_NODES, STATUS_INTERNAL_TIMEOUT = 16, 32, 64, 128
+STATUS_BAD_TABLE_IDX = 256
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 COST_QUADRATIC, COST_TABLE, COST_TABLE_INTERP = 0, 1, 2
 FLAG_EMIT_DENSE_MASK, FLAG_EMIT_TOPK, FLAG_FIXED_BUDGET = 1, 2, 4

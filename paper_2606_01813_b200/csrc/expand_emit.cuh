@@ -223,11 +223,19 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
         cm.kind = p.cost_kind; cm.row0 = cm.row1 = nullptr; cm.alpha = 0.0;
         cm.q[0] = cm.q[1] = cm.q[2] = cm.q[3] = 0.0;
         double C_d;
+        int st = 0;
+        bool ok = true;
         if (p.cost_kind == CADD_COST_QUADRATIC) {
             for (int c = 0; c < 4; ++c) cm.q[c] = p.cost_coef[(int64_t)b * 4 + c];
             C_d = cm.q[0];
         } else if (p.cost_kind == CADD_COST_TABLE) {
-            cm.row0 = p.cost_table + (int64_t)p.table_idx[b] * (B_max + 1);
+            int ti = p.table_idx[b];
+            if (ti < 0 || ti >= p.n_tables) {               // no such table: flagged, empty tree, nothing of it is read
+                st |= CADD_STATUS_BAD_TABLE_IDX;
+                ok = false;
+                ti = 0;
+            }
+            cm.row0 = p.cost_table + (int64_t)ti * (B_max + 1);
             C_d = p.t_draft[b];
         } else {                                            // Eq. 13: the two profiled context lengths around l
             const int l = p.ctx_len ? p.ctx_len[b] : 0;
@@ -240,11 +248,9 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
             cm.alpha = jhi == jlo ? 0.0 : ((double)l - (double)p.ctx_grid[jlo]) / ((double)p.ctx_grid[jhi] - (double)p.ctx_grid[jlo]);
             C_d = p.t_draft[b];
         }
-        int st = 0;
-        bool ok = true;
         double theta_prev = 0.0, Phi = 0.0;
         const double den0 = C_d + cost_verify(cm, 0);
-        if (!(den0 > 0.0)) { st |= CADD_STATUS_COST_NONPOSITIVE; ok = false; }
+        if (ok && !(den0 > 0.0)) { st |= CADD_STATUS_COST_NONPOSITIVE; ok = false; }
         else theta_prev = 1.0 / den0;
         if (s_pinf) ok = false;
 

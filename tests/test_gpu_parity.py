@@ -168,6 +168,23 @@ def test_table_cost_and_limits():
     assert int(ot.n_nodes[0]) == 2048
 
 
+def test_table_index_out_of_range_is_flagged_and_reads_nothing():
+    """A table index that names no table must not be dereferenced: the request is flagged and gets the empty tree,
+    its neighbours are untouched."""
+    g = torch.Generator().manual_seed(12)
+    x = (torch.randn(4, 5, 700, generator=g) * 2).to(torch.bfloat16)
+    n = torch.arange(41, dtype=torch.float64)
+    table = torch.stack([0.9 + 0.01 * n + 0.0004 * n * n, 0.5 + 0.002 * n])
+    kw = dict(cost_kind=G.COST_TABLE, cost_table=table, table_idx=torch.tensor([-1, 1, 2, 1 << 30], dtype=torch.int32),
+              t_draft=torch.tensor([0.3, 0.2, 0.3, 0.3], dtype=torch.float64))
+    for flags in (0, G.FLAG_FIXED_BUDGET):
+        gt, ot = run_both_build(x, 6, 40, **kw, flags=flags)
+        assert not compare_build(gt, ot, 6)["exempt"]
+        st = to_cpu(gt.status)
+        assert [bool(int(v) & G.STATUS_BAD_TABLE_IDX) for v in st] == [True, False, True, True]
+        assert to_cpu(gt.n_nodes)[[0, 2, 3]].tolist() == [0, 0, 0] and int(gt.n_nodes[1]) > 0
+
+
 def test_argmax_ties_nan_and_walk():
     g = torch.Generator().manual_seed(11)
     batch, R, V, L = 3, 40, 151936, 6

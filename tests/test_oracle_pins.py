@@ -579,6 +579,16 @@ def test_edge_cases_and_status():
     assert int(t.n_nodes[0]) == 12 and int(t.status[0]) & O.ST_FEWER_THAN_K
     with pytest.raises(ValueError):
         O.build_tree(x, 4, 20, R=20, cost_coef=coef)                             # R < B_max + 1
+    # a table index that names no table: flagged, empty tree, the other requests as with a valid index
+    n = torch.arange(21, dtype=torch.float64)
+    table = torch.stack([1.0 + 0.01 * n, 1.0 + 0.2 * n])
+    td = torch.full((3,), 1.0, dtype=torch.float64)
+    t = O.build_tree(x, 4, 20, cost_kind=O.COST_TABLE, cost_table=table, t_draft=td,
+                     table_idx=torch.tensor([2, 0, -1], dtype=torch.int32))
+    assert [bool(int(v) & O.ST_BAD_TABLE_IDX) for v in t.status] == [True, False, True]
+    assert int(t.n_nodes[0]) == 0 == int(t.n_nodes[2]) and int(t.token_ids[0, 1:].max()) == -1
+    ref = O.build_tree(x, 4, 20, cost_coef=coef)                                 # table 0 is that quadratic
+    assert int(t.n_nodes[1]) == int(ref.n_nodes[1]) > 0 and torch.equal(t.token_ids[1], ref.token_ids[1])
 
 
 def test_cross_depth_exact_tie_prefers_lower_depth():
