@@ -4,13 +4,16 @@
 A *step* is one decoding round of the whole hot path over one batch of synthetic input:
     cadd_build_tree   (softmax + top-K over every live draft position, expansion, emission)
     cadd_verify_tree  (argmax over every target row, accepted-path walk)
-The default workload is benchmark configuration 2 (batch 32, L 16, V 151936, bf16, K 8, B_max 256) with
-verification over the dense [batch, B_max+1, V] target tensor.  Inputs are seeded synthetic logits
-(paper_2606_01813_b200.synth); they are far larger than L2, so no flush is needed between steps.
+The default workload is the largest benchmark configuration that fits one GPU: configuration 5 (batch 256, L 16 with
+4..16 live positions per request, V 151936, bf16, K 8, B_max 384) with verification over the dense
+[batch, B_max+1, V] target tensor, 30.7 GB of logits per round.  Configurations 2 and 4 (budget stress) are measured
+the same way afterwards and reported as extra keys of the same line (`other_workloads`).  Inputs are seeded synthetic
+logits (paper_2606_01813_b200.synth); they are far larger than L2, so no flush is needed between steps.
 
-`python bench.py --gpus N --steps K --warmup W` prints ONE JSON line (rank 0).  With N > 1 (under
-torchrun) every rank runs an independent replica of the workload (requests are independent; there is no
-exchange step), and the value is the rounds all ranks completed per second of the slowest rank.
+`python bench.py --gpus N --steps K --warmup W` prints ONE JSON line (rank 0).  With N > 1 every rank runs an
+independent replica of the workload (requests are independent; there is no exchange step), and the value is the
+rounds all ranks completed per second of the slowest rank; the N ranks come from torchrun, or, when the command is
+started by hand, from this script starting N copies of itself.
 `--impl reference` times the CPU oracle instead (the only baseline there is: the paper ships no code).
 """
 from __future__ import annotations
@@ -40,6 +43,10 @@ KERNELS_PER_STEP = 4          # softmax_topk_partial, expand_emit, row_argmax, a
 # algorithmic bytes, from an ncu capture of the config-2 launch (summary kept under profiles/)
 # (2.5037 GB for 2.4990 GB).  Traffic grows in proportion to the rows read, so other workloads scale it.
 ARGMAX_TRAFFIC_RATIO = 1.0019
+# The same for one softmax_topk_partial launch (159.5 MB read + written for 155.6 MB of logits: the per-row records are
+# the extra), profiles/softmax_topk_partial_config2.md.
+TOPK_TRAFFIC_RATIO = 1.025
+NOMINAL_HBM_GBS = 8000.0      # the nominal HBM3e figure the bandwidth target is stated against
 
 
 def measured_peak_gbs():
@@ -107,6 +114,148 @@ def cost_kwargs(G, c):
     return dict(cost_kind=G.COST_QUADRATIC, cost_coef=c.coef)
 
 
+def workload_string(cfg, rows_mode):
+    return (f"config {cfg.index} ({cfg.name}): batch={cfg.batch} L={cfg.L} V={cfg.V} {cfg.dtype} "
+            f"K={cfg.K} B_max={cfg.B_max} R={cfg.R}, verify rows_mode={rows_mode}")
+
+
+def config_block(cfg, rows_mode, world):
+    """The `config` object of the JSON line; the same for the CUDA arm and the reference arm."""
+    dense_bytes = (cfg.batch * cfg.L + cfg.batch * cfg.R) * cfg.V * cfg.elem_bytes
+    big = rows_mode == "dense" and dense_bytes > (126 << 20)
+    return {"workload": workload_string(cfg, rows_mode),
+            "l2": ("inputs larger than L2 (no flush needed)" if big else
+                   "inputs may fit in L2 and are not flushed between steps (a launch-bound or live-rows case)"),
+            "parallelism": f"replicas x{world}"}
+
+
+def hbm_roofline(kernel, nbytes, ms, traffic_ratio, profile):
+    """Roofline block of one streaming kernel: algorithmic bytes of one launch over its CUDA-event duration."""
+    peak, peak_kind = measured_peak_gbs()
+    ach = nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+    return {"kernel": kernel, "bound": "hbm", "achieved": round(ach, 1), "peak": peak, "peak_kind": f"of {peak_kind}",
+            "unit": "GB/s", "frac": round(ach / peak, 4), "frac_of_nominal_8tbs": round(ach / NOMINAL_HBM_GBS, 4),
+            "traffic": int(nbytes * traffic_ratio), "traffic_source": profile,
+            "algorithmic_bytes": int(nbytes), "ms": round(ms, 5)}
+
+
+class Workload:
+    """One benchmark configuration resident in HBM: inputs, reusable outputs, and the step that is timed."""
+
+    def __init__(self, G, cfg, rows_mode, rank, dev):
+        self.G, self.cfg, self.dev = G, cfg, dev
+        self.rows_mode_name = rows_mode
+        self.rows_mode = G.ROWS_DENSE if rows_mode == "dense" else G.ROWS_LIVE
+        self.flags = G.FLAG_FIXED_BUDGET if cfg.fixed_budget else 0
+        seed = replicas.replica_seed(synth.config_seed(cfg), rank)
+        self.d = d = synth.make_draft_inputs(cfg, seed, device=str(dev))
+        self.c = c = synth.make_cost_inputs(cfg, seed)
+        self.kw = dict(l_eff=d.l_eff.to(dev), bonus_token=d.bonus_token.to(dev), ctx_len=d.ctx_len.to(dev))
+        self.ck = {k: (v.to(dev) if torch.is_tensor(v) else v) for k, v in cost_kwargs(G, c).items()}
+        self.ws = torch.empty(G.cadd_build_workspace_bytes(cfg.batch, cfg.L, cfg.V, cfg.K, cfg.B_max, cfg.R, cfg.torch_dtype),
+                              dtype=torch.uint8, device=dev)
+        self.tree = G.cadd_build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, workspace=self.ws, flags=self.flags, **self.kw, **self.ck)
+        torch.cuda.synchronize()
+        self.y = synth.make_target_logits(cfg, seed, d, self.tree.depth.cpu(), device=str(dev))
+        self.verdict = G.cadd_verify_tree(self.y, cfg.L, self.tree.n_nodes, self.tree.token_ids, self.tree.parent_idx, self.rows_mode)
+        torch.cuda.synchronize()
+        n_star = self.tree.n_nodes.cpu()
+        es = cfg.elem_bytes
+        self.n_star = n_star
+        self.build_bytes = int(d.l_eff.clamp(0, cfg.L).sum().item()) * cfg.V * es
+        rows_read = cfg.batch * cfg.R if self.rows_mode == G.ROWS_DENSE else int((n_star + 1).sum().item())
+        self.verify_bytes = rows_read * cfg.V * es
+
+    def build(self, x=None, extra_flags=0):
+        cfg = self.cfg
+        self.G.cadd_build_tree(self.d.logits if x is None else x, cfg.K, cfg.B_max, cfg.R, workspace=self.ws, out=self.tree,
+                               flags=self.flags | extra_flags, **self.kw, **self.ck)
+
+    def verify(self, y=None, flags=0):
+        t = self.tree
+        self.G.cadd_verify_tree(self.y if y is None else y, self.cfg.L, t.n_nodes, t.token_ids, t.parent_idx, self.rows_mode,
+                                out=self.verdict, flags=flags)
+
+    def step(self):
+        self.build()
+        self.verify()
+
+
+def barrier():
+    replicas.barrier()
+    torch.cuda.synchronize()
+
+
+def timed_region(w, K, Wm, world):
+    """Wm untimed steps, then exactly K steps between one pair of CUDA events on the launching stream, bracketed by
+    barrier + synchronize; MAX over ranks.  Returns (total ms, wall seconds)."""
+    for _ in range(Wm):
+        w.step()
+    e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.perf_counter()
+    e_start.record()
+    for _ in range(K):
+        w.step()
+    e_end.record()
+    barrier()
+    return replicas.max_over_ranks(e_start.elapsed_time(e_end), w.dev), time.perf_counter() - t0
+
+
+def per_kernel_pass(w, K):
+    """K more steps, each kernel of the step launched by a call of its own (the single-kernel flags of the C ABI) with a
+    CUDA event on either side, so that every kernel is timed alone on the launching stream.  Kept out of the timed
+    region: the events keep a kernel from being set up while the one before it drains."""
+    G = w.G
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(5 * K)]
+    for i in range(K):
+        ev[5 * i].record()
+        w.build(extra_flags=G.FLAG_ONLY_TOPK)
+        ev[5 * i + 1].record()
+        w.build(extra_flags=G.FLAG_ONLY_EXPAND)
+        ev[5 * i + 2].record()
+        w.verify(flags=G.VERIFY_ONLY_ARGMAX)
+        ev[5 * i + 3].record()
+        w.verify(flags=G.VERIFY_ONLY_WALK)
+        ev[5 * i + 4].record()
+    barrier()
+    mean = lambda a, b: sum(ev[5 * i + a].elapsed_time(ev[5 * i + b]) for i in range(K)) / K
+    steps = sorted(ev[5 * i].elapsed_time(ev[5 * i + 4]) for i in range(K))
+    return {"softmax_topk_partial": mean(0, 1), "expand_emit": mean(1, 2), "row_argmax": mean(2, 3), "accept_walk": mean(3, 4),
+            "step_mean": mean(0, 4), "step_median": steps[K // 2], "step_min": steps[0]}
+
+
+def kernel_blocks(w, km):
+    """Roofline blocks of the two streaming kernels and the absolute times of the two latency-bound ones."""
+    topk = hbm_roofline("softmax_topk_partial", w.build_bytes, km["softmax_topk_partial"], TOPK_TRAFFIC_RATIO,
+                        "profiles/softmax_topk_partial_config2.md, scaled by rows")
+    argmax = hbm_roofline("row_argmax", w.verify_bytes, km["row_argmax"], ARGMAX_TRAFFIC_RATIO,
+                          "profiles/row_argmax_config2.md, scaled by rows")
+    return topk, argmax, {k: round(km[k], 5) for k in ("softmax_topk_partial", "expand_emit", "row_argmax", "accept_walk",
+                                                         "step_mean", "step_median", "step_min")}
+
+
+def tree_stats(w):
+    n = w.n_star
+    return {"n_star_mean": round(float(n.float().mean()), 2), "n_star_max": int(n.max()), "n_star_hist": n_star_histogram(n),
+            "accepted_mean": round(float(w.verdict.accepted_len.float().mean().item()), 2)}
+
+
+def side_workload(G, name, rows_mode, rank, world, dev, K, Wm):
+    """Another benchmark configuration measured the same way (timed region + per-kernel pass), reported as an extra key."""
+    cfg = synth.CONFIGS[name]
+    w = Workload(G, cfg, rows_mode, rank, dev)
+    total_ms, _ = timed_region(w, K, Wm, world)
+    km = per_kernel_pass(w, K)
+    topk, argmax, kms = kernel_blocks(w, km)
+    out = {"workload": workload_string(cfg, rows_mode), "value": round(replicas.whole_job_rounds_per_second(K, world, total_ms), 3),
+           "unit": UNIT, "steps": K, "ms_per_step": round(total_ms / K, 5), "kernel_ms": kms,
+           "roofline_softmax_topk": topk, "roofline_row_argmax": argmax, "trees": tree_stats(w)}
+    del w
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, rank, world):
     from paper_2606_01813_b200 import binding as G
     from paper_2606_01813_b200 import build as cuda_build
@@ -118,126 +267,35 @@ def run_ours(args, rank, world):
     cfg = synth.CONFIGS[args.workload]
     if args.batch:
         cfg = synth.scaled(cfg, batch=args.batch)        # reduced case of the same workload (profiling captures)
-    seed = replicas.replica_seed(synth.config_seed(cfg), rank)
-    rows_mode = G.ROWS_DENSE if args.rows_mode == "dense" else G.ROWS_LIVE
-    flags = G.FLAG_FIXED_BUDGET if cfg.fixed_budget else 0
-
-    # ---- inputs resident in HBM ----
-    d = synth.make_draft_inputs(cfg, seed, device=str(dev))
-    c = synth.make_cost_inputs(cfg, seed)
-    kw = dict(l_eff=d.l_eff.to(dev), bonus_token=d.bonus_token.to(dev), ctx_len=d.ctx_len.to(dev), flags=flags)
-    ck = {k: (v.to(dev) if torch.is_tensor(v) else v) for k, v in cost_kwargs(G, c).items()}
-    ws = torch.empty(G.cadd_build_workspace_bytes(cfg.batch, cfg.L, cfg.V, cfg.K, cfg.B_max, cfg.R, cfg.torch_dtype),
-                     dtype=torch.uint8, device=dev)
-    tree = G.cadd_build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, workspace=ws, **kw, **ck)
-    torch.cuda.synchronize()
-    y = synth.make_target_logits(cfg, seed, d, tree.depth.cpu(), device=str(dev))
-    verdict = G.cadd_verify_tree(y, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode)
-    torch.cuda.synchronize()
-
-    def step():
-        G.cadd_build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=tree, **kw, **ck)
-        G.cadd_verify_tree(y, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, out=verdict)
-
-    def barrier():
-        replicas.barrier()
-        torch.cuda.synchronize()
+    w = Workload(G, cfg, args.rows_mode, rank, dev)      # inputs resident in HBM
+    d, c, y, tree, verdict, ws, kw, ck = w.d, w.c, w.y, w.tree, w.verdict, w.ws, dict(w.kw, flags=w.flags), w.ck
+    rows_mode = w.rows_mode
 
     # ---- device-resident timing ----
     K, Wm = args.steps, max(args.warmup, 3)
     sampler = ClockSampler(dev) if rank == 0 else None
-    for _ in range(Wm):
-        step()
-    # The timed region: exactly K steps between one pair of events (barrier + synchronize on both sides).
-    e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    t_wall0 = time.perf_counter()
-    e_start.record()
-    for i in range(K):
-        step()
-    e_end.record()
-    barrier()
-    total_ms = e_start.elapsed_time(e_end)
-    # A second pass of K steps with an event around every call gives the per-call breakdown (build / verify) the
-    # roofline block needs.  It is kept out of the timed region because the events cost about 10 us per step on this
-    # workload: an event between two calls keeps the second call's first kernel from being set up while the first
-    # call's last kernel drains.
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * K)]
-    for i in range(K):
-        ev[3 * i].record()
-        G.cadd_build_tree(d.logits, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=tree, **kw, **ck)
-        ev[3 * i + 1].record()
-        G.cadd_verify_tree(y, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, out=verdict)
-        ev[3 * i + 2].record()
-    barrier()
-    t_wall = time.perf_counter() - t_wall0
+    total_ms, t_wall = timed_region(w, K, Wm, world)
+    km = per_kernel_pass(w, K)
     # keep the GPU busy long enough for a few clock samples if the timed region was very short
     if sampler is not None:
         t_end = time.perf_counter() + max(0.0, 0.6 - t_wall)
         while time.perf_counter() < t_end:
-            step()
+            w.step()
         torch.cuda.synchronize()
     clocks = sampler.stop() if sampler is not None else None
-    instrumented_ms = ev[0].elapsed_time(ev[3 * K - 1]) / K
-    per_step = sorted(ev[3 * i].elapsed_time(ev[3 * i + 2]) for i in range(K))
-    step_median_ms, step_min_ms = per_step[K // 2], per_step[0]
-    build_ms = sum(ev[3 * i].elapsed_time(ev[3 * i + 1]) for i in range(K)) / K
-    verify_ms = sum(ev[3 * i + 1].elapsed_time(ev[3 * i + 2]) for i in range(K)) / K
-    total_ms = replicas.max_over_ranks(total_ms, dev)
     value = replicas.whole_job_rounds_per_second(K, world, total_ms)
-
-    # ---- algorithmic bytes (logit bytes the kernels must read) ----
-    n_star = tree.n_nodes.cpu()
-    es = cfg.elem_bytes
-    build_bytes = int(d.l_eff.clamp(0, cfg.L).sum().item()) * cfg.V * es
-    rows_read = cfg.batch * cfg.R if rows_mode == G.ROWS_DENSE else int((n_star + 1).sum().item())
-    verify_bytes = rows_read * cfg.V * es
-    peak, peak_kind = measured_peak_gbs()
-    achieved = verify_bytes / (verify_ms * 1e-3) / 1e9
-    roofline = {"kernel": "row_argmax (+accept_walk, timed together)", "bound": "hbm", "achieved": round(achieved, 1),
-                "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(achieved / peak, 4),
-                "traffic": None if ARGMAX_TRAFFIC_RATIO is None else int(verify_bytes * ARGMAX_TRAFFIC_RATIO),
-                "algorithmic_bytes": verify_bytes, "ms": round(verify_ms, 4)}
-    build_gbs = build_bytes / (build_ms * 1e-3) / 1e9
-    build_info = {"kernels": "softmax_topk_partial + expand_emit", "ms": round(build_ms, 4), "algorithmic_bytes": build_bytes,
-                  "achieved": round(build_gbs, 1), "unit": "GB/s", "frac": round(build_gbs / peak, 4)}
+    roofline_topk, roofline, kernel_ms = kernel_blocks(w, km)
+    verify_bytes = w.verify_bytes
+    step = w.step
 
     # ---- end to end through the public API with HOST buffers ----
     e2e = None
     if not args.no_e2e:
-        hx = d.logits.cpu().pin_memory()
-        hy = torch.empty(y.shape, dtype=y.dtype, pin_memory=True)
-        hy.copy_(y)
-        h_tree = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (tree.n_nodes, tree.token_ids, tree.parent_idx, tree.depth)]
-        h_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (verdict.accepted_len, verdict.accepted_nodes, verdict.next_bonus)]
-        dx = torch.empty_like(d.logits)
-        dy = torch.empty_like(y)
-
-        def e2e_step():
-            dx.copy_(hx, non_blocking=True)
-            G.cadd_build_tree(dx, cfg.K, cfg.B_max, cfg.R, workspace=ws, out=tree, **kw, **ck)
-            for h, t in zip(h_tree, (tree.n_nodes, tree.token_ids, tree.parent_idx, tree.depth)):
-                h.copy_(t, non_blocking=True)
-            dy.copy_(hy, non_blocking=True)
-            G.cadd_verify_tree(dy, cfg.L, tree.n_nodes, tree.token_ids, tree.parent_idx, rows_mode, out=verdict)
-            for h, t in zip(h_out, (verdict.accepted_len, verdict.accepted_nodes, verdict.next_bonus)):
-                h.copy_(t, non_blocking=True)
-
-        ke = max(1, min(K, args.e2e_steps))
-        e2e_step()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(ke):
-            e2e_step()
-        e1.record()
-        barrier()
-        ems = replicas.max_over_ranks(e0.elapsed_time(e1), dev)
-        h2d = hx.numel() * hx.element_size() + hy.numel() * hy.element_size()
-        d2h = sum(h.numel() * h.element_size() for h in h_tree + h_out)
-        e2e = {"value": round(replicas.whole_job_rounds_per_second(ke, world, ems), 3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": ke, "ms_per_step": round(ems / ke, 3)}
-        del hx, hy, dx, dy
+        try:
+            e2e = e2e_block(G, w, world, max(1, min(K, args.e2e_steps)))
+        except Exception as ex:      # e.g. the host cannot pin a copy of the target logits
+            e2e = {"error": str(ex)[:200]}
+        torch.cuda.empty_cache()
 
     # ---- verification under sampling (T = 1) over the same target logits: one draw per row instead of the arg-max ----
     sampled = None
@@ -305,32 +363,87 @@ def run_ours(args, rank, world):
     fresh = None
     if args.fresh_rounds > 0:
         try:
-            fresh = fresh_rounds_block(G, cfg, rank, rows_mode, flags, ws, tree, verdict, y, dev, args.fresh_rounds)
+            fresh = fresh_rounds_block(G, cfg, rank, rows_mode, w.flags, ws, tree, verdict, y, dev, args.fresh_rounds)
         except Exception as ex:
             fresh = {"error": str(ex)[:200]}
 
     # ---- the oracle timed on this machine's host cores, on a bounded sample (rank 0, N = 1 only) ----
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu_baseline = oracle_sample(cfg, d, c, y, tree, rows_mode == G.ROWS_DENSE, args.cpu_requests)
+        cpu_baseline = oracle_sample(cfg, d, c, y, tree, w.rows_mode == G.ROWS_DENSE, args.cpu_requests)
+
+    # ---- two more of the V = 151936 configurations, measured the same way, as extra keys of the line ----
+    others = {}
+    for name in [n for n in args.also.split(",") if n and n != "none"]:
+        if name == args.workload or args.batch:
+            continue
+        try:
+            settle()
+            if name in ("c3", "c4", "c4_stress", "c5"):          # tens of GB each: make room first
+                w.y = None
+                y = None
+                torch.cuda.empty_cache()
+            others[name] = side_workload(G, name, args.rows_mode, rank, world, dev, min(K, 50), 3)
+        except Exception as ex:
+            others[name] = {"error": str(ex)[:200]}
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-            "ms_per_step": round(total_ms / K, 5), "instrumented_ms_per_step": round(instrumented_ms, 5), "instrumented_step_median_ms": round(step_median_ms, 5), "instrumented_step_min_ms": round(step_min_ms, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": cfg.dtype, "data": "synthetic",
-            "config": {"workload": f"config {cfg.index} ({cfg.name}): batch={cfg.batch} L={cfg.L} V={cfg.V} {cfg.dtype} "
-                                   f"K={cfg.K} B_max={cfg.B_max} R={cfg.R}, verify rows_mode={args.rows_mode}",
-                       "l2": ("inputs larger than L2 (no flush needed)" if build_bytes + verify_bytes > (126 << 20)
-                              else "inputs fit in L2 and are not flushed between steps (a launch-bound case, not the headline workload)"),
-                       "timing": "value: K steps between one pair of CUDA events; roofline/build: a second pass of K steps with events around every call (instrumented_ms_per_step)", "parallelism": f"replicas x{world}",
-                       "n_star_mean": round(float(n_star.float().mean()), 2), "n_star_max": int(n_star.max()), "n_star_hist": n_star_histogram(n_star),
-                       "accepted_mean": round(float(verdict.accepted_len.float().mean().item()), 2)},
-            "roofline": roofline, "build": build_info, "cuda_graph": graph, "fused_head": fused_head, "fused_draft_head": fused_draft, "sampled_verify": sampled, "fresh_seed_rounds": fresh, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "config": config_block(cfg, args.rows_mode, world),
+            "timing": "value: K steps between one pair of CUDA events; roofline blocks and kernel_ms: a second pass of K steps in "
+                      "which every kernel is launched by a call of its own with a CUDA event on either side",
+            "trees": tree_stats(w),
+            "roofline": roofline, "roofline_softmax_topk": roofline_topk, "kernel_ms": kernel_ms,
+            "other_workloads": others, "cuda_graph": graph, "fused_head": fused_head, "fused_draft_head": fused_draft,
+            "sampled_verify": sampled, "fresh_seed_rounds": fresh, "cost_fit": cost_fit, "e2e": e2e, "cpu_baseline": cpu_baseline,
             "gpu_launches": KERNELS_PER_STEP * K, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
     replicas.shutdown()
+
+
+def e2e_block(G, w, world, ke):
+    """The same step through the public API with HOST buffers: every step copies the draft and target logits from pinned
+    host memory to the device and reads the tree arrays and the verdict back, all inside the timed region."""
+    d, y, tree, verdict = w.d, w.y, w.tree, w.verdict
+    hx = torch.empty(d.logits.shape, dtype=d.logits.dtype, pin_memory=True)
+    hx.copy_(d.logits)
+    hy = torch.empty(y.shape, dtype=y.dtype, pin_memory=True)
+    hy.copy_(y)
+    tree_t = (tree.n_nodes, tree.token_ids, tree.parent_idx, tree.depth)
+    out_t = (verdict.accepted_len, verdict.accepted_nodes, verdict.next_bonus)
+    h_tree = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in tree_t]
+    h_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in out_t]
+    dx = torch.empty_like(d.logits)
+    dy = y                                   # the resident copy is overwritten with the same bits
+
+    def e2e_step():
+        dx.copy_(hx, non_blocking=True)
+        w.build(x=dx)
+        for h, t in zip(h_tree, tree_t):
+            h.copy_(t, non_blocking=True)
+        dy.copy_(hy, non_blocking=True)
+        w.verify(y=dy)
+        for h, t in zip(h_out, out_t):
+            h.copy_(t, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(ke):
+        e2e_step()
+    e1.record()
+    barrier()
+    ems = replicas.max_over_ranks(e0.elapsed_time(e1), w.dev)
+    h2d = hx.numel() * hx.element_size() + hy.numel() * hy.element_size()
+    d2h = sum(h.numel() * h.element_size() for h in h_tree + h_out)
+    same = bool(torch.equal(h_tree[0], w.n_star))
+    return {"value": round(replicas.whole_job_rounds_per_second(ke, world, ems), 3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "steps": ke, "ms_per_step": round(ems / ke, 3), "trees_match_resident_run": same}
 
 
 def n_star_histogram(n_star):
@@ -512,31 +625,57 @@ def fit_block(G, dev, iters=5):
 
 def oracle_sample(cfg, d, c, y, tree, dense, n_req, target_cpu_seconds=15.0):
     """Time the CPU oracle, as it stands, on the first n_req requests of the workload, repeated until about
-    target_cpu_seconds of CPU work (wall time x threads) have been spent."""
+    target_cpu_seconds of CPU work (wall time x threads) have been spent; then once more on one thread, on fewer
+    requests.  The oracle's trees are compared with the CUDA path's on the way (requests that differ, and how many of
+    those differ at a decision the oracle itself made with a margin below 1e-6)."""
     from oracle import cadd_oracle as O
     nb = min(n_req, cfg.batch)
     x = d.logits[:nb].cpu()
     yy = y[:nb].cpu()
-    kw = dict(l_eff=d.l_eff[:nb], bonus_token=d.bonus_token[:nb], ctx_len=d.ctx_len[:nb],
-              flags=O.FLAG_FIXED_BUDGET if cfg.fixed_budget else 0)
-    if c.kind == synth.COST_TABLE:
-        kw.update(cost_kind=O.COST_TABLE, cost_table=c.table, table_idx=c.table_idx[:nb], t_draft=c.t_draft[:nb])
-    else:
-        kw.update(cost_coef=c.coef[:nb])
+    mode = O.ROWS_DENSE if dense else O.ROWS_LIVE
+
+    def kwargs(n):
+        kw = dict(l_eff=d.l_eff[:n], bonus_token=d.bonus_token[:n], ctx_len=d.ctx_len[:n],
+                  flags=O.FLAG_FIXED_BUDGET if cfg.fixed_budget else 0)
+        if c.kind == synth.COST_TABLE:
+            kw.update(cost_kind=O.COST_TABLE, cost_table=c.table, table_idx=c.table_idx[:n], t_draft=c.t_draft[:n])
+        else:
+            kw.update(cost_coef=c.coef[:n])
+        return kw
+
     cores = O.num_threads()
     reps, dt = 0, 0.0
     t0 = time.perf_counter()
     while True:
-        ot = O.build_tree(x, cfg.K, cfg.B_max, cfg.R, **kw)
-        O.verify_tree(yy, cfg.L, ot.n_nodes, ot.token_ids, ot.parent_idx, O.ROWS_DENSE if dense else O.ROWS_LIVE)
+        ot = O.build_tree(x, cfg.K, cfg.B_max, cfg.R, **kwargs(nb))
+        O.verify_tree(yy, cfg.L, ot.n_nodes, ot.token_ids, ot.parent_idx, mode)
         reps += 1
         dt = time.perf_counter() - t0
         if dt * cores >= target_cpu_seconds or reps >= 50:
             break
-    same = bool(torch.equal(ot.n_nodes, tree.n_nodes[:nb].cpu()) and torch.equal(ot.token_ids, tree.token_ids[:nb].cpu()))
+    # the same code on one thread, on a smaller sample (about a third of the CPU work above)
+    n1 = max(1, min(nb, int(nb * (target_cpu_seconds / 3.0) / max(dt / reps * cores, 1e-9))))
+    O.set_num_threads(1)
+    t1 = time.perf_counter()
+    o1 = O.build_tree(x[:n1], cfg.K, cfg.B_max, cfg.R, **kwargs(n1))
+    O.verify_tree(yy[:n1], cfg.L, o1.n_nodes, o1.token_ids, o1.parent_idx, mode)
+    dt1 = time.perf_counter() - t1
+    O.set_num_threads(cores)
+    g_n, g_tok, g_par = tree.n_nodes[:nb].cpu(), tree.token_ids[:nb].cpu(), tree.parent_idx[:nb].cpu()
+    differ = [b for b in range(nb) if not (int(ot.n_nodes[b]) == int(g_n[b]) and torch.equal(ot.token_ids[b], g_tok[b])
+                                           and torch.equal(ot.parent_idx[b], g_par[b]))]
+    inside = 0
+    for b in differ:
+        k = min(int(ot.n_nodes[b]), int(g_n[b])) + 1
+        rows = [j for j in range(k) if int(ot.token_ids[b, j]) != int(g_tok[b, j]) or int(ot.parent_idx[b, j]) != int(g_par[b, j])]
+        margin = float(ot.pop_gap[b, rows[0]]) if rows else float(ot.stop_gap[b])
+        inside += margin < 1e-6
     return {"value": round(reps * (nb / cfg.batch) / dt, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{reps} x ({nb} of {cfg.batch} requests of the same workload, one build + verify each), "
-                      f"{dt:.2f} s wall on {cores} threads; value scaled to whole rounds", "trees_match_gpu": same}
+                      f"{dt:.2f} s wall on {cores} threads; value scaled to whole rounds",
+            "single_thread_value": round((n1 / cfg.batch) / dt1, 5),
+            "single_thread_sample": f"1 x ({n1} of {cfg.batch} requests), {dt1:.2f} s on 1 thread; value scaled to whole rounds",
+            "trees_match_gpu": not differ, "requests_differing_from_gpu": len(differ), "of_which_inside_oracle_margin_1e-6": int(inside)}
 
 
 def run_reference(args, rank, world):
@@ -577,12 +716,49 @@ def run_reference(args, rank, world):
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": Wm, "ms_per_step": round(dt / K * 1e3, 3), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"config {cfg.index} ({cfg.name}): batch={cfg.batch} L={cfg.L} V={cfg.V} {cfg.dtype} "
-                                   f"K={cfg.K} B_max={cfg.B_max} R={cfg.R}, verify rows_mode={args.rows_mode}"},
+            "config": config_block(cfg, args.rows_mode, world),
             "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def run_stub(args, rank, world):
+    """The launcher and the replica plumbing without a GPU: every rank joins a gloo group, 'steps' are short sleeps,
+    rank 0 prints a line with the contract's base keys.  Used by the CPU tests of `--gpus N`."""
+    replicas.init_replicas("gloo")
+    cpu = torch.device("cpu")
+    K, Wm = args.steps, max(args.warmup, 3)
+    for _ in range(Wm):
+        time.sleep(0.001)
+    replicas.barrier()
+    t0 = time.perf_counter()
+    for _ in range(K):
+        time.sleep(0.002 * (1 + rank))                   # the last rank is the slow one
+    ms = replicas.max_over_ranks((time.perf_counter() - t0) * 1e3, cpu)
+    replicas.barrier()
+    if rank == 0:
+        cfg = synth.CONFIGS[args.workload]
+        print(json.dumps({"metric": METRIC, "value": round(replicas.whole_job_rounds_per_second(K, world, ms), 3), "unit": UNIT,
+                          "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": round(ms / K, 5), "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "stub (no GPU work)",
+                          "config": config_block(cfg, args.rows_mode, world), "gpu_launches": 0}), flush=True)
+    replicas.shutdown()
+
+
+def launch_replicas(n):
+    """`python bench.py --gpus N` started by hand (no torchrun): start N copies of this command, one per GPU, with the
+    rendezvous variables torchrun would set; rank 0 prints the line.  Returns the worst exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    return max(p.wait() for p in procs)
 
 
 def main():
@@ -591,9 +767,13 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--workload", default="c5", choices=sorted(synth.CONFIGS),
+                    help="the timed configuration; default: the largest one that fits a GPU (config 5, 30.7 GB per round)")
+    ap.add_argument("--also", default="c2,c4_stress",
+                    help="comma-separated configurations measured the same way after the main one and reported under "
+                         "other_workloads ('none' to skip)")
     ap.add_argument("--rows-mode", default="dense", choices=["dense", "live"])
-    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-requests", type=int, default=32)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -605,17 +785,20 @@ def main():
     ap.add_argument("--no-fit", action="store_true", help="skip the offline cost-fitting measurement")
     ap.add_argument("--head-hidden", type=int, default=4096,
                     help="hidden size for the fused output-projection verification measurement (0 = skip)")
+    ap.add_argument("--stub", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(launch_replicas(args.gpus))           # not under torchrun: become the launcher
     rank = int(os.environ.get("RANK", 0))
-    world = int(os.environ.get("WORLD_SIZE", 1))
+    world = int(os.environ.get("WORLD_SIZE", args.gpus if args.impl == "reference" else 1))
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args, rank, world)
     else:
-        args.steps = 500 if args.steps is None else args.steps
-        args.warmup = 10 if args.warmup is None else args.warmup
-        run_ours(args, rank, world)
+        args.steps = 100 if args.steps is None else args.steps
+        args.warmup = 5 if args.warmup is None else args.warmup
+        (run_stub if args.stub else run_ours)(args, rank, world)
 
 
 if __name__ == "__main__":

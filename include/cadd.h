@@ -76,6 +76,18 @@ extern "C" {
 #define CADD_FLAG_EMIT_TOPK       2u   /* also write topk_token / topk_logprob */
 #define CADD_FLAG_FIXED_BUDGET    4u   /* ignore the stopping rule: expand to B_max (DDTree; the paper's constant-cost ablation, Table 2) */
 
+/* Measurement aids: a call with one of these enqueues only one of the two kernels of cadd_build_tree, so that each can
+   be timed alone with events on the caller's stream.  ONLY_TOPK runs the softmax/top-K pass (Eq. 1; Algorithm 1,
+   Require) and leaves its per-position records in the workspace, writing no output; ONLY_EXPAND runs Algorithm 1 and
+   the emission on the records an earlier call left in the SAME workspace for the same shape.  Both together:
+   CADD_ERR_DTYPE.  ONLY_TOPK followed by ONLY_EXPAND gives exactly the outputs of one plain call. */
+#define CADD_FLAG_ONLY_TOPK       8u
+#define CADD_FLAG_ONLY_EXPAND    16u
+/* The same for cadd_verify_tree (its `flags` field): only the per-node argmax, or only the walk on a node_argmax
+   array that an earlier call filled. */
+#define CADD_VERIFY_ONLY_ARGMAX   1u
+#define CADD_VERIFY_ONLY_WALK     2u
+
 #define CADD_ROWS_LIVE  0        /* verify reads target rows 0..n_nodes[b] only */
 #define CADD_ROWS_DENSE 1        /* verify takes the argmax of all R rows */
 
@@ -140,7 +152,7 @@ typedef struct cadd_build_args {
  */
 typedef struct cadd_verify_args {
     uint32_t struct_size;          /* = sizeof(cadd_verify_args) */
-    uint32_t flags;                /* reserved, 0 */
+    uint32_t flags;                /* 0, or one of CADD_VERIFY_ONLY_* */
     int32_t  batch, L, R;
     int32_t  logits_dtype;         /* CADD_DTYPE_* */
     int32_t  rows_mode;            /* CADD_ROWS_* */

@@ -74,6 +74,16 @@ int cadd_oracle_num_threads(void)
 #endif
 }
 
+/* Threads the batch loops below may use from now on (timing aid: the same code on one core). */
+void cadd_oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 /* Exact widening of one stored logit to double. */
 static double logit_at(const void *base, int dtype, int64_t idx)
 {

@@ -50,6 +50,11 @@ def num_threads() -> int:
     return int(lib().cadd_oracle_num_threads())
 
 
+def set_num_threads(n: int) -> None:
+    """Threads the oracle's per-request loops use from now on (for timing the same code on one core)."""
+    lib().cadd_oracle_set_num_threads(int(n))
+
+
 def _dt(t: torch.Tensor) -> int:
     if t.dtype == torch.bfloat16:
         return DT_BF16

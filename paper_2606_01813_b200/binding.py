@@ -24,6 +24,8 @@ STATUS_BAD_TABLE_IDX = 256
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 COST_QUADRATIC, COST_TABLE, COST_TABLE_INTERP = 0, 1, 2
 FLAG_EMIT_DENSE_MASK, FLAG_EMIT_TOPK, FLAG_FIXED_BUDGET = 1, 2, 4
+FLAG_ONLY_TOPK, FLAG_ONLY_EXPAND = 8, 16          # measurement aids: one of the two build kernels alone
+VERIFY_ONLY_ARGMAX, VERIFY_ONLY_WALK = 1, 2       # the same for cadd_verify_tree
 ROWS_LIVE, ROWS_DENSE = 0, 1
 
 EXPORTS = ("cadd_version", "cadd_status_string", "cadd_build_workspace_bytes", "cadd_verify_workspace_bytes",
@@ -164,9 +166,10 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
     return None if t is None else t.data_ptr()
 
 
-def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
-    s = torch.cuda.current_stream() if stream is None else stream
-    return s.cuda_stream
+def _stream_of(stream: Optional[torch.cuda.Stream], dev) -> torch.cuda.Stream:
+    """The stream a call is enqueued on: the given one, else the current stream OF THE TENSORS' DEVICE (which need
+    not be the current device).  The same object serves the C call and record_stream."""
+    return torch.cuda.current_stream(dev) if stream is None else stream
 
 
 def _dev(t: Optional[torch.Tensor], device, dtype) -> Optional[torch.Tensor]:
@@ -285,20 +288,21 @@ def cadd_build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[
         nbytes = cadd_build_workspace_bytes(batch, L, V, K, B_max, R, x.dtype)
         workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=dev)
     a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    st = _stream_of(stream, dev)
     with torch.cuda.device(dev):
-        rc = lib().cadd_build_tree(C.byref(a), _stream_ptr(stream))
+        rc = lib().cadd_build_tree(C.byref(a), st.cuda_stream)
     if rc != OK:
         raise CaddError(rc)
     # the call is asynchronous: keep temporaries alive until the stream has consumed them
     for t in keep + [workspace]:
         if t is not None:
-            t.record_stream(torch.cuda.current_stream() if stream is None else stream)
+            t.record_stream(st)
     return out
 
 
 def cadd_verify_tree(target_logits: torch.Tensor, L: int, n_nodes: torch.Tensor, token_ids: torch.Tensor,
                      parent_idx: torch.Tensor, rows_mode: int = ROWS_LIVE, *, out: Optional[Verdict] = None,
-                     stream: Optional[torch.cuda.Stream] = None) -> Verdict:
+                     flags: int = 0, stream: Optional[torch.cuda.Stream] = None) -> Verdict:
     """Greedy tree verification (Sections 3.1, 3.3): per-node argmax of target_logits [batch, R, V]
     and the walk along the longest accepted path, on the current CUDA stream."""
     y = target_logits
@@ -313,6 +317,7 @@ def cadd_verify_tree(target_logits: torch.Tensor, L: int, n_nodes: torch.Tensor,
             raise ValueError("tree arrays must be contiguous int32 CUDA tensors")
     a = VerifyArgs()
     a.struct_size = C.sizeof(VerifyArgs)
+    a.flags = flags
     a.batch, a.L, a.R, a.V = batch, L, R, V
     a.logits_dtype = _dtype_code(y)
     a.rows_mode = rows_mode
@@ -325,8 +330,9 @@ def cadd_verify_tree(target_logits: torch.Tensor, L: int, n_nodes: torch.Tensor,
                       next_bonus=i32(batch), status=i32(batch))
     a.node_argmax, a.accepted_len, a.accepted_nodes = _ptr(out.node_argmax), _ptr(out.accepted_len), _ptr(out.accepted_nodes)
     a.next_bonus, a.status = _ptr(out.next_bonus), _ptr(out.status)
+    st = _stream_of(stream, dev)
     with torch.cuda.device(dev):
-        rc = lib().cadd_verify_tree(C.byref(a), _stream_ptr(stream))
+        rc = lib().cadd_verify_tree(C.byref(a), st.cuda_stream)
     if rc != OK:
         raise CaddError(rc)
     return out
@@ -384,11 +390,12 @@ def cadd_verify_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tenso
     if workspace is None:
         workspace = torch.empty(cadd_head_workspace_bytes(batch, R, hidden, V, L, rows_mode), dtype=torch.uint8, device=dev)
     a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    st = _stream_of(stream, dev)
     with torch.cuda.device(dev):
-        rc = lib().cadd_verify_tree_fused_head(C.byref(a), _stream_ptr(stream))
+        rc = lib().cadd_verify_tree_fused_head(C.byref(a), st.cuda_stream)
     if rc != OK:
         raise CaddError(rc)
-    workspace.record_stream(torch.cuda.current_stream() if stream is None else stream)
+    workspace.record_stream(st)
     return out
 
 
@@ -445,13 +452,14 @@ def cadd_build_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor
     if workspace is None:
         workspace = torch.empty(cadd_build_head_workspace_bytes(batch, L, V, hidden, K, B_max, R), dtype=torch.uint8, device=dev)
     h.build.workspace, h.build.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    st = _stream_of(stream, dev)
     with torch.cuda.device(dev):
-        rc = lib().cadd_build_tree_fused_head(C.byref(h), _stream_ptr(stream))
+        rc = lib().cadd_build_tree_fused_head(C.byref(h), st.cuda_stream)
     if rc != OK:
         raise CaddError(rc)
     for t in keep + [workspace]:
         if t is not None:
-            t.record_stream(torch.cuda.current_stream() if stream is None else stream)
+            t.record_stream(st)
     return out
 
 
@@ -490,8 +498,9 @@ def cadd_verify_tree_sampled(target_logits: torch.Tensor, uniforms: torch.Tensor
                       next_bonus=i32(batch), status=i32(batch))
     a.node_token, a.accepted_len, a.accepted_nodes = _ptr(out.node_argmax), _ptr(out.accepted_len), _ptr(out.accepted_nodes)
     a.next_bonus, a.status = _ptr(out.next_bonus), _ptr(out.status)
+    st = _stream_of(stream, dev)
     with torch.cuda.device(dev):
-        rc = lib().cadd_verify_tree_sampled(C.byref(a), _stream_ptr(stream))
+        rc = lib().cadd_verify_tree_sampled(C.byref(a), st.cuda_stream)
     if rc != OK:
         raise CaddError(rc)
     return out
@@ -512,7 +521,7 @@ def cadd_fit_cost_tables(y: torch.Tensor, *, stream: Optional[torch.cuda.Stream]
     st = torch.empty(y.shape[0], dtype=torch.int32, device=y.device)
     a.y, a.fit, a.n_breaks, a.status = y.data_ptr(), fit.data_ptr(), nb.data_ptr(), st.data_ptr()
     with torch.cuda.device(y.device):
-        rc = lib().cadd_fit_cost_tables(C.byref(a), _stream_ptr(stream))
+        rc = lib().cadd_fit_cost_tables(C.byref(a), _stream_of(stream, y.device).cuda_stream)
     if rc != OK:
         raise CaddError(rc)
     return fit, nb, st
@@ -565,11 +574,12 @@ def cadd_build_tree_static_scratch(draft_logits: torch.Tensor, K: int, B_max: in
     a.position_ids, a.node_logprob, a.phi, a.theta = _ptr(out.position_ids), _ptr(out.node_logprob), _ptr(out.phi), _ptr(out.theta)
     a.mask_bits, a.mask_dense = _ptr(out.mask_bits), _ptr(out.mask_dense)
     a.topk_token, a.topk_logprob, a.status = _ptr(out.topk_token), _ptr(out.topk_logprob), _ptr(out.status)
+    st = _stream_of(stream, dev)
     with torch.cuda.device(dev):
-        rc = lib().cadd_build_tree_static_scratch(C.byref(a), _stream_ptr(stream))
+        rc = lib().cadd_build_tree_static_scratch(C.byref(a), st.cuda_stream)
     if rc != OK:
         raise CaddError(rc)
     for t in keep:
         if t is not None:
-            t.record_stream(torch.cuda.current_stream() if stream is None else stream)
+            t.record_stream(st)
     return out

@@ -42,6 +42,7 @@ static int check_build_shape(const cadd_build_args* a) {
     if ((int64_t)a->batch * a->L * 8 >= ((int64_t)1 << 31) || (int64_t)a->batch * a->R >= ((int64_t)1 << 31)) return CADD_ERR_SHAPE;
     if (a->logits_dtype != CADD_DTYPE_BF16 && a->logits_dtype != CADD_DTYPE_FP32) return CADD_ERR_DTYPE;
     if (a->cost_kind != CADD_COST_QUADRATIC && a->cost_kind != CADD_COST_TABLE && a->cost_kind != CADD_COST_TABLE_INTERP) return CADD_ERR_DTYPE;
+    if ((a->flags & CADD_FLAG_ONLY_TOPK) && (a->flags & CADD_FLAG_ONLY_EXPAND)) return CADD_ERR_DTYPE;
     return CADD_OK;
 }
 
@@ -206,11 +207,13 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
     tp.L = a->L; tp.S = pl.S; tp.KP = pl.KP; tp.l_eff = a->l_eff; tp.partials = (unsigned char*)a->workspace;
     const unsigned items = (unsigned)((int64_t)a->batch * a->L * pl.S);
     const bool overlap = (int64_t)a->batch * a->L * a->V * (int64_t)es >= kOverlapMinBytes;
-    const cudaError_t le = a->logits_dtype == CADD_DTYPE_BF16
-        ? launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, dim3(items), dim3(kThreads), topk_smem_bytes(), st, tp)
-        : launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, dim3(items), dim3(kThreads), topk_smem_bytes(), st, tp);
-    if (le != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
-
+    if (!(a->flags & CADD_FLAG_ONLY_EXPAND)) {
+        const cudaError_t le = a->logits_dtype == CADD_DTYPE_BF16
+            ? launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, dim3(items), dim3(kThreads), topk_smem_bytes(), st, tp)
+            : launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, dim3(items), dim3(kThreads), topk_smem_bytes(), st, tp);
+        if (le != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+    }
+    if (a->flags & CADD_FLAG_ONLY_TOPK) return CADD_OK;
     return launch_expand(a, pl.KP, pl.S, (const unsigned char*)a->workspace, st, overlap);
 }
 
@@ -222,6 +225,7 @@ static int check_verify_shape(const cadd_verify_args* a) {
         return CADD_ERR_SHAPE;
     if (a->logits_dtype != CADD_DTYPE_BF16 && a->logits_dtype != CADD_DTYPE_FP32) return CADD_ERR_DTYPE;
     if (a->rows_mode != CADD_ROWS_LIVE && a->rows_mode != CADD_ROWS_DENSE) return CADD_ERR_DTYPE;
+    if ((a->flags & CADD_VERIFY_ONLY_ARGMAX) && (a->flags & CADD_VERIFY_ONLY_WALK)) return CADD_ERR_DTYPE;
     return CADD_OK;
 }
 
@@ -262,10 +266,13 @@ int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream) {
         cudaGetLastError();
         return CADD_ERR_LAUNCH;
     }
-    const cudaError_t le = a->logits_dtype == CADD_DTYPE_BF16
-        ? launch_dependent(overlap, row_argmax_kernel<CADD_DTYPE_BF16>, dim3(rows), dim3(kThreads), argmax_smem_bytes(), st, ap)
-        : launch_dependent(overlap, row_argmax_kernel<CADD_DTYPE_FP32>, dim3(rows), dim3(kThreads), argmax_smem_bytes(), st, ap);
-    if (le != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+    if (!(a->flags & CADD_VERIFY_ONLY_WALK)) {
+        const cudaError_t le = a->logits_dtype == CADD_DTYPE_BF16
+            ? launch_dependent(overlap, row_argmax_kernel<CADD_DTYPE_BF16>, dim3(rows), dim3(kThreads), argmax_smem_bytes(), st, ap)
+            : launch_dependent(overlap, row_argmax_kernel<CADD_DTYPE_FP32>, dim3(rows), dim3(kThreads), argmax_smem_bytes(), st, ap);
+        if (le != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+    }
+    if (a->flags & CADD_VERIFY_ONLY_ARGMAX) return CADD_OK;
 
     WalkParams wp;
     wp.batch = a->batch; wp.L = a->L; wp.R = a->R; wp.n_nodes = a->n_nodes; wp.token_ids = a->token_ids;

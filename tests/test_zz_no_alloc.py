@@ -71,3 +71,29 @@ def test_static_scratch_matches_regular_entry_point_twice():
     torch.cuda.synchronize()
     for f in INT_FIELDS:
         assert torch.equal(getattr(results[0][1], f), getattr(again, f)), f
+
+
+@pytest.mark.gpu
+def test_static_scratch_calls_allocate_nothing():
+    """With every input already on the device and the outputs preallocated, calls of the scratch-free entry point
+    must leave the device's memory exactly as it was: neither torch's allocator nor the driver hands anything out
+    (the one-time address look-up happened in the warm-up call)."""
+    cfg = synth.scaled(synth.CONFIGS["c2"], batch=2)
+    d = synth.make_draft_inputs(cfg, 13)
+    c = synth.make_cost_inputs(cfg, 13)
+    dev = torch.device("cuda")
+    x = d.logits.to(dev)
+    kw = dict(l_eff=d.l_eff.to(dev, torch.int32), bonus_token=d.bonus_token.to(dev, torch.int32),
+              ctx_len=d.ctx_len.to(dev, torch.int32), cost_coef=c.coef.to(dev, torch.float64), flags=G.FLAG_EMIT_TOPK)
+    out = G.cadd_build_tree_static_scratch(x, cfg.K, cfg.B_max, cfg.R, **kw)          # warm-up: allocates `out`
+    torch.cuda.synchronize()
+    first = out.token_ids.clone()
+    allocated, reserved = torch.cuda.memory_allocated(dev), torch.cuda.memory_reserved(dev)
+    free_before, _ = torch.cuda.mem_get_info(dev)
+    for _ in range(5):
+        G.cadd_build_tree_static_scratch(x, cfg.K, cfg.B_max, cfg.R, out=out, **kw)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info(dev)
+    assert torch.cuda.memory_allocated(dev) == allocated and torch.cuda.memory_reserved(dev) == reserved
+    assert free_after == free_before
+    assert torch.equal(out.token_ids, first)
