@@ -87,6 +87,12 @@ extern "C" {
    array that an earlier call filled. */
 #define CADD_VERIFY_ONLY_ARGMAX   1u
 #define CADD_VERIFY_ONLY_WALK     2u
+/* Test hook, accepted in the `flags` of cadd_build_tree, cadd_verify_tree and cadd_verify_tree_sampled: the streaming
+   kernel never issues the asynchronous copy of the second tile (16 KB) of each row it reads (the first, if the row has
+   only one), and its wait for that one tile gives up after a few tries.  Nothing hangs and nothing faults: the call
+   exercises the library's bounded-wait exit (copies already in flight are waited for, then the CTA leaves) and every
+   request reports CADD_STATUS_INTERNAL_TIMEOUT with the empty tree (build) or accepted_len 0 (verify).  For tests only. */
+#define CADD_FLAG_TEST_DROP_TILE  0x80000000u
 
 #define CADD_ROWS_LIVE  0        /* verify reads target rows 0..n_nodes[b] only */
 #define CADD_ROWS_DENSE 1        /* verify takes the argmax of all R rows */

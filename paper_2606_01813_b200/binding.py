@@ -26,6 +26,7 @@ COST_QUADRATIC, COST_TABLE, COST_TABLE_INTERP = 0, 1, 2
 FLAG_EMIT_DENSE_MASK, FLAG_EMIT_TOPK, FLAG_FIXED_BUDGET = 1, 2, 4
 FLAG_ONLY_TOPK, FLAG_ONLY_EXPAND = 8, 16          # measurement aids: one of the two build kernels alone
 VERIFY_ONLY_ARGMAX, VERIFY_ONLY_WALK = 1, 2       # the same for cadd_verify_tree
+FLAG_TEST_DROP_TILE = 0x80000000                  # test hook: one tile per row is never copied, its wait gives up
 ROWS_LIVE, ROWS_DENSE = 0, 1
 
 EXPORTS = ("cadd_version", "cadd_status_string", "cadd_build_workspace_bytes", "cadd_verify_workspace_bytes",
@@ -465,7 +466,7 @@ def cadd_build_tree_fused_head(hidden_states: torch.Tensor, weight: torch.Tensor
 
 def cadd_verify_tree_sampled(target_logits: torch.Tensor, uniforms: torch.Tensor, L: int, n_nodes: torch.Tensor,
                              token_ids: torch.Tensor, parent_idx: torch.Tensor, rows_mode: int = ROWS_LIVE, *,
-                             temperature: float = 1.0, out: Optional[Verdict] = None,
+                             temperature: float = 1.0, out: Optional[Verdict] = None, flags: int = 0,
                              stream: Optional[torch.cuda.Stream] = None) -> Verdict:
     """Tree verification under sampling: one token is drawn per node from softmax(target_logits / temperature) by the
     inverse CDF at uniforms[b, j]; the walk follows the child that carries the drawn token.  Verdict.node_argmax holds
@@ -484,6 +485,7 @@ def cadd_verify_tree_sampled(target_logits: torch.Tensor, uniforms: torch.Tensor
             raise ValueError("tree arrays must be contiguous int32 CUDA tensors")
     a = SampleArgs()
     a.struct_size = C.sizeof(SampleArgs)
+    a.flags = flags
     a.batch, a.L, a.R, a.V = batch, L, R, V
     a.logits_dtype = _dtype_code(y)
     a.rows_mode = rows_mode

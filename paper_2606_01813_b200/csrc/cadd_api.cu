@@ -205,6 +205,7 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
     TopkParams tp;
     tp.logits = a->draft_logits; tp.V = a->V; tp.stride_b = a->stride_b; tp.stride_l = a->stride_l;
     tp.L = a->L; tp.S = pl.S; tp.KP = pl.KP; tp.l_eff = a->l_eff; tp.partials = (unsigned char*)a->workspace;
+    tp.fault_tile = (a->flags & CADD_FLAG_TEST_DROP_TILE) ? 1 : -1;
     const unsigned items = (unsigned)((int64_t)a->batch * a->L * pl.S);
     const bool overlap = (int64_t)a->batch * a->L * a->V * (int64_t)es >= kOverlapMinBytes;
     if (!(a->flags & CADD_FLAG_ONLY_EXPAND)) {
@@ -254,6 +255,7 @@ int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream) {
     ArgmaxParams ap;
     ap.logits = a->target_logits; ap.V = a->V; ap.stride_b = a->stride_b; ap.stride_row = a->stride_row;
     ap.R = a->R; ap.rows_mode = a->rows_mode; ap.n_nodes = a->n_nodes; ap.node_argmax = a->node_argmax;
+    ap.fault_tile = (a->flags & CADD_FLAG_TEST_DROP_TILE) ? 1 : -1;
     // LIVE with a small node cap: most rows are padding on typical trees, so eight rows share a CTA (interleaved, so
     // that a request's live rows, which come first, still spread over its CTAs) and few CTAs are launched only to exit.
     // Large caps and DENSE keep one row per CTA: every row is work there and short CTAs keep the last wave short.
@@ -582,6 +584,7 @@ int cadd_verify_tree_sampled(const cadd_sample_args* a, void* cuda_stream) {
     sp.logits = a->target_logits; sp.V = a->V; sp.stride_b = a->stride_b; sp.stride_row = a->stride_row;
     sp.R = a->R; sp.rows_mode = a->rows_mode; sp.c = (float)(1.4426950408889634 / a->temperature);
     sp.n_nodes = a->n_nodes; sp.uniforms = a->uniforms; sp.node_token = a->node_token;
+    sp.fault_tile = (a->flags & CADD_FLAG_TEST_DROP_TILE) ? 1 : -1;
     // LIVE with a small node cap: eight rows of a request share a CTA (as in cadd_verify_tree)
     const bool shared_rows = a->rows_mode == CADD_ROWS_LIVE && a->R <= kLiveSharedRowsMaxR;
     sp.ctas_per_request = shared_rows ? (a->R + 7) / 8 : a->R;

@@ -191,10 +191,10 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
             lz[i] = logZ;
             int st = 0;
             if (fl & kPartNonfinite) st |= CADD_STATUS_NONFINITE_INPUT;
-            if (ke < K) st |= CADD_STATUS_FEWER_THAN_K_FINITE;
+            if (fl & kPartTimeout) { st |= CADD_STATUS_INTERNAL_TIMEOUT; s_pinf = 1; }   // nothing is known of the row: empty tree
+            else if (ke < K) st |= CADD_STATUS_FEWER_THAN_K_FINITE;
             if (st) atomicOr(&s_status, st);
             if (fl & kPartPosInf) s_pinf = 1;
-            if (fl & kPartTimeout) { atomicOr(&s_status, CADD_STATUS_INTERNAL_TIMEOUT); s_pinf = 1; }   // empty tree
         }
         if (emit) for (int k = lane; k < K; k += 32) {
             if (out_tok) out_tok[k] = k < ke ? tok_list[i * K + k] : -1;

@@ -33,11 +33,13 @@ struct SampleParams {
     const int32_t* n_nodes;    // [batch]
     const double* uniforms;    // [batch, R]
     int32_t* node_token;       // [batch, R]
+    int fault_tile;            // test hook: this tile of every row is never copied (-1: none)
 };
 
 struct SampleShared {
     alignas(8) uint64_t full[kStages];
     unsigned released[kStages];
+    unsigned last_seq[kStages];           // last tile issued into the stage (see ring_drain)
     unsigned timeout;
     int n_runs;
     float run_ref[kMaxRuns];              // per run: reference exponent = fp32(max * log2(e) / T) over its finite elements; -Inf if none
@@ -178,10 +180,13 @@ __device__ __forceinline__ bool sample_one_row(SampleShared& sh, const SamplePar
 
     const unsigned base = issued;                        // stage of tile t of this row: (base + t) % kStages
     issued += (unsigned)n_tiles;
+    const int fault_tile = p.fault_tile < 0 ? -1 : min(p.fault_tile, n_tiles - 1);
     auto issue_tile = [&](int t) {
+        if (t == fault_tile) return;                     // test hook: this copy is never made
         const int c0 = t * kTileChunks;
         const unsigned bytes = (unsigned)min(kTileChunks, nc - c0) * 16u;
         const unsigned st = (base + (unsigned)t) % kStages;
+        *(volatile unsigned*)&sh.last_seq[st] = base + (unsigned)t;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive_expect_tx(&sh.full[st], bytes);
         bulk_load(&sh.ring[st][0], body + c0, bytes, &sh.full[st]);
@@ -207,7 +212,7 @@ __device__ __forceinline__ bool sample_one_row(SampleShared& sh, const SamplePar
 
     const uint64_t c2 = pack2(p.c, p.c);
     for (int t = 0; t < n_tiles; ++t) {
-        if (!__all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase))) { sh.timeout = 1; break; }
+        if (!__all_sync(kFullMask, mbar_wait_limited(&sh.full[st], phase, tile_wait_limit(t, fault_tile)))) { sh.timeout = 1; break; }
         // this warp's run of the tile: chunks [c0, c0 + kRunChunks), four per lane
         const int c0 = t * kTileChunks + warp * kRunChunks;
         const int nvw = max(0, min(kRunChunks, nc - c0));
@@ -290,6 +295,7 @@ __device__ __forceinline__ bool sample_one_row(SampleShared& sh, const SamplePar
 
     // ---- combine the runs (warp 0): total, the run that holds the crossing, the token inside it ----
     const bool ok = sh.timeout == 0;
+    if (!ok && tid == 32) ring_drain(sh.full, sh.last_seq);        // every warp has left the tile loop: let the copies in flight land
     if (warp == 0) {
         int32_t ans = -2;                                          // a wait ran out: no draw
         if (ok) ans = sample_combine<DT>(sh, n_runs, p.c, p.uniforms[(int64_t)b * p.R + j], row, sp, body, p.V);
@@ -317,7 +323,7 @@ __global__ void __launch_bounds__(kThreads, 4) row_sample_kernel(SampleParams p)
         }
     }
     if (tid == 0) {
-        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
+        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; sh.last_seq[q] = kNoTile; }
         sh.timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -345,7 +351,7 @@ __global__ void __launch_bounds__(kThreads, 4) row_sample_shared_rows_kernel(Sam
         return;
     }
     if (tid == 0) {
-        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
+        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; sh.last_seq[q] = kNoTile; }
         sh.timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }

@@ -61,6 +61,7 @@ struct TopkParams {
     int L, S, KP;
     const int32_t* l_eff;
     unsigned char* partials;     // [batch*L*S] records of seg_partial_stride(KP) bytes
+    int fault_tile;              // test hook: this tile of every segment is never copied (-1: none)
 };
 
 constexpr float kLog2eHi = 1.44269502162933349609375f;     // float(log2 e)
@@ -115,6 +116,7 @@ struct TopkShared {
     unsigned red_u[kThreads / 32];
     alignas(8) uint64_t full[kStages];                 // mbarriers: tile landed
     unsigned released[kStages];                        // warps done with the stage's current tile
+    unsigned last_seq[kStages];                        // last tile issued into the stage (see ring_drain)
     alignas(128) uint4 ring[kStages][kTileChunks];     // tiles of logits
 };
 
@@ -449,7 +451,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
 
     for (int q = tid; q < kCandCap; q += kThreads) sh.keys[q] = 0ull;
     if (tid == 0) {
-        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
+        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; sh.last_seq[q] = kNoTile; }
         sh.timeout = 0; sh.overflow = 0; sh.pushed = 0; sh.nwin = 0;
         sh.count = 0; sh.thr_key = 0; sh.thr_val = -INFINITY;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -457,10 +459,13 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
     __syncthreads();
     // one thread issues tile t into stage t % kStages: thread 0 for the first kStages tiles, afterwards
     // lane 0 of whichever warp is the last to finish with the tile that occupied the stage
+    const int fault_tile = p.fault_tile < 0 ? -1 : min(p.fault_tile, n_tiles - 1);
     auto issue_tile = [&](int t) {
+        if (t == fault_tile) return;                                   // test hook: this copy is never made
         const int c0 = c_begin + t * kTileChunks;
         const unsigned bytes = (unsigned)min(kTileChunks, c_end - c0) * 16u;
         const unsigned st = (unsigned)t % kStages;
+        *(volatile unsigned*)&sh.last_seq[st] = (unsigned)t;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic reads of the stage are done
         mbar_arrive_expect_tx(&sh.full[st], bytes);
         bulk_load(&sh.ring[st][0], body + c0, bytes, &sh.full[st]);
@@ -495,7 +500,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
         float* seeds = (float*)sh.hist;
         float gm = -INFINITY;
         if (n_tiles > 0) {
-            landed = mbar_wait_bounded(&sh.full[0], 0);
+            landed = mbar_wait_limited(&sh.full[0], 0, tile_wait_limit(0, fault_tile));
             if (landed) {
 #pragma unroll
                 for (int u = 0; u < kTopkUnroll; ++u)
@@ -545,7 +550,7 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
         const bool timed_out = sh.timeout != 0;
         unsigned st = 0, phase = 0;
         for (int t = 0; t < n_tiles && !timed_out; ++t, st = (st + 1 == kStages ? 0u : st + 1), phase ^= (st == 0 ? 1u : 0u)) {
-            const bool here = __all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase));
+            const bool here = __all_sync(kFullMask, mbar_wait_limited(&sh.full[st], phase, tile_wait_limit(t, fault_tile)));
             if (!here) { sh.timeout = 1; break; }
             const uint64_t thrk = *(volatile uint64_t*)&sh.thr_key;          // only ever rises; stale is safe
             const float thrv = thrk ? key_value(thrk) : -INFINITY;
@@ -645,7 +650,10 @@ __global__ void __launch_bounds__(kThreads, 4) softmax_topk_partial_kernel(TopkP
         }
         __syncthreads();
         // keep the KP best of the buffer, fold the rest into the sums (CTA-wide), sort the survivors into win[]
-        if (tid == 0) sh.count = min(sh.pushed, (unsigned)kCandCap);
+        if (tid == 0) {
+            sh.count = min(sh.pushed, (unsigned)kCandCap);
+            if (sh.timeout) ring_drain(sh.full, sh.last_seq);          // a wait ran out: let the copies still in flight land
+        }
         __syncthreads();
         if (!sh.overflow && !sh.timeout) {
             s = refresh_candidates(sh, s, KP);

@@ -38,12 +38,32 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity, un
     return ok != 0;
 }
 // Wait for a phase with an iteration limit; false = gave up (the caller flags an error and leaves).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity) {
-    for (int it = 0; it < kSpinLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t* bar, unsigned parity, int limit) {
+    for (int it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         __nanosleep(200);          // a waiting warp must not take issue slots from the warps that still work
     }
     return false;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity) { return mbar_wait_limited(bar, parity, kSpinLimit); }
+
+// Test hook of the streaming kernels (the TEST_DROP_TILE flags of the C ABI): the copy of one tile per row is never
+// issued, and the wait for that tile alone gives up after kTestSpinLimit tries, so that the time-out path runs with
+// nothing in flight for the barrier that is given up on.  Every other wait keeps the full limit.
+constexpr int kTestSpinLimit = 4;
+__device__ __forceinline__ int tile_wait_limit(int t, int fault_tile) { return t == fault_tile ? kTestSpinLimit : kSpinLimit; }
+
+// Ring bookkeeping for the exit path after a wait ran out: last_seq[s] is the sequence number g of the last tile issued
+// into stage s (tile g goes to stage g % kStages and completes phase (g / kStages) & 1 of that stage's barrier), kNoTile
+// if none.  ring_drain, called by ONE thread once every warp of the CTA has left its tile loop, waits (with the full
+// limit per stage) until every issued copy has landed, so that the CTA never exits with a bulk copy still writing into
+// its shared memory.  A tile that has landed already, consumed or not, costs one successful try.
+constexpr unsigned kNoTile = 0xffffffffu;
+__device__ __forceinline__ void ring_drain(uint64_t* full, const volatile unsigned* last_seq) {
+    for (int s = 0; s < kStages; ++s) {
+        const unsigned g = last_seq[s];
+        if (g != kNoTile) mbar_wait_bounded(&full[s], (g / kStages) & 1u);
+    }
 }
 // 1-D bulk copy global -> this CTA's shared memory; both addresses 16-byte aligned, bytes % 16 == 0.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {

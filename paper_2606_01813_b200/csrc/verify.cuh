@@ -13,12 +13,14 @@ struct ArgmaxParams {
     int ctas_per_request;      // CTA g of a request reads rows g, g + ctas_per_request, ... (= R: one row per CTA)
     const int32_t* n_nodes;    // [batch]
     int32_t* node_argmax;      // [batch, R]
+    int fault_tile;            // test hook: this tile of every row is never copied (-1: none)
 };
 
 // Shared memory of row_argmax_kernel.
 struct ArgmaxRing {
     alignas(8) uint64_t full[kStages];                 // mbarriers: tile landed
     unsigned released[kStages];                        // warps done with the stage's current tile
+    unsigned last_seq[kStages];                        // last tile issued into the stage (see ring_drain)
     unsigned timeout;
     float red_m[kThreads / 32];
     int64_t red_p[kThreads / 32];
@@ -56,7 +58,7 @@ __global__ void __launch_bounds__(kThreads, 4) row_argmax_kernel(ArgmaxParams p)
         }
     }
     if (tid == 0) {
-        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; }
+        for (int q = 0; q < kStages; ++q) { mbar_init(&sh.full[q], 1); sh.released[q] = 0; sh.last_seq[q] = kNoTile; }
         sh.timeout = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -75,10 +77,13 @@ __global__ void __launch_bounds__(kThreads, 4) row_argmax_kernel(ArgmaxParams p)
         const int nc = sp.n_chunks;
         const int n_tiles = (nc + kTileChunks - 1) / kTileChunks;
         const unsigned base = issued;                    // stage of tile t of this row: (base + t) % kStages
+        const int fault_tile = p.fault_tile < 0 ? -1 : min(p.fault_tile, n_tiles - 1);
         auto issue_tile = [&](int t) {
+            if (t == fault_tile) return;                 // test hook: this copy is never made
             const int c0 = t * kTileChunks;
             const unsigned bytes = (unsigned)min(kTileChunks, nc - c0) * 16u;
             const unsigned stg = (base + (unsigned)t) % kStages;
+            *(volatile unsigned*)&sh.last_seq[stg] = base + (unsigned)t;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive_expect_tx(&sh.full[stg], bytes);
             bulk_load(&sh.ring[stg][0], body + c0, bytes, &sh.full[stg]);
@@ -94,7 +99,7 @@ __global__ void __launch_bounds__(kThreads, 4) row_argmax_kernel(ArgmaxParams p)
             if (x > rm) { rm = x; rpos = tid; }
         }
         for (int t = 0; t < n_tiles; ++t) {
-            if (!__all_sync(kFullMask, mbar_wait_bounded(&sh.full[st], phase))) { sh.timeout = 1; break; }
+            if (!__all_sync(kFullMask, mbar_wait_limited(&sh.full[st], phase, tile_wait_limit(t, fault_tile)))) { sh.timeout = 1; break; }
             const uint4* tile = &sh.ring[st][tid];
             const int cbase = t * kTileChunks + tid;
 #pragma unroll
@@ -152,6 +157,7 @@ __global__ void __launch_bounds__(kThreads, 4) row_argmax_kernel(ArgmaxParams p)
         if (timed_out) {                                      // the ring's state is unknown: give up on this CTA's other rows too
             for (int jj = j + p.ctas_per_request + tid * p.ctas_per_request; jj < p.R; jj += kThreads * p.ctas_per_request)
                 p.node_argmax[(int64_t)b * p.R + jj] = jj > n ? -1 : -2;
+            if (tid == 0) ring_drain(sh.full, sh.last_seq);   // every warp is past the barrier above: let the copies in flight land
             return;
         }
         __syncthreads();                                      // red_m / red_p and the ring are free for the next row
