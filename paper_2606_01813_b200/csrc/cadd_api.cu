@@ -50,14 +50,22 @@ static int check_build_shape(const cadd_build_args* a) {
 // grid must fill the resident-CTA slots of the machine evenly: take the smallest cut whose last wave
 // is at least 85 % full (else the fullest), never making a segment shorter than 4 iterations.
 constexpr int kMaxSegments = 8;
+// Rows are cut only while the grid stays within kSlotsCap CTAs (more than any device has resident slots for), so that the
+// workspace -- sized for the largest cut whatever the device -- stays small for large batches.
+constexpr int64_t kSlotsCap = 1024;
+static int max_segments(int64_t rows) {
+    const int64_t s = (kSlotsCap + rows - 1) / rows;
+    return (int)(s < 1 ? 1 : (s > kMaxSegments ? kMaxSegments : s));
+}
 static BuildPlan plan_build(const cadd_build_args* a, int slots) {
     BuildPlan pl;
     pl.KP = a->K > kPreciseMin ? a->K : kPreciseMin;
     const int epc = a->logits_dtype == CADD_DTYPE_BF16 ? 8 : 4;
     const int64_t rows = (int64_t)a->batch * a->L;
     const int64_t chunks = a->V / epc;
-    int64_t cap = chunks / (4 * kTopkUnroll * kThreads);
-    if (cap > kMaxSegments) cap = kMaxSegments;
+    int64_t cap = chunks / (4 * kTkTileChunks);
+    if (cap > max_segments(rows)) cap = max_segments(rows);
+    if (cap > 512 / seg_key_cap(pl.KP)) cap = 512 / seg_key_cap(pl.KP);   // the expansion kernel holds every key of a row's records per warp
     if (cap < 1) cap = 1;
     int best = 1;
     double best_eff = 0.0;
@@ -69,8 +77,8 @@ static BuildPlan plan_build(const cadd_build_args* a, int slots) {
         if (eff >= 0.85) { best = S; break; }
     }
     pl.S = best;
-    pl.partial_bytes = (size_t)rows * pl.S * seg_partial_stride(pl.KP);
-    pl.lay = expand_layout(a->L, a->K, pl.KP, pl.S, a->B_max);
+    pl.partial_bytes = (size_t)rows * pl.S * seg_record_stride(pl.KP);
+    pl.lay = expand_layout(a->L, a->K, seg_key_cap(pl.KP), pl.S, a->B_max);
     return pl;
 }
 
@@ -84,9 +92,9 @@ static int topk_slots(int dtype) {
         return -1;
     }
     cudaError_t e = dtype == CADD_DTYPE_BF16
-        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, kThreads, topk_smem_bytes())
-        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, kThreads, topk_smem_bytes());
-    if (e != cudaSuccess || per_sm < 1) { cudaGetLastError(); per_sm = 3; }
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, kTkThreads, topk_smem_bytes())
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, kTkThreads, topk_smem_bytes());
+    if (e != cudaSuccess || per_sm < 1) { cudaGetLastError(); per_sm = 4; }
     return per_sm * sm_count();
 }
 
@@ -121,10 +129,11 @@ static cudaError_t launch_dependent(bool overlap, void (*kernel)(KArgs...), dim3
 }
 
 // Launches the expansion + emission kernel on the per-row partial records at `partials` (S records per row).
-static int launch_expand(const cadd_build_args* a, int KP, int S, const unsigned char* partials, cudaStream_t st, bool overlap) {
-    const ExpandLayout lay = expand_layout(a->L, a->K, KP, S, a->B_max);
+static int launch_expand(const cadd_build_args* a, int KP, int S, int rec_fmt, const unsigned char* partials, cudaStream_t st, bool overlap) {
+    const ExpandLayout lay = expand_layout(a->L, a->K, rec_key_cap(rec_fmt, KP), S, a->B_max);
     ExpandParams ep;
     ep.batch = a->batch; ep.L = a->L; ep.K = a->K; ep.KP = KP; ep.S = S; ep.B_max = a->B_max; ep.R = a->R;
+    ep.rec_fmt = rec_fmt;
     ep.flags = a->flags; ep.partials = partials;
     ep.l_eff = a->l_eff; ep.bonus_token = a->bonus_token; ep.ctx_len = a->ctx_len;
     ep.cost_kind = a->cost_kind; ep.cost_coef = a->cost_coef; ep.cost_table = a->cost_table;
@@ -170,7 +179,7 @@ int cadd_build_workspace_bytes(const cadd_build_args* a, size_t* out) {
     BuildPlan pl = plan_build(a, 148 * 3);
     BuildPlan worst = pl;
     worst.S = kMaxSegments;
-    worst.partial_bytes = (size_t)a->batch * a->L * kMaxSegments * seg_partial_stride(pl.KP);
+    worst.partial_bytes = (size_t)a->batch * a->L * max_segments((int64_t)a->batch * a->L) * seg_record_stride(pl.KP);
     *out = build_workspace_bytes(worst);
     return CADD_OK;
 }
@@ -210,12 +219,12 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
     const bool overlap = (int64_t)a->batch * a->L * a->V * (int64_t)es >= kOverlapMinBytes;
     if (!(a->flags & CADD_FLAG_ONLY_EXPAND)) {
         const cudaError_t le = a->logits_dtype == CADD_DTYPE_BF16
-            ? launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, dim3(items), dim3(kThreads), topk_smem_bytes(), st, tp)
-            : launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, dim3(items), dim3(kThreads), topk_smem_bytes(), st, tp);
+            ? launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_BF16>, dim3(items), dim3(kTkThreads), topk_smem_bytes(), st, tp)
+            : launch_dependent(overlap, softmax_topk_partial_kernel<CADD_DTYPE_FP32>, dim3(items), dim3(kTkThreads), topk_smem_bytes(), st, tp);
         if (le != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
     }
     if (a->flags & CADD_FLAG_ONLY_TOPK) return CADD_OK;
-    return launch_expand(a, pl.KP, pl.S, (const unsigned char*)a->workspace, st, overlap);
+    return launch_expand(a, pl.KP, pl.S, kRecSegRecord, (const unsigned char*)a->workspace, st, overlap);
 }
 
 static int check_verify_shape(const cadd_verify_args* a) {
@@ -554,7 +563,7 @@ int cadd_build_tree_fused_head(const cadd_build_head_args* h, void* cuda_stream)
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
     draft_merge_kernel<<<(unsigned)((M + 3) / 4), 128, 0, st>>>(dp, merged);
     if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
-    return launch_expand(a, pl.KP, 1, merged, st, false);
+    return launch_expand(a, pl.KP, 1, kRecSegPartial, merged, st, false);
 }
 
 // ---------------- tree verification under sampling ----------------

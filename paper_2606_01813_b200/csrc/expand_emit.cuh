@@ -25,6 +25,7 @@ namespace cadd {
 
 struct ExpandParams {
     int batch, L, K, KP, S, B_max, R;
+    int rec_fmt;               // records at `partials`: kRecSegRecord (softmax_topk_partial_kernel) or kRecSegPartial (draft_merge_kernel)
     uint32_t flags;
     const unsigned char* partials;
     const int32_t* l_eff;
@@ -53,6 +54,10 @@ struct ExpandParams {
     int32_t* status;
 };
 
+constexpr int kRecSegPartial = 0, kRecSegRecord = 1;
+// candidate keys a record of the given format holds at most
+__host__ __device__ inline int rec_key_cap(int rec_fmt, int KP) { return rec_fmt == kRecSegRecord ? seg_key_cap(KP) : KP; }
+
 constexpr int kExpandThreads = 512;        // sixteen warps: one per draft position in the merge phase for L <= 16
 constexpr int kExpandWarps = kExpandThreads / 32;
 
@@ -72,13 +77,13 @@ struct ExpandLayout {
     size_t a_list, lz, S, nHi, nLo, region, tok_list, keff, total;
     int fr_cap;        // frontier slots per lane
 };
-__host__ __device__ inline ExpandLayout expand_layout(int L, int K, int KP, int S, int B_max) {
+__host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap, int S, int B_max) {
     ExpandLayout o;
     const size_t NR = (size_t)B_max + 1;
     // every pop adds at most one entry (the sibling reuses the popped slot, the child is dealt round-robin)
     o.fr_cap = (B_max + 1 + 31) / 32 + 1;
     size_t frontier = (size_t)o.fr_cap * 32 * (8 + 8 + 8);
-    size_t scratch = (size_t)kExpandWarps * S * KP * 8;
+    size_t scratch = (size_t)kExpandWarps * S * key_cap * 8;     // phase 0: every key of a row's records, per warp
     size_t region = frontier > scratch ? frontier : scratch;
     region = (region + 7) & ~(size_t)7;
     size_t p = 0;
@@ -113,7 +118,8 @@ __device__ __forceinline__ double cost_verify(const CostModel& cm, int n) {
 __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandParams p) {
     grid_dependency_wait();
     extern __shared__ __align__(16) unsigned char smem[];
-    const ExpandLayout lay = expand_layout(p.L, p.K, p.KP, p.S, p.B_max);
+    const int key_cap = rec_key_cap(p.rec_fmt, p.KP);
+    const ExpandLayout lay = expand_layout(p.L, p.K, key_cap, p.S, p.B_max);
     double* a_list = (double*)(smem + lay.a_list);
     double* lz = (double*)(smem + lay.lz);
     double* Sd = (double*)(smem + lay.S);
@@ -137,8 +143,12 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
     for (int d = tid; d < L + 2; d += kExpandThreads) keff[d] = 0;
     __syncthreads();
 
-    // ---------------- phase 0: merge partials, one warp per position ----------------
-    const size_t pstride = seg_partial_stride(p.KP);
+    // ---------------- phase 0: merge the records of every live position, one warp per position ----------------
+    // A record lists candidate keys (a superset of the K best of its part of the row) and one or more pairs (W, C) with
+    // the mass of everything else as W * 2^C.  All keys of the row are ranked by counting (they are unique); every listed
+    // key's exponential is taken in fp64.
+    const bool seg_records = p.rec_fmt == kRecSegRecord;
+    const size_t pstride = seg_records ? seg_record_stride(p.KP) : seg_partial_stride(p.KP);
     for (int i = warp; i < L; i += kExpandWarps) {
         int32_t* out_tok = p.topk_token ? p.topk_token + ((int64_t)b * L + i) * K : nullptr;
         double* out_lp = p.topk_logprob ? p.topk_logprob + ((int64_t)b * L + i) * K : nullptr;
@@ -150,15 +160,23 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
             }
             continue;
         }
-        uint64_t* scr = (uint64_t*)(smem + lay.region) + (size_t)warp * p.S * p.KP;
+        uint64_t* scr = (uint64_t*)(smem + lay.region) + (size_t)warp * p.S * key_cap;
         const unsigned char* rec0 = p.partials + ((size_t)((int64_t)b * L + i) * p.S) * pstride;
         int n = 0;
         uint32_t fl = 0;
         for (int s = 0; s < p.S; ++s) {
-            const SegPartial* h = (const SegPartial*)(rec0 + (size_t)s * pstride);
-            const uint64_t* keys = (const uint64_t*)(h + 1);
-            const int cnt = h->cnt;
-            fl |= h->flags;
+            const unsigned char* rec = rec0 + (size_t)s * pstride;
+            int cnt;
+            const uint64_t* keys;
+            if (seg_records) {
+                const SegRecord* h = (const SegRecord*)rec;
+                cnt = min(h->cnt, key_cap); fl |= h->flags;
+                keys = (const uint64_t*)(rec + sizeof(SegRecord) + (size_t)kSegSums * 16);
+            } else {
+                const SegPartial* h = (const SegPartial*)rec;
+                cnt = min(h->cnt, key_cap); fl |= h->flags;
+                keys = (const uint64_t*)(h + 1);
+            }
             for (int q = lane; q < cnt; q += 32) scr[n + q] = keys[q];
             n += cnt;
         }
@@ -177,9 +195,24 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
             zsum += exp(x - m);
             if (rank < K) { tok_list[i * K + rank] = (int32_t)key_id(k); a_list[i * K + rank] = x - m; }
         }
-        for (int s = lane; s < p.S; s += 32) {
-            const SegPartial* h = (const SegPartial*)(rec0 + (size_t)s * pstride);
-            if (h->W > 0.0) zsum += h->W * exp(h->C * 0.6931471805599453094 - m);
+        // the mass outside the lists: one (W, C) per record, or one per warp of the CTA that wrote it
+        const int spr = seg_records ? kSegSums : 1;
+        for (int t = lane; t < p.S * spr; t += 32) {
+            const unsigned char* rec = rec0 + (size_t)(t / spr) * pstride;
+            double W, C;
+            if (seg_records) {
+                const SegRecord* h = (const SegRecord*)rec;
+                const double* sums = (const double*)(rec + sizeof(SegRecord));
+                const int q = t % spr;
+                W = q < h->n_sums ? sums[2 * q] : 0.0;
+                C = q < h->n_sums ? sums[2 * q + 1] : 0.0;
+            } else {
+                const SegPartial* h = (const SegPartial*)rec;
+                W = h->W; C = h->C;
+            }
+            // (a warp's W can be negative: the warp that takes a candidate's term out of the sums need not be the one that
+            // added it; only the total over a record's warps is a sum of terms)
+            if (W != 0.0) zsum += W * exp(C * 0.6931471805599453094 - m);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) zsum += __shfl_xor_sync(kFullMask, zsum, o);
