@@ -2,18 +2,18 @@
 // of the tree arrays and the ancestor mask (Algorithm 1; Eq. 5-7, Eq. 11, Corollary 1; Section 3.3).
 //
 // One CTA per request.
-//   phase 0  all warps: merge the per-segment softmax/top-K partials of each live position into the
-//            sorted top-K list (token, a = logit - row max) and log Z, all in fp64
+//   phase 0  all warps: merge the softmax/top-K records of each live position (candidate keys in no order,
+//            plus the mass of everything else as pairs W * 2^C) into the sorted top-K list (token,
+//            a = logit - row max) and log Z, all in fp64
 //   phase 1  one thread: running log-partition sums S_d and the reachable depth
-//   phase 2  warp 0: the pop loop.  The frontier (Algorithm 1's heap) is striped over the 32 lanes;
-//            each lane caches the best entry of its stripe in registers.  A pop is a warp arg-max over
-//            the cached bests on a 128-bit key (score, then the packed tie-break), taken 32 bits at a
-//            time with redux.sync and stopped as soon as one lane is left.  The popped entry's next
-//            sibling overwrites it in place, only the winner lane rescans its stripe, the first child
-//            goes to the next lane round-robin.  Nodes are popped speculatively in groups; the group's
-//            exp(sigma), prefix sums Phi and throughput tests are then evaluated lane-parallel, and the
-//            first failing test fixes n*.  The pop order does not depend on the cost model, so this
-//            yields exactly Algorithm 1's tree.
+//   phase 2  warp 0: the pop loop.  The best 32 entries of the frontier (Algorithm 1's heap) sit in the
+//            warp's registers, sorted over the lanes on a 128-bit key (score, then the packed tie-break);
+//            what does not fit waits, unsorted, in a shared-memory pool whose best key is tracked.  A pop
+//            takes lane 0's entry and moves the others up; the popped node's next sibling and first
+//            child are inserted by one ballot (how many entries stay ahead) and one shuffle each.  Nodes
+//            are popped speculatively in groups; the group's exp(sigma), prefix sums Phi and throughput
+//            tests are then evaluated lane-parallel, and the first failing test fixes n*.  The pop order
+//            does not depend on the cost model, so this yields exactly Algorithm 1's tree.
 //   phase 3  all threads: write token / parent / depth / position / log-prob rows and padding; zero
 //            the mask rows with coalesced stores, then one thread per node walks its ancestors and
 //            writes the few non-zero words (bytes for the dense form).
@@ -74,15 +74,15 @@ __device__ __forceinline__ int tb_rank(uint64_t tb) { return (int)(tb & 0x7fu); 
 
 // Dynamic shared memory layout of the expansion kernel (byte offsets), same arithmetic on host and device.
 struct ExpandLayout {
-    size_t a_list, lz, S, nHi, nLo, region, tok_list, keff, total;
-    int fr_cap;        // frontier slots per lane
+    size_t a_list, lz, S, nHi, nLo, nA, region, tok_list, keff, total;
+    int pool_cap;      // entries of the frontier's pool
 };
 __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap, int S, int B_max) {
     ExpandLayout o;
     const size_t NR = (size_t)B_max + 1;
-    // every pop adds at most one entry (the sibling reuses the popped slot, the child is dealt round-robin)
-    o.fr_cap = (B_max + 1 + 31) / 32 + 1;
-    size_t frontier = (size_t)o.fr_cap * 32 * (8 + 8 + 8);
+    // every pop takes one entry out of the frontier and puts at most two in
+    o.pool_cap = B_max + 2;
+    size_t frontier = (size_t)o.pool_cap * (8 + 8);
     size_t scratch = (size_t)kExpandWarps * S * key_cap * 8;     // phase 0: every key of a row's records, per warp
     size_t region = frontier > scratch ? frontier : scratch;
     region = (region + 7) & ~(size_t)7;
@@ -92,6 +92,7 @@ __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap,
     o.S = p;        p += ((size_t)L + 1) * 8;
     o.nHi = p;      p += NR * 8;
     o.nLo = p;      p += NR * 8;
+    o.nA = p;       p += NR * 8;
     o.region = p;   p += region;
     o.tok_list = p; p += (size_t)L * K * 4;
     o.keff = p;     p += ((size_t)L + 2) * 4;
@@ -127,9 +128,9 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
     uint64_t* nLo = (uint64_t*)(smem + lay.nLo);          // ~pack_tiebreak(depth, token, parent, rank)
     int32_t* tok_list = (int32_t*)(smem + lay.tok_list);
     int32_t* keff = (int32_t*)(smem + lay.keff);          // keff[d], d = 1..L
-    uint64_t* fHi = (uint64_t*)(smem + lay.region);       // frontier, lane-major: [lane * fr_cap + slot]
-    uint64_t* fLo = fHi + (size_t)lay.fr_cap * 32;
-    double* fAp = (double*)(fLo + (size_t)lay.fr_cap * 32);  // the entry's parent's sum of (logit - row max)
+    double* nA = (double*)(smem + lay.nA);                // the node's sum of (logit - row max) along its path
+    uint64_t* pHi = (uint64_t*)(smem + lay.region);       // the frontier's pool (see phase 2), in no order
+    uint64_t* pLo = pHi + lay.pool_cap;
 
     __shared__ int s_status, s_pinf, s_Lr, s_n;
     __shared__ double s_phi, s_theta, s_theta0;
@@ -287,77 +288,109 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
         else theta_prev = 1.0 / den0;
         if (s_pinf) ok = false;
 
-        // Lane-private view of the frontier.  This lane's stripe holds cnt entries in shared memory; its
-        // best entry (b1) and, when b2ok, its exact second best (b2) are cached in registers, so that most
-        // pops need no look at the stripe at all.  (0,0) stands for "no entry": every real key is larger.
-        const int fbase = lane * lay.fr_cap;
-        int cnt = 0, b1slot = 0, b2slot = 0;
-        uint64_t b1hi = 0, b1lo = 0, b2hi = 0, b2lo = 0;
-        double b1ap = 0.0;
-        bool b2ok = true;
+        // The frontier (Algorithm 1's heap) in two parts.  The WINDOW is its best entries, at most 32, sorted best
+        // first over the lanes of the warp (lane i holds the i-th best; a key of (0,0) is an empty lane: every real key
+        // is larger).  The POOL, in shared memory and in no order, holds what did not fit: an entry goes there only if
+        // the window is full and all 32 of its entries are better, or by falling off the window's end.  pmax is the
+        // best key of the pool.  A pop takes the window's head unless the pool's best beats it (or the window is empty).
+        // Every step is a handful of shuffles and compares on the 128-bit key (score, then the packed tie-break); the
+        // parent's sum A, needed for the successors, is read from the node table instead of travelling with the entry.
+        uint64_t whi = 0, wlo = 0;                          // this lane's window entry
+        int wn = 0;                                         // entries in the window
+        int pn = 0;                                         // entries in the pool
+        uint64_t pmax_hi = 0, pmax_lo = 0;
         int fsize = 0;
-        unsigned pushctr = 0;
         auto key_gt = [](uint64_t ahi, uint64_t alo, uint64_t bhi, uint64_t blo) { return ahi > bhi || (ahi == bhi && alo > blo); };
-        // recompute b1 and b2 from the stripe (only this lane runs it, reading its own earlier writes)
-        auto rescan_top2 = [&]() {
-            b1hi = b1lo = b2hi = b2lo = 0; b1slot = b2slot = 0;
-            for (int s2 = 0; s2 < cnt; ++s2) {
-                const uint64_t hi = fHi[fbase + s2], lo = fLo[fbase + s2];
-                if (key_gt(hi, lo, b1hi, b1lo)) { b2hi = b1hi; b2lo = b1lo; b2slot = b1slot; b1hi = hi; b1lo = lo; b1slot = s2; }
-                else if (key_gt(hi, lo, b2hi, b2lo)) { b2hi = hi; b2lo = lo; b2slot = s2; }
+        // a new entry joins the frontier
+        auto push = [&](uint64_t khi, uint64_t klo) {
+            const int pos = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, khi, klo)));   // window entries that stay ahead of it
+            if (pos >= 32) {                                // a full window of better entries: to the pool
+                if (lane == 0) { pHi[pn] = khi; pLo[pn] = klo; }
+                if (key_gt(khi, klo, pmax_hi, pmax_lo)) { pmax_hi = khi; pmax_lo = klo; }
+                ++pn;
+                return;
             }
-            b1ap = cnt > 0 ? fAp[fbase + b1slot] : 0.0;
-            b2ok = true;
+            if (wn == 32) {                                 // the window's last entry makes room
+                const uint64_t lhi = __shfl_sync(kFullMask, whi, 31), llo = __shfl_sync(kFullMask, wlo, 31);
+                if (lane == 0) { pHi[pn] = lhi; pLo[pn] = llo; }
+                if (key_gt(lhi, llo, pmax_hi, pmax_lo)) { pmax_hi = lhi; pmax_lo = llo; }
+                ++pn;
+            } else {
+                ++wn;
+            }
+            const uint64_t uhi = __shfl_up_sync(kFullMask, whi, 1), ulo = __shfl_up_sync(kFullMask, wlo, 1);
+            if (lane > pos) { whi = uhi; wlo = ulo; }
+            else if (lane == pos) { whi = khi; wlo = klo; }
         };
         if (ok && Lr >= 1) {                                // Algorithm 1, line 3: the heap starts with node (1)
-            if (lane == 0) {
-                b1hi = ord64(a_list[0] - Sd[1]);
-                b1lo = ~pack_tiebreak(1, tok_list[0], 0, 1);
-                b1ap = 0.0;
-                fHi[fbase] = b1hi; fLo[fbase] = b1lo; fAp[fbase] = 0.0;
-                cnt = 1;
-            }
+            push(ord64(a_list[0] - Sd[1]), ~pack_tiebreak(1, tok_list[0], 0, 1));
             fsize = 1;
-            pushctr = 1;
         }
+        if (lane == 0) nA[0] = 0.0;
+        __syncwarp();
 
         int n = 0, popped = 0;
         bool stopped = false;
         while (ok && !stopped) {
             // group sizes grow with the tree: a stop is usually found within the group that contains it, and what a
-            // group pops beyond the stop is wasted (a pop costs about four group evaluations)
+            // group pops beyond the stop is wasted
             const int G = popped < 8 ? 4 : (popped < 32 ? 8 : (popped < 64 ? 16 : 32));
             int g = 0;
             while (g < G && popped < B_max && fsize > 0) {
-                // ---- arg-max of the 128-bit keys cached per lane, 32 bits at a time ----
-                uint32_t v = (uint32_t)(b1hi >> 32);        // empty lanes hold 0
-                uint32_t mx = __reduce_max_sync(kFullMask, v);
-                unsigned m = __ballot_sync(kFullMask, cnt > 0 && v == mx);
-                if (m & (m - 1)) {
-                    v = ((m >> lane) & 1u) ? (uint32_t)b1hi : 0u;
-                    mx = __reduce_max_sync(kFullMask, v);
-                    m &= __ballot_sync(kFullMask, v == mx);
-                    if (m & (m - 1)) {                      // equal scores: the tie-break decides
-                        v = ((m >> lane) & 1u) ? (uint32_t)(b1lo >> 32) : 0u;
-                        mx = __reduce_max_sync(kFullMask, v);
-                        m &= __ballot_sync(kFullMask, v == mx);
+                // ---- the best entry of the frontier ----
+                __syncwarp();                               // lane 0's writes to the node table and the pool are visible to all
+                uint64_t khi = __shfl_sync(kFullMask, whi, 0), klo = __shfl_sync(kFullMask, wlo, 0);
+                if (wn == 0 || key_gt(pmax_hi, pmax_lo, khi, klo)) {
+                    // rare: the best entry sits in the pool.  Find it (lanes scan stripes of the pool, then the warp's
+                    // arg-max 32 bits at a time), fill its slot with the pool's last entry, and find the new best.
+                    uint64_t bhi = 0, blo = 0;
+                    int bi = -1;
+                    for (int q = lane; q < pn; q += 32) {
+                        const uint64_t hi = pHi[q], lo = pLo[q];
+                        if (key_gt(hi, lo, bhi, blo)) { bhi = hi; blo = lo; bi = q; }
+                    }
+                    uint32_t v = (uint32_t)(bhi >> 32);
+                    unsigned m = __ballot_sync(kFullMask, bi >= 0 && v == __reduce_max_sync(kFullMask, v));
+                    if (m & (m - 1)) {
+                        v = ((m >> lane) & 1u) ? (uint32_t)bhi : 0u;
+                        m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
                         if (m & (m - 1)) {
-                            v = ((m >> lane) & 1u) ? (uint32_t)b1lo : 0u;
-                            mx = __reduce_max_sync(kFullMask, v);
-                            m &= __ballot_sync(kFullMask, v == mx);
+                            v = ((m >> lane) & 1u) ? (uint32_t)(blo >> 32) : 0u;
+                            m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
+                            if (m & (m - 1)) {
+                                v = ((m >> lane) & 1u) ? (uint32_t)blo : 0u;
+                                m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
+                            }
                         }
                     }
+                    const int win = __ffs(m) - 1;
+                    khi = __shfl_sync(kFullMask, bhi, win); klo = __shfl_sync(kFullMask, blo, win);
+                    const int slot = __shfl_sync(kFullMask, bi, win);
+                    --pn;
+                    if (lane == 0 && slot != pn) { pHi[slot] = pHi[pn]; pLo[slot] = pLo[pn]; }
+                    __syncwarp();
+                    bhi = blo = 0;
+                    for (int q = lane; q < pn; q += 32) {
+                        const uint64_t hi = pHi[q], lo = pLo[q];
+                        if (key_gt(hi, lo, bhi, blo)) { bhi = hi; blo = lo; }
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o), olo = __shfl_xor_sync(kFullMask, blo, o);
+                        if (key_gt(ohi, olo, bhi, blo)) { bhi = ohi; blo = olo; }
+                    }
+                    pmax_hi = bhi; pmax_lo = blo;
+                } else {                                    // the window's head; the others move up
+                    whi = __shfl_down_sync(kFullMask, whi, 1); wlo = __shfl_down_sync(kFullMask, wlo, 1);
+                    if (lane == 31) { whi = 0; wlo = 0; }
+                    --wn;
                 }
-                const int win = __ffs(m) - 1;
-                const uint64_t whi = __shfl_sync(kFullMask, b1hi, win);
-                const uint64_t wlo = __shfl_sync(kFullMask, b1lo, win);
-                const double Apar = __shfl_sync(kFullMask, b1ap, win);
-                const uint64_t tb = ~wlo;
+                const uint64_t tb = ~klo;
                 const int d = tb_depth(tb), par = tb_parent(tb), r = tb_rank(tb);
                 const int j = ++popped;
-                // ---- the popped node and its two successors (Algorithm 1, lines 12-19); every lane forms
-                //      both successor keys so that all shared-memory reads are issued together ----
+                // ---- the popped node and its two successors (Algorithm 1, lines 12-19) ----
                 const double* arow = a_list + (d - 1) * K;
+                const double Apar = nA[par];
                 const double a_cur = arow[r - 1];
                 const int rs = r < K ? r : K - 1;                       // index of the next sibling (clamped)
                 const int dc = d < L ? d : L - 1;                       // row of the first child (clamped)
@@ -367,68 +400,11 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
                 const bool has_sib = r < keff[d];
                 const bool has_child = d < Lr;
                 const double A = Apar + a_cur;
-                const uint64_t sib_hi = ord64((Apar + a_sib) - S_d);
-                const uint64_t sib_lo = ~pack_tiebreak(d, tok_sib, par, r + 1);
-                const uint64_t chi_hi = ord64((A + a_chi) - S_c);
-                const uint64_t chi_lo = ~pack_tiebreak(d + 1, tok_chi, j, 1);
-                if (lane == 1) nHi[j] = whi;
-                if (lane == 2) nLo[j] = wlo;
-                const bool w = lane == win;
-                if (has_sib) {
-                    // The next sibling takes the popped entry's slot (same parent).  Written without
-                    // divergent branches: every lane evaluates the selects, only the winner's take effect.
-                    const int s1 = b1slot;
-                    if (w) { fHi[fbase + s1] = sib_hi; fLo[fbase + s1] = sib_lo; }
-                    if (w && cnt > 1 && !b2ok) {
-                        rescan_top2();                      // rare: the second best was not known
-                    } else {
-                        // an empty b2 is (0,0), so a lone sibling always wins
-                        const bool sib_wins = key_gt(sib_hi, sib_lo, b2hi, b2lo);
-                        const bool promote = w && !sib_wins;        // the cached second best moves up and the
-                        const bool keep = w && sib_wins;            // sibling becomes a candidate second
-                        const double ap2 = promote ? fAp[fbase + b2slot] : b1ap;
-                        const uint64_t o2hi = b2hi, o2lo = b2lo;
-                        const int o2slot = b2slot;
-                        b1hi = keep ? sib_hi : (promote ? o2hi : b1hi);
-                        b1lo = keep ? sib_lo : (promote ? o2lo : b1lo);
-                        b1slot = promote ? o2slot : b1slot;
-                        b1ap = ap2;
-                        b2hi = promote ? sib_hi : b2hi;
-                        b2lo = promote ? sib_lo : b2lo;
-                        b2slot = promote ? s1 : b2slot;
-                        b2ok = promote ? (cnt == 2) : b2ok;
-                    }
-                } else if (w) {                             // no sibling: the last entry moves into the hole
-                    const int s1 = b1slot;
-                    const int last = --cnt;
-                    if (s1 != last) {
-                        fHi[fbase + s1] = fHi[fbase + last]; fLo[fbase + s1] = fLo[fbase + last]; fAp[fbase + s1] = fAp[fbase + last];
-                        if (b2slot == last) b2slot = s1;
-                    }
-                    if (cnt == 0) { b1hi = b1lo = b2hi = b2lo = 0; b2ok = true; }
-                    else if (!b2ok) rescan_top2();
-                    else {
-                        b1hi = b2hi; b1lo = b2lo; b1slot = b2slot; b1ap = fAp[fbase + b2slot];
-                        b2hi = b2lo = 0;
-                        b2ok = cnt == 1;
-                    }
-                }
-                if (has_child) {                            // the first child goes to the next lane in turn
-                    const bool mine = lane == (int)(pushctr & 31);
-                    ++pushctr;
-                    if (mine) { fHi[fbase + cnt] = chi_hi; fLo[fbase + cnt] = chi_lo; fAp[fbase + cnt] = A; }
-                    const bool first = mine && key_gt(chi_hi, chi_lo, b1hi, b1lo);   // new best: the old best is the exact second
-                    const bool second = mine && !first && b2ok && key_gt(chi_hi, chi_lo, b2hi, b2lo);
-                    b2hi = first ? b1hi : (second ? chi_hi : b2hi);
-                    b2lo = first ? b1lo : (second ? chi_lo : b2lo);
-                    b2slot = first ? b1slot : (second ? cnt : b2slot);
-                    b2ok = first ? true : b2ok;
-                    b1hi = first ? chi_hi : b1hi;
-                    b1lo = first ? chi_lo : b1lo;
-                    b1slot = first ? cnt : b1slot;
-                    b1ap = first ? A : b1ap;
-                    cnt += mine ? 1 : 0;
-                }
+                if (lane == 0) nA[j] = A;
+                if (lane == 1) nHi[j] = khi;
+                if (lane == 2) nLo[j] = klo;
+                if (has_sib) push(ord64((Apar + a_sib) - S_d), ~pack_tiebreak(d, tok_sib, par, r + 1));
+                if (has_child) push(ord64((A + a_chi) - S_c), ~pack_tiebreak(d + 1, tok_chi, j, 1));
                 fsize += (int)has_sib + (int)has_child - 1;
                 ++g;
             }
