@@ -43,9 +43,10 @@ KERNELS_PER_STEP = 4          # softmax_topk_partial, expand_emit, row_argmax, a
 # algorithmic bytes, from an ncu capture of the config-2 launch (summary kept under profiles/)
 # (2.5037 GB for 2.4990 GB).  Traffic grows in proportion to the rows read, so other workloads scale it.
 ARGMAX_TRAFFIC_RATIO = 1.0019
-# The same for one softmax_topk_partial launch (159.5 MB read + written for 155.6 MB of logits: the per-row records are
-# the extra), profiles/softmax_topk_partial_config2.md.
-TOPK_TRAFFIC_RATIO = 1.025
+# The same for one softmax_topk_partial launch (171.5 MB read + written for 155.6 MB of logits: the records it writes and
+# the part of its second look at ~16 two-kilobyte pieces per segment that misses L2),
+# profiles/softmax_topk_partial_config2_config3.md.
+TOPK_TRAFFIC_RATIO = 1.102
 NOMINAL_HBM_GBS = 8000.0      # the nominal HBM3e figure the bandwidth target is stated against
 
 
@@ -228,11 +229,41 @@ def per_kernel_pass(w, K):
 def kernel_blocks(w, km):
     """Roofline blocks of the two streaming kernels and the absolute times of the two latency-bound ones."""
     topk = hbm_roofline("softmax_topk_partial", w.build_bytes, km["softmax_topk_partial"], TOPK_TRAFFIC_RATIO,
-                        "profiles/softmax_topk_partial_config2.md, scaled by rows")
+                        "profiles/softmax_topk_partial_config2_config3.md, scaled by rows")
     argmax = hbm_roofline("row_argmax", w.verify_bytes, km["row_argmax"], ARGMAX_TRAFFIC_RATIO,
                           "profiles/row_argmax_config2.md, scaled by rows")
     return topk, argmax, {k: round(km[k], 5) for k in ("softmax_topk_partial", "expand_emit", "row_argmax", "accept_walk",
                                                          "step_mean", "step_median", "step_min")}
+
+
+def topk_alone_block(w, dev, iters=20):
+    """The softmax/top-K kernel launched alone, back to back, after a pause that lets the clocks recover from the
+    30 GB steps before it: this kernel is bound by instruction issue, so its time follows the SM clock (which a long
+    streaming step pulls down to the power cap), while the arg-max's does not."""
+    G = w.G
+    torch.cuda.synchronize()
+    time.sleep(0.5)
+    for _ in range(3):
+        w.build(extra_flags=G.FLAG_ONLY_TOPK)
+    sampler = ClockSampler(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(iters):
+        w.build(extra_flags=G.FLAG_ONLY_TOPK)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    while time.perf_counter() - t0 < 0.35:                 # long enough for a few clock samples
+        w.build(extra_flags=G.FLAG_ONLY_TOPK)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    blk = hbm_roofline("softmax_topk_partial (launched alone, back to back)", w.build_bytes, ms, TOPK_TRAFFIC_RATIO,
+                       "profiles/softmax_topk_partial_config2_config3.md, scaled by rows")
+    blk["launches"] = iters
+    blk["sm_mhz"] = clocks.get("sm_mhz")
+    return blk
 
 
 def tree_stats(w):
@@ -285,6 +316,10 @@ def run_ours(args, rank, world):
     clocks = sampler.stop() if sampler is not None else None
     value = replicas.whole_job_rounds_per_second(K, world, total_ms)
     roofline_topk, roofline, kernel_ms = kernel_blocks(w, km)
+    try:
+        roofline_topk["alone"] = topk_alone_block(w, dev)
+    except Exception as ex:
+        roofline_topk["alone"] = {"error": str(ex)[:200]}
     verify_bytes = w.verify_bytes
     step = w.step
 
