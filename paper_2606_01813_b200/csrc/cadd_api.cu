@@ -15,7 +15,7 @@
 
 namespace cadd {
 
-constexpr int kPreciseMin = 16;   // candidates per position whose exponentials are taken in fp64 (>= K)
+constexpr int kPreciseMin = 8;    // KP = max(K, 8): candidates per position singled out by the softmax/top-K kernel, exponentials in fp64
 
 static inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 
