@@ -87,6 +87,10 @@ extern "C" {
    array that an earlier call filled. */
 #define CADD_VERIFY_ONLY_ARGMAX   1u
 #define CADD_VERIFY_ONLY_WALK     2u
+/* Small problems are served by one kernel per call (see cadd_build_tree / cadd_verify_tree); these flags make a call
+   take the regular two-kernel path whatever its size (results are the same; for measurements and tests). */
+#define CADD_FLAG_REGULAR_PATH   32u   /* cadd_build_tree */
+#define CADD_VERIFY_REGULAR_PATH  4u   /* cadd_verify_tree */
 /* Test hook, accepted in the `flags` of cadd_build_tree, cadd_verify_tree and cadd_verify_tree_sampled: the streaming
    kernel never issues the asynchronous copy of the second tile (16 KB) of each row it reads (the first, if the row has
    only one), and its wait for that one tile gives up after a few tries.  Nothing hangs and nothing faults: the call
@@ -304,11 +308,19 @@ const char* cadd_status_string(int code);
 int cadd_build_workspace_bytes(const cadd_build_args* a, size_t* out);
 int cadd_verify_workspace_bytes(const cadd_verify_args* a, size_t* out);
 
-/* Tree construction (Eq. 1, Algorithm 1, Section 3.3).  Asynchronous on `cuda_stream`. */
+/* Tree construction (Eq. 1, Algorithm 1, Section 3.3).  Asynchronous on `cuda_stream`: two kernels (softmax/top-K
+ * over the rows, then expansion + emission), or ONE for small problems (rows of at most 8192 logits, 2 MiB of draft
+ * logits in all), where the expansion kernel reads the rows itself. */
 int cadd_build_tree(const cadd_build_args* a, void* cuda_stream);
 
-/* Tree verification (Sections 3.1 and 3.3).  Asynchronous on `cuda_stream`. */
+/* Tree verification (Sections 3.1 and 3.3).  Asynchronous on `cuda_stream`: two kernels (arg-max of the rows, then the
+ * walk), or ONE for small problems (rows of at most 8192 logits, 4 MiB of target logits in all). */
 int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream);
+
+/* Kernels the call with these arguments enqueues (pure host arithmetic on the shape fields and flags; pointers are
+ * ignored): 1 or 2, or a negative CADD_ERR_* code for arguments the call itself would reject. */
+int cadd_build_launches(const cadd_build_args* a);
+int cadd_verify_launches(const cadd_verify_args* a);
 
 /* Scratch size of cadd_verify_tree_fused_head: pure host arithmetic on batch, R, hidden and rows_mode (LIVE mode
  * needs room for a packed copy of the hidden states). */

@@ -27,10 +27,13 @@ FLAG_EMIT_DENSE_MASK, FLAG_EMIT_TOPK, FLAG_FIXED_BUDGET = 1, 2, 4
 FLAG_ONLY_TOPK, FLAG_ONLY_EXPAND = 8, 16          # measurement aids: one of the two build kernels alone
 VERIFY_ONLY_ARGMAX, VERIFY_ONLY_WALK = 1, 2       # the same for cadd_verify_tree
 FLAG_TEST_DROP_TILE = 0x80000000                  # test hook: one tile per row is never copied, its wait gives up
+FLAG_REGULAR_PATH, VERIFY_REGULAR_PATH = 32, 4    # small problems too take the two-kernel path
+# Tests set this to run small shapes through the regular two-kernel path as well (it only adds the two flags above).
+FORCE_REGULAR_PATH = False
 ROWS_LIVE, ROWS_DENSE = 0, 1
 
 EXPORTS = ("cadd_version", "cadd_status_string", "cadd_build_workspace_bytes", "cadd_verify_workspace_bytes",
-           "cadd_build_tree", "cadd_verify_tree", "cadd_build_tree_static_scratch",
+           "cadd_build_tree", "cadd_verify_tree", "cadd_build_tree_static_scratch", "cadd_build_launches", "cadd_verify_launches",
            "cadd_head_workspace_bytes", "cadd_verify_tree_fused_head", "cadd_fit_cost_tables",
            "cadd_build_head_workspace_bytes", "cadd_build_tree_fused_head", "cadd_verify_tree_sampled")
 ERR_STATIC_SCRATCH = -8
@@ -137,6 +140,8 @@ def lib() -> C.CDLL:
         l.cadd_build_head_workspace_bytes.argtypes = [C.POINTER(BuildHeadArgs), C.POINTER(C.c_size_t)]
         l.cadd_build_tree_fused_head.argtypes = [C.POINTER(BuildHeadArgs), C.c_void_p]
         l.cadd_build_tree_static_scratch.argtypes = [C.POINTER(BuildArgs), C.c_void_p]
+        l.cadd_build_launches.argtypes = [C.POINTER(BuildArgs)]
+        l.cadd_verify_launches.argtypes = [C.POINTER(VerifyArgs)]
         _lib = l
     return _lib
 
@@ -260,6 +265,22 @@ def cadd_build_workspace_bytes(batch: int, L: int, V: int, K: int, B_max: int, R
     return int(out.value)
 
 
+def cadd_round_launches(batch: int, L: int, V: int, K: int, B_max: int, R: int, dtype: torch.dtype, rows_mode: int = ROWS_LIVE) -> int:
+    """Kernels one round (cadd_build_tree + cadd_verify_tree) enqueues for this shape: 4, or 2 for small problems."""
+    a = BuildArgs()
+    a.struct_size = C.sizeof(BuildArgs)
+    a.batch, a.L, a.V, a.K, a.B_max, a.R = batch, L, V, K, B_max, R
+    a.logits_dtype = DTYPE_BF16 if dtype == torch.bfloat16 else DTYPE_FP32
+    v = VerifyArgs()
+    v.struct_size = C.sizeof(VerifyArgs)
+    v.batch, v.L, v.R, v.V = batch, L, R, V
+    v.logits_dtype, v.rows_mode = a.logits_dtype, rows_mode
+    nb, nv = lib().cadd_build_launches(C.byref(a)), lib().cadd_verify_launches(C.byref(v))
+    if nb < 0 or nv < 0:
+        raise CaddError(min(nb, nv))
+    return int(nb + nv)
+
+
 def cadd_build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[int] = None, *,
                     l_eff=None, bonus_token=None, ctx_len=None,
                     cost_kind: int = COST_QUADRATIC, cost_coef=None, cost_table=None, table_idx=None,
@@ -280,7 +301,7 @@ def cadd_build_tree(draft_logits: torch.Tensor, K: int, B_max: int, R: Optional[
     dev = x.device
     batch, L, V = x.shape
     R = B_max + 1 if R is None else R
-    a = _build_args(x, K, B_max, R, flags, cost_kind)
+    a = _build_args(x, K, B_max, R, flags | (FLAG_REGULAR_PATH if FORCE_REGULAR_PATH else 0), cost_kind)
     a.draft_logits = x.data_ptr()
     a.stride_b, a.stride_l = x.stride(0), x.stride(1)
     out, keep = _marshal_build(a, dev, batch, L, K, R, flags, theta_curve, out, l_eff, bonus_token, ctx_len, cost_coef,
@@ -318,7 +339,7 @@ def cadd_verify_tree(target_logits: torch.Tensor, L: int, n_nodes: torch.Tensor,
             raise ValueError("tree arrays must be contiguous int32 CUDA tensors")
     a = VerifyArgs()
     a.struct_size = C.sizeof(VerifyArgs)
-    a.flags = flags
+    a.flags = flags | (VERIFY_REGULAR_PATH if FORCE_REGULAR_PATH else 0)
     a.batch, a.L, a.R, a.V = batch, L, R, V
     a.logits_dtype = _dtype_code(y)
     a.rows_mode = rows_mode

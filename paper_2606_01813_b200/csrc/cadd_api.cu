@@ -128,12 +128,30 @@ static cudaError_t launch_dependent(bool overlap, void (*kernel)(KArgs...), dim3
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+// Small problems are launch-bound: below these sizes tree construction is ONE kernel (the expansion kernel reads the
+// short rows itself, one warp per row) and verification is ONE kernel (one CTA per request: arg-max of its rows, then
+// the walk).  The single-kernel measurement flags and the test hook always take the regular path.
+constexpr int64_t kSmallMaxV = 8192;                 // elements per row
+constexpr int64_t kSmallBuildBytes = 2ll << 20;      // draft logits of the whole call
+constexpr int64_t kSmallVerifyBytes = 4ll << 20;     // target logits the call reads at most
+static bool build_is_small(const cadd_build_args* a) {
+    if (a->flags & (CADD_FLAG_ONLY_TOPK | CADD_FLAG_ONLY_EXPAND | CADD_FLAG_TEST_DROP_TILE | CADD_FLAG_REGULAR_PATH)) return false;
+    const int64_t es = a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
+    return a->V <= kSmallMaxV && (int64_t)a->batch * a->L * a->V * es <= kSmallBuildBytes;
+}
+static bool verify_is_small(const cadd_verify_args* a) {
+    if (a->flags & (CADD_VERIFY_ONLY_ARGMAX | CADD_VERIFY_ONLY_WALK | CADD_FLAG_TEST_DROP_TILE | CADD_VERIFY_REGULAR_PATH)) return false;
+    const int64_t es = a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
+    return a->V <= kSmallMaxV && (int64_t)a->batch * a->R * a->V * es <= kSmallVerifyBytes;
+}
+
 // Launches the expansion + emission kernel on the per-row partial records at `partials` (S records per row).
 static int launch_expand(const cadd_build_args* a, int KP, int S, int rec_fmt, const unsigned char* partials, cudaStream_t st, bool overlap) {
     const ExpandLayout lay = expand_layout(a->L, a->K, rec_key_cap(rec_fmt, KP), S, a->B_max);
     ExpandParams ep;
     ep.batch = a->batch; ep.L = a->L; ep.K = a->K; ep.KP = KP; ep.S = S; ep.B_max = a->B_max; ep.R = a->R;
     ep.rec_fmt = rec_fmt;
+    ep.logits = a->draft_logits; ep.V = a->V; ep.stride_b = a->stride_b; ep.stride_l = a->stride_l; ep.logits_dtype = a->logits_dtype;
     ep.flags = a->flags; ep.partials = partials;
     ep.l_eff = a->l_eff; ep.bonus_token = a->bonus_token; ep.ctx_len = a->ctx_len;
     ep.cost_kind = a->cost_kind; ep.cost_coef = a->cost_coef; ep.cost_table = a->cost_table;
@@ -210,6 +228,7 @@ int cadd_build_tree(const cadd_build_args* a, void* cuda_stream) {
     const BuildPlan pl = plan_build(a, slots);
     if (!a->workspace || !aligned(a->workspace, 256) || a->workspace_bytes < build_workspace_bytes(pl)) return CADD_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (build_is_small(a)) return launch_expand(a, pl.KP, 1, kRecDirect, nullptr, st, false);
 
     TopkParams tp;
     tp.logits = a->draft_logits; tp.V = a->V; tp.stride_b = a->stride_b; tp.stride_l = a->stride_l;
@@ -239,12 +258,26 @@ static int check_verify_shape(const cadd_verify_args* a) {
     return CADD_OK;
 }
 
+int cadd_build_launches(const cadd_build_args* a) {
+    int rc = check_build_shape(a);
+    if (rc != CADD_OK) return rc;
+    if (a->flags & (CADD_FLAG_ONLY_TOPK | CADD_FLAG_ONLY_EXPAND)) return 1;
+    return build_is_small(a) ? 1 : 2;
+}
+
 int cadd_verify_workspace_bytes(const cadd_verify_args* a, size_t* out) {
     int rc = check_verify_shape(a);
     if (rc != CADD_OK) return rc;
     if (!out) return CADD_ERR_NULL;
     *out = 0;
     return CADD_OK;
+}
+
+int cadd_verify_launches(const cadd_verify_args* a) {
+    int rc = check_verify_shape(a);
+    if (rc != CADD_OK) return rc;
+    if (a->flags & (CADD_VERIFY_ONLY_ARGMAX | CADD_VERIFY_ONLY_WALK)) return 1;
+    return verify_is_small(a) ? 1 : 2;
 }
 
 int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream) {
@@ -265,6 +298,17 @@ int cadd_verify_tree(const cadd_verify_args* a, void* cuda_stream) {
     ap.logits = a->target_logits; ap.V = a->V; ap.stride_b = a->stride_b; ap.stride_row = a->stride_row;
     ap.R = a->R; ap.rows_mode = a->rows_mode; ap.n_nodes = a->n_nodes; ap.node_argmax = a->node_argmax;
     ap.fault_tile = (a->flags & CADD_FLAG_TEST_DROP_TILE) ? 1 : -1;
+    if (verify_is_small(a)) {
+        WalkParams wp;
+        wp.batch = a->batch; wp.L = a->L; wp.R = a->R; wp.n_nodes = a->n_nodes; wp.token_ids = a->token_ids;
+        wp.parent_idx = a->parent_idx; wp.node_argmax = a->node_argmax; wp.accepted_len = a->accepted_len;
+        wp.accepted_nodes = a->accepted_nodes; wp.next_bonus = a->next_bonus; wp.status = a->status;
+        ap.ctas_per_request = 1;
+        if (a->logits_dtype == CADD_DTYPE_BF16) verify_small_kernel<CADD_DTYPE_BF16><<<(unsigned)a->batch, kVerifySmallThreads, 0, st>>>(ap, wp);
+        else verify_small_kernel<CADD_DTYPE_FP32><<<(unsigned)a->batch, kVerifySmallThreads, 0, st>>>(ap, wp);
+        if (cudaGetLastError() != cudaSuccess) return CADD_ERR_LAUNCH;
+        return CADD_OK;
+    }
     // LIVE with a small node cap: most rows are padding on typical trees, so eight rows share a CTA (interleaved, so
     // that a request's live rows, which come first, still spread over its CTAs) and few CTAs are launched only to exit.
     // Large caps and DENSE keep one row per CTA: every row is work there and short CTAs keep the last wave short.

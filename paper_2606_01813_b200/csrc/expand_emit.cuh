@@ -25,7 +25,11 @@ namespace cadd {
 
 struct ExpandParams {
     int batch, L, K, KP, S, B_max, R;
-    int rec_fmt;               // records at `partials`: kRecSegRecord (softmax_topk_partial_kernel) or kRecSegPartial (draft_merge_kernel)
+    int rec_fmt;               // records at `partials`: kRecSegRecord (softmax_topk_partial_kernel) or kRecSegPartial (draft_merge_kernel);
+                               // kRecDirect: no records, the kernel reads the (short) rows of logits itself
+    const void* logits;        // kRecDirect: [batch, L, V]
+    int64_t V, stride_b, stride_l;
+    int logits_dtype;
     uint32_t flags;
     const unsigned char* partials;
     const int32_t* l_eff;
@@ -54,9 +58,9 @@ struct ExpandParams {
     int32_t* status;
 };
 
-constexpr int kRecSegPartial = 0, kRecSegRecord = 1;
+constexpr int kRecSegPartial = 0, kRecSegRecord = 1, kRecDirect = 2;
 // candidate keys a record of the given format holds at most
-__host__ __device__ inline int rec_key_cap(int rec_fmt, int KP) { return rec_fmt == kRecSegRecord ? seg_key_cap(KP) : KP; }
+__host__ __device__ inline int rec_key_cap(int rec_fmt, int KP) { return rec_fmt == kRecSegRecord ? seg_key_cap(KP) : (rec_fmt == kRecDirect ? 0 : KP); }
 
 constexpr int kExpandThreads = 512;        // sixteen warps: one per draft position in the merge phase for L <= 16
 constexpr int kExpandWarps = kExpandThreads / 32;
@@ -116,6 +120,66 @@ __device__ __forceinline__ double cost_verify(const CostModel& cm, int n) {
     return cm.q[1] + cm.q[2] * x + cm.q[3] * (x * x);
 }
 
+// Small problems (a few thousand logits per row): one warp turns one row into the sorted top-K list and log Z by itself
+// (Eq. 1; Algorithm 1, Require), reading the row K + 2 times from L1/L2: the largest finite logit m; then the K best
+// keys one after the other (each the largest key below the one before; keys are unique); then the mass of everything
+// else as fp32 exponentials against the reference exponent ceil(m * log2e) + 1, summed in fp64.  The K best go through
+// the fp64 exponential, as on the large path.  NaN and infinities carry no mass and are flagged.
+template <int DT>
+__device__ __forceinline__ void row_lists_warp(const void* row, int64_t V, int K, int32_t* tok_out, double* a_out,
+                                               double* logZ_out, int32_t* keff_out, uint32_t* flags_out) {
+    using E = Elem<DT>;
+    const int lane = threadIdx.x & 31;
+    float m = -INFINITY;
+    uint32_t fl = 0;
+    int nfin = 0;
+    for (int64_t i = lane; i < V; i += 32) {
+        const float x = E::load(row, i);
+        const uint32_t b = __float_as_uint(x);
+        if ((b & 0x7f800000u) == 0x7f800000u) {
+            if (b != 0xff800000u) fl |= kPartNonfinite;
+            if (b == 0x7f800000u) fl |= kPartPosInf;
+            continue;
+        }
+        m = fmaxf(m, x);
+        ++nfin;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, o));
+    nfin = __reduce_add_sync(kFullMask, nfin);
+    fl = __reduce_or_sync(kFullMask, fl);
+    const int ke = nfin < K ? nfin : K;
+    uint64_t prev = ~0ull;                                   // above every key
+    for (int r = 0; r < ke; ++r) {
+        uint64_t best = 0;
+        for (int64_t i = lane; i < V; i += 32) {
+            const float x = E::load(row, i);
+            if (fabsf(x) < INFINITY) {
+                const uint64_t key = make_key(x, (uint32_t)i);
+                if (key < prev && key > best) best = key;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(kFullMask, best, o));
+        if (lane == 0) { tok_out[r] = (int32_t)key_id(best); a_out[r] = (double)key_value(best) - (double)m; }
+        prev = best;
+    }
+    const float negc = m > -INFINITY ? -(ceilf(fminf(m, 2.0e38f) * kLog2eHi) + 1.0f) : 0.0f;
+    double acc = 0.0;
+    for (int64_t i = lane; i < V; i += 32) {
+        const float x = E::load(row, i);
+        if (fabsf(x) < INFINITY && (ke == 0 || make_key(x, (uint32_t)i) < prev)) acc += (double)exp2_term(x, negc);
+    }
+    __syncwarp();
+    double zsum = lane < ke ? exp(a_out[lane]) : 0.0;
+    for (int r = lane + 32; r < ke; r += 32) zsum += exp(a_out[r]);
+    if (acc != 0.0) zsum += acc * kEx2BiasFix * exp((double)(-negc) * 0.6931471805599453094 - (double)m);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) zsum += __shfl_xor_sync(kFullMask, zsum, o);
+    if (lane == 0) { *logZ_out = log(zsum); *keff_out = ke; *flags_out = fl; }
+    __syncwarp();
+}
+
 __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandParams p) {
     grid_dependency_wait();
     extern __shared__ __align__(16) unsigned char smem[];
@@ -158,6 +222,27 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
             if (emit) for (int k = lane; k < K; k += 32) {
                 if (out_tok) out_tok[k] = -1;
                 if (out_lp) out_lp[k] = -INFINITY;
+            }
+            continue;
+        }
+        if (p.rec_fmt == kRecDirect) {                      // small problem: this warp reads the row itself
+            const size_t es = p.logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
+            const char* row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)i * p.stride_l) * (int64_t)es;
+            uint32_t fl = 0;
+            if (p.logits_dtype == CADD_DTYPE_BF16) row_lists_warp<CADD_DTYPE_BF16>(row, p.V, K, tok_list + i * K, a_list + i * K, &lz[i], &keff[i + 1], &fl);
+            else row_lists_warp<CADD_DTYPE_FP32>(row, p.V, K, tok_list + i * K, a_list + i * K, &lz[i], &keff[i + 1], &fl);
+            fl = __shfl_sync(kFullMask, fl, 0);
+            const int ke = keff[i + 1];
+            if (lane == 0) {
+                int st = 0;
+                if (fl & kPartNonfinite) st |= CADD_STATUS_NONFINITE_INPUT;
+                if (ke < K) st |= CADD_STATUS_FEWER_THAN_K_FINITE;
+                if (st) atomicOr(&s_status, st);
+                if (fl & kPartPosInf) s_pinf = 1;
+            }
+            if (emit) for (int k = lane; k < K; k += 32) {
+                if (out_tok) out_tok[k] = k < ke ? tok_list[i * K + k] : -1;
+                if (out_lp) out_lp[k] = k < ke ? a_list[i * K + k] - lz[i] : -INFINITY;
             }
             continue;
         }

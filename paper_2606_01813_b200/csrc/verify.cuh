@@ -176,13 +176,10 @@ struct WalkParams {
     int32_t* status;           // may be NULL
 };
 
-// One warp per request: from the root, move to the child whose token equals the target's argmax at
+// The walk of one request by one warp: from the root, move to the child whose token equals the target's argmax at
 // the current node (children always have a larger row index than their parent); stop at the first miss.
-__global__ void __launch_bounds__(128) accept_walk_kernel(WalkParams p) {
-    grid_dependency_wait();
-    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+__device__ __forceinline__ void accept_walk_warp(const WalkParams& p, int b) {
     const int lane = threadIdx.x & 31;
-    if (b >= p.batch) return;
     int st = 0;
     int n = p.n_nodes[b];
     if (n < 0) { n = 0; st |= CADD_STATUS_BAD_N_NODES; }
@@ -217,6 +214,55 @@ __global__ void __launch_bounds__(128) accept_walk_kernel(WalkParams p) {
         p.next_bonus[b] = gmx[cur];
         if (p.status) p.status[b] = st;
     }
+}
+
+// One warp per request.
+__global__ void __launch_bounds__(128) accept_walk_kernel(WalkParams p) {
+    grid_dependency_wait();
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (b >= p.batch) return;
+    accept_walk_warp(p, b);
+}
+
+// Small problems (short rows, few of them): the whole verification of a request in one CTA and one launch.  Every warp
+// takes rows of the request in turn and finds the row's first maximal element by itself (lanes read elements
+// lane, lane + 32, ... in ascending order, so a lane's first maximum is its lowest index; the warp reduces on
+// (value descending, index ascending)); after a CTA barrier warp 0 walks the accepted path.
+constexpr int kVerifySmallThreads = 512;
+template <int DT>
+__global__ void __launch_bounds__(kVerifySmallThreads) verify_small_kernel(ArgmaxParams p, WalkParams wp) {
+    using E = Elem<DT>;
+    grid_dependency_wait();
+    const int b = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int n = p.R - 1;
+    if (p.rows_mode == CADD_ROWS_LIVE) {
+        n = p.n_nodes[b];
+        n = n < 0 ? 0 : (n > p.R - 1 ? p.R - 1 : n);
+    }
+    for (int j = warp; j < p.R; j += kVerifySmallThreads / 32) {
+        int32_t* out = p.node_argmax + (int64_t)b * p.R + j;
+        if (j > n) {
+            if (lane == 0) *out = -1;
+            continue;
+        }
+        const char* row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)j * p.stride_row) * E::ES;
+        float rm = -INFINITY;            // running maximum (NaN never enters: only strict '>' updates it)
+        int64_t rpos = INT64_MAX;        // first position where rm was reached
+        for (int64_t i = lane; i < p.V; i += 32) {
+            const float x = E::load(row, i);
+            if (x > rm) { rm = x; rpos = i; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(kFullMask, rm, o);
+            const int64_t op = __shfl_xor_sync(kFullMask, rpos, o);
+            if (om > rm || (om == rm && op < rpos)) { rm = om; rpos = op; }
+        }
+        if (lane == 0) *out = rpos == INT64_MAX ? 0 : (int32_t)rpos;      // every logit is -Inf or NaN: lowest id
+    }
+    __syncthreads();
+    if (warp == 0) accept_walk_warp(wp, b);
 }
 
 }  // namespace cadd

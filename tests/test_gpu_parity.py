@@ -21,6 +21,15 @@ def cost_kwargs(c: synth.CostInputs):
     return dict(cost_kind=G.COST_QUADRATIC, cost_coef=c.coef)
 
 
+@pytest.fixture(autouse=True, params=["one-launch where small", "regular"])
+def launch_path(request):
+    """Small problems are served by one kernel per call; every test of this file runs once as a caller would and once
+    with all calls forced onto the regular two-kernel path, so that both are held to the oracle on the same cases."""
+    G.FORCE_REGULAR_PATH = request.param == "regular"
+    yield
+    G.FORCE_REGULAR_PATH = False
+
+
 def round_trip(cfg, seed, rows_mode=G.ROWS_LIVE, dense_mask=False):
     """One full round (build, target logits for the built tree, verify) on both sides."""
     d = synth.make_draft_inputs(cfg, seed)
