@@ -62,8 +62,9 @@ constexpr int kRecSegPartial = 0, kRecSegRecord = 1, kRecDirect = 2;
 // candidate keys a record of the given format holds at most
 __host__ __device__ inline int rec_key_cap(int rec_fmt, int KP) { return rec_fmt == kRecSegRecord ? seg_key_cap(KP) : (rec_fmt == kRecDirect ? 0 : KP); }
 
-constexpr int kExpandThreads = 512;        // sixteen warps: one per draft position in the merge phase for L <= 16
-constexpr int kExpandWarps = kExpandThreads / 32;
+constexpr int kMergeWarps = 8;             // sixteen half-warps: one per draft position in the merge phase for L <= 16
+constexpr int kExpandWarps = kMergeWarps + 2;      // and the two warps of the expansion proper
+constexpr int kExpandThreads = kExpandWarps * 32;
 
 // Tie-break half of a frontier / node key.  Smaller packed value = earlier in the pop order
 // (depth, then token id, then parent row); the rank within the position's top-K list rides along in
@@ -78,16 +79,16 @@ __device__ __forceinline__ int tb_rank(uint64_t tb) { return (int)(tb & 0x7fu); 
 
 // Dynamic shared memory layout of the expansion kernel (byte offsets), same arithmetic on host and device.
 struct ExpandLayout {
-    size_t a_list, lz, S, nHi, nLo, nA, region, tok_list, keff, total;
+    size_t a_list, lz, S, nHi, nLo, nA, cv, region, tok_list, keff, total;
     int pool_cap;      // entries of the frontier's pool
 };
 __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap, int S, int B_max) {
     ExpandLayout o;
-    const size_t NR = (size_t)B_max + 1;
+    const size_t NR = (size_t)B_max + 2;                         // rows 0..B_max, and one that the trial pass writes
     // every pop takes one entry out of the frontier and puts at most two in
     o.pool_cap = B_max + 2;
     size_t frontier = (size_t)o.pool_cap * (8 + 8);
-    size_t scratch = (size_t)kExpandWarps * S * key_cap * 8;     // phase 0: every key of a row's records, per warp
+    size_t scratch = (size_t)kMergeWarps * 2 * S * key_cap * 8;     // phase 0: every key of a row's records, per warp
     size_t region = frontier > scratch ? frontier : scratch;
     region = (region + 7) & ~(size_t)7;
     size_t p = 0;
@@ -97,6 +98,7 @@ __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap,
     o.nHi = p;      p += NR * 8;
     o.nLo = p;      p += NR * 8;
     o.nA = p;       p += NR * 8;
+    o.cv = p;       p += NR * 8;
     o.region = p;   p += region;
     o.tok_list = p; p += (size_t)L * K * 4;
     o.keff = p;     p += ((size_t)L + 2) * 4;
@@ -180,8 +182,15 @@ __device__ __forceinline__ void row_lists_warp(const void* row, int64_t V, int K
     __syncwarp();
 }
 
-__global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandParams p) {
-    grid_dependency_wait();
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// Barrier 1 of the CTA: every warp arrives once, the merging warps when their lists are complete, the popping and the
+// evaluating warp before their real pass.
+__device__ __forceinline__ void lists_ready_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kExpandThreads) : "memory"); }
+
+__global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandParams p) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int key_cap = rec_key_cap(p.rec_fmt, p.KP);
     const ExpandLayout lay = expand_layout(p.L, p.K, key_cap, p.S, p.B_max);
@@ -193,42 +202,46 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
     int32_t* tok_list = (int32_t*)(smem + lay.tok_list);
     int32_t* keff = (int32_t*)(smem + lay.keff);          // keff[d], d = 1..L
     double* nA = (double*)(smem + lay.nA);                // the node's sum of (logit - row max) along its path
+    double* cv = (double*)(smem + lay.cv);                // C_v(n), n = 0..B_max
     uint64_t* pHi = (uint64_t*)(smem + lay.region);       // the frontier's pool (see phase 2), in no order
     uint64_t* pLo = pHi + lay.pool_cap;
 
-    __shared__ int s_status, s_pinf, s_Lr, s_n;
+    __shared__ int s_status, s_pinf, s_n;
+    __shared__ int s_cost_ok, s_pop_done, s_stop, s_fsize_end;   // between the popping warp and the evaluating warp
     __shared__ double s_phi, s_theta, s_theta0;
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int L = p.L, K = p.K, R = p.R;
+    const int L = p.L, K = p.K, R = p.R, B_max = p.B_max;
     int clamped;
-    const int Le = clamp_l_eff(p.l_eff, b, L, &clamped);
-    if (tid == 0) { s_status = clamped ? CADD_STATUS_L_EFF_CLAMPED : 0; s_pinf = 0; }
+    int Le = clamp_l_eff(p.l_eff, b, L, &clamped);         // (not written by the kernel before this one: read at once)
+    asm volatile("" : "+r"(Le));                          // a register from here on: never read from memory again
+    if (tid == 0) { s_status = 0; s_pinf = 0; s_pop_done = 0; s_stop = 0; s_fsize_end = 0; s_cost_ok = 0; }
     for (int d = tid; d < L + 2; d += kExpandThreads) keff[d] = 0;
+    for (int j = tid; j <= B_max + 1; j += kExpandThreads) nHi[j] = 0;   // "not popped yet" (see phase 2)
     __syncthreads();
+    if (tid == 0 && clamped) atomicOr(&s_status, CADD_STATUS_L_EFF_CLAMPED);
 
-    // ---------------- phase 0: merge the records of every live position, one warp per position ----------------
-    // A record lists candidate keys (a superset of the K best of its part of the row) and one or more pairs (W, C) with
-    // the mass of everything else as W * 2^C.  All keys of the row are ranked by counting (they are unique); every listed
-    // key's exponential is taken in fp64.
-    const bool seg_records = p.rec_fmt == kRecSegRecord;
-    const size_t pstride = seg_records ? seg_record_stride(p.KP) : seg_partial_stride(p.KP);
-    for (int i = warp; i < L; i += kExpandWarps) {
-        int32_t* out_tok = p.topk_token ? p.topk_token + ((int64_t)b * L + i) * K : nullptr;
-        double* out_lp = p.topk_logprob ? p.topk_logprob + ((int64_t)b * L + i) * K : nullptr;
-        const bool emit = (p.flags & CADD_FLAG_EMIT_TOPK) != 0;
-        if (i >= Le) {
-            if (emit) for (int k = lane; k < K; k += 32) {
-                if (out_tok) out_tok[k] = -1;
-                if (out_lp) out_lp[k] = -INFINITY;
+    const int kPopWarp = kMergeWarps;                       // the last warp evaluates
+    if (warp < kMergeWarps) {
+    // ---------------- phase 0: the sorted top-K list and log Z of every live position ----------------
+    grid_dependency_wait();                                 // the records are the previous kernel's
+    const bool emit = (p.flags & CADD_FLAG_EMIT_TOPK) != 0;
+    if (p.rec_fmt == kRecDirect) {
+        // small problem: there are no records, one warp per position reads the (short) row itself
+        for (int i = warp; i < L; i += kMergeWarps) {
+            int32_t* out_tok = p.topk_token ? p.topk_token + ((int64_t)b * L + i) * K : nullptr;
+            double* out_lp = p.topk_logprob ? p.topk_logprob + ((int64_t)b * L + i) * K : nullptr;
+            if (i >= Le) {
+                if (emit) for (int k = lane; k < K; k += 32) {
+                    if (out_tok) out_tok[k] = -1;
+                    if (out_lp) out_lp[k] = -INFINITY;
+                }
+                continue;
             }
-            continue;
-        }
-        if (p.rec_fmt == kRecDirect) {                      // small problem: this warp reads the row itself
             const size_t es = p.logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
             const char* row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)i * p.stride_l) * (int64_t)es;
-            uint32_t fl = 0;
+            uint32_t fl;
             if (p.logits_dtype == CADD_DTYPE_BF16) row_lists_warp<CADD_DTYPE_BF16>(row, p.V, K, tok_list + i * K, a_list + i * K, &lz[i], &keff[i + 1], &fl);
             else row_lists_warp<CADD_DTYPE_FP32>(row, p.V, K, tok_list + i * K, a_list + i * K, &lz[i], &keff[i + 1], &fl);
             fl = __shfl_sync(kFullMask, fl, 0);
@@ -244,36 +257,78 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
                 if (out_tok) out_tok[k] = k < ke ? tok_list[i * K + k] : -1;
                 if (out_lp) out_lp[k] = k < ke ? a_list[i * K + k] - lz[i] : -INFINITY;
             }
-            continue;
         }
-        uint64_t* scr = (uint64_t*)(smem + lay.region) + (size_t)warp * p.S * key_cap;
-        const unsigned char* rec0 = p.partials + ((size_t)((int64_t)b * L + i) * p.S) * pstride;
-        int n = 0;
-        uint32_t fl = 0;
+    } else {
+    // Merge of the softmax/top-K records, one HALF-warp per position (a row's records hold a few dozen keys and at most
+    // sixteen headers).  A record lists candidate keys (a superset of the K best of its part of the row) and one or more
+    // pairs (W, C) with the mass of everything else as W * 2^C.  All keys of the row are ranked by counting (they are
+    // unique); every listed key's exponential is taken in fp64.  Every key slot of the row's records is copied to shared
+    // memory asynchronously and the headers and first sums are read in the same round trip; what a record does not use
+    // is dropped afterwards.  Shuffles below move data within a half only (offsets below 16, or an explicit lane).
+    const bool seg_records = p.rec_fmt == kRecSegRecord;
+    const size_t pstride = seg_records ? seg_record_stride(p.KP) : seg_partial_stride(p.KP);
+    const size_t keys_at = seg_records ? sizeof(SegRecord) + (size_t)kSegSums * 16 : sizeof(SegPartial);
+    const int slots = p.S * key_cap;                        // at most 512, and at most 16 records
+    const int n_pairs = seg_records ? p.S * kSegSums : p.S; // (W, C) pairs of a row
+    const int hl = lane & 15, half = lane >> 4, lane0 = half << 4;
+    for (int i0 = 2 * warp; i0 < L; i0 += 2 * kMergeWarps) {
+        const int i = i0 + half;                            // this half-warp's position
+        const bool has_row = i < L;
+        const int ii = has_row ? i : L - 1;                 // (addresses stay inside the arrays; nothing of it is kept)
+        int32_t* out_tok = p.topk_token ? p.topk_token + ((int64_t)b * L + ii) * K : nullptr;
+        double* out_lp = p.topk_logprob ? p.topk_logprob + ((int64_t)b * L + ii) * K : nullptr;
+        uint64_t* scr = (uint64_t*)(smem + lay.region) + (size_t)(2 * warp + half) * slots;
+        const unsigned char* rec0 = p.partials + ((size_t)((int64_t)b * L + ii) * p.S) * pstride;
         for (int s = 0; s < p.S; ++s) {
-            const unsigned char* rec = rec0 + (size_t)s * pstride;
-            int cnt;
-            const uint64_t* keys;
-            if (seg_records) {
-                const SegRecord* h = (const SegRecord*)rec;
-                cnt = min(h->cnt, key_cap); fl |= h->flags;
-                keys = (const uint64_t*)(rec + sizeof(SegRecord) + (size_t)kSegSums * 16);
-            } else {
-                const SegPartial* h = (const SegPartial*)rec;
-                cnt = min(h->cnt, key_cap); fl |= h->flags;
-                keys = (const uint64_t*)(h + 1);
+            const uint64_t* keys = (const uint64_t*)(rec0 + (size_t)s * pstride + keys_at);
+            for (int q = hl; q < key_cap; q += 16) cp_async8(&scr[s * key_cap + q], keys + q);
+        }
+        // lane s of the half reads the header of record s, lane t the row's pair t (pair t % 8 of record t / 8)
+        int my_cnt = 0, my_ns = 0;
+        uint32_t my_fl = 0;
+        double W0 = 0.0, C0 = 0.0;
+        if (seg_records) {
+            if (hl < p.S) {
+                const int4 h = *(const int4*)(rec0 + (size_t)hl * pstride);
+                my_cnt = h.x; my_fl = (uint32_t)h.y; my_ns = h.z;
             }
-            for (int q = lane; q < cnt; q += 32) scr[n + q] = keys[q];
-            n += cnt;
+            if (hl < n_pairs) {
+                const double2 wc = *(const double2*)(rec0 + (size_t)(hl / kSegSums) * pstride + sizeof(SegRecord) + (size_t)(hl % kSegSums) * 16);
+                W0 = wc.x; C0 = wc.y;
+            }
+        } else if (hl < p.S) {
+            const SegPartial* h = (const SegPartial*)(rec0 + (size_t)hl * pstride);
+            my_cnt = h->cnt; my_fl = h->flags; my_ns = 1;
+            W0 = h->W; C0 = h->C;
+        }
+        cp_async_wait_all();
+        __syncwarp();
+        const bool live = has_row && i < Le;                // a masked position: whatever its records hold is not looked at
+        my_cnt = live ? min(max(my_cnt, 0), key_cap) : 0;
+        uint32_t fl = live ? my_fl : 0u;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) fl |= __shfl_xor_sync(kFullMask, fl, o);
+        // keep the slots that are in use, in place (a batch of 16 is read before its survivors are written below it)
+        int n = 0;
+        for (int base = 0; base < slots; base += 16) {
+            const int e = base + hl;
+            const int s = min(e / key_cap, p.S - 1);
+            const int cnt_s = __shfl_sync(kFullMask, my_cnt, lane0 + s);
+            const bool valid = e < slots && e - s * key_cap < cnt_s;
+            const uint64_t key = valid ? scr[e] : 0ull;
+            const unsigned m = (__ballot_sync(kFullMask, valid) >> lane0) & 0xffffu;
+            __syncwarp();
+            if (valid) scr[n + __popc(m & ((1u << hl) - 1u))] = key;
+            n += __popc(m);
         }
         __syncwarp();
         uint64_t mk = 0;
-        for (int q = lane; q < n; q += 32) mk = max(mk, scr[q]);
+        for (int q = hl; q < n; q += 16) mk = max(mk, scr[q]);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mk = max(mk, __shfl_xor_sync(kFullMask, mk, o));
+        for (int o = 8; o > 0; o >>= 1) mk = max(mk, __shfl_xor_sync(kFullMask, mk, o));
         const double m = (double)key_value(mk);
         double zsum = 0.0;
-        for (int q = lane; q < n; q += 32) {
+        for (int q = hl; q < n; q += 16) {
             const uint64_t k = scr[q];
             int rank = 0;
             for (int r = 0; r < n; ++r) rank += scr[r] > k;
@@ -282,30 +337,26 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
             if (rank < K) { tok_list[i * K + rank] = (int32_t)key_id(k); a_list[i * K + rank] = x - m; }
         }
         // the mass outside the lists: one (W, C) per record, or one per warp of the CTA that wrote it
-        const int spr = seg_records ? kSegSums : 1;
-        for (int t = lane; t < p.S * spr; t += 32) {
-            const unsigned char* rec = rec0 + (size_t)(t / spr) * pstride;
-            double W, C;
-            if (seg_records) {
-                const SegRecord* h = (const SegRecord*)rec;
-                const double* sums = (const double*)(rec + sizeof(SegRecord));
-                const int q = t % spr;
-                W = q < h->n_sums ? sums[2 * q] : 0.0;
-                C = q < h->n_sums ? sums[2 * q + 1] : 0.0;
-            } else {
-                const SegPartial* h = (const SegPartial*)rec;
-                W = h->W; C = h->C;
+        // (a warp's W can be negative: the warp that takes a candidate's term out of the sums need not be the one that
+        // added it; only the total over a record's warps is a sum of terms)
+        for (int t0 = 0; t0 < n_pairs; t0 += 16) {
+            const int t = t0 + hl;
+            const int rec = seg_records ? t / kSegSums : t;
+            const int ns = __shfl_sync(kFullMask, my_ns, lane0 + (rec & 15));
+            double W = W0, C = C0;
+            if (seg_records && t0 > 0 && t < n_pairs) {                     // (more than two records to a row: rare)
+                const double2 wc = *(const double2*)(rec0 + (size_t)rec * pstride + sizeof(SegRecord) + (size_t)(t % kSegSums) * 16);
+                W = wc.x; C = wc.y;
             }
-            // (a warp's W can be negative: the warp that takes a candidate's term out of the sums need not be the one that
-            // added it; only the total over a record's warps is a sum of terms)
-            if (W != 0.0) zsum += W * exp(C * 0.6931471805599453094 - m);
+            const bool used = live && t < n_pairs && (seg_records ? t % kSegSums < ns : true);
+            if (used && W != 0.0) zsum += W * exp(C * 0.6931471805599453094 - m);
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) zsum += __shfl_xor_sync(kFullMask, zsum, o);
+        for (int o = 8; o > 0; o >>= 1) zsum += __shfl_xor_sync(kFullMask, zsum, o);
         const double logZ = log(zsum);
         const int ke = n < K ? n : K;
         __syncwarp();
-        if (lane == 0) {
+        if (hl == 0 && live) {
             keff[i + 1] = ke;
             lz[i] = logZ;
             int st = 0;
@@ -315,29 +366,189 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
             if (st) atomicOr(&s_status, st);
             if (fl & kPartPosInf) s_pinf = 1;
         }
-        if (emit) for (int k = lane; k < K; k += 32) {
-            if (out_tok) out_tok[k] = k < ke ? tok_list[i * K + k] : -1;
-            if (out_lp) out_lp[k] = k < ke ? a_list[i * K + k] - logZ : -INFINITY;
+        if (emit && has_row) for (int k = hl; k < K; k += 16) {
+            if (out_tok) out_tok[k] = (live && k < ke) ? tok_list[i * K + k] : -1;
+            if (out_lp) out_lp[k] = (live && k < ke) ? a_list[i * K + k] - logZ : -INFINITY;
         }
     }
-    __syncthreads();
-    // ---------------- phase 1: S_d and the reachable depth ----------------
-    if (tid == 0) {
-        Sd[0] = 0.0;
-        int Lr = Le;
-        for (int d = 1; d <= Le; ++d) {
-            Sd[d] = Sd[d - 1] + lz[d - 1];
-            if (keff[d] == 0 && Lr == Le) Lr = d - 1;
-        }
-        s_Lr = Lr;
-        nHi[0] = ord64(0.0); nLo[0] = ~0ull;
     }
-    __syncthreads();
-    // ---------------- phase 2: the pop loop (warp 0) ----------------
-    if (warp == 0) {
-        const int Lr = s_Lr;
-        const int B_max = p.B_max;
-        const bool fixed = (p.flags & CADD_FLAG_FIXED_BUDGET) != 0;
+    lists_ready_barrier();
+    }
+    // ---------------- phase 2: the pop loop (one warp) and the throughput tests (another) ----------------
+    // The popping warp pops; the evaluating warp follows it through the node table, taking exp(sigma), the prefix sums
+    // Phi and the throughput tests of whatever has been popped since it last looked, up to 32 nodes at a time, one per
+    // lane.  The first failing test fixes n* and tells the popping warp to stop.  The pop order does not depend on the
+    // cost model, so what is popped beyond n* (as many nodes as fit into one evaluation's latency) is simply left unused.
+    // While the lists are being merged both warps go once through their loops on a made-up node (row B_max + 1 of the
+    // node table, nothing of it is kept): a trial pass that brings the loops' instructions into the SM's caches, since a
+    // CTA of this kernel lives for some tens of microseconds and its first pops would otherwise wait for their code.
+    else if (warp == kPopWarp) {
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+            const bool trial = pass == 0;
+            if (!trial) lists_ready_barrier();
+            // phase 1: running log-partition sums S_d (each lane adds up its own prefix, in position order) and the
+            // reachable depth (the trial pass does the same on whatever the arrays hold)
+            int Lr = Le;
+            for (int d0 = 0; d0 < Le; d0 += 32) {
+                const int d = d0 + lane + 1;
+                double acc = 0.0;
+                for (int i = 0; i < Le; ++i) {                     // (the same trip count for every lane)
+                    const double v = lz[i];
+                    if (i < d) acc += v;
+                }
+                if (d <= Le) Sd[d] = acc;
+                const unsigned z = __ballot_sync(kFullMask, d <= Le && keff[d] == 0);   // positions without a finite logit
+                if (z != 0 && Lr == Le) Lr = d0 + __ffs(z) - 1;
+            }
+            if (lane == 0) Sd[0] = 0.0;
+            bool ok = *(volatile int*)&s_cost_ok != 0 && *(volatile int*)&s_pinf == 0;
+            if (trial) { ok = true; Lr = 1; }
+            nA[0] = 0.0;
+            nHi[0] = ord64(0.0); nLo[0] = ~0ull;
+            __syncwarp();
+            // The frontier (Algorithm 1's heap) in two parts.  The WINDOW is its best entries, at most 32, sorted best
+            // first over the lanes of the warp (lane i holds the i-th best; a key of (0,0) is an empty lane: every real key
+            // is larger).  The POOL, in shared memory and in no order, holds what did not fit: an entry goes there only if
+            // the window is full and all of its entries are better, or by falling off the window's end.  pmax is the
+            // best key of the pool.  A pop takes the window's head unless the pool's best beats it (or the window is empty).
+            // In the usual case (the head is popped) the window changes once per pop: the head leaves and the node's next
+            // sibling and first child enter, each lane taking its new entry from its old one or a neighbour's according to
+            // two ballots on the old window.  The parent's sum A, needed for the successors, is read from the node table
+            // instead of travelling with the entry.  All lanes hold the same scalars and write the same values to the node
+            // table and the pool, so a lane only ever reads back what it has written itself.
+            uint64_t whi = 0, wlo = 0;                          // this lane's window entry
+            int wn = 0;                                         // entries in the window
+            int pn = 0;                                         // entries in the pool
+            uint64_t pmax_hi = 0, pmax_lo = 0;
+            auto key_gt = [](uint64_t ahi, uint64_t alo, uint64_t bhi, uint64_t blo) { return ahi > bhi || (ahi == bhi && alo > blo); };
+            auto to_pool = [&](uint64_t khi, uint64_t klo) {
+                pHi[pn] = khi; pLo[pn] = klo;
+                if (key_gt(khi, klo, pmax_hi, pmax_lo)) { pmax_hi = khi; pmax_lo = klo; }
+                ++pn;
+            };
+            // a new entry joins the frontier (the general form: any state of the window)
+            auto push = [&](uint64_t khi, uint64_t klo) {
+                const int pos = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, khi, klo)));   // window entries that stay ahead of it
+                if (pos >= 32) {                                // a full window of better entries: to the pool
+                    to_pool(khi, klo);
+                    return;
+                }
+                if (wn == 32) to_pool(__shfl_sync(kFullMask, whi, 31), __shfl_sync(kFullMask, wlo, 31));   // the last entry makes room
+                else ++wn;
+                const uint64_t uhi = __shfl_up_sync(kFullMask, whi, 1), ulo = __shfl_up_sync(kFullMask, wlo, 1);
+                if (lane > pos) { whi = uhi; wlo = ulo; }
+                else if (lane == pos) { whi = khi; wlo = klo; }
+            };
+            if (trial) push(ord64(-1.0), ~pack_tiebreak(1, 0, 0, 1));
+            else if (ok && Lr >= 1)                             // Algorithm 1, line 3: the heap starts with node (1)
+                push(ord64(a_list[0] - Sd[1]), ~pack_tiebreak(1, tok_list[0], 0, 1));
+            const int limit = trial ? 1 : B_max;
+
+            int popped = 0;
+            int stop_now = 0;
+            while (ok && popped < limit && (wn | pn) != 0 && !stop_now) {
+                stop_now = *(volatile int*)&s_stop;         // looked at when this pop is over
+                // ---- the best entry of the frontier ----
+                uint64_t khi = __shfl_sync(kFullMask, whi, 0), klo = __shfl_sync(kFullMask, wlo, 0);
+                const bool from_pool = wn == 0 || key_gt(pmax_hi, pmax_lo, khi, klo);
+                if (from_pool) {
+                    // rare: the best entry sits in the pool.  Find it (lanes scan stripes of the pool, then the warp's
+                    // arg-max 32 bits at a time), fill its slot with the pool's last entry, and find the new best.
+                    __syncwarp();
+                    uint64_t bhi = 0, blo = 0;
+                    int bi = -1;
+                    for (int q = lane; q < pn; q += 32) {
+                        const uint64_t hi = pHi[q], lo = pLo[q];
+                        if (key_gt(hi, lo, bhi, blo)) { bhi = hi; blo = lo; bi = q; }
+                    }
+                    uint32_t v = (uint32_t)(bhi >> 32);
+                    unsigned m = __ballot_sync(kFullMask, bi >= 0 && v == __reduce_max_sync(kFullMask, v));
+                    if (m & (m - 1)) {
+                        v = ((m >> lane) & 1u) ? (uint32_t)bhi : 0u;
+                        m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
+                        if (m & (m - 1)) {
+                            v = ((m >> lane) & 1u) ? (uint32_t)(blo >> 32) : 0u;
+                            m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
+                            if (m & (m - 1)) {
+                                v = ((m >> lane) & 1u) ? (uint32_t)blo : 0u;
+                                m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
+                            }
+                        }
+                    }
+                    const int win = __ffs(m) - 1;
+                    khi = __shfl_sync(kFullMask, bhi, win); klo = __shfl_sync(kFullMask, blo, win);
+                    const int slot = __shfl_sync(kFullMask, bi, win);
+                    --pn;
+                    __syncwarp();
+                    if (slot != pn) { const uint64_t lhi = pHi[pn], llo = pLo[pn]; __syncwarp(); pHi[slot] = lhi; pLo[slot] = llo; }
+                    __syncwarp();
+                    bhi = blo = 0;
+                    for (int q = lane; q < pn; q += 32) {
+                        const uint64_t hi = pHi[q], lo = pLo[q];
+                        if (key_gt(hi, lo, bhi, blo)) { bhi = hi; blo = lo; }
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o), olo = __shfl_xor_sync(kFullMask, blo, o);
+                        if (key_gt(ohi, olo, bhi, blo)) { bhi = ohi; blo = olo; }
+                    }
+                    pmax_hi = bhi; pmax_lo = blo;
+                }
+                const uint64_t tb = ~klo;
+                const int d = tb_depth(tb), par = tb_parent(tb), r = tb_rank(tb);
+                const int j = trial ? B_max + 1 : popped + 1;
+                ++popped;
+                // ---- the popped node and its two successors (Algorithm 1, lines 12-19) ----
+                const double* arow = a_list + (d - 1) * K;
+                const double Apar = nA[par];
+                const double a_cur = arow[r - 1];
+                const int rs = r < K ? r : K - 1;                       // index of the next sibling (clamped)
+                const int dc = d < L ? d : L - 1;                       // row of the first child (clamped)
+                const double a_sib = arow[rs], a_chi = a_list[dc * K];
+                const int tok_sib = tok_list[(d - 1) * K + rs], tok_chi = tok_list[dc * K];
+                const double S_d = Sd[d], S_c = Sd[dc + 1];
+                const bool has_sib = r < keff[d];
+                const bool has_child = d < Lr;
+                const double A = Apar + a_cur;
+                nA[j] = A;
+                nLo[j] = klo;
+                *(volatile uint64_t*)&nHi[j] = khi;                     // the evaluating warp's signal that node j exists
+                const uint64_t shi = has_sib ? ord64((Apar + a_sib) - S_d) : 0ull;
+                const uint64_t slo = has_sib ? ~pack_tiebreak(d, tok_sib, par, r + 1) : 0ull;
+                const uint64_t chi = has_child ? ord64((A + a_chi) - S_c) : 0ull;
+                const uint64_t clo = has_child ? ~pack_tiebreak(d + 1, tok_chi, j, 1) : 0ull;
+                if (from_pool) {                                        // the window kept its head: one entry after the other
+                    if (has_sib) push(shi, slo);
+                    if (has_child) push(chi, clo);
+                    continue;
+                }
+                // The head leaves; a (the better of the two successors) and b enter; a missing one is (0,0), which lands on
+                // the first empty lane.  Old entries ahead of a move up one lane, those between a and b stay, those behind b
+                // move down one.  Every successor is behind its node in the order, so the head counts in both ballots.
+                const bool sib_first = key_gt(shi, slo, chi, clo);
+                const uint64_t ahi = sib_first ? shi : chi, alo = sib_first ? slo : clo;
+                const uint64_t bhi = sib_first ? chi : shi, blo = sib_first ? clo : slo;
+                const int pa = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, ahi, alo))) - 1;
+                const int pb = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, bhi, blo)));
+                uint64_t nhi = __shfl_down_sync(kFullMask, whi, 1), nlo = __shfl_down_sync(kFullMask, wlo, 1);   // old[lane + 1]
+                const uint64_t phi_ = __shfl_up_sync(kFullMask, whi, 1), plo_ = __shfl_up_sync(kFullMask, wlo, 1); // old[lane - 1]
+                if (lane == 31) { nhi = 0; nlo = 0; }
+                if (wn == 32 && bhi != 0ull) {                          // 33 entries: the one that does not fit goes to the pool
+                    const uint64_t lhi = __shfl_sync(kFullMask, whi, 31), llo = __shfl_sync(kFullMask, wlo, 31);
+                    if (pb == 32) to_pool(bhi, blo); else to_pool(lhi, llo);
+                }
+                wn = min(32, wn - 1 + (int)(ahi != 0ull) + (int)(bhi != 0ull));
+                if (lane < pa) { whi = nhi; wlo = nlo; }
+                else if (lane == pa) { whi = ahi; wlo = alo; }
+                else if (lane == pb) { whi = bhi; wlo = blo; }
+                else if (lane > pb) { whi = phi_; wlo = plo_; }
+            }
+            __syncwarp();
+            if (!trial && lane == 0) { s_fsize_end = wn + pn; __threadfence_block(); *(volatile int*)&s_pop_done = 1; }
+        }
+    } else {
+        // the cost model of this request as a table: C_v(n) for every n the tree can reach, and the draft cost C_d
         CostModel cm;
         cm.kind = p.cost_kind; cm.row0 = cm.row1 = nullptr; cm.alpha = 0.0;
         cm.q[0] = cm.q[1] = cm.q[2] = cm.q[3] = 0.0;
@@ -367,171 +578,88 @@ __global__ void __launch_bounds__(kExpandThreads, 1) expand_emit_kernel(ExpandPa
             cm.alpha = jhi == jlo ? 0.0 : ((double)l - (double)p.ctx_grid[jlo]) / ((double)p.ctx_grid[jhi] - (double)p.ctx_grid[jlo]);
             C_d = p.t_draft[b];
         }
-        double theta_prev = 0.0, Phi = 0.0;
-        const double den0 = C_d + cost_verify(cm, 0);
-        if (ok && !(den0 > 0.0)) { st |= CADD_STATUS_COST_NONPOSITIVE; ok = false; }
-        else theta_prev = 1.0 / den0;
-        if (s_pinf) ok = false;
-
-        // The frontier (Algorithm 1's heap) in two parts.  The WINDOW is its best entries, at most 32, sorted best
-        // first over the lanes of the warp (lane i holds the i-th best; a key of (0,0) is an empty lane: every real key
-        // is larger).  The POOL, in shared memory and in no order, holds what did not fit: an entry goes there only if
-        // the window is full and all 32 of its entries are better, or by falling off the window's end.  pmax is the
-        // best key of the pool.  A pop takes the window's head unless the pool's best beats it (or the window is empty).
-        // Every step is a handful of shuffles and compares on the 128-bit key (score, then the packed tie-break); the
-        // parent's sum A, needed for the successors, is read from the node table instead of travelling with the entry.
-        uint64_t whi = 0, wlo = 0;                          // this lane's window entry
-        int wn = 0;                                         // entries in the window
-        int pn = 0;                                         // entries in the pool
-        uint64_t pmax_hi = 0, pmax_lo = 0;
-        int fsize = 0;
-        auto key_gt = [](uint64_t ahi, uint64_t alo, uint64_t bhi, uint64_t blo) { return ahi > bhi || (ahi == bhi && alo > blo); };
-        // a new entry joins the frontier
-        auto push = [&](uint64_t khi, uint64_t klo) {
-            const int pos = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, khi, klo)));   // window entries that stay ahead of it
-            if (pos >= 32) {                                // a full window of better entries: to the pool
-                if (lane == 0) { pHi[pn] = khi; pLo[pn] = klo; }
-                if (key_gt(khi, klo, pmax_hi, pmax_lo)) { pmax_hi = khi; pmax_lo = klo; }
-                ++pn;
-                return;
-            }
-            if (wn == 32) {                                 // the window's last entry makes room
-                const uint64_t lhi = __shfl_sync(kFullMask, whi, 31), llo = __shfl_sync(kFullMask, wlo, 31);
-                if (lane == 0) { pHi[pn] = lhi; pLo[pn] = llo; }
-                if (key_gt(lhi, llo, pmax_hi, pmax_lo)) { pmax_hi = lhi; pmax_lo = llo; }
-                ++pn;
-            } else {
-                ++wn;
-            }
-            const uint64_t uhi = __shfl_up_sync(kFullMask, whi, 1), ulo = __shfl_up_sync(kFullMask, wlo, 1);
-            if (lane > pos) { whi = uhi; wlo = ulo; }
-            else if (lane == pos) { whi = khi; wlo = klo; }
-        };
-        if (ok && Lr >= 1) {                                // Algorithm 1, line 3: the heap starts with node (1)
-            push(ord64(a_list[0] - Sd[1]), ~pack_tiebreak(1, tok_list[0], 0, 1));
-            fsize = 1;
+        for (int n0 = lane; n0 <= B_max; n0 += 32 * 16) {       // (sixteen loads in flight: the rows may come from DRAM)
+            double v[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) v[u] = n0 + 32 * u <= B_max ? cost_verify(cm, n0 + 32 * u) : 0.0;
+#pragma unroll
+            for (int u = 0; u < 16; ++u) if (n0 + 32 * u <= B_max) cv[n0 + 32 * u] = v[u];
         }
-        if (lane == 0) nA[0] = 0.0;
+        if (lane == 0) cv[B_max + 1] = 1.0;
         __syncwarp();
+        const double den0 = C_d + cv[0];
+        double theta_first = 0.0;                               // theta*(0) as the stopping rule sees it
+        if (ok && !(den0 > 0.0)) { st |= CADD_STATUS_COST_NONPOSITIVE; ok = false; }
+        else theta_first = 1.0 / den0;
+        const double theta0 = (den0 > 0.0) ? 1.0 / den0 : 0.0;
+        const bool fixed = (p.flags & CADD_FLAG_FIXED_BUDGET) != 0;
+        if (lane == 0) *(volatile int*)&s_cost_ok = ok ? 1 : 0;          // (ahead of the barrier the popping warp waits at)
 
-        int n = 0, popped = 0;
+        int n = 0;
+        double Phi = 0.0, theta_prev = theta_first;
         bool stopped = false;
-        while (ok && !stopped) {
-            // group sizes grow with the tree: a stop is usually found within the group that contains it, and what a
-            // group pops beyond the stop is wasted
-            const int G = popped < 8 ? 4 : (popped < 32 ? 8 : (popped < 64 ? 16 : 32));
-            int g = 0;
-            while (g < G && popped < B_max && fsize > 0) {
-                // ---- the best entry of the frontier ----
-                __syncwarp();                               // lane 0's writes to the node table and the pool are visible to all
-                uint64_t khi = __shfl_sync(kFullMask, whi, 0), klo = __shfl_sync(kFullMask, wlo, 0);
-                if (wn == 0 || key_gt(pmax_hi, pmax_lo, khi, klo)) {
-                    // rare: the best entry sits in the pool.  Find it (lanes scan stripes of the pool, then the warp's
-                    // arg-max 32 bits at a time), fill its slot with the pool's last entry, and find the new best.
-                    uint64_t bhi = 0, blo = 0;
-                    int bi = -1;
-                    for (int q = lane; q < pn; q += 32) {
-                        const uint64_t hi = pHi[q], lo = pLo[q];
-                        if (key_gt(hi, lo, bhi, blo)) { bhi = hi; blo = lo; bi = q; }
-                    }
-                    uint32_t v = (uint32_t)(bhi >> 32);
-                    unsigned m = __ballot_sync(kFullMask, bi >= 0 && v == __reduce_max_sync(kFullMask, v));
-                    if (m & (m - 1)) {
-                        v = ((m >> lane) & 1u) ? (uint32_t)bhi : 0u;
-                        m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
-                        if (m & (m - 1)) {
-                            v = ((m >> lane) & 1u) ? (uint32_t)(blo >> 32) : 0u;
-                            m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
-                            if (m & (m - 1)) {
-                                v = ((m >> lane) & 1u) ? (uint32_t)blo : 0u;
-                                m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
-                            }
-                        }
-                    }
-                    const int win = __ffs(m) - 1;
-                    khi = __shfl_sync(kFullMask, bhi, win); klo = __shfl_sync(kFullMask, blo, win);
-                    const int slot = __shfl_sync(kFullMask, bi, win);
-                    --pn;
-                    if (lane == 0 && slot != pn) { pHi[slot] = pHi[pn]; pLo[slot] = pLo[pn]; }
-                    __syncwarp();
-                    bhi = blo = 0;
-                    for (int q = lane; q < pn; q += 32) {
-                        const uint64_t hi = pHi[q], lo = pLo[q];
-                        if (key_gt(hi, lo, bhi, blo)) { bhi = hi; blo = lo; }
-                    }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o), olo = __shfl_xor_sync(kFullMask, blo, o);
-                        if (key_gt(ohi, olo, bhi, blo)) { bhi = ohi; blo = olo; }
-                    }
-                    pmax_hi = bhi; pmax_lo = blo;
-                } else {                                    // the window's head; the others move up
-                    whi = __shfl_down_sync(kFullMask, whi, 1); wlo = __shfl_down_sync(kFullMask, wlo, 1);
-                    if (lane == 31) { whi = 0; wlo = 0; }
-                    --wn;
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+            const bool trial = pass == 0;
+            if (!trial) {
+                lists_ready_barrier();
+                if (*(volatile int*)&s_pinf) ok = false;
+            }
+            n = 0; Phi = 0.0; theta_prev = theta_first; stopped = false;
+            while ((ok || trial) && !stopped) {
+                // rows n+1 .. n+32, one per lane: a non-zero score word says the node has been popped (no score's ordered
+                // image is zero); the rows that are there form a prefix
+                const int done = trial ? 1 : *(volatile int*)&s_pop_done;   // read before the table: once set, nothing more will come
+                const int j = trial ? B_max + 1 : n + 1 + lane;
+                uint64_t sw = j <= B_max ? *(volatile uint64_t*)&nHi[j] : 0ull;
+                if (trial && lane == 0) sw = ord64(-1.0);
+                const unsigned have = __ballot_sync(kFullMask, sw != 0ull);
+                const int g = have == 0xffffffffu ? 32 : __ffs(~have) - 1;
+                if (g == 0) {
+                    if (done) break;
+                    __nanosleep(20);
+                    continue;
                 }
-                const uint64_t tb = ~klo;
-                const int d = tb_depth(tb), par = tb_parent(tb), r = tb_rank(tb);
-                const int j = ++popped;
-                // ---- the popped node and its two successors (Algorithm 1, lines 12-19) ----
-                const double* arow = a_list + (d - 1) * K;
-                const double Apar = nA[par];
-                const double a_cur = arow[r - 1];
-                const int rs = r < K ? r : K - 1;                       // index of the next sibling (clamped)
-                const int dc = d < L ? d : L - 1;                       // row of the first child (clamped)
-                const double a_sib = arow[rs], a_chi = a_list[dc * K];
-                const int tok_sib = tok_list[(d - 1) * K + rs], tok_chi = tok_list[dc * K];
-                const double S_d = Sd[d], S_c = Sd[dc + 1];
-                const bool has_sib = r < keff[d];
-                const bool has_child = d < Lr;
-                const double A = Apar + a_cur;
-                if (lane == 0) nA[j] = A;
-                if (lane == 1) nHi[j] = khi;
-                if (lane == 2) nLo[j] = klo;
-                if (has_sib) push(ord64((Apar + a_sib) - S_d), ~pack_tiebreak(d, tok_sib, par, r + 1));
-                if (has_child) push(ord64((A + a_chi) - S_c), ~pack_tiebreak(d + 1, tok_chi, j, 1));
-                fsize += (int)has_sib + (int)has_child - 1;
-                ++g;
-            }
-            __syncwarp();                                   // the node records written above are read below
-            if (g == 0) break;
-            // evaluate the group: rows n+1 .. n+g, one per lane
-            const int j = n + 1 + lane;
-            const bool act = lane < g;
-            const double delta = act ? exp(unord64(nHi[j])) : 0.0;
-            double cum = delta;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const double t = __shfl_up_sync(kFullMask, cum, o);
-                if (lane >= o) cum += t;
-            }
-            const double Phi_j = Phi + cum;
-            const double den = act ? C_d + cost_verify(cm, j) : 1.0;
-            const bool bad = !(den > 0.0);
-            const double theta_j = (1.0 + Phi_j) / den;
-            double theta_jm1 = __shfl_up_sync(kFullMask, theta_j, 1);
-            if (lane == 0) theta_jm1 = theta_prev;
-            const bool stop = act && (bad || (!fixed && theta_j <= theta_jm1));
-            const unsigned sm = __ballot_sync(kFullMask, stop);
-            if (p.theta_curve && act && (sm == 0 || lane < __ffs(sm) - 1))
-                p.theta_curve[(int64_t)b * R + j] = theta_j;        // theta*(n) of every accepted n (Prop. 1)
-            if (sm) {
-                const int f = __ffs(sm) - 1;                // rows n+1 .. n+f are accepted
-                if (__shfl_sync(kFullMask, (int)bad, f)) st |= CADD_STATUS_COST_NONPOSITIVE;
-                const double ph = __shfl_sync(kFullMask, Phi_j, f > 0 ? f - 1 : 0);
-                const double th = __shfl_sync(kFullMask, theta_j, f > 0 ? f - 1 : 0);
-                if (f > 0) { Phi = ph; theta_prev = th; }
-                n += f;
-                stopped = true;
-            } else {
-                Phi = __shfl_sync(kFullMask, Phi_j, g - 1);
-                theta_prev = __shfl_sync(kFullMask, theta_j, g - 1);
-                n += g;
+                const bool act = lane < g;
+                const double delta = act ? exp(unord64(sw)) : 0.0;
+                double cum = delta;
+                for (int o = 1; o < g; o <<= 1) {
+                    const double t = __shfl_up_sync(kFullMask, cum, o);
+                    if (lane >= o) cum += t;
+                }
+                const double Phi_j = Phi + cum;
+                const double den = act ? C_d + cv[j] : 1.0;
+                const bool bad = !(den > 0.0);
+                const double theta_j = (1.0 + Phi_j) / den;
+                double theta_jm1 = __shfl_up_sync(kFullMask, theta_j, 1);
+                if (lane == 0) theta_jm1 = theta_prev;
+                const bool stop = act && (bad || (!fixed && theta_j <= theta_jm1));
+                const unsigned sm = __ballot_sync(kFullMask, stop);
+                if (trial) break;
+                if (sm && lane == 0) *(volatile int*)&s_stop = 1;      // first thing: the popping warp need not go on
+                if (p.theta_curve && act && (sm == 0 || lane < __ffs(sm) - 1))
+                    p.theta_curve[(int64_t)b * R + j] = theta_j;        // theta*(n) of every accepted n (Prop. 1)
+                if (sm) {
+                    const int f = __ffs(sm) - 1;                // rows n+1 .. n+f are accepted
+                    if (__shfl_sync(kFullMask, (int)bad, f)) st |= CADD_STATUS_COST_NONPOSITIVE;
+                    const double ph = __shfl_sync(kFullMask, Phi_j, f > 0 ? f - 1 : 0);
+                    const double th = __shfl_sync(kFullMask, theta_j, f > 0 ? f - 1 : 0);
+                    if (f > 0) { Phi = ph; theta_prev = th; }
+                    n += f;
+                    stopped = true;
+                } else {
+                    Phi = __shfl_sync(kFullMask, Phi_j, g - 1);
+                    theta_prev = __shfl_sync(kFullMask, theta_j, g - 1);
+                    n += g;
+                }
             }
         }
-        if (ok && !stopped) st |= (fsize == 0) ? CADD_STATUS_FRONTIER_EXHAUSTED : CADD_STATUS_CAP_HIT;
+        if (ok && !stopped) {
+            while (!*(volatile int*)&s_pop_done) __nanosleep(40);      // (it is set: the loop above only ends that way)
+            st |= (*(volatile int*)&s_fsize_end == 0) ? CADD_STATUS_FRONTIER_EXHAUSTED : CADD_STATUS_CAP_HIT;
+        }
         if (lane == 0) {
-            s_n = n; s_phi = Phi; s_theta = theta_prev; s_theta0 = (den0 > 0.0) ? 1.0 / den0 : 0.0;
+            s_n = n; s_phi = Phi; s_theta = theta_prev; s_theta0 = theta0;
             if (st) atomicOr(&s_status, st);
         }
     }
