@@ -309,7 +309,7 @@ int cadd_build_workspace_bytes(const cadd_build_args* a, size_t* out);
 int cadd_verify_workspace_bytes(const cadd_verify_args* a, size_t* out);
 
 /* Tree construction (Eq. 1, Algorithm 1, Section 3.3).  Asynchronous on `cuda_stream`: two kernels (softmax/top-K
- * over the rows, then expansion + emission), or ONE for small problems (rows of at most 8192 logits, 2 MiB of draft
+ * over the rows, then expansion + emission), or ONE for small problems (rows of at most 2048 logits, 2 MiB of draft
  * logits in all), where the expansion kernel reads the rows itself. */
 int cadd_build_tree(const cadd_build_args* a, void* cuda_stream);
 

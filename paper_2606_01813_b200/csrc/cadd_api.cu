@@ -78,7 +78,7 @@ static BuildPlan plan_build(const cadd_build_args* a, int slots) {
     }
     pl.S = best;
     pl.partial_bytes = (size_t)rows * pl.S * seg_record_stride(pl.KP);
-    pl.lay = expand_layout(a->L, a->K, seg_key_cap(pl.KP), pl.S, a->B_max);
+    pl.lay = expand_layout(a->L, a->K, seg_key_cap(pl.KP), pl.S, a->B_max, 0);
     return pl;
 }
 
@@ -131,13 +131,14 @@ static cudaError_t launch_dependent(bool overlap, void (*kernel)(KArgs...), dim3
 // Small problems are launch-bound: below these sizes tree construction is ONE kernel (the expansion kernel reads the
 // short rows itself, one warp per row) and verification is ONE kernel (one CTA per request: arg-max of its rows, then
 // the walk).  The single-kernel measurement flags and the test hook always take the regular path.
-constexpr int64_t kSmallMaxV = 8192;                 // elements per row
+constexpr int64_t kSmallMaxV = 8192;                 // elements per row (verification)
+constexpr int64_t kSmallBuildMaxV = 2048;            // elements per row (construction: eight staged rows fit in shared memory)
 constexpr int64_t kSmallBuildBytes = 2ll << 20;      // draft logits of the whole call
 constexpr int64_t kSmallVerifyBytes = 4ll << 20;     // target logits the call reads at most
 static bool build_is_small(const cadd_build_args* a) {
     if (a->flags & (CADD_FLAG_ONLY_TOPK | CADD_FLAG_ONLY_EXPAND | CADD_FLAG_TEST_DROP_TILE | CADD_FLAG_REGULAR_PATH)) return false;
     const int64_t es = a->logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
-    return a->V <= kSmallMaxV && (int64_t)a->batch * a->L * a->V * es <= kSmallBuildBytes;
+    return a->V <= kSmallBuildMaxV && (int64_t)a->batch * a->L * a->V * es <= kSmallBuildBytes;
 }
 static bool verify_is_small(const cadd_verify_args* a) {
     if (a->flags & (CADD_VERIFY_ONLY_ARGMAX | CADD_VERIFY_ONLY_WALK | CADD_FLAG_TEST_DROP_TILE | CADD_VERIFY_REGULAR_PATH)) return false;
@@ -147,7 +148,7 @@ static bool verify_is_small(const cadd_verify_args* a) {
 
 // Launches the expansion + emission kernel on the per-row partial records at `partials` (S records per row).
 static int launch_expand(const cadd_build_args* a, int KP, int S, int rec_fmt, const unsigned char* partials, cudaStream_t st, bool overlap) {
-    const ExpandLayout lay = expand_layout(a->L, a->K, rec_key_cap(rec_fmt, KP), S, a->B_max);
+    const ExpandLayout lay = expand_layout(a->L, a->K, rec_key_cap(rec_fmt, KP), S, a->B_max, rec_fmt == kRecDirect ? direct_stage_bytes(a->V, a->logits_dtype) : 0);
     ExpandParams ep;
     ep.batch = a->batch; ep.L = a->L; ep.K = a->K; ep.KP = KP; ep.S = S; ep.B_max = a->B_max; ep.R = a->R;
     ep.rec_fmt = rec_fmt;
@@ -160,13 +161,14 @@ static int launch_expand(const cadd_build_args* a, int KP, int S, int rec_fmt, c
     ep.position_ids = a->position_ids; ep.node_logprob = a->node_logprob; ep.phi = a->phi; ep.theta = a->theta; ep.theta_curve = a->theta_curve;
     ep.mask_bits = a->mask_bits; ep.mask_dense = a->mask_dense; ep.topk_token = a->topk_token;
     ep.topk_logprob = a->topk_logprob; ep.status = a->status;
+    void (*kernel)(ExpandParams) = rec_fmt == kRecDirect ? expand_emit_kernel<true> : expand_emit_kernel<false>;
     if (lay.total > 48 * 1024) {
-        if (cudaFuncSetAttribute(expand_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lay.total) != cudaSuccess) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lay.total) != cudaSuccess) {
             cudaGetLastError();
             return CADD_ERR_LAUNCH;
         }
     }
-    if (launch_dependent(overlap, expand_emit_kernel, dim3((unsigned)a->batch), dim3(kExpandThreads), lay.total, st, ep) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
+    if (launch_dependent(overlap, kernel, dim3((unsigned)a->batch), dim3(kExpandThreads), lay.total, st, ep) != cudaSuccess) { cudaGetLastError(); return CADD_ERR_LAUNCH; }
     return CADD_OK;
 }
 

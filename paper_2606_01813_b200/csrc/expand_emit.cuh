@@ -82,7 +82,10 @@ struct ExpandLayout {
     size_t a_list, lz, S, nHi, nLo, nA, cv, region, tok_list, keff, total;
     int pool_cap;      // entries of the frontier's pool
 };
-__host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap, int S, int B_max) {
+// kRecDirect: bytes of shared memory for one staged row (the row, the up to 15 bytes before it back to a 16-byte boundary,
+// rounded up to whole 16-byte pieces)
+__host__ __device__ inline size_t direct_row_bytes(int64_t V, int dtype) { return (((size_t)V * (dtype == CADD_DTYPE_BF16 ? 2 : 4)) + 31) & ~(size_t)15; }
+__host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap, int S, int B_max, size_t row_bytes) {
     ExpandLayout o;
     const size_t NR = (size_t)B_max + 2;                         // rows 0..B_max, and one that the trial pass writes
     // every pop takes one entry out of the frontier and puts at most two in
@@ -90,17 +93,20 @@ __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap,
     size_t frontier = (size_t)o.pool_cap * (8 + 8);
     size_t scratch = (size_t)kMergeWarps * 2 * S * key_cap * 8;     // phase 0: every key of a row's records, per warp
     size_t region = frontier > scratch ? frontier : scratch;
-    region = (region + 7) & ~(size_t)7;
+    if ((size_t)kMergeWarps * row_bytes > region) region = (size_t)kMergeWarps * row_bytes;   // kRecDirect: a staged row per warp
+    region = (region + 15) & ~(size_t)15;
     size_t p = 0;
-    o.a_list = p;   p += (size_t)L * K * 8;
+    o.a_list = p;   p += ((size_t)L + 1) * K * 8;                 // one row more than there are positions: indices one past
+                                                                 // a list's or the tree's end stay inside (what they read is never used)
     o.lz = p;       p += (size_t)L * 8;
-    o.S = p;        p += ((size_t)L + 1) * 8;
+    o.S = p;        p += ((size_t)L + 2) * 8;
     o.nHi = p;      p += NR * 8;
     o.nLo = p;      p += NR * 8;
     o.nA = p;       p += NR * 8;
     o.cv = p;       p += NR * 8;
+    p = (p + 15) & ~(size_t)15;
     o.region = p;   p += region;
-    o.tok_list = p; p += (size_t)L * K * 4;
+    o.tok_list = p; p += ((size_t)L + 1) * K * 4;
     o.keff = p;     p += ((size_t)L + 2) * 4;
     o.total = (p + 15) & ~(size_t)15;
     return o;
@@ -122,17 +128,42 @@ __device__ __forceinline__ double cost_verify(const CostModel& cm, int n) {
     return cm.q[1] + cm.q[2] * x + cm.q[3] * (x * x);
 }
 
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 // Small problems (a few thousand logits per row): one warp turns one row into the sorted top-K list and log Z by itself
-// (Eq. 1; Algorithm 1, Require), reading the row K + 2 times from L1/L2: the largest finite logit m; then the K best
-// keys one after the other (each the largest key below the one before; keys are unique); then the mass of everything
-// else as fp32 exponentials against the reference exponent ceil(m * log2e) + 1, summed in fp64.  The K best go through
-// the fp64 exponential, as on the large path.  NaN and infinities carry no mass and are flagged.
+// (Eq. 1; Algorithm 1, Require).  The row comes to shared memory in one round trip and is read there twice:
+//   first pass   every lane's largest finite key (and with it the row maximum m), the number of finite logits, flags
+//   bound        the K-th largest of the 32 lanes' maxima: at least K keys are at or above it, so the K best are
+//   second pass  every key at or above the bound goes to a candidate list (a handful for most rows); the mass of all
+//                others is summed as fp32 exponentials against the reference exponent ceil(m * log2e) + 1, in fp64
+//   selection    the candidates are ranked by counting (keys are unique); the K best go through the fp64 exponential, as
+//                on the large path, the others join the mass
+// For K above 32, or if the candidates do not fit, the K best are taken one after the other instead (each the largest
+// key below the one before: K more passes).  NaN and infinities carry no mass and are flagged.
+constexpr int kDirectCandCap = 256;
+__host__ __device__ inline size_t direct_stage_bytes(int64_t V, int dtype) { return direct_row_bytes(V, dtype) + (size_t)kDirectCandCap * 8; }
+
 template <int DT>
-__device__ __forceinline__ void row_lists_warp(const void* row, int64_t V, int K, int32_t* tok_out, double* a_out,
+__device__ __forceinline__ void row_lists_warp(const void* grow, unsigned char* buf, int64_t V, int K, int32_t* tok_out, double* a_out,
                                                double* logZ_out, int32_t* keff_out, uint32_t* flags_out) {
     using E = Elem<DT>;
     const int lane = threadIdx.x & 31;
-    float m = -INFINITY;
+    // whole 16-byte pieces from the boundary at or below the row's start
+    const size_t lead = (size_t)((uintptr_t)grow & 15);
+    const char* g0 = (const char*)grow - lead;
+    const int pieces = (int)((lead + (size_t)V * (DT == CADD_DTYPE_BF16 ? 2 : 4) + 15) >> 4);
+    for (int c = lane; c < pieces; c += 32) cp_async16(buf + 16 * c, g0 + 16 * (size_t)c);
+    cp_async_wait_all();
+    __syncwarp();
+    const void* row = buf + lead;
+    uint64_t* cand = (uint64_t*)(buf + direct_row_bytes(V, DT));
+
+    uint64_t mine = 0;                                       // this lane's largest finite key (0: none)
     uint32_t fl = 0;
     int nfin = 0;
     for (int64_t i = lane; i < V; i += 32) {
@@ -143,34 +174,78 @@ __device__ __forceinline__ void row_lists_warp(const void* row, int64_t V, int K
             if (b == 0x7f800000u) fl |= kPartPosInf;
             continue;
         }
-        m = fmaxf(m, x);
+        mine = max(mine, make_key(x, (uint32_t)i));
         ++nfin;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFullMask, m, o));
     nfin = __reduce_add_sync(kFullMask, nfin);
     fl = __reduce_or_sync(kFullMask, fl);
     const int ke = nfin < K ? nfin : K;
-    uint64_t prev = ~0ull;                                   // above every key
-    for (int r = 0; r < ke; ++r) {
-        uint64_t best = 0;
-        for (int64_t i = lane; i < V; i += 32) {
-            const float x = E::load(row, i);
-            if (fabsf(x) < INFINITY) {
-                const uint64_t key = make_key(x, (uint32_t)i);
-                if (key < prev && key > best) best = key;
-            }
-        }
+    uint64_t top = mine;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(kFullMask, best, o));
-        if (lane == 0) { tok_out[r] = (int32_t)key_id(best); a_out[r] = (double)key_value(best) - (double)m; }
-        prev = best;
-    }
+    for (int o = 16; o > 0; o >>= 1) top = max(top, __shfl_xor_sync(kFullMask, top, o));
+    const float m = nfin > 0 ? key_value(top) : -INFINITY;
     const float negc = m > -INFINITY ? -(ceilf(fminf(m, 2.0e38f) * kLog2eHi) + 1.0f) : 0.0f;
     double acc = 0.0;
-    for (int64_t i = lane; i < V; i += 32) {
-        const float x = E::load(row, i);
-        if (fabsf(x) < INFINITY && (ke == 0 || make_key(x, (uint32_t)i) < prev)) acc += (double)exp2_term(x, negc);
+    bool listed = false;
+    if (K <= 32) {
+        // the K-th largest of the lanes' maxima (0 if fewer lanes than that hold a finite logit: then everything is listed)
+        uint64_t bound = top, left = mine == top ? 0ull : mine;
+        for (int r = 1; r < K; ++r) {
+            uint64_t nx = left;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) nx = max(nx, __shfl_xor_sync(kFullMask, nx, o));
+            bound = nx;
+            if (left == nx) left = 0ull;
+        }
+        int nc = 0;
+        for (int64_t i0 = 0; i0 < V; i0 += 32) {
+            const int64_t i = i0 + lane;
+            const float x = i < V ? E::load(row, i) : INFINITY;
+            const bool fin = fabsf(x) < INFINITY;
+            const uint64_t key = fin ? make_key(x, (uint32_t)i) : 0ull;
+            const bool is_cand = fin && key >= bound;
+            const unsigned cm = __ballot_sync(kFullMask, is_cand);
+            if (is_cand) {
+                const int at = nc + __popc(cm & ((1u << lane) - 1u));
+                if (at < kDirectCandCap) cand[at] = key;
+            } else if (fin) {
+                acc += (double)exp2_term(x, negc);
+            }
+            nc += __popc(cm);
+        }
+        __syncwarp();
+        if (nc <= kDirectCandCap) {
+            listed = true;
+            for (int q = lane; q < nc; q += 32) {
+                const uint64_t k = cand[q];
+                int rank = 0;
+                for (int r = 0; r < nc; ++r) rank += cand[r] > k;
+                if (rank < K) { tok_out[rank] = (int32_t)key_id(k); a_out[rank] = (double)key_value(k) - (double)m; }
+                else acc += (double)exp2_term(key_value(k), negc);
+            }
+        }
+    }
+    if (!listed) {
+        acc = 0.0;
+        uint64_t prev = ~0ull;                               // above every key
+        for (int r = 0; r < ke; ++r) {
+            uint64_t best = 0;
+            for (int64_t i = lane; i < V; i += 32) {
+                const float x = E::load(row, i);
+                if (fabsf(x) < INFINITY) {
+                    const uint64_t key = make_key(x, (uint32_t)i);
+                    if (key < prev && key > best) best = key;
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(kFullMask, best, o));
+            if (lane == 0) { tok_out[r] = (int32_t)key_id(best); a_out[r] = (double)key_value(best) - (double)m; }
+            prev = best;
+        }
+        for (int64_t i = lane; i < V; i += 32) {
+            const float x = E::load(row, i);
+            if (fabsf(x) < INFINITY && (ke == 0 || make_key(x, (uint32_t)i) < prev)) acc += (double)exp2_term(x, negc);
+        }
     }
     __syncwarp();
     double zsum = lane < ke ? exp(a_out[lane]) : 0.0;
@@ -182,18 +257,16 @@ __device__ __forceinline__ void row_lists_warp(const void* row, int64_t V, int K
     __syncwarp();
 }
 
-__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 // Barrier 1 of the CTA: every warp arrives once, the merging warps when their lists are complete, the popping and the
 // evaluating warp before their real pass.
 __device__ __forceinline__ void lists_ready_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kExpandThreads) : "memory"); }
 
+// kDirect: the kernel for p.rec_fmt == kRecDirect (its own instantiation, so that neither carries the other's phase 0)
+template <bool kDirect>
 __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandParams p) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int key_cap = rec_key_cap(p.rec_fmt, p.KP);
-    const ExpandLayout lay = expand_layout(p.L, p.K, key_cap, p.S, p.B_max);
+    const ExpandLayout lay = expand_layout(p.L, p.K, key_cap, p.S, p.B_max, kDirect ? direct_stage_bytes(p.V, p.logits_dtype) : 0);
     double* a_list = (double*)(smem + lay.a_list);
     double* lz = (double*)(smem + lay.lz);
     double* Sd = (double*)(smem + lay.S);
@@ -227,7 +300,7 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
     // ---------------- phase 0: the sorted top-K list and log Z of every live position ----------------
     grid_dependency_wait();                                 // the records are the previous kernel's
     const bool emit = (p.flags & CADD_FLAG_EMIT_TOPK) != 0;
-    if (p.rec_fmt == kRecDirect) {
+    if constexpr (kDirect) {
         // small problem: there are no records, one warp per position reads the (short) row itself
         for (int i = warp; i < L; i += kMergeWarps) {
             int32_t* out_tok = p.topk_token ? p.topk_token + ((int64_t)b * L + i) * K : nullptr;
@@ -241,9 +314,10 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             }
             const size_t es = p.logits_dtype == CADD_DTYPE_BF16 ? 2 : 4;
             const char* row = (const char*)p.logits + ((int64_t)b * p.stride_b + (int64_t)i * p.stride_l) * (int64_t)es;
+            unsigned char* stage = smem + lay.region + (size_t)warp * direct_stage_bytes(p.V, p.logits_dtype);
             uint32_t fl;
-            if (p.logits_dtype == CADD_DTYPE_BF16) row_lists_warp<CADD_DTYPE_BF16>(row, p.V, K, tok_list + i * K, a_list + i * K, &lz[i], &keff[i + 1], &fl);
-            else row_lists_warp<CADD_DTYPE_FP32>(row, p.V, K, tok_list + i * K, a_list + i * K, &lz[i], &keff[i + 1], &fl);
+            if (p.logits_dtype == CADD_DTYPE_BF16) row_lists_warp<CADD_DTYPE_BF16>(row, stage, p.V, K, tok_list + i * K, a_list + i * K, &lz[i], &keff[i + 1], &fl);
+            else row_lists_warp<CADD_DTYPE_FP32>(row, stage, p.V, K, tok_list + i * K, a_list + i * K, &lz[i], &keff[i + 1], &fl);
             fl = __shfl_sync(kFullMask, fl, 0);
             const int ke = keff[i + 1];
             if (lane == 0) {
@@ -448,10 +522,9 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             int popped = 0;
             int stop_now = 0;
             while (ok && popped < limit && (wn | pn) != 0 && !stop_now) {
-                stop_now = *(volatile int*)&s_stop;         // looked at when this pop is over
                 // ---- the best entry of the frontier ----
                 uint64_t khi = __shfl_sync(kFullMask, whi, 0), klo = __shfl_sync(kFullMask, wlo, 0);
-                const bool from_pool = wn == 0 || key_gt(pmax_hi, pmax_lo, khi, klo);
+                const bool from_pool = key_gt(pmax_hi, pmax_lo, khi, klo);   // (an empty window's head is (0,0))
                 if (from_pool) {
                     // rare: the best entry sits in the pool.  Find it (lanes scan stripes of the pool, then the warp's
                     // arg-max 32 bits at a time), fill its slot with the pool's last entry, and find the new best.
@@ -499,25 +572,25 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 const int d = tb_depth(tb), par = tb_parent(tb), r = tb_rank(tb);
                 const int j = trial ? B_max + 1 : popped + 1;
                 ++popped;
+                *(volatile uint64_t*)&nHi[j] = khi;                     // at once: the evaluating warp waits for this word
                 // ---- the popped node and its two successors (Algorithm 1, lines 12-19) ----
                 const double* arow = a_list + (d - 1) * K;
                 const double Apar = nA[par];
                 const double a_cur = arow[r - 1];
-                const int rs = r < K ? r : K - 1;                       // index of the next sibling (clamped)
-                const int dc = d < L ? d : L - 1;                       // row of the first child (clamped)
-                const double a_sib = arow[rs], a_chi = a_list[dc * K];
-                const int tok_sib = tok_list[(d - 1) * K + rs], tok_chi = tok_list[dc * K];
-                const double S_d = Sd[d], S_c = Sd[dc + 1];
+                // (the next sibling and the first child are read whether they exist or not: the arrays have room)
+                const double a_sib = arow[r], a_chi = a_list[d * K];
+                const int tok_sib = tok_list[(d - 1) * K + r], tok_chi = tok_list[d * K];
+                const double S_d = Sd[d], S_c = Sd[d + 1];
                 const bool has_sib = r < keff[d];
                 const bool has_child = d < Lr;
                 const double A = Apar + a_cur;
                 nA[j] = A;
                 nLo[j] = klo;
-                *(volatile uint64_t*)&nHi[j] = khi;                     // the evaluating warp's signal that node j exists
                 const uint64_t shi = has_sib ? ord64((Apar + a_sib) - S_d) : 0ull;
                 const uint64_t slo = has_sib ? ~pack_tiebreak(d, tok_sib, par, r + 1) : 0ull;
                 const uint64_t chi = has_child ? ord64((A + a_chi) - S_c) : 0ull;
                 const uint64_t clo = has_child ? ~pack_tiebreak(d + 1, tok_chi, j, 1) : 0ull;
+                stop_now = *(volatile int*)&s_stop;                     // looked at when this pop is over
                 if (from_pool) {                                        // the window kept its head: one entry after the other
                     if (has_sib) push(shi, slo);
                     if (has_child) push(chi, clo);
@@ -525,24 +598,21 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 }
                 // The head leaves; a (the better of the two successors) and b enter; a missing one is (0,0), which lands on
                 // the first empty lane.  Old entries ahead of a move up one lane, those between a and b stay, those behind b
-                // move down one.  Every successor is behind its node in the order, so the head counts in both ballots.
+                // move down one: one gathering shuffle.  Every successor is behind its node in the order, so the head counts in both ballots.
                 const bool sib_first = key_gt(shi, slo, chi, clo);
                 const uint64_t ahi = sib_first ? shi : chi, alo = sib_first ? slo : clo;
                 const uint64_t bhi = sib_first ? chi : shi, blo = sib_first ? clo : slo;
                 const int pa = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, ahi, alo))) - 1;
                 const int pb = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, bhi, blo)));
-                uint64_t nhi = __shfl_down_sync(kFullMask, whi, 1), nlo = __shfl_down_sync(kFullMask, wlo, 1);   // old[lane + 1]
-                const uint64_t phi_ = __shfl_up_sync(kFullMask, whi, 1), plo_ = __shfl_up_sync(kFullMask, wlo, 1); // old[lane - 1]
-                if (lane == 31) { nhi = 0; nlo = 0; }
+                const int src = lane + (lane < pa ? 1 : 0) - (lane > pb ? 1 : 0);      // whose old entry this lane takes
+                const uint64_t ghi = __shfl_sync(kFullMask, whi, src), glo = __shfl_sync(kFullMask, wlo, src);
                 if (wn == 32 && bhi != 0ull) {                          // 33 entries: the one that does not fit goes to the pool
                     const uint64_t lhi = __shfl_sync(kFullMask, whi, 31), llo = __shfl_sync(kFullMask, wlo, 31);
                     if (pb == 32) to_pool(bhi, blo); else to_pool(lhi, llo);
                 }
                 wn = min(32, wn - 1 + (int)(ahi != 0ull) + (int)(bhi != 0ull));
-                if (lane < pa) { whi = nhi; wlo = nlo; }
-                else if (lane == pa) { whi = ahi; wlo = alo; }
-                else if (lane == pb) { whi = bhi; wlo = blo; }
-                else if (lane > pb) { whi = phi_; wlo = plo_; }
+                whi = lane == pa ? ahi : (lane == pb ? bhi : ghi);
+                wlo = lane == pa ? alo : (lane == pb ? blo : glo);
             }
             __syncwarp();
             if (!trial && lane == 0) { s_fsize_end = wn + pn; __threadfence_block(); *(volatile int*)&s_pop_done = 1; }
@@ -606,51 +676,37 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 if (*(volatile int*)&s_pinf) ok = false;
             }
             n = 0; Phi = 0.0; theta_prev = theta_first; stopped = false;
+            // one node after the other, as soon as its score word is there (no score's ordered image is zero); every
+            // lane does the same arithmetic, so nothing has to be exchanged
+            int j = trial ? B_max + 1 : 1;
             while ((ok || trial) && !stopped) {
-                // rows n+1 .. n+32, one per lane: a non-zero score word says the node has been popped (no score's ordered
-                // image is zero); the rows that are there form a prefix
-                const int done = trial ? 1 : *(volatile int*)&s_pop_done;   // read before the table: once set, nothing more will come
-                const int j = trial ? B_max + 1 : n + 1 + lane;
-                uint64_t sw = j <= B_max ? *(volatile uint64_t*)&nHi[j] : 0ull;
-                if (trial && lane == 0) sw = ord64(-1.0);
-                const unsigned have = __ballot_sync(kFullMask, sw != 0ull);
-                const int g = have == 0xffffffffu ? 32 : __ffs(~have) - 1;
-                if (g == 0) {
-                    if (done) break;
-                    __nanosleep(20);
-                    continue;
+                uint64_t sw;
+                if (trial) sw = ord64(-1.0);
+                else {
+                    if (j > B_max) break;                               // the cap: every node was worth its cost
+                    sw = *(volatile uint64_t*)&nHi[j];
+                    if (sw == 0ull) {
+                        if (!*(volatile int*)&s_pop_done) continue;     // not popped yet
+                        __threadfence_block();
+                        sw = *(volatile uint64_t*)&nHi[j];              // the popping warp is through: what is there now is final
+                        if (sw == 0ull) break;
+                    }
                 }
-                const bool act = lane < g;
-                const double delta = act ? exp(unord64(sw)) : 0.0;
-                double cum = delta;
-                for (int o = 1; o < g; o <<= 1) {
-                    const double t = __shfl_up_sync(kFullMask, cum, o);
-                    if (lane >= o) cum += t;
-                }
-                const double Phi_j = Phi + cum;
-                const double den = act ? C_d + cv[j] : 1.0;
+                const double Phi_j = Phi + exp(unord64(sw));
+                const double den = C_d + cv[j];
                 const bool bad = !(den > 0.0);
                 const double theta_j = (1.0 + Phi_j) / den;
-                double theta_jm1 = __shfl_up_sync(kFullMask, theta_j, 1);
-                if (lane == 0) theta_jm1 = theta_prev;
-                const bool stop = act && (bad || (!fixed && theta_j <= theta_jm1));
-                const unsigned sm = __ballot_sync(kFullMask, stop);
+                const bool stop = bad || (!fixed && theta_j <= theta_prev);
                 if (trial) break;
-                if (sm && lane == 0) *(volatile int*)&s_stop = 1;      // first thing: the popping warp need not go on
-                if (p.theta_curve && act && (sm == 0 || lane < __ffs(sm) - 1))
-                    p.theta_curve[(int64_t)b * R + j] = theta_j;        // theta*(n) of every accepted n (Prop. 1)
-                if (sm) {
-                    const int f = __ffs(sm) - 1;                // rows n+1 .. n+f are accepted
-                    if (__shfl_sync(kFullMask, (int)bad, f)) st |= CADD_STATUS_COST_NONPOSITIVE;
-                    const double ph = __shfl_sync(kFullMask, Phi_j, f > 0 ? f - 1 : 0);
-                    const double th = __shfl_sync(kFullMask, theta_j, f > 0 ? f - 1 : 0);
-                    if (f > 0) { Phi = ph; theta_prev = th; }
-                    n += f;
+                if (stop) {
+                    if (lane == 0) *(volatile int*)&s_stop = 1;         // the popping warp need not go on
+                    if (bad) st |= CADD_STATUS_COST_NONPOSITIVE;
                     stopped = true;
                 } else {
-                    Phi = __shfl_sync(kFullMask, Phi_j, g - 1);
-                    theta_prev = __shfl_sync(kFullMask, theta_j, g - 1);
-                    n += g;
+                    if (p.theta_curve && lane == 0) p.theta_curve[(int64_t)b * R + j] = theta_j;   // theta*(n) of every accepted n (Prop. 1)
+                    Phi = Phi_j; theta_prev = theta_j;
+                    n = j;
+                    ++j;
                 }
             }
         }
