@@ -66,20 +66,21 @@ constexpr int kMergeWarps = 8;             // sixteen half-warps: one per draft 
 constexpr int kExpandWarps = kMergeWarps + 2;      // and the two warps of the expansion proper
 constexpr int kExpandThreads = kExpandWarps * 32;
 
-// Tie-break half of a frontier / node key.  Smaller packed value = earlier in the pop order
-// (depth, then token id, then parent row); the rank within the position's top-K list rides along in
-// the low bits (it never decides: depth, token and parent already identify a node).
-__device__ __forceinline__ uint64_t pack_tiebreak(int depth, int token, int parent, int rank) {
-    return ((uint64_t)depth << 50) | ((uint64_t)(uint32_t)token << 19) | ((uint64_t)parent << 7) | (uint64_t)rank;
+// A frontier entry / node besides its score, in 30 bits, most significant first: depth - 1 (6 bits), the token's place
+// among the tokens of its position's top-K list in token-id order (6 bits), parent row (12 bits), rank - 1 in the
+// list (6 bits).  Between entries of equal score a SMALLER word comes first: that is (depth, token id, parent row) in this
+// order, because two entries of one depth compare their tokens like the tokens' places; the rank never decides (depth,
+// token and parent already identify a node).
+__device__ __forceinline__ uint32_t pack_meta(int depth, int place, int parent, int rank) {
+    return ((uint32_t)(depth - 1) << 24) | ((uint32_t)place << 18) | ((uint32_t)parent << 6) | (uint32_t)(rank - 1);
 }
-__device__ __forceinline__ int tb_depth(uint64_t tb) { return (int)(tb >> 50); }
-__device__ __forceinline__ int tb_token(uint64_t tb) { return (int)((tb >> 19) & 0x7fffffffu); }
-__device__ __forceinline__ int tb_parent(uint64_t tb) { return (int)((tb >> 7) & 0xfffu); }
-__device__ __forceinline__ int tb_rank(uint64_t tb) { return (int)(tb & 0x7fu); }
+__device__ __forceinline__ int me_depth(uint32_t me) { return (int)(me >> 24) + 1; }
+__device__ __forceinline__ int me_parent(uint32_t me) { return (int)((me >> 6) & 0xfffu); }
+__device__ __forceinline__ int me_rank(uint32_t me) { return (int)(me & 0x3fu) + 1; }
 
 // Dynamic shared memory layout of the expansion kernel (byte offsets), same arithmetic on host and device.
 struct ExpandLayout {
-    size_t a_list, lz, S, nHi, nLo, nA, cv, region, tok_list, keff, total;
+    size_t a_list, lz, S, nHi, nMe, nA, cv, region, tok_list, keff, place, total;
     int pool_cap;      // entries of the frontier's pool
 };
 // kRecDirect: bytes of shared memory for one staged row (the row, the up to 15 bytes before it back to a 16-byte boundary,
@@ -90,7 +91,7 @@ __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap,
     const size_t NR = (size_t)B_max + 2;                         // rows 0..B_max, and one that the trial pass writes
     // every pop takes one entry out of the frontier and puts at most two in
     o.pool_cap = B_max + 2;
-    size_t frontier = (size_t)o.pool_cap * (8 + 8);
+    size_t frontier = (size_t)o.pool_cap * (8 + 4);
     size_t scratch = (size_t)kMergeWarps * 2 * S * key_cap * 8;     // phase 0: every key of a row's records, per warp
     size_t region = frontier > scratch ? frontier : scratch;
     if ((size_t)kMergeWarps * row_bytes > region) region = (size_t)kMergeWarps * row_bytes;   // kRecDirect: a staged row per warp
@@ -101,13 +102,14 @@ __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap,
     o.lz = p;       p += (size_t)L * 8;
     o.S = p;        p += ((size_t)L + 2) * 8;
     o.nHi = p;      p += NR * 8;
-    o.nLo = p;      p += NR * 8;
+    o.nMe = p;      p += ((NR * 4) + 7) & ~(size_t)7;
     o.nA = p;       p += NR * 8;
     o.cv = p;       p += NR * 8;
     p = (p + 15) & ~(size_t)15;
     o.region = p;   p += region;
     o.tok_list = p; p += ((size_t)L + 1) * K * 4;
     o.keff = p;     p += ((size_t)L + 2) * 4;
+    o.place = p;    p += ((size_t)L + 1) * K;
     o.total = (p + 15) & ~(size_t)15;
     return o;
 }
@@ -271,13 +273,14 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
     double* lz = (double*)(smem + lay.lz);
     double* Sd = (double*)(smem + lay.S);
     uint64_t* nHi = (uint64_t*)(smem + lay.nHi);          // ordered image of the node's score sigma
-    uint64_t* nLo = (uint64_t*)(smem + lay.nLo);          // ~pack_tiebreak(depth, token, parent, rank)
+    uint32_t* nMe = (uint32_t*)(smem + lay.nMe);          // pack_meta(depth, parent row, rank)
     int32_t* tok_list = (int32_t*)(smem + lay.tok_list);
     int32_t* keff = (int32_t*)(smem + lay.keff);          // keff[d], d = 1..L
+    uint8_t* place = smem + lay.place;                    // of each listed token among its list's tokens, by token id
     double* nA = (double*)(smem + lay.nA);                // the node's sum of (logit - row max) along its path
     double* cv = (double*)(smem + lay.cv);                // C_v(n), n = 0..B_max
     uint64_t* pHi = (uint64_t*)(smem + lay.region);       // the frontier's pool (see phase 2), in no order
-    uint64_t* pLo = pHi + lay.pool_cap;
+    uint32_t* pMe = (uint32_t*)(pHi + lay.pool_cap);
 
     __shared__ int s_status, s_pinf, s_n;
     __shared__ int s_cost_ok, s_pop_done, s_stop, s_fsize_end;   // between the popping warp and the evaluating warp
@@ -320,6 +323,12 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             else row_lists_warp<CADD_DTYPE_FP32>(row, stage, p.V, K, tok_list + i * K, a_list + i * K, &lz[i], &keff[i + 1], &fl);
             fl = __shfl_sync(kFullMask, fl, 0);
             const int ke = keff[i + 1];
+            for (int k = lane; k < ke; k += 32) {
+                const int t = tok_list[i * K + k];
+                int c = 0;
+                for (int q = 0; q < ke; ++q) c += tok_list[i * K + q] < t;
+                place[i * K + k] = (uint8_t)c;
+            }
             if (lane == 0) {
                 int st = 0;
                 if (fl & kPartNonfinite) st |= CADD_STATUS_NONFINITE_INPUT;
@@ -430,6 +439,12 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
         const double logZ = log(zsum);
         const int ke = n < K ? n : K;
         __syncwarp();
+        for (int k = hl; k < ke; k += 16) {
+            const int t = tok_list[i * K + k];
+            int c = 0;
+            for (int q = 0; q < ke; ++q) c += tok_list[i * K + q] < t;
+            place[i * K + k] = (uint8_t)c;
+        }
         if (hl == 0 && live) {
             keff[i + 1] = ke;
             lz[i] = logZ;
@@ -479,97 +494,100 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             bool ok = *(volatile int*)&s_cost_ok != 0 && *(volatile int*)&s_pinf == 0;
             if (trial) { ok = true; Lr = 1; }
             nA[0] = 0.0;
-            nHi[0] = ord64(0.0); nLo[0] = ~0ull;
+            nHi[0] = ord64(0.0); nMe[0] = 0u;
             __syncwarp();
             // The frontier (Algorithm 1's heap) in two parts.  The WINDOW is its best entries, at most 32, sorted best
-            // first over the lanes of the warp (lane i holds the i-th best; a key of (0,0) is an empty lane: every real key
-            // is larger).  The POOL, in shared memory and in no order, holds what did not fit: an entry goes there only if
-            // the window is full and all of its entries are better, or by falling off the window's end.  pmax is the
-            // best key of the pool.  A pop takes the window's head unless the pool's best beats it (or the window is empty).
-            // In the usual case (the head is popped) the window changes once per pop: the head leaves and the node's next
-            // sibling and first child enter, each lane taking its new entry from its old one or a neighbour's according to
-            // two ballots on the old window.  The parent's sum A, needed for the successors, is read from the node table
-            // instead of travelling with the entry.  All lanes hold the same scalars and write the same values to the node
-            // table and the pool, so a lane only ever reads back what it has written itself.
-            uint64_t whi = 0, wlo = 0;                          // this lane's window entry
+            // first over the lanes of the warp: lane i holds the i-th best as the ordered image of its score and a 32-bit
+            // word (depth, place of its token, parent row, rank: see pack_meta); a score word of 0 is an empty lane (no
+            // score's image is 0).  Entry A comes before entry B if its score word is larger or, at equal scores, its second
+            // word is smaller: the total order (score, depth, token id, parent row).  The POOL, in shared memory and in no
+            // order, holds what did not fit: an entry goes there only if the window is full and all of its entries are
+            // better, or by falling off the window's end; (pmax_hi, pmax_me) is the pool's best.  A pop takes the window's
+            // head unless the pool's best comes before it.  In the usual case (the head is popped) the window changes once
+            // per pop: the head leaves and the node's next sibling and first child enter, each lane taking its new entry
+            // from its old one or a neighbour's according to two ballots on the old window.  The parent's sum A is read
+            // from the node table instead of travelling with the entry.  All lanes hold the same scalars and write the same
+            // values to the node table and the pool, so a lane only ever reads back what it has written itself.
+            uint64_t whi = 0;                                   // this lane's window entry
+            uint32_t wme = 0;
             int wn = 0;                                         // entries in the window
             int pn = 0;                                         // entries in the pool
-            uint64_t pmax_hi = 0, pmax_lo = 0;
-            auto key_gt = [](uint64_t ahi, uint64_t alo, uint64_t bhi, uint64_t blo) { return ahi > bhi || (ahi == bhi && alo > blo); };
-            auto to_pool = [&](uint64_t khi, uint64_t klo) {
-                pHi[pn] = khi; pLo[pn] = klo;
-                if (key_gt(khi, klo, pmax_hi, pmax_lo)) { pmax_hi = khi; pmax_lo = klo; }
+            uint64_t pmax_hi = 0;
+            uint32_t pmax_me = 0;
+            auto before = [](uint64_t ahi, uint32_t ame, uint64_t bhi, uint32_t bme) { return ahi > bhi || (ahi == bhi && ame < bme); };
+            auto to_pool = [&](uint64_t khi, uint32_t kme) {
+                pHi[pn] = khi; pMe[pn] = kme;
+                if (before(khi, kme, pmax_hi, pmax_me)) { pmax_hi = khi; pmax_me = kme; }
                 ++pn;
             };
-            // a new entry joins the frontier (the general form: any state of the window)
-            auto push = [&](uint64_t khi, uint64_t klo) {
-                const int pos = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, khi, klo)));   // window entries that stay ahead of it
+            // a new entry joins the frontier (the general form: any state of the window, full comparisons)
+            auto push = [&](uint64_t khi, uint32_t kme) {
+                const int pos = __popc(__ballot_sync(kFullMask, before(whi, wme, khi, kme)));   // window entries that stay ahead of it
                 if (pos >= 32) {                                // a full window of better entries: to the pool
-                    to_pool(khi, klo);
+                    to_pool(khi, kme);
                     return;
                 }
-                if (wn == 32) to_pool(__shfl_sync(kFullMask, whi, 31), __shfl_sync(kFullMask, wlo, 31));   // the last entry makes room
+                if (wn == 32) to_pool(__shfl_sync(kFullMask, whi, 31), __shfl_sync(kFullMask, wme, 31));   // the last entry makes room
                 else ++wn;
-                const uint64_t uhi = __shfl_up_sync(kFullMask, whi, 1), ulo = __shfl_up_sync(kFullMask, wlo, 1);
-                if (lane > pos) { whi = uhi; wlo = ulo; }
-                else if (lane == pos) { whi = khi; wlo = klo; }
+                const uint64_t uhi = __shfl_up_sync(kFullMask, whi, 1);
+                const uint32_t ume = __shfl_up_sync(kFullMask, wme, 1);
+                if (lane > pos) { whi = uhi; wme = ume; }
+                else if (lane == pos) { whi = khi; wme = kme; }
             };
-            if (trial) push(ord64(-1.0), ~pack_tiebreak(1, 0, 0, 1));
+            if (trial) push(ord64(-1.0), pack_meta(1, 0, 0, 1));
             else if (ok && Lr >= 1)                             // Algorithm 1, line 3: the heap starts with node (1)
-                push(ord64(a_list[0] - Sd[1]), ~pack_tiebreak(1, tok_list[0], 0, 1));
+                push(ord64(a_list[0] - Sd[1]), pack_meta(1, place[0], 0, 1));
             const int limit = trial ? 1 : B_max;
 
             int popped = 0;
             int stop_now = 0;
             while (ok && popped < limit && (wn | pn) != 0 && !stop_now) {
                 // ---- the best entry of the frontier ----
-                uint64_t khi = __shfl_sync(kFullMask, whi, 0), klo = __shfl_sync(kFullMask, wlo, 0);
-                const bool from_pool = key_gt(pmax_hi, pmax_lo, khi, klo);   // (an empty window's head is (0,0))
-                if (from_pool) {
-                    // rare: the best entry sits in the pool.  Find it (lanes scan stripes of the pool, then the warp's
-                    // arg-max 32 bits at a time), fill its slot with the pool's last entry, and find the new best.
+                uint64_t khi = __shfl_sync(kFullMask, whi, 0);
+                uint32_t kme = __shfl_sync(kFullMask, wme, 0);
+                const bool general = before(pmax_hi, pmax_me, khi, kme);   // the pool holds the best entry (always, if the window is empty)
+                bool head_popped = true;
+                if (general) {
+                    // rare.  The pool's best under the total order: lanes scan stripes of the pool, then a butterfly.
                     __syncwarp();
-                    uint64_t bhi = 0, blo = 0;
+                    uint64_t bhi = 0;
+                    uint32_t bme = 0;
                     int bi = -1;
                     for (int q = lane; q < pn; q += 32) {
-                        const uint64_t hi = pHi[q], lo = pLo[q];
-                        if (key_gt(hi, lo, bhi, blo)) { bhi = hi; blo = lo; bi = q; }
-                    }
-                    uint32_t v = (uint32_t)(bhi >> 32);
-                    unsigned m = __ballot_sync(kFullMask, bi >= 0 && v == __reduce_max_sync(kFullMask, v));
-                    if (m & (m - 1)) {
-                        v = ((m >> lane) & 1u) ? (uint32_t)bhi : 0u;
-                        m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
-                        if (m & (m - 1)) {
-                            v = ((m >> lane) & 1u) ? (uint32_t)(blo >> 32) : 0u;
-                            m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
-                            if (m & (m - 1)) {
-                                v = ((m >> lane) & 1u) ? (uint32_t)blo : 0u;
-                                m &= __ballot_sync(kFullMask, v == __reduce_max_sync(kFullMask, v));
-                            }
-                        }
-                    }
-                    const int win = __ffs(m) - 1;
-                    khi = __shfl_sync(kFullMask, bhi, win); klo = __shfl_sync(kFullMask, blo, win);
-                    const int slot = __shfl_sync(kFullMask, bi, win);
-                    --pn;
-                    __syncwarp();
-                    if (slot != pn) { const uint64_t lhi = pHi[pn], llo = pLo[pn]; __syncwarp(); pHi[slot] = lhi; pLo[slot] = llo; }
-                    __syncwarp();
-                    bhi = blo = 0;
-                    for (int q = lane; q < pn; q += 32) {
-                        const uint64_t hi = pHi[q], lo = pLo[q];
-                        if (key_gt(hi, lo, bhi, blo)) { bhi = hi; blo = lo; }
+                        const uint64_t hi = pHi[q];
+                        const uint32_t me = pMe[q];
+                        if (before(hi, me, bhi, bme)) { bhi = hi; bme = me; bi = q; }
                     }
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) {
-                        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o), olo = __shfl_xor_sync(kFullMask, blo, o);
-                        if (key_gt(ohi, olo, bhi, blo)) { bhi = ohi; blo = olo; }
+                        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o);
+                        const uint32_t ome = __shfl_xor_sync(kFullMask, bme, o);
+                        const int oi = __shfl_xor_sync(kFullMask, bi, o);
+                        if (before(ohi, ome, bhi, bme)) { bhi = ohi; bme = ome; bi = oi; }
                     }
-                    pmax_hi = bhi; pmax_lo = blo;
+                    if (bi >= 0 && before(bhi, bme, khi, kme)) {        // it beats the window's head: take it out of the pool
+                        head_popped = false;
+                        khi = bhi; kme = bme;
+                        --pn;
+                        __syncwarp();
+                        if (bi != pn) { const uint64_t lhi = pHi[pn]; const uint32_t lme = pMe[pn]; __syncwarp(); pHi[bi] = lhi; pMe[bi] = lme; }
+                        __syncwarp();
+                        bhi = 0; bme = 0;
+                        for (int q = lane; q < pn; q += 32) {
+                            const uint64_t hi = pHi[q];
+                            const uint32_t me = pMe[q];
+                            if (before(hi, me, bhi, bme)) { bhi = hi; bme = me; }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o);
+                            const uint32_t ome = __shfl_xor_sync(kFullMask, bme, o);
+                            if (before(ohi, ome, bhi, bme)) { bhi = ohi; bme = ome; }
+                        }
+                        pmax_hi = bhi; pmax_me = bme;
+                    }
                 }
-                const uint64_t tb = ~klo;
-                const int d = tb_depth(tb), par = tb_parent(tb), r = tb_rank(tb);
+                const int d = me_depth(kme), par = me_parent(kme), r = me_rank(kme);
                 const int j = trial ? B_max + 1 : popped + 1;
                 ++popped;
                 *(volatile uint64_t*)&nHi[j] = khi;                     // at once: the evaluating warp waits for this word
@@ -579,40 +597,49 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 const double a_cur = arow[r - 1];
                 // (the next sibling and the first child are read whether they exist or not: the arrays have room)
                 const double a_sib = arow[r], a_chi = a_list[d * K];
-                const int tok_sib = tok_list[(d - 1) * K + r], tok_chi = tok_list[d * K];
                 const double S_d = Sd[d], S_c = Sd[d + 1];
                 const bool has_sib = r < keff[d];
+                const uint32_t pl_sib = place[(d - 1) * K + r], pl_chi = place[d * K];
                 const bool has_child = d < Lr;
                 const double A = Apar + a_cur;
                 nA[j] = A;
-                nLo[j] = klo;
+                nMe[j] = kme;
                 const uint64_t shi = has_sib ? ord64((Apar + a_sib) - S_d) : 0ull;
-                const uint64_t slo = has_sib ? ~pack_tiebreak(d, tok_sib, par, r + 1) : 0ull;
+                const uint32_t sme = has_sib ? ((kme & 0x3f03ffc0u) | (pl_sib << 18) | (uint32_t)r) : 0u;   // same depth and parent, next rank
                 const uint64_t chi = has_child ? ord64((A + a_chi) - S_c) : 0ull;
-                const uint64_t clo = has_child ? ~pack_tiebreak(d + 1, tok_chi, j, 1) : 0ull;
+                const uint32_t cme = has_child ? (((uint32_t)d << 24) | (pl_chi << 18) | ((uint32_t)j << 6)) : 0u;   // pack_meta(d + 1, place, j, 1)
                 stop_now = *(volatile int*)&s_stop;                     // looked at when this pop is over
-                if (from_pool) {                                        // the window kept its head: one entry after the other
-                    if (has_sib) push(shi, slo);
-                    if (has_child) push(chi, clo);
+                // a is the better of the two successors (equal scores: the sibling, which is less deep), b the other; a
+                // missing one is all zero
+                const bool sib_first = shi >= chi;
+                const uint64_t ahi = sib_first ? shi : chi, bhi = sib_first ? chi : shi;
+                const uint32_t ame = sib_first ? sme : cme, bme = sib_first ? cme : sme;
+                if (general) {                                          // one entry after the other
+                    if (head_popped) {
+                        whi = __shfl_down_sync(kFullMask, whi, 1); wme = __shfl_down_sync(kFullMask, wme, 1);
+                        if (lane == 31) { whi = 0; wme = 0; }
+                        --wn;
+                    }
+                    if (ahi != 0ull) push(ahi, ame);
+                    if (bhi != 0ull) push(bhi, bme);
                     continue;
                 }
-                // The head leaves; a (the better of the two successors) and b enter; a missing one is (0,0), which lands on
-                // the first empty lane.  Old entries ahead of a move up one lane, those between a and b stay, those behind b
-                // move down one: one gathering shuffle.  Every successor is behind its node in the order, so the head counts in both ballots.
-                const bool sib_first = key_gt(shi, slo, chi, clo);
-                const uint64_t ahi = sib_first ? shi : chi, alo = sib_first ? slo : clo;
-                const uint64_t bhi = sib_first ? chi : shi, blo = sib_first ? clo : slo;
-                const int pa = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, ahi, alo))) - 1;
-                const int pb = __popc(__ballot_sync(kFullMask, key_gt(whi, wlo, bhi, blo)));
+                // The head leaves, a and b enter; a missing one lands on the first empty lane.  Old entries ahead of a move up
+                // one lane, those between a and b stay, those behind b move down one: one gathering shuffle.  Every successor
+                // is behind its node in the order, so the head counts in both ballots.
+                const int pa = __popc(__ballot_sync(kFullMask, before(whi, wme, ahi, ame))) - 1;
+                const int pb = __popc(__ballot_sync(kFullMask, before(whi, wme, bhi, bme)));
                 const int src = lane + (lane < pa ? 1 : 0) - (lane > pb ? 1 : 0);      // whose old entry this lane takes
-                const uint64_t ghi = __shfl_sync(kFullMask, whi, src), glo = __shfl_sync(kFullMask, wlo, src);
+                const uint64_t ghi = __shfl_sync(kFullMask, whi, src);
+                const uint32_t gme = __shfl_sync(kFullMask, wme, src);
                 if (wn == 32 && bhi != 0ull) {                          // 33 entries: the one that does not fit goes to the pool
-                    const uint64_t lhi = __shfl_sync(kFullMask, whi, 31), llo = __shfl_sync(kFullMask, wlo, 31);
-                    if (pb == 32) to_pool(bhi, blo); else to_pool(lhi, llo);
+                    const uint64_t lhi = __shfl_sync(kFullMask, whi, 31);
+                    const uint32_t lme = __shfl_sync(kFullMask, wme, 31);
+                    if (pb == 32) to_pool(bhi, bme); else to_pool(lhi, lme);
                 }
                 wn = min(32, wn - 1 + (int)(ahi != 0ull) + (int)(bhi != 0ull));
                 whi = lane == pa ? ahi : (lane == pb ? bhi : ghi);
-                wlo = lane == pa ? alo : (lane == pb ? blo : glo);
+                wme = lane == pa ? ame : (lane == pb ? bme : gme);
             }
             __syncwarp();
             if (!trial && lane == 0) { s_fsize_end = wn + pn; __threadfence_block(); *(volatile int*)&s_pop_done = 1; }
@@ -739,8 +766,8 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
         double lp = 0.0;
         if (j == 0) { t = bonus; pos = ctx; }
         else if (j <= n) {
-            const uint64_t tb = ~nLo[j];
-            t = tb_token(tb); par = tb_parent(tb); d = tb_depth(tb); pos = ctx + d; lp = unord64(nHi[j]);
+            const uint32_t me = nMe[j];
+            d = me_depth(me); par = me_parent(me); t = tok_list[(d - 1) * K + me_rank(me) - 1]; pos = ctx + d; lp = unord64(nHi[j]);
         }
         p.token_ids[o] = t;
         p.parent_idx[o] = par;
@@ -776,7 +803,7 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             acc |= 1u << (cur & 31);
             if (brow) brow[cur] = 1;
             if (cur == 0) break;
-            const int next = tb_parent(~nLo[cur]);
+            const int next = me_parent(nMe[cur]);
             if ((next >> 5) != word) {
                 if (wrow) wrow[word] = acc;
                 acc = 0;
