@@ -1,19 +1,22 @@
 // Best-first expansion of the candidate tree with the greedy throughput stopping rule, and emission
 // of the tree arrays and the ancestor mask (Algorithm 1; Eq. 5-7, Eq. 11, Corollary 1; Section 3.3).
 //
-// One CTA per request.
-//   phase 0  all warps: merge the softmax/top-K records of each live position (candidate keys in no order,
-//            plus the mass of everything else as pairs W * 2^C) into the sorted top-K list (token,
-//            a = logit - row max) and log Z, all in fp64
-//   phase 1  one thread: running log-partition sums S_d and the reachable depth
-//   phase 2  warp 0: the pop loop.  The best 32 entries of the frontier (Algorithm 1's heap) sit in the
-//            warp's registers, sorted over the lanes on a 128-bit key (score, then the packed tie-break);
-//            what does not fit waits, unsorted, in a shared-memory pool whose best key is tracked.  A pop
-//            takes lane 0's entry and moves the others up; the popped node's next sibling and first
-//            child are inserted by one ballot (how many entries stay ahead) and one shuffle each.  Nodes
-//            are popped speculatively in groups; the group's exp(sigma), prefix sums Phi and throughput
-//            tests are then evaluated lane-parallel, and the first failing test fixes n*.  The pop order
-//            does not depend on the cost model, so this yields exactly Algorithm 1's tree.
+// One CTA of ten warps per request: eight prepare the lists, one pops, one evaluates.
+//   phase 0  eight warps, one half-warp per position: merge the softmax/top-K records of each live position (candidate
+//            keys in no order, plus the mass of everything else as pairs W * 2^C) into the sorted top-K list (token,
+//            a = logit - row max) and log Z, all in fp64.  (Small problems: there are no records, one warp per position
+//            reads the short row itself.)  Meanwhile the evaluating warp turns the cost model into a table C_v(0..B_max),
+//            and both it and the popping warp go once through their loops on a made-up node, so that the loops' code is
+//            in the SM's caches when the lists are ready.
+//   phase 1  popping warp: running log-partition sums S_d and the reachable depth
+//   phase 2  popping warp: the best 32 entries of the frontier (Algorithm 1's heap) sit in the warp's registers, sorted
+//            over the lanes on a 96-bit key (score, then depth / token / parent packed in 32 bits); what does not fit
+//            waits, unsorted, in a shared-memory pool whose best key is tracked.  A pop takes lane 0's entry; the popped
+//            node's next sibling and first child enter by two ballots (how many entries stay ahead of each) and one
+//            gathering shuffle.
+//            evaluating warp: follows through the node table; exp(sigma), Phi and the throughput test of one node after
+//            the other; the first failing test fixes n* and stops the popping warp.  The pop order does not depend on
+//            the cost model, so this yields exactly Algorithm 1's tree.
 //   phase 3  all threads: write token / parent / depth / position / log-prob rows and padding; zero
 //            the mask rows with coalesced stores, then one thread per node walks its ancestors and
 //            writes the few non-zero words (bytes for the dense form).

@@ -69,6 +69,42 @@ def test_host_validation_codes(lib):
     assert G.cadd_version() == 4
 
 
+def test_launch_counts_are_host_arithmetic(lib):
+    """cadd_build_launches / cadd_verify_launches: one kernel per call below the small-problem sizes, two above; the flags
+    that ask for the regular path or for a single kernel of it are honoured; bad shapes give the usual codes."""
+    import torch
+    # the five benchmark shapes: only configuration 1 is small
+    assert G.cadd_round_launches(1, 8, 1024, 4, 32, 33, torch.float32) == 2
+    for batch, L, K, B_max in ((32, 16, 8, 256), (128, 16, 16, 512), (64, 32, 32, 1024), (256, 16, 8, 384)):
+        assert G.cadd_round_launches(batch, L, 151936, K, B_max, B_max + 1, torch.bfloat16) == 4
+    a = G.BuildArgs(); a.struct_size = C.sizeof(G.BuildArgs)
+    a.batch, a.L, a.V, a.K, a.B_max, a.R = 1, 8, 1024, 4, 32, 33
+    a.logits_dtype = G.DTYPE_FP32
+    assert lib.cadd_build_launches(C.byref(a)) == 1
+    a.flags = G.FLAG_REGULAR_PATH
+    assert lib.cadd_build_launches(C.byref(a)) == 2
+    a.flags = G.FLAG_ONLY_TOPK
+    assert lib.cadd_build_launches(C.byref(a)) == 1          # the one kernel that was asked for
+    a.flags = 0
+    a.V = 2049                                               # rows too long to stage: regular path
+    assert lib.cadd_build_launches(C.byref(a)) == 2
+    a.V, a.batch, a.L = 2048, 64, 8                          # 64 * 8 * 2048 * 4 B = 4 MiB of draft logits: regular path
+    assert lib.cadd_build_launches(C.byref(a)) == 2
+    a.batch = 0
+    assert lib.cadd_build_launches(C.byref(a)) == G.ERR_SHAPE
+    assert lib.cadd_build_launches(None) == G.ERR_NULL
+    v = G.VerifyArgs(); v.struct_size = C.sizeof(G.VerifyArgs)
+    v.batch, v.L, v.R, v.V = 1, 8, 33, 1024
+    v.logits_dtype = G.DTYPE_FP32
+    assert lib.cadd_verify_launches(C.byref(v)) == 1
+    v.flags = G.VERIFY_REGULAR_PATH
+    assert lib.cadd_verify_launches(C.byref(v)) == 2
+    v.flags = 0
+    v.V = 8193
+    assert lib.cadd_verify_launches(C.byref(v)) == 2
+    assert lib.cadd_verify_launches(None) == G.ERR_NULL
+
+
 def test_binding_refuses_cpu_tensors():
     import torch
     with pytest.raises(ValueError):
