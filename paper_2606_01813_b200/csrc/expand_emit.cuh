@@ -168,19 +168,30 @@ __device__ __forceinline__ void row_lists_warp(const void* grow, unsigned char* 
     const void* row = buf + lead;
     uint64_t* cand = (uint64_t*)(buf + direct_row_bytes(V, DT));
 
+    // (four elements per turn in both passes, each with its own running values: one warp is alone with this row, and
+    // what it waits for is its own previous instruction)
     uint64_t mine = 0;                                       // this lane's largest finite key (0: none)
     uint32_t fl = 0;
     int nfin = 0;
-    for (int64_t i = lane; i < V; i += 32) {
-        const float x = E::load(row, i);
-        const uint32_t b = __float_as_uint(x);
-        if ((b & 0x7f800000u) == 0x7f800000u) {
-            if (b != 0xff800000u) fl |= kPartNonfinite;
-            if (b == 0x7f800000u) fl |= kPartPosInf;
-            continue;
+    {
+        uint64_t best[4] = {0ull, 0ull, 0ull, 0ull};
+        for (int64_t i0 = lane; i0 < V; i0 += 128) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int64_t i = i0 + 32 * u;
+                const float x = i < V ? E::load(row, i) : -INFINITY;
+                const uint32_t b = __float_as_uint(x);
+                const bool fin = (b & 0x7f800000u) != 0x7f800000u;
+                if (!fin && i < V) {
+                    if (b != 0xff800000u) fl |= kPartNonfinite;
+                    if (b == 0x7f800000u) fl |= kPartPosInf;
+                }
+                const uint64_t key = fin ? make_key(x, (uint32_t)i) : 0ull;
+                best[u] = max(best[u], key);
+                nfin += fin ? 1 : 0;
+            }
         }
-        mine = max(mine, make_key(x, (uint32_t)i));
-        ++nfin;
+        mine = max(max(best[0], best[1]), max(best[2], best[3]));
     }
     nfin = __reduce_add_sync(kFullMask, nfin);
     fl = __reduce_or_sync(kFullMask, fl);
@@ -203,20 +214,31 @@ __device__ __forceinline__ void row_lists_warp(const void* grow, unsigned char* 
             if (left == nx) left = 0ull;
         }
         int nc = 0;
-        for (int64_t i0 = 0; i0 < V; i0 += 32) {
-            const int64_t i = i0 + lane;
-            const float x = i < V ? E::load(row, i) : INFINITY;
-            const bool fin = fabsf(x) < INFINITY;
-            const uint64_t key = fin ? make_key(x, (uint32_t)i) : 0ull;
-            const bool is_cand = fin && key >= bound;
-            const unsigned cm = __ballot_sync(kFullMask, is_cand);
-            if (is_cand) {
-                const int at = nc + __popc(cm & ((1u << lane) - 1u));
-                if (at < kDirectCandCap) cand[at] = key;
-            } else if (fin) {
-                acc += (double)exp2_term(x, negc);
+        for (int64_t i0 = 0; i0 < V; i0 += 128) {
+            float part[4];
+            bool is_cand[4];
+            uint64_t key[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int64_t i = i0 + 32 * u + lane;
+                const float x = i < V ? E::load(row, i) : INFINITY;
+                const bool fin = fabsf(x) < INFINITY;
+                key[u] = fin ? make_key(x, (uint32_t)i) : 0ull;
+                is_cand[u] = fin && key[u] >= bound;
+                part[u] = exp2_term((fin && !is_cand[u]) ? x : -INFINITY, negc);      // 2^-inf = 0
             }
-            nc += __popc(cm);
+            acc += (double)((part[0] + part[1]) + (part[2] + part[3]));
+            if (__any_sync(kFullMask, is_cand[0] || is_cand[1] || is_cand[2] || is_cand[3])) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const unsigned cm = __ballot_sync(kFullMask, is_cand[u]);
+                    if (is_cand[u]) {
+                        const int at = nc + __popc(cm & ((1u << lane) - 1u));
+                        if (at < kDirectCandCap) cand[at] = key[u];
+                    }
+                    nc += __popc(cm);
+                }
+            }
         }
         __syncwarp();
         if (nc <= kDirectCandCap) {
@@ -300,6 +322,9 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
     for (int j = tid; j <= B_max + 1; j += kExpandThreads) nHi[j] = 0;   // "not popped yet" (see phase 2)
     __syncthreads();
     if (tid == 0 && clamped) atomicOr(&s_status, CADD_STATUS_L_EFF_CLAMPED);
+    // (used by the emission only; read here so that the emission does not start with a trip to DRAM)
+    const int ctx = p.ctx_len ? p.ctx_len[b] : 0;
+    const int bonus = p.bonus_token ? p.bonus_token[b] : -1;
 
     const int kPopWarp = kMergeWarps;                       // the last warp evaluates
     if (warp < kMergeWarps) {
@@ -752,8 +777,6 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
     __syncthreads();
     // ---------------- phase 3: emission ----------------
     const int n = s_n;
-    const int ctx = p.ctx_len ? p.ctx_len[b] : 0;
-    const int bonus = p.bonus_token ? p.bonus_token[b] : -1;
     if (tid == 0) {
         p.n_nodes[b] = n;
         if (p.phi) p.phi[b] = s_phi;
