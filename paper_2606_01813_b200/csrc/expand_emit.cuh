@@ -65,6 +65,7 @@ constexpr int kRecSegPartial = 0, kRecSegRecord = 1, kRecDirect = 2;
 // candidate keys a record of the given format holds at most
 __host__ __device__ inline int rec_key_cap(int rec_fmt, int KP) { return rec_fmt == kRecSegRecord ? seg_key_cap(KP) : (rec_fmt == kRecDirect ? 0 : KP); }
 
+constexpr int kEvalPollLimit = 1 << 20;    // polls of one node's score word before the evaluating warp gives up (tens of milliseconds)
 constexpr int kMergeWarps = 8;             // sixteen half-warps: one per draft position in the merge phase for L <= 16
 constexpr int kExpandWarps = kMergeWarps + 2;      // and the two warps of the expansion proper
 constexpr int kExpandThreads = kExpandWarps * 32;
@@ -722,7 +723,7 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
 
         int n = 0;
         double Phi = 0.0, theta_prev = theta_first;
-        bool stopped = false;
+        bool stopped = false, gave_up = false;
 #pragma unroll 1
         for (int pass = 0; pass < 2; ++pass) {
             const bool trial = pass == 0;
@@ -734,6 +735,7 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             // one node after the other, as soon as its score word is there (no score's ordered image is zero); every
             // lane does the same arithmetic, so nothing has to be exchanged
             int j = trial ? B_max + 1 : 1;
+            int polls = 0;                                          // looks at a score word that was not there yet
             while ((ok || trial) && !stopped) {
                 uint64_t sw;
                 if (trial) sw = ord64(-1.0);
@@ -741,12 +743,18 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                     if (j > B_max) break;                               // the cap: every node was worth its cost
                     sw = *(volatile uint64_t*)&nHi[j];
                     if (sw == 0ull) {
-                        if (!*(volatile int*)&s_pop_done) continue;     // not popped yet
+                        if (!*(volatile int*)&s_pop_done) {             // not popped yet
+                            // (the popping warp waits for nobody and a pop is some hundred cycles; the limit is there so
+                            // that no wait in this library is without one)
+                            if (++polls > kEvalPollLimit) { gave_up = true; break; }
+                            continue;
+                        }
                         __threadfence_block();
                         sw = *(volatile uint64_t*)&nHi[j];              // the popping warp is through: what is there now is final
                         if (sw == 0ull) break;
                     }
                 }
+                polls = 0;
                 const double Phi_j = Phi + exp(unord64(sw));
                 const double den = C_d + cv[j];
                 const bool bad = !(den > 0.0);
@@ -765,8 +773,13 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 }
             }
         }
-        if (ok && !stopped) {
-            while (!*(volatile int*)&s_pop_done) __nanosleep(40);      // (it is set: the loop above only ends that way)
+        if (gave_up) {                                              // flagged, empty tree; the popping warp is told to stop
+            if (lane == 0) *(volatile int*)&s_stop = 1;
+            st = CADD_STATUS_INTERNAL_TIMEOUT;
+            n = 0; Phi = 0.0; theta_prev = theta_first;
+        } else if (ok && !stopped) {
+            // the loop above only ends this way after it has seen the flag set (or at the cap, a pop or two before it is)
+            for (int q = 0; !*(volatile int*)&s_pop_done && q < kEvalPollLimit; ++q) __nanosleep(40);
             st |= (*(volatile int*)&s_fsize_end == 0) ? CADD_STATUS_FRONTIER_EXHAUSTED : CADD_STATUS_CAP_HIT;
         }
         if (lane == 0) {
