@@ -570,14 +570,52 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
 
             int popped = 0;
             int stop_now = 0;
+            // What a pop reads about its node: fetched as soon as the node is known, which for the usual pop is before the
+            // previous pop has finished with the window (the next head is the window's second entry or the better
+            // successor), so that the loads are under way while the window is put in order.
+            struct NodeIn { double Apar, a_cur, a_sib, a_chi, S_d, S_c; int keff_d; uint32_t pl_sib, pl_chi; };
+            auto load_node = [&](uint32_t kme) {
+                const int d = me_depth(kme), par = me_parent(kme), r = me_rank(kme);
+                const double* arow = a_list + (d - 1) * K;
+                NodeIn in;
+                in.Apar = nA[par];
+                in.a_cur = arow[r - 1];
+                // (the next sibling and the first child are read whether they exist or not: the arrays have room)
+                in.a_sib = arow[r]; in.a_chi = a_list[d * K];
+                in.S_d = Sd[d]; in.S_c = Sd[d + 1];
+                in.keff_d = keff[d];
+                in.pl_sib = place[(d - 1) * K + r]; in.pl_chi = place[d * K];
+                return in;
+            };
+            // The popped node (khi, kme) becomes row j: its score word at once (the evaluating warp waits for it), then
+            // its two successors (Algorithm 1, lines 12-19): a is the better one (equal scores: the sibling, which is
+            // less deep), b the other; a missing one is all zero.
+            auto node_and_successors = [&](uint64_t khi, uint32_t kme, const NodeIn& in, int j, uint64_t& ahi, uint32_t& ame, uint64_t& bhi, uint32_t& bme) {
+                const int d = me_depth(kme), r = me_rank(kme);
+                *(volatile uint64_t*)&nHi[j] = khi;
+                const bool has_sib = r < in.keff_d;
+                const bool has_child = d < Lr;
+                const double A = in.Apar + in.a_cur;
+                nA[j] = A;
+                nMe[j] = kme;
+                const uint64_t shi = has_sib ? ord64((in.Apar + in.a_sib) - in.S_d) : 0ull;
+                const uint32_t sme = has_sib ? ((kme & 0x3f03ffc0u) | (in.pl_sib << 18) | (uint32_t)r) : 0u;   // same depth and parent, next rank
+                const uint64_t chi = has_child ? ord64((A + in.a_chi) - in.S_c) : 0ull;
+                const uint32_t cme = has_child ? (((uint32_t)d << 24) | (in.pl_chi << 18) | ((uint32_t)j << 6)) : 0u;   // pack_meta(d + 1, place, j, 1)
+                const bool sib_first = shi >= chi;
+                ahi = sib_first ? shi : chi; bhi = sib_first ? chi : shi;
+                ame = sib_first ? sme : cme; bme = sib_first ? cme : sme;
+            };
+            uint64_t khi = __shfl_sync(kFullMask, whi, 0);          // the window's head, and what its pop will read
+            uint32_t kme = __shfl_sync(kFullMask, wme, 0);
+            NodeIn in = load_node(kme);
             while (ok && popped < limit && (wn | pn) != 0 && !stop_now) {
-                // ---- the best entry of the frontier ----
-                uint64_t khi = __shfl_sync(kFullMask, whi, 0);
-                uint32_t kme = __shfl_sync(kFullMask, wme, 0);
-                const bool general = before(pmax_hi, pmax_me, khi, kme);   // the pool holds the best entry (always, if the window is empty)
-                bool head_popped = true;
-                if (general) {
-                    // rare.  The pool's best under the total order: lanes scan stripes of the pool, then a butterfly.
+                const int j = trial ? B_max + 1 : popped + 1;
+                ++popped;
+                if (before(pmax_hi, pmax_me, khi, kme)) {
+                    // Rare: the pool holds the best entry (always, if the window is empty).  Find it (lanes scan stripes
+                    // of the pool, then a butterfly), take it out, find the pool's new best; the node's successors enter
+                    // one after the other.
                     __syncwarp();
                     uint64_t bhi = 0;
                     uint32_t bme = 0;
@@ -594,78 +632,65 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                         const int oi = __shfl_xor_sync(kFullMask, bi, o);
                         if (before(ohi, ome, bhi, bme)) { bhi = ohi; bme = ome; bi = oi; }
                     }
-                    if (bi >= 0 && before(bhi, bme, khi, kme)) {        // it beats the window's head: take it out of the pool
-                        head_popped = false;
-                        khi = bhi; kme = bme;
-                        --pn;
-                        __syncwarp();
-                        if (bi != pn) { const uint64_t lhi = pHi[pn]; const uint32_t lme = pMe[pn]; __syncwarp(); pHi[bi] = lhi; pMe[bi] = lme; }
-                        __syncwarp();
-                        bhi = 0; bme = 0;
-                        for (int q = lane; q < pn; q += 32) {
-                            const uint64_t hi = pHi[q];
-                            const uint32_t me = pMe[q];
-                            if (before(hi, me, bhi, bme)) { bhi = hi; bme = me; }
-                        }
+                    const uint64_t qhi = bhi;
+                    const uint32_t qme = bme;
+                    --pn;
+                    __syncwarp();
+                    if (bi != pn) { const uint64_t lhi = pHi[pn]; const uint32_t lme = pMe[pn]; __syncwarp(); pHi[bi] = lhi; pMe[bi] = lme; }
+                    __syncwarp();
+                    bhi = 0; bme = 0;
+                    for (int q = lane; q < pn; q += 32) {
+                        const uint64_t hi = pHi[q];
+                        const uint32_t me = pMe[q];
+                        if (before(hi, me, bhi, bme)) { bhi = hi; bme = me; }
+                    }
 #pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) {
-                            const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o);
-                            const uint32_t ome = __shfl_xor_sync(kFullMask, bme, o);
-                            if (before(ohi, ome, bhi, bme)) { bhi = ohi; bme = ome; }
-                        }
-                        pmax_hi = bhi; pmax_me = bme;
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o);
+                        const uint32_t ome = __shfl_xor_sync(kFullMask, bme, o);
+                        if (before(ohi, ome, bhi, bme)) { bhi = ohi; bme = ome; }
                     }
-                }
-                const int d = me_depth(kme), par = me_parent(kme), r = me_rank(kme);
-                const int j = trial ? B_max + 1 : popped + 1;
-                ++popped;
-                *(volatile uint64_t*)&nHi[j] = khi;                     // at once: the evaluating warp waits for this word
-                // ---- the popped node and its two successors (Algorithm 1, lines 12-19) ----
-                const double* arow = a_list + (d - 1) * K;
-                const double Apar = nA[par];
-                const double a_cur = arow[r - 1];
-                // (the next sibling and the first child are read whether they exist or not: the arrays have room)
-                const double a_sib = arow[r], a_chi = a_list[d * K];
-                const double S_d = Sd[d], S_c = Sd[d + 1];
-                const bool has_sib = r < keff[d];
-                const uint32_t pl_sib = place[(d - 1) * K + r], pl_chi = place[d * K];
-                const bool has_child = d < Lr;
-                const double A = Apar + a_cur;
-                nA[j] = A;
-                nMe[j] = kme;
-                const uint64_t shi = has_sib ? ord64((Apar + a_sib) - S_d) : 0ull;
-                const uint32_t sme = has_sib ? ((kme & 0x3f03ffc0u) | (pl_sib << 18) | (uint32_t)r) : 0u;   // same depth and parent, next rank
-                const uint64_t chi = has_child ? ord64((A + a_chi) - S_c) : 0ull;
-                const uint32_t cme = has_child ? (((uint32_t)d << 24) | (pl_chi << 18) | ((uint32_t)j << 6)) : 0u;   // pack_meta(d + 1, place, j, 1)
-                stop_now = *(volatile int*)&s_stop;                     // looked at when this pop is over
-                // a is the better of the two successors (equal scores: the sibling, which is less deep), b the other; a
-                // missing one is all zero
-                const bool sib_first = shi >= chi;
-                const uint64_t ahi = sib_first ? shi : chi, bhi = sib_first ? chi : shi;
-                const uint32_t ame = sib_first ? sme : cme, bme = sib_first ? cme : sme;
-                if (general) {                                          // one entry after the other
-                    if (head_popped) {
-                        whi = __shfl_down_sync(kFullMask, whi, 1); wme = __shfl_down_sync(kFullMask, wme, 1);
-                        if (lane == 31) { whi = 0; wme = 0; }
-                        --wn;
-                    }
+                    pmax_hi = bhi; pmax_me = bme;
+                    uint64_t ahi, b2hi;
+                    uint32_t ame, b2me;
+                    node_and_successors(qhi, qme, load_node(qme), j, ahi, ame, b2hi, b2me);
                     if (ahi != 0ull) push(ahi, ame);
-                    if (bhi != 0ull) push(bhi, bme);
+                    if (b2hi != 0ull) push(b2hi, b2me);
+                    stop_now = *(volatile int*)&s_stop;
+                    khi = __shfl_sync(kFullMask, whi, 0);
+                    kme = __shfl_sync(kFullMask, wme, 0);
+                    in = load_node(kme);
                     continue;
                 }
+                const uint64_t o1hi = __shfl_sync(kFullMask, whi, 1);      // the window's second entry: the next head unless a is
+                const uint32_t o1me = __shfl_sync(kFullMask, wme, 1);
+                uint64_t ahi, bhi;
+                uint32_t ame, bme;
+                node_and_successors(khi, kme, in, j, ahi, ame, bhi, bme);
+                stop_now = *(volatile int*)&s_stop;                     // looked at when this pop is over
                 // The head leaves, a and b enter; a missing one lands on the first empty lane.  Old entries ahead of a move up
                 // one lane, those between a and b stay, those behind b move down one: one gathering shuffle.  Every successor
                 // is behind its node in the order, so the head counts in both ballots.
                 const int pa = __popc(__ballot_sync(kFullMask, before(whi, wme, ahi, ame))) - 1;
                 const int pb = __popc(__ballot_sync(kFullMask, before(whi, wme, bhi, bme)));
+                khi = pa == 0 ? ahi : o1hi;                             // the new head; its loads go out now
+                kme = pa == 0 ? ame : o1me;
+                in = load_node(kme);
                 const int src = lane + (lane < pa ? 1 : 0) - (lane > pb ? 1 : 0);      // whose old entry this lane takes
                 const uint64_t ghi = __shfl_sync(kFullMask, whi, src);
                 const uint32_t gme = __shfl_sync(kFullMask, wme, src);
-                if (wn == 32 && bhi != 0ull) {                          // 33 entries: the one that does not fit goes to the pool
-                    const uint64_t lhi = __shfl_sync(kFullMask, whi, 31);
-                    const uint32_t lme = __shfl_sync(kFullMask, wme, 31);
-                    if (pb == 32) to_pool(bhi, bme); else to_pool(lhi, lme);
-                }
+                // 33 entries: the one that does not fit (b, if all 32 old entries come before it, else the window's last)
+                // goes to the pool; written without a branch, the stress regime spills on every pop
+                const uint64_t lhi = __shfl_sync(kFullMask, whi, 31);
+                const uint32_t lme = __shfl_sync(kFullMask, wme, 31);
+                const bool spill = wn == 32 && bhi != 0ull;
+                const uint64_t xhi = pb == 32 ? bhi : lhi;
+                const uint32_t xme = pb == 32 ? bme : lme;
+                if (spill) { pHi[pn] = xhi; pMe[pn] = xme; }
+                const bool new_best = spill && before(xhi, xme, pmax_hi, pmax_me);
+                pmax_hi = new_best ? xhi : pmax_hi;
+                pmax_me = new_best ? xme : pmax_me;
+                pn += spill ? 1 : 0;
                 wn = min(32, wn - 1 + (int)(ahi != 0ull) + (int)(bhi != 0ull));
                 whi = lane == pa ? ahi : (lane == pb ? bhi : ghi);
                 wme = lane == pa ? ame : (lane == pb ? bme : gme);
