@@ -65,6 +65,7 @@ constexpr int kRecSegPartial = 0, kRecSegRecord = 1, kRecDirect = 2;
 // candidate keys a record of the given format holds at most
 __host__ __device__ inline int rec_key_cap(int rec_fmt, int KP) { return rec_fmt == kRecSegRecord ? seg_key_cap(KP) : (rec_fmt == kRecDirect ? 0 : KP); }
 
+constexpr int kLateStopPops = 24;          // pops that look at the stop flag a second time, at their end
 constexpr int kEvalPollLimit = 1 << 20;    // polls of one node's score word before the evaluating warp gives up (tens of milliseconds)
 constexpr int kMergeWarps = 8;             // sixteen half-warps: one per draft position in the merge phase for L <= 16
 constexpr int kExpandWarps = kMergeWarps + 2;      // and the two warps of the expansion proper
@@ -543,7 +544,8 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             int pn = 0;                                         // entries in the pool
             uint64_t pmax_hi = 0;
             uint32_t pmax_me = 0;
-            auto before = [](uint64_t ahi, uint32_t ame, uint64_t bhi, uint32_t bme) { return ahi > bhi || (ahi == bhi && ame < bme); };
+            // (bitwise on purpose: three comparisons and two logic operations, no branch)
+            auto before = [](uint64_t ahi, uint32_t ame, uint64_t bhi, uint32_t bme) { return (bool)((int)(ahi > bhi) | ((int)(ahi == bhi) & (int)(ame < bme))); };
             auto to_pool = [&](uint64_t khi, uint32_t kme) {
                 pHi[pn] = khi; pMe[pn] = kme;
                 if (before(khi, kme, pmax_hi, pmax_me)) { pmax_hi = khi; pmax_me = kme; }
@@ -598,10 +600,12 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 const double A = in.Apar + in.a_cur;
                 nA[j] = A;
                 nMe[j] = kme;
-                const uint64_t shi = has_sib ? ord64((in.Apar + in.a_sib) - in.S_d) : 0ull;
-                const uint32_t sme = has_sib ? ((kme & 0x3f03ffc0u) | (in.pl_sib << 18) | (uint32_t)r) : 0u;   // same depth and parent, next rank
-                const uint64_t chi = has_child ? ord64((A + in.a_chi) - in.S_c) : 0ull;
-                const uint32_t cme = has_child ? (((uint32_t)d << 24) | (in.pl_chi << 18) | ((uint32_t)j << 6)) : 0u;   // pack_meta(d + 1, place, j, 1)
+                // (both are computed whether they exist or not and masked afterwards: no branch)
+                const uint64_t ms = 0ull - (uint64_t)has_sib, mc = 0ull - (uint64_t)has_child;
+                const uint64_t shi = ord64((in.Apar + in.a_sib) - in.S_d) & ms;
+                const uint32_t sme = ((kme & 0x3f03ffc0u) | (in.pl_sib << 18) | (uint32_t)r) & (uint32_t)ms;   // same depth and parent, next rank
+                const uint64_t chi = ord64((A + in.a_chi) - in.S_c) & mc;
+                const uint32_t cme = (((uint32_t)d << 24) | (in.pl_chi << 18) | ((uint32_t)j << 6)) & (uint32_t)mc;   // pack_meta(d + 1, place, j, 1)
                 const bool sib_first = shi >= chi;
                 ahi = sib_first ? shi : chi; bhi = sib_first ? chi : shi;
                 ame = sib_first ? sme : cme; bme = sib_first ? cme : sme;
@@ -687,13 +691,17 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 const uint64_t xhi = pb == 32 ? bhi : lhi;
                 const uint32_t xme = pb == 32 ? bme : lme;
                 if (spill) { pHi[pn] = xhi; pMe[pn] = xme; }
-                const bool new_best = spill && before(xhi, xme, pmax_hi, pmax_me);
+                const bool new_best = (bool)((int)spill & (int)before(xhi, xme, pmax_hi, pmax_me));
                 pmax_hi = new_best ? xhi : pmax_hi;
                 pmax_me = new_best ? xme : pmax_me;
                 pn += spill ? 1 : 0;
                 wn = min(32, wn - 1 + (int)(ahi != 0ull) + (int)(bhi != 0ull));
                 whi = lane == pa ? ahi : (lane == pb ? bhi : ghi);
                 wme = lane == pa ? ame : (lane == pb ? bme : gme);
+                // On the first pops the flag is read once more at the very end: the verdict on this pop's node arrives about
+                // now, and a small tree should not pay for a pop it does not need.  (Later the wait for this load would
+                // cost more than the occasional extra pop.)
+                if (popped <= kLateStopPops) stop_now |= *(volatile int*)&s_stop;
             }
             __syncwarp();
             if (!trial && lane == 0) { s_fsize_end = wn + pn; __threadfence_block(); *(volatile int*)&s_pop_done = 1; }
