@@ -440,28 +440,38 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) mk = max(mk, __shfl_xor_sync(kFullMask, mk, o));
         const double m = (double)key_value(mk);
+        // This lane's terms of Z: its keys (ranked by counting on the way), then its pair of the mass outside the lists,
+        // one (W, C) per record or per warp of the CTA that wrote it -- all through one exponential, so that its code is
+        // there once.  (A warp's W can be negative: the warp that takes a candidate's term out of the sums need not be the
+        // one that added it; only the total over a record's warps is a sum of terms.)
+        const int ns0 = __shfl_sync(kFullMask, my_ns, lane0 + ((seg_records ? hl / kSegSums : hl) & 15));
+        const bool used0 = live && hl < n_pairs && (seg_records ? hl % kSegSums < ns0 : true);
+        const int nk = n > hl ? (n - hl + 15) >> 4 : 0;        // keys of this lane
         double zsum = 0.0;
-        for (int q = hl; q < n; q += 16) {
-            const uint64_t k = scr[q];
-            int rank = 0;
-            for (int r = 0; r < n; ++r) rank += scr[r] > k;
-            const double x = (double)key_value(k);
-            zsum += exp(x - m);
-            if (rank < K) { tok_list[i * K + rank] = (int32_t)key_id(k); a_list[i * K + rank] = x - m; }
+        for (int k = 0; k <= nk; ++k) {
+            double arg, w;
+            if (k < nk) {
+                const uint64_t key = scr[hl + 16 * k];
+                int rank = 0;
+                for (int r = 0; r < n; ++r) rank += scr[r] > key;
+                const double x = (double)key_value(key);
+                arg = x - m; w = 1.0;
+                if (rank < K) { tok_list[i * K + rank] = (int32_t)key_id(key); a_list[i * K + rank] = arg; }
+            } else {
+                arg = C0 * 0.6931471805599453094 - m; w = used0 ? W0 : 0.0;
+            }
+            if (w != 0.0) zsum += w * exp(arg);
         }
-        // the mass outside the lists: one (W, C) per record, or one per warp of the CTA that wrote it
-        // (a warp's W can be negative: the warp that takes a candidate's term out of the sums need not be the one that
-        // added it; only the total over a record's warps is a sum of terms)
-        for (int t0 = 0; t0 < n_pairs; t0 += 16) {
+        for (int t0 = 16; t0 < n_pairs; t0 += 16) {             // (more than two records to a row: rare)
             const int t = t0 + hl;
             const int rec = seg_records ? t / kSegSums : t;
             const int ns = __shfl_sync(kFullMask, my_ns, lane0 + (rec & 15));
-            double W = W0, C = C0;
-            if (seg_records && t0 > 0 && t < n_pairs) {                     // (more than two records to a row: rare)
+            double W = 0.0, C = 0.0;
+            if (seg_records && t < n_pairs) {
                 const double2 wc = *(const double2*)(rec0 + (size_t)rec * pstride + sizeof(SegRecord) + (size_t)(t % kSegSums) * 16);
                 W = wc.x; C = wc.y;
             }
-            const bool used = live && t < n_pairs && (seg_records ? t % kSegSums < ns : true);
+            const bool used = live && t < n_pairs && (seg_records ? t % kSegSums < ns : false);
             if (used && W != 0.0) zsum += W * exp(C * 0.6931471805599453094 - m);
         }
 #pragma unroll
