@@ -65,6 +65,7 @@ constexpr int kRecSegPartial = 0, kRecSegRecord = 1, kRecDirect = 2;
 // candidate keys a record of the given format holds at most
 __host__ __device__ inline int rec_key_cap(int rec_fmt, int KP) { return rec_fmt == kRecSegRecord ? seg_key_cap(KP) : (rec_fmt == kRecDirect ? 0 : KP); }
 
+constexpr int kEvalOneByOne = 64;          // nodes the evaluating warp takes one at a time before it turns to batches
 constexpr int kLateStopPops = 24;          // pops that look at the stop flag a second time, at their end
 constexpr int kEvalPollLimit = 1 << 20;    // polls of one node's score word before the evaluating warp gives up (tens of milliseconds)
 constexpr int kMergeWarps = 8;             // sixteen half-warps: one per draft position in the merge phase for L <= 16
@@ -550,7 +551,6 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             // values to the node table and the pool, so a lane only ever reads back what it has written itself.
             uint64_t whi = 0;                                   // this lane's window entry
             uint32_t wme = 0;
-            int wn = 0;                                         // entries in the window
             int pn = 0;                                         // entries in the pool
             uint64_t pmax_hi = 0;
             uint32_t pmax_me = 0;
@@ -568,8 +568,9 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                     to_pool(khi, kme);
                     return;
                 }
-                if (wn == 32) to_pool(__shfl_sync(kFullMask, whi, 31), __shfl_sync(kFullMask, wme, 31));   // the last entry makes room
-                else ++wn;
+                const uint64_t lhi = __shfl_sync(kFullMask, whi, 31);     // a full window: its last entry makes room
+                const uint32_t lme = __shfl_sync(kFullMask, wme, 31);
+                if (lhi != 0ull) to_pool(lhi, lme);
                 const uint64_t uhi = __shfl_up_sync(kFullMask, whi, 1);
                 const uint32_t ume = __shfl_up_sync(kFullMask, wme, 1);
                 if (lane > pos) { whi = uhi; wme = ume; }
@@ -578,7 +579,8 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             if (trial) push(ord64(-1.0), pack_meta(1, 0, 0, 1));
             else if (ok && Lr >= 1)                             // Algorithm 1, line 3: the heap starts with node (1)
                 push(ord64(a_list[0] - Sd[1]), pack_meta(1, place[0], 0, 1));
-            const int limit = trial ? 1 : B_max;
+            const int limit = !ok ? 0 : (trial ? 1 : B_max);
+            const int jbase = trial ? B_max + 1 : 1;               // row of the first popped node
 
             int popped = 0;
             int stop_now = 0;
@@ -623,8 +625,9 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
             uint64_t khi = __shfl_sync(kFullMask, whi, 0);          // the window's head, and what its pop will read
             uint32_t kme = __shfl_sync(kFullMask, wme, 0);
             NodeIn in = load_node(kme);
-            while (ok && popped < limit && (wn | pn) != 0 && !stop_now) {
-                const int j = trial ? B_max + 1 : popped + 1;
+            // (the frontier is empty when the window's head is and the pool holds nothing)
+            while (popped < limit && (khi != 0ull || pn != 0) && !stop_now) {
+                const int j = popped + jbase;
                 ++popped;
                 if (before(pmax_hi, pmax_me, khi, kme)) {
                     // Rare: the pool holds the best entry (always, if the window is empty).  Find it (lanes scan stripes
@@ -685,11 +688,14 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 // The head leaves, a and b enter; a missing one lands on the first empty lane.  Old entries ahead of a move up
                 // one lane, those between a and b stay, those behind b move down one: one gathering shuffle.  Every successor
                 // is behind its node in the order, so the head counts in both ballots.
+                // the new head is the window's second entry unless a comes before it (known without the ballots); its
+                // loads go out now
+                const bool second_stays = before(o1hi, o1me, ahi, ame);
+                khi = second_stays ? o1hi : ahi;
+                kme = second_stays ? o1me : ame;
+                in = load_node(kme);
                 const int pa = __popc(__ballot_sync(kFullMask, before(whi, wme, ahi, ame))) - 1;
                 const int pb = __popc(__ballot_sync(kFullMask, before(whi, wme, bhi, bme)));
-                khi = pa == 0 ? ahi : o1hi;                             // the new head; its loads go out now
-                kme = pa == 0 ? ame : o1me;
-                in = load_node(kme);
                 const int src = lane + (lane < pa ? 1 : 0) - (lane > pb ? 1 : 0);      // whose old entry this lane takes
                 const uint64_t ghi = __shfl_sync(kFullMask, whi, src);
                 const uint32_t gme = __shfl_sync(kFullMask, wme, src);
@@ -697,7 +703,7 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 // goes to the pool; written without a branch, the stress regime spills on every pop
                 const uint64_t lhi = __shfl_sync(kFullMask, whi, 31);
                 const uint32_t lme = __shfl_sync(kFullMask, wme, 31);
-                const bool spill = wn == 32 && bhi != 0ull;
+                const bool spill = lhi != 0ull && bhi != 0ull;          // a full window and two new entries
                 const uint64_t xhi = pb == 32 ? bhi : lhi;
                 const uint32_t xme = pb == 32 ? bme : lme;
                 if (spill) { pHi[pn] = xhi; pMe[pn] = xme; }
@@ -705,7 +711,6 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 pmax_hi = new_best ? xhi : pmax_hi;
                 pmax_me = new_best ? xme : pmax_me;
                 pn += spill ? 1 : 0;
-                wn = min(32, wn - 1 + (int)(ahi != 0ull) + (int)(bhi != 0ull));
                 whi = lane == pa ? ahi : (lane == pb ? bhi : ghi);
                 wme = lane == pa ? ame : (lane == pb ? bme : gme);
                 // On the first pops the flag is read once more at the very end: the verdict on this pop's node arrives about
@@ -714,7 +719,7 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 if (popped <= kLateStopPops) stop_now |= *(volatile int*)&s_stop;
             }
             __syncwarp();
-            if (!trial && lane == 0) { s_fsize_end = wn + pn; __threadfence_block(); *(volatile int*)&s_pop_done = 1; }
+            if (!trial && lane == 0) { s_fsize_end = (khi != 0ull ? 1 : 0) + pn; __threadfence_block(); *(volatile int*)&s_pop_done = 1; }
         }
     } else {
         // the cost model of this request as a table: C_v(n) for every n the tree can reach, and the draft cost C_d
@@ -775,15 +780,16 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 if (*(volatile int*)&s_pinf) ok = false;
             }
             n = 0; Phi = 0.0; theta_prev = theta_first; stopped = false;
-            // one node after the other, as soon as its score word is there (no score's ordered image is zero); every
-            // lane does the same arithmetic, so nothing has to be exchanged
+            // The first nodes one after the other, as soon as a node's score word is there (no score's ordered image is
+            // zero); every lane does the same arithmetic, so nothing has to be exchanged and the verdict on a node is out
+            // within a pop.  (Small trees end here.)
             int j = trial ? B_max + 1 : 1;
             int polls = 0;                                          // looks at a score word that was not there yet
             while ((ok || trial) && !stopped) {
                 uint64_t sw;
                 if (trial) sw = ord64(-1.0);
                 else {
-                    if (j > B_max) break;                               // the cap: every node was worth its cost
+                    if (j > B_max || j > kEvalOneByOne) break;          // the cap (every node was worth its cost), or the batches' turn
                     sw = *(volatile uint64_t*)&nHi[j];
                     if (sw == 0ull) {
                         if (!*(volatile int*)&s_pop_done) {             // not popped yet
@@ -814,6 +820,51 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                     n = j;
                     ++j;
                 }
+            }
+            // A large tree: whatever has been popped since the last look, up to 32 nodes at a time, one per lane: the
+            // exponentials and the divisions side by side, so that this warp keeps ahead of the popping warp whatever
+            // that one's pace; Phi is still summed in node order (every lane adds up its own prefix).
+            while (!trial && ok && !stopped && !gave_up && j <= B_max) {
+                const int jj = j + lane;
+                uint64_t sw = jj <= B_max ? *(volatile uint64_t*)&nHi[jj] : 0ull;
+                unsigned have = __ballot_sync(kFullMask, sw != 0ull);
+                if ((have & 1u) == 0u) {
+                    if (!*(volatile int*)&s_pop_done) {
+                        if (++polls > kEvalPollLimit) gave_up = true;
+                        continue;
+                    }
+                    __threadfence_block();
+                    sw = jj <= B_max ? *(volatile uint64_t*)&nHi[jj] : 0ull;   // the popping warp is through: what is there now is final
+                    have = __ballot_sync(kFullMask, sw != 0ull);
+                    if ((have & 1u) == 0u) break;
+                }
+                polls = 0;
+                const int g = have == 0xffffffffu ? 32 : __ffs(~have) - 1;      // the nodes that are there form a prefix
+                const bool act = lane < g;
+                const double delta = act ? exp(unord64(sw)) : 0.0;
+                double Phi_l = Phi;
+                for (int i = 0; i < g; ++i) {
+                    const double di = __shfl_sync(kFullMask, delta, i);
+                    if (i <= lane) Phi_l += di;
+                }
+                const double den = act ? C_d + cv[jj] : 1.0;
+                const bool bad = !(den > 0.0);
+                const double theta_l = (1.0 + Phi_l) / den;
+                double theta_before = __shfl_up_sync(kFullMask, theta_l, 1);
+                if (lane == 0) theta_before = theta_prev;
+                const unsigned sm = __ballot_sync(kFullMask, act && (bad || (!fixed && theta_l <= theta_before)));
+                const int f = sm ? __ffs(sm) - 1 : g;                           // nodes j .. j + f - 1 are accepted
+                if (sm && lane == 0) *(volatile int*)&s_stop = 1;
+                if (p.theta_curve && lane < f) p.theta_curve[(int64_t)b * R + jj] = theta_l;
+                if (sm) {
+                    if (__shfl_sync(kFullMask, (int)bad, f)) st |= CADD_STATUS_COST_NONPOSITIVE;
+                    stopped = true;
+                }
+                if (f > 0) {
+                    Phi = __shfl_sync(kFullMask, Phi_l, f - 1);
+                    theta_prev = __shfl_sync(kFullMask, theta_l, f - 1);
+                }
+                n += f; j += f;
             }
         }
         if (gave_up) {                                              // flagged, empty tree; the popping warp is told to stop
