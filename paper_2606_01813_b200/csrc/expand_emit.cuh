@@ -291,6 +291,52 @@ __device__ __forceinline__ void row_lists_warp(const void* grow, unsigned char* 
 // evaluating warp before their real pass.
 __device__ __forceinline__ void lists_ready_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kExpandThreads) : "memory"); }
 
+// The pool's turn (rare): finds the pool's best entry under the order of the frontier (lanes scan stripes of the pool, then
+// a butterfly), takes it out (the last entry fills its slot) and finds the new best.  Out of line: the usual pop should
+// not carry this code.
+struct PoolTake { uint64_t qhi, pmax_hi; uint32_t qme, pmax_me; };   // the entry taken, and the pool's best after it
+__device__ __noinline__ PoolTake pool_take_best(uint64_t* pHi, uint32_t* pMe, int pn) {   // pn: entries before the call (one fewer after)
+    const int lane = threadIdx.x & 31;
+    auto before = [](uint64_t ahi, uint32_t ame, uint64_t bhi, uint32_t bme) { return (bool)((int)(ahi > bhi) | ((int)(ahi == bhi) & (int)(ame < bme))); };
+    __syncwarp();
+    uint64_t bhi = 0;
+    uint32_t bme = 0;
+    int bi = -1;
+    for (int q = lane; q < pn; q += 32) {
+        const uint64_t hi = pHi[q];
+        const uint32_t me = pMe[q];
+        if (before(hi, me, bhi, bme)) { bhi = hi; bme = me; bi = q; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o);
+        const uint32_t ome = __shfl_xor_sync(kFullMask, bme, o);
+        const int oi = __shfl_xor_sync(kFullMask, bi, o);
+        if (before(ohi, ome, bhi, bme)) { bhi = ohi; bme = ome; bi = oi; }
+    }
+    PoolTake out;
+    out.qhi = bhi;
+    out.qme = bme;
+    --pn;
+    __syncwarp();
+    if (bi != pn) { const uint64_t lhi = pHi[pn]; const uint32_t lme = pMe[pn]; __syncwarp(); pHi[bi] = lhi; pMe[bi] = lme; }
+    __syncwarp();
+    bhi = 0; bme = 0;
+    for (int q = lane; q < pn; q += 32) {
+        const uint64_t hi = pHi[q];
+        const uint32_t me = pMe[q];
+        if (before(hi, me, bhi, bme)) { bhi = hi; bme = me; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o);
+        const uint32_t ome = __shfl_xor_sync(kFullMask, bme, o);
+        if (before(ohi, ome, bhi, bme)) { bhi = ohi; bme = ome; }
+    }
+    out.pmax_hi = bhi; out.pmax_me = bme;
+    return out;
+}
+
 // kDirect: the kernel for p.rec_fmt == kRecDirect (its own instantiation, so that neither carries the other's phase 0)
 template <bool kDirect>
 __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandParams p) {
@@ -633,41 +679,11 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                     // Rare: the pool holds the best entry (always, if the window is empty).  Find it (lanes scan stripes
                     // of the pool, then a butterfly), take it out, find the pool's new best; the node's successors enter
                     // one after the other.
-                    __syncwarp();
-                    uint64_t bhi = 0;
-                    uint32_t bme = 0;
-                    int bi = -1;
-                    for (int q = lane; q < pn; q += 32) {
-                        const uint64_t hi = pHi[q];
-                        const uint32_t me = pMe[q];
-                        if (before(hi, me, bhi, bme)) { bhi = hi; bme = me; bi = q; }
-                    }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o);
-                        const uint32_t ome = __shfl_xor_sync(kFullMask, bme, o);
-                        const int oi = __shfl_xor_sync(kFullMask, bi, o);
-                        if (before(ohi, ome, bhi, bme)) { bhi = ohi; bme = ome; bi = oi; }
-                    }
-                    const uint64_t qhi = bhi;
-                    const uint32_t qme = bme;
+                    const PoolTake took = pool_take_best(pHi, pMe, pn);
                     --pn;
-                    __syncwarp();
-                    if (bi != pn) { const uint64_t lhi = pHi[pn]; const uint32_t lme = pMe[pn]; __syncwarp(); pHi[bi] = lhi; pMe[bi] = lme; }
-                    __syncwarp();
-                    bhi = 0; bme = 0;
-                    for (int q = lane; q < pn; q += 32) {
-                        const uint64_t hi = pHi[q];
-                        const uint32_t me = pMe[q];
-                        if (before(hi, me, bhi, bme)) { bhi = hi; bme = me; }
-                    }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        const uint64_t ohi = __shfl_xor_sync(kFullMask, bhi, o);
-                        const uint32_t ome = __shfl_xor_sync(kFullMask, bme, o);
-                        if (before(ohi, ome, bhi, bme)) { bhi = ohi; bme = ome; }
-                    }
-                    pmax_hi = bhi; pmax_me = bme;
+                    pmax_hi = took.pmax_hi; pmax_me = took.pmax_me;
+                    const uint64_t qhi = took.qhi;
+                    const uint32_t qme = took.qme;
                     uint64_t ahi, b2hi;
                     uint32_t ame, b2me;
                     node_and_successors(qhi, qme, load_node(qme), j, ahi, ame, b2hi, b2me);
