@@ -291,6 +291,61 @@ __device__ __forceinline__ void row_lists_warp(const void* grow, unsigned char* 
 // evaluating warp before their real pass.
 __device__ __forceinline__ void lists_ready_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kExpandThreads) : "memory"); }
 
+// The evaluating warp on a large tree: whatever has been popped since the last look, up to 32 nodes at a time, one per
+// lane: the exponentials and the divisions side by side, so that this warp keeps ahead of the popping warp whatever that
+// one's pace; Phi is still summed in node order (every lane adds up its own prefix).  Takes over at node es.j with es.n
+// nodes accepted; returns when the stopping rule fires (end & 1), the popping warp is through, or a wait ran out (end & 2).
+struct EvalState { double Phi, theta_prev; int j, n, st, end; };
+__device__ __noinline__ EvalState evaluate_in_batches(EvalState es, const uint64_t* nHi, const double* cv, double* theta_curve_row,
+                                                      int B_max, double C_d, bool fixed, int* s_stop, int* s_pop_done) {
+    const int lane = threadIdx.x & 31;
+    int polls = 0;
+    while (es.j <= B_max) {
+        const int jj = es.j + lane;
+        uint64_t sw = jj <= B_max ? *(volatile const uint64_t*)&nHi[jj] : 0ull;
+        unsigned have = __ballot_sync(kFullMask, sw != 0ull);
+        if ((have & 1u) == 0u) {
+            if (!*(volatile int*)s_pop_done) {
+                if (++polls > kEvalPollLimit) { es.end |= 2; break; }
+                continue;
+            }
+            __threadfence_block();
+            sw = jj <= B_max ? *(volatile const uint64_t*)&nHi[jj] : 0ull;   // the popping warp is through: what is there now is final
+            have = __ballot_sync(kFullMask, sw != 0ull);
+            if ((have & 1u) == 0u) break;
+        }
+        polls = 0;
+        const int g = have == 0xffffffffu ? 32 : __ffs(~have) - 1;      // the nodes that are there form a prefix
+        const bool act = lane < g;
+        const double delta = act ? exp(unord64(sw)) : 0.0;
+        double Phi_l = es.Phi;
+        for (int i = 0; i < g; ++i) {
+            const double di = __shfl_sync(kFullMask, delta, i);
+            if (i <= lane) Phi_l += di;
+        }
+        const double den = act ? C_d + cv[jj] : 1.0;
+        const bool bad = !(den > 0.0);
+        const double theta_l = (1.0 + Phi_l) / den;
+        double theta_before = __shfl_up_sync(kFullMask, theta_l, 1);
+        if (lane == 0) theta_before = es.theta_prev;
+        const unsigned sm = __ballot_sync(kFullMask, act && (bad || (!fixed && theta_l <= theta_before)));
+        const int f = sm ? __ffs(sm) - 1 : g;                           // nodes j .. j + f - 1 are accepted
+        if (sm && lane == 0) *(volatile int*)s_stop = 1;
+        if (theta_curve_row && lane < f) theta_curve_row[jj] = theta_l;
+        if (f > 0) {
+            es.Phi = __shfl_sync(kFullMask, Phi_l, f - 1);
+            es.theta_prev = __shfl_sync(kFullMask, theta_l, f - 1);
+        }
+        es.n += f; es.j += f;
+        if (sm) {
+            if (__shfl_sync(kFullMask, (int)bad, f)) es.st |= CADD_STATUS_COST_NONPOSITIVE;
+            es.end |= 1;
+            break;
+        }
+    }
+    return es;
+}
+
 // The pool's turn (rare): finds the pool's best entry under the order of the frontier (lanes scan stripes of the pool, then
 // a butterfly), takes it out (the last entry fills its slot) and finds the new best.  Out of line: the usual pop should
 // not carry this code.
@@ -837,50 +892,12 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                     ++j;
                 }
             }
-            // A large tree: whatever has been popped since the last look, up to 32 nodes at a time, one per lane: the
-            // exponentials and the divisions side by side, so that this warp keeps ahead of the popping warp whatever
-            // that one's pace; Phi is still summed in node order (every lane adds up its own prefix).
-            while (!trial && ok && !stopped && !gave_up && j <= B_max) {
-                const int jj = j + lane;
-                uint64_t sw = jj <= B_max ? *(volatile uint64_t*)&nHi[jj] : 0ull;
-                unsigned have = __ballot_sync(kFullMask, sw != 0ull);
-                if ((have & 1u) == 0u) {
-                    if (!*(volatile int*)&s_pop_done) {
-                        if (++polls > kEvalPollLimit) gave_up = true;
-                        continue;
-                    }
-                    __threadfence_block();
-                    sw = jj <= B_max ? *(volatile uint64_t*)&nHi[jj] : 0ull;   // the popping warp is through: what is there now is final
-                    have = __ballot_sync(kFullMask, sw != 0ull);
-                    if ((have & 1u) == 0u) break;
-                }
-                polls = 0;
-                const int g = have == 0xffffffffu ? 32 : __ffs(~have) - 1;      // the nodes that are there form a prefix
-                const bool act = lane < g;
-                const double delta = act ? exp(unord64(sw)) : 0.0;
-                double Phi_l = Phi;
-                for (int i = 0; i < g; ++i) {
-                    const double di = __shfl_sync(kFullMask, delta, i);
-                    if (i <= lane) Phi_l += di;
-                }
-                const double den = act ? C_d + cv[jj] : 1.0;
-                const bool bad = !(den > 0.0);
-                const double theta_l = (1.0 + Phi_l) / den;
-                double theta_before = __shfl_up_sync(kFullMask, theta_l, 1);
-                if (lane == 0) theta_before = theta_prev;
-                const unsigned sm = __ballot_sync(kFullMask, act && (bad || (!fixed && theta_l <= theta_before)));
-                const int f = sm ? __ffs(sm) - 1 : g;                           // nodes j .. j + f - 1 are accepted
-                if (sm && lane == 0) *(volatile int*)&s_stop = 1;
-                if (p.theta_curve && lane < f) p.theta_curve[(int64_t)b * R + jj] = theta_l;
-                if (sm) {
-                    if (__shfl_sync(kFullMask, (int)bad, f)) st |= CADD_STATUS_COST_NONPOSITIVE;
-                    stopped = true;
-                }
-                if (f > 0) {
-                    Phi = __shfl_sync(kFullMask, Phi_l, f - 1);
-                    theta_prev = __shfl_sync(kFullMask, theta_l, f - 1);
-                }
-                n += f; j += f;
+            // A large tree goes on in batches (out of line: small trees never get there).
+            if (!trial && ok && !stopped && !gave_up && j <= B_max) {
+                const EvalState es = evaluate_in_batches(EvalState{Phi, theta_prev, j, n, st, 0}, nHi, cv, p.theta_curve ? p.theta_curve + (int64_t)b * R : nullptr,
+                                                         B_max, C_d, fixed, &s_stop, &s_pop_done);
+                Phi = es.Phi; theta_prev = es.theta_prev; j = es.j; n = es.n; st = es.st;
+                stopped = (es.end & 1) != 0; gave_up = (es.end & 2) != 0;
             }
         }
         if (gave_up) {                                              // flagged, empty tree; the popping warp is told to stop
