@@ -142,7 +142,9 @@ def test_random_small_problems_wide_lists_masked_positions_offsets(seed):
             x[m < 0.05] = float("-inf")
             x[(m > 0.05) & (m < 0.07)] = float("nan")
         x = x.to(dtype)
-        coef = torch.tensor([[rng.choice([0.3, 1.0]), rng.choice([0.5, 2.0]), rng.choice([0.0, 0.01, 0.05]), rng.choice([0.0, 0.0005])]
+        # (the marginal cost is kept positive: with a constant cost the rule stops where a node's probability drops below
+        # the rounding of 1 + Phi, which is not a property of the tree)
+        coef = torch.tensor([[rng.choice([0.3, 1.0]), rng.choice([0.5, 2.0]), rng.choice([0.002, 0.01, 0.05]), rng.choice([0.0, 0.0005])]
                              for _ in range(batch)], dtype=torch.float64)
         le = torch.tensor(rng.integers(0, L + 1, size=batch), dtype=torch.int32)
         flags = G.FLAG_FIXED_BUDGET if rng.integers(0, 2) else 0
