@@ -15,8 +15,9 @@
 //            node's next sibling and first child enter by two ballots (how many entries stay ahead of each) and one
 //            gathering shuffle.
 //            evaluating warp: follows through the node table; exp(sigma), Phi and the throughput test of one node after
-//            the other; the first failing test fixes n* and stops the popping warp.  The pop order does not depend on
-//            the cost model, so this yields exactly Algorithm 1's tree.
+//            the other (past the first 64: of up to 32 nodes at a time, one per lane); the first failing test fixes n*
+//            and stops the popping warp.  The pop order does not depend on the cost model, so this yields exactly
+//            Algorithm 1's tree.
 //   phase 3  all threads: write token / parent / depth / position / log-prob rows and padding; zero
 //            the mask rows with coalesced stores, then one thread per node walks its ancestors and
 //            writes the few non-zero words (bytes for the dense form).
