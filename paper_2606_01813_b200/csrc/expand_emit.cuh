@@ -549,17 +549,30 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
         // one that added it; only the total over a record's warps is a sum of terms.)
         const int ns0 = __shfl_sync(kFullMask, my_ns, lane0 + ((seg_records ? hl / kSegSums : hl) & 15));
         const bool used0 = live && hl < n_pairs && (seg_records ? hl % kSegSums < ns0 : true);
+        // ranks by counting, four of this lane's keys against each key of the row at a time (one load serves four compares)
+        for (int q0 = hl; q0 < n; q0 += 64) {
+            uint64_t key[4];
+            int rank[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) key[u] = q0 + 16 * u < n ? scr[q0 + 16 * u] : ~0ull;   // (nothing is above ~0: no rank, no store)
+            for (int r = 0; r < n; ++r) {
+                const uint64_t v = scr[r];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) rank[u] += v > key[u] ? 1 : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (q0 + 16 * u < n && rank[u] < K) {
+                    tok_list[i * K + rank[u]] = (int32_t)key_id(key[u]);
+                    a_list[i * K + rank[u]] = (double)key_value(key[u]) - m;
+                }
+        }
         const int nk = n > hl ? (n - hl + 15) >> 4 : 0;        // keys of this lane
         double zsum = 0.0;
         for (int k = 0; k <= nk; ++k) {
             double arg, w;
             if (k < nk) {
-                const uint64_t key = scr[hl + 16 * k];
-                int rank = 0;
-                for (int r = 0; r < n; ++r) rank += scr[r] > key;
-                const double x = (double)key_value(key);
-                arg = x - m; w = 1.0;
-                if (rank < K) { tok_list[i * K + rank] = (int32_t)key_id(key); a_list[i * K + rank] = arg; }
+                arg = (double)key_value(scr[hl + 16 * k]) - m; w = 1.0;
             } else {
                 arg = C0 * 0.6931471805599453094 - m; w = used0 ? W0 : 0.0;
             }
