@@ -957,22 +957,18 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
     }
     const bool dense = (p.flags & CADD_FLAG_EMIT_DENSE_MASK) && p.mask_dense;
     const int W = (R + 31) >> 5;
-    // all rows zero first (coalesced), then the few non-zero words / bytes of the live rows
-    if (p.mask_bits) {
-        uint32_t* base = p.mask_bits + (int64_t)b * R * W;
-        for (int64_t q = tid; q < (int64_t)R * W; q += kExpandThreads) base[q] = 0u;
-    }
-    if (dense) {
-        uint8_t* base = p.mask_dense + (int64_t)b * R * R;
-        const int64_t total = (int64_t)R * R;
-        int64_t head = (4 - (int64_t)((uintptr_t)base & 3)) & 3;
+    // all rows zero first (16 bytes per store between the ragged ends), then the few non-zero words / bytes of the live rows
+    auto zero_bytes = [&](unsigned char* base, int64_t total) {
+        int64_t head = (16 - (int64_t)((uintptr_t)base & 15)) & 15;
         if (head > total) head = total;
-        const int64_t words = (total - head) >> 2;
+        const int64_t chunks = (total - head) >> 4;
         if (tid < head) base[tid] = 0;
-        uint32_t* mid = (uint32_t*)(base + head);
-        for (int64_t q = tid; q < words; q += kExpandThreads) mid[q] = 0u;
-        for (int64_t q = head + words * 4 + tid; q < total; q += kExpandThreads) base[q] = 0;
-    }
+        uint4* mid = (uint4*)(base + head);
+        for (int64_t q = tid; q < chunks; q += kExpandThreads) mid[q] = make_uint4(0u, 0u, 0u, 0u);
+        for (int64_t q = head + chunks * 16 + tid; q < total; q += kExpandThreads) base[q] = 0;
+    };
+    if (p.mask_bits) zero_bytes((unsigned char*)(p.mask_bits + (int64_t)b * R * W), (int64_t)R * W * 4);
+    if (dense) zero_bytes(p.mask_dense + (int64_t)b * R * R, (int64_t)R * R);
     __syncthreads();
     for (int j = tid; j <= n; j += kExpandThreads) {              // self and ancestors: at most L+1 bits, rows descending
         uint32_t* wrow = p.mask_bits ? p.mask_bits + ((int64_t)b * R + j) * W : nullptr;
