@@ -116,7 +116,8 @@ __host__ __device__ inline ExpandLayout expand_layout(int L, int K, int key_cap,
     o.region = p;   p += region;
     o.tok_list = p; p += ((size_t)L + 1) * K * 4;
     o.keff = p;     p += ((size_t)L + 2) * 4;
-    o.place = p;    p += ((size_t)L + 1) * K;
+    o.place = p;    p += ((size_t)L + 2) * K + 8;               // (the last array: room for the reads one past a list's end and
+                                                                 // for the rank the trial pass may make up)
     o.total = (p + 15) & ~(size_t)15;
     return o;
 }
@@ -713,7 +714,8 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
                 in.a_sib = arow[r]; in.a_chi = a_list[d * K];
                 in.S_d = Sd[d]; in.S_c = Sd[d + 1];
                 in.keff_d = keff[d];
-                in.pl_sib = place[(d - 1) * K + r]; in.pl_chi = place[d * K];
+                // (six bits each: what the trial pass reads here is whatever the memory holds, and must stay in its field)
+                in.pl_sib = place[(d - 1) * K + r] & 63u; in.pl_chi = place[d * K] & 63u;
                 return in;
             };
             // The popped node (khi, kme) becomes row j: its score word at once (the evaluating warp waits for it), then
