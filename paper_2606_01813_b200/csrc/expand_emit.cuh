@@ -527,16 +527,17 @@ __global__ void __launch_bounds__(kExpandThreads, 2) expand_emit_kernel(ExpandPa
         for (int o = 8; o > 0; o >>= 1) fl |= __shfl_xor_sync(kFullMask, fl, o);
         // keep the slots that are in use, in place (a batch of 16 is read before its survivors are written below it)
         int n = 0;
-        for (int base = 0; base < slots; base += 16) {
-            const int e = base + hl;
-            const int s = min(e / key_cap, p.S - 1);
+        for (int s = 0; s < p.S; ++s) {
             const int cnt_s = __shfl_sync(kFullMask, my_cnt, lane0 + s);
-            const bool valid = e < slots && e - s * key_cap < cnt_s;
-            const uint64_t key = valid ? scr[e] : 0ull;
-            const unsigned m = (__ballot_sync(kFullMask, valid) >> lane0) & 0xffffu;
-            __syncwarp();
-            if (valid) scr[n + __popc(m & ((1u << hl) - 1u))] = key;
-            n += __popc(m);
+            for (int q0 = 0; q0 < key_cap; q0 += 16) {
+                const int q = q0 + hl;
+                const bool valid = q < cnt_s;                   // (cnt_s <= key_cap)
+                const uint64_t key = valid ? scr[s * key_cap + q] : 0ull;
+                const unsigned m = (__ballot_sync(kFullMask, valid) >> lane0) & 0xffffu;
+                __syncwarp();
+                if (valid) scr[n + __popc(m & ((1u << hl) - 1u))] = key;
+                n += __popc(m);
+            }
         }
         __syncwarp();
         uint64_t mk = 0;
