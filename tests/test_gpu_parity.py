@@ -156,6 +156,41 @@ def test_random_small_problems_wide_lists_masked_positions_offsets(seed):
         assert diag["max_logZ_err"] < 1e-6
 
 
+@pytest.mark.parametrize("seed", [0, 1])
+def test_random_midsize_problems_wide_lists_masked_positions_offsets(seed):
+    """The same mix on vocabularies of thousands to 150 thousand tokens (several tiles and segments per row, records of up
+    to 256 keys), where every call takes the two-kernel path."""
+    rng = np.random.default_rng(777 + seed)
+    g = torch.Generator().manual_seed(5 + seed)
+    for trial in range(10):
+        batch, L = int(rng.choice([1, 2, 3])), int(rng.choice([1, 2, 5, 8, 16, 32]))
+        V = int(rng.choice([2049, 3000, 8192, 20000, 50001, 151936]))
+        K, B = int(rng.choice([1, 2, 4, 8, 13, 32, 40, 64])), int(rng.choice([0, 1, 5, 32, 100, 300]))
+        dtype = torch.float32 if rng.integers(0, 2) else torch.bfloat16
+        off = int(rng.choice([0, 1, 3, 4, 5]))
+        mode = ["normal", "ties", "flat", "nonfinite"][int(rng.integers(0, 4))]
+        x = torch.randn(batch, L, V + 8, generator=g) * float(rng.choice([0.5, 1.0, 3.0]))
+        if mode == "ties":
+            x = torch.round(x * 2) / 2
+        elif mode == "flat":
+            x = torch.zeros_like(x)
+        elif mode == "nonfinite":
+            m = torch.rand(x.shape, generator=g)
+            x[m < 0.05] = float("-inf")
+            x[(m > 0.05) & (m < 0.07)] = float("nan")
+        x = x.to(dtype)
+        coef = torch.tensor([[rng.choice([0.3, 1.0]), rng.choice([0.5, 2.0]), rng.choice([0.002, 0.01, 0.05]), rng.choice([0.0, 0.0005])]
+                             for _ in range(batch)], dtype=torch.float64)
+        le = torch.tensor(rng.integers(0, L + 1, size=batch), dtype=torch.int32)
+        flags = G.FLAG_FIXED_BUDGET if rng.integers(0, 2) else 0
+        ot = O.build_tree(x[:, :, off:off + V].contiguous(), K, B, cost_coef=coef, l_eff=le, flags=flags)
+        gt = G.cadd_build_tree(x.cuda()[:, :, off:off + V], K, B, cost_coef=coef, l_eff=le, flags=flags | G.FLAG_EMIT_TOPK)
+        torch.cuda.synchronize()
+        diag = compare_build(gt, ot, K)
+        assert not diag["exempt"], (diag, batch, L, V, K, B, dtype, off, mode)
+        assert diag["max_logZ_err"] < 1e-6
+
+
 def test_unaligned_rows_and_strides():
     """Row starts that are not 16-byte aligned (odd V, offset base) go through the scalar head/tail path."""
     g = torch.Generator().manual_seed(5)
