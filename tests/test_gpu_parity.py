@@ -191,6 +191,41 @@ def test_random_midsize_problems_wide_lists_masked_positions_offsets(seed):
         assert diag["max_logZ_err"] < 1e-6
 
 
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_random_rounds_verification_both_row_modes(seed):
+    """Random full rounds on small and mid-size vocabularies: the tree from the builder, target logits that agree with the
+    tree's tokens at a random share of the nodes (and tie, or hold NaN, in places), verification in both row modes."""
+    rng = np.random.default_rng(31337 + seed)
+    g = torch.Generator().manual_seed(17 + seed)
+    for trial in range(8):
+        batch, L = int(rng.choice([1, 2, 4])), int(rng.choice([1, 3, 8, 16]))
+        V = int(rng.choice([2, 33, 257, 1024, 4099, 8192, 20000]))
+        K, B = int(rng.choice([1, 2, 4, 8])), int(rng.choice([1, 8, 32, 100]))
+        dtype = torch.float32 if rng.integers(0, 2) else torch.bfloat16
+        x = (torch.randn(batch, L, V, generator=g) * 2.0).to(dtype)
+        coef = torch.tensor([[0.3, 0.5, 0.002, 0.0]] * batch, dtype=torch.float64)
+        gt, ot = run_both_build(x, K, B, cost_coef=coef, flags=G.FLAG_FIXED_BUDGET if trial % 2 else 0)
+        assert not compare_build(gt, ot, K)["exempt"]
+        R = B + 1
+        y = torch.randn(batch, R, V, generator=g)
+        if trial % 3 == 0:
+            y = torch.round(y)                                  # arg-max ties: the lowest id wins
+        agree = float(rng.choice([0.3, 0.7, 1.0]))
+        tok, par = ot.token_ids, ot.parent_idx
+        for b in range(batch):                                  # plant the child's token at its parent's row
+            for j in range(1, int(ot.n_nodes[b]) + 1):
+                if rng.random() < agree:
+                    y[b, int(par[b, j]), int(tok[b, j])] = 50.0 + j
+        if trial % 4 == 1:
+            y[:, :, 0] = float("nan")
+        y = y.to(dtype)
+        for rows_mode in (G.ROWS_LIVE, G.ROWS_DENSE):
+            ov = O.verify_tree(y, L, ot.n_nodes, ot.token_ids, ot.parent_idx, rows_mode)
+            gv = G.cadd_verify_tree(y.cuda(), L, gt.n_nodes, gt.token_ids, gt.parent_idx, rows_mode)
+            torch.cuda.synchronize()
+            compare_verify(gv, ov)
+
+
 def test_unaligned_rows_and_strides():
     """Row starts that are not 16-byte aligned (odd V, offset base) go through the scalar head/tail path."""
     g = torch.Generator().manual_seed(5)
